@@ -1,0 +1,13 @@
+"""CPU oracle for the DReSD retrieval path: test infrastructure only.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package.  It never imports the CUDA package.
+"""
+from .dresd_oracle import (  # noqa: F401
+    build,
+    decode,
+    preprocess,
+    scores,
+    retrieve,
+    OracleResult,
+)

@@ -1,0 +1,209 @@
+/*
+ * DReSD dense-retrieval oracle: TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, brute-force CPU statement of what one DReSD draft-model call
+ * computes (Algorithm 1 steps 4-7 of the paper): the query is z-scored
+ * (Eq. 1), projected with the PCA matrix (Section 3.3, v_l <- v W_l),
+ * scaled to unit length (Eq. 2), compared by inner product with EVERY key of
+ * the datastore (Eq. 3; on unit-length vectors cosine similarity is the inner
+ * product), the n most similar keys are taken, and each one's stored
+ * continuation is looked up (Section 3.5, the key -> value map f_D).
+ *
+ * Everything floating point is done in float64, one term after another, in
+ * the order the formulas are written; selection is a full sort of all N row
+ * indices.  No blocking, no fusion, no early exit.  Only tests, the smoke
+ * check and the benchmark's CPU-baseline leg may call this file; the CUDA
+ * library shares no code, header, table or constant with it.
+ *
+ * Readings where the paper is silent:
+ *   - epsilon of Eq. 1 and Eq. 2 are parameters (eps_z, eps_n);
+ *   - Eq. 3's arg max is extended to the n best (drafts are n x L matrices,
+ *     Section 5.4), ordered by score descending, ties by row index ascending;
+ *   - keys are used as stored (they are unit length by construction), so the
+ *     similarity is the inner product of the unit query with the stored key;
+ *   - no PCA centring unless a pca_mean vector is supplied;
+ *   - the value lookup copies the first draft_len stored tokens verbatim.
+ *
+ * Pins (tests/test_oracle_*.py): hand-computed cases, closed forms
+ * (unit norm, scale invariance, identity keys), brute-force cross-check
+ * against an independent numpy float64 formulation, and the invariants
+ * self-retrieval / permutation / shard-merge.  The paper prints no worked
+ * numeric example of a retrieval, so there is no paper-printed value to pin.
+ */
+#define _GNU_SOURCE
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORACLE_F32 = 0, ORACLE_F16 = 1, ORACLE_BF16 = 2 };
+
+/* ---- exact decoding of stored bit patterns to float64 ------------------- */
+
+static double decode_f16(uint16_t h)
+{
+    int sign = (h >> 15) & 1;
+    int expo = (h >> 10) & 0x1F;
+    int mant = h & 0x3FF;
+    double v;
+    if (expo == 0)
+        v = ldexp((double)mant, -24);               /* subnormal or zero   */
+    else if (expo == 31)
+        v = mant ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + (double)mant / 1024.0, expo - 15);
+    return sign ? -v : v;
+}
+
+static double decode_bf16(uint16_t b)
+{
+    /* bfloat16 is the upper half of an IEEE-754 binary32. */
+    int sign = (b >> 15) & 1;
+    int expo = (b >> 7) & 0xFF;
+    int mant = b & 0x7F;
+    double v;
+    if (expo == 0)
+        v = ldexp((double)mant, -133);              /* 2^-126 * mant/128   */
+    else if (expo == 255)
+        v = mant ? NAN : INFINITY;
+    else
+        v = ldexp(1.0 + (double)mant / 128.0, expo - 127);
+    return sign ? -v : v;
+}
+
+static double load_elem(const void *base, int64_t idx, int dtype)
+{
+    switch (dtype) {
+    case ORACLE_F32: return (double)((const float *)base)[idx];
+    case ORACLE_F16: return decode_f16(((const uint16_t *)base)[idx]);
+    default:         return decode_bf16(((const uint16_t *)base)[idx]);
+    }
+}
+
+double dresd_oracle_decode(uint32_t bits, int dtype)
+{
+    if (dtype == ORACLE_F32) {
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+    return dtype == ORACLE_F16 ? decode_f16((uint16_t)bits) : decode_bf16((uint16_t)bits);
+}
+
+/* ---- query preprocessing: Eq. 1 -> v W_l -> Eq. 2 ------------------------
+ * queries [B][d_in] in `dtype`; mean/var/pca_mean fp32 [d_in] or NULL;
+ * W [d_in][d] in `dtype` or NULL (then d must equal d_in).
+ * qhat [B][d] float64 out.  Returns 0, or -1 on bad arguments.            */
+int dresd_oracle_preprocess(const void *queries, int B, int d_in, int dtype,
+                            const float *mean, const float *var, double eps_z,
+                            const void *W, int d, const float *pca_mean,
+                            double eps_n, double *qhat)
+{
+    if (B < 0 || d_in <= 0 || d <= 0) return -1;
+    if (!W && d != d_in) return -1;
+    if ((mean == NULL) != (var == NULL)) return -1;
+    double *v = (double *)malloc(sizeof(double) * (size_t)d_in);
+    if (!v) return -1;
+    for (int b = 0; b < B; ++b) {
+        for (int j = 0; j < d_in; ++j)
+            v[j] = load_elem(queries, (int64_t)b * d_in + j, dtype);
+        if (mean)                                              /* Eq. 1 */
+            for (int j = 0; j < d_in; ++j)
+                v[j] = (v[j] - (double)mean[j]) / sqrt((double)var[j] + eps_z);
+        double *vl = qhat + (size_t)b * d;
+        if (W) {                                               /* v_l <- v W_l */
+            if (pca_mean)
+                for (int j = 0; j < d_in; ++j) v[j] -= (double)pca_mean[j];
+            for (int c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int j = 0; j < d_in; ++j)
+                    acc += v[j] * load_elem(W, (int64_t)j * d + c, dtype);
+                vl[c] = acc;
+            }
+        } else {
+            for (int c = 0; c < d; ++c) vl[c] = v[c];
+        }
+        double ss = 0.0;                                       /* Eq. 2 */
+        for (int c = 0; c < d; ++c) ss += vl[c] * vl[c];
+        double nrm = sqrt(ss);
+        double den = nrm > eps_n ? nrm : eps_n;
+        for (int c = 0; c < d; ++c) vl[c] /= den;
+    }
+    free(v);
+    return 0;
+}
+
+/* ---- scoring: s[i] = sum_c qhat[c] * k[i][c] for every row -------------
+ * Rows are independent; `threads` > 1 only splits the row loop, the
+ * arithmetic of each row is unchanged.                                      */
+int dresd_oracle_scores(const void *keys, int64_t N, int d, int dtype,
+                        const double *qhat, double *s, int threads)
+{
+    if (N < 0 || d <= 0) return -1;
+    if (threads < 1) threads = 1;
+#pragma omp parallel for num_threads(threads) schedule(static)
+    for (int64_t i = 0; i < N; ++i) {
+        double acc = 0.0;
+        for (int c = 0; c < d; ++c)
+            acc += qhat[c] * load_elem(keys, i * d + c, dtype);
+        s[i] = acc;
+    }
+    return 0;
+}
+
+/* ---- ordering: score descending, then row index ascending --------------- */
+static int by_score_then_id(const void *pa, const void *pb, void *ctx)
+{
+    const double *s = (const double *)ctx;
+    int64_t a = *(const int64_t *)pa, b = *(const int64_t *)pb;
+    if (s[a] > s[b]) return -1;
+    if (s[a] < s[b]) return 1;
+    return (a > b) - (a < b);
+}
+
+/* ---- the whole call ------------------------------------------------------
+ * keys [N][d] dtype; next_tokens [N][stored_len] int32; queries [B][d_in].
+ * out_ids [B][top_n] int32, out_scores [B][top_n] float64,
+ * out_tokens [B][top_n][draft_len] int32; full_scores [B][N] float64 or NULL.
+ * Returns 0, or -1 on bad arguments / allocation failure.                   */
+int dresd_oracle_retrieve(const void *keys, const int32_t *next_tokens, int64_t N, int d,
+                          int dtype, int stored_len,
+                          const void *queries, int B, int d_in,
+                          const float *mean, const float *var, double eps_z,
+                          const void *W, const float *pca_mean, double eps_n,
+                          int top_n, int draft_len,
+                          int32_t *out_ids, double *out_scores, int32_t *out_tokens,
+                          double *full_scores, int threads)
+{
+    if (N <= 0 || top_n < 1 || top_n > N) return -1;
+    if (draft_len < 1 || draft_len > stored_len) return -1;
+    if (B < 0) return -1;
+    double *qhat = (double *)malloc(sizeof(double) * (size_t)(B > 0 ? B : 1) * d);
+    double *s = (double *)malloc(sizeof(double) * (size_t)N);
+    int64_t *order = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+    int rc = -1;
+    if (!qhat || !s || !order) goto done;
+    if (dresd_oracle_preprocess(queries, B, d_in, dtype, mean, var, eps_z, W, d,
+                                pca_mean, eps_n, qhat) != 0)
+        goto done;
+    for (int b = 0; b < B; ++b) {
+        dresd_oracle_scores(keys, N, d, dtype, qhat + (size_t)b * d, s, threads);
+        for (int64_t i = 0; i < N; ++i) order[i] = i;
+        qsort_r(order, (size_t)N, sizeof(int64_t), by_score_then_id, s);
+        for (int r = 0; r < top_n; ++r) {
+            int64_t id = order[r];
+            out_ids[(size_t)b * top_n + r] = (int32_t)id;
+            out_scores[(size_t)b * top_n + r] = s[id];
+            for (int t = 0; t < draft_len; ++t)                 /* f_D lookup */
+                out_tokens[((size_t)b * top_n + r) * draft_len + t] =
+                    next_tokens[id * stored_len + t];
+        }
+        if (full_scores) memcpy(full_scores + (size_t)b * N, s, sizeof(double) * (size_t)N);
+    }
+    rc = 0;
+done:
+    free(qhat);
+    free(s);
+    free(order);
+    return rc;
+}

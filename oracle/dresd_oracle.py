@@ -1,0 +1,163 @@
+"""ctypes front end of the brute-force C oracle (``dresd_oracle.c``).
+
+TEST INFRASTRUCTURE: argument marshalling only; all arithmetic is in the C
+file, which restates Algorithm 1 steps 4-7 / Eq. 1-3 / Section 3.5 of the
+paper in float64 with a full sort.  Arrays of 16-bit values are passed as
+their bit patterns (numpy ``float16`` for f16, ``uint16`` for bf16).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dresd_oracle.c")
+_LIB = os.path.join(_HERE, "libdresd_oracle.so")
+_DTYPE_CODE = {"f32": 0, "f16": 1, "bf16": 2}
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fPIC", "-shared", "-fopenmp", "-std=gnu11",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        c = ctypes
+        lib.dresd_oracle_decode.restype = c.c_double
+        lib.dresd_oracle_decode.argtypes = [c.c_uint32, c.c_int]
+        lib.dresd_oracle_preprocess.restype = c.c_int
+        lib.dresd_oracle_preprocess.argtypes = [
+            c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_double,
+            c.c_void_p, c.c_int, c.c_void_p, c.c_double, c.c_void_p]
+        lib.dresd_oracle_scores.restype = c.c_int
+        lib.dresd_oracle_scores.argtypes = [c.c_void_p, c.c_int64, c.c_int, c.c_int,
+                                            c.c_void_p, c.c_void_p, c.c_int]
+        lib.dresd_oracle_retrieve.restype = c.c_int
+        lib.dresd_oracle_retrieve.argtypes = [
+            c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_int,
+            c.c_void_p, c.c_int, c.c_int,
+            c.c_void_p, c.c_void_p, c.c_double, c.c_void_p, c.c_void_p, c.c_double,
+            c.c_int, c.c_int,
+            c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int]
+        _lib = lib
+    return _lib
+
+
+def _store_array(x, dtype: str) -> np.ndarray:
+    want = {"f32": np.float32, "f16": np.float16, "bf16": np.uint16}[dtype]
+    a = np.asarray(x)
+    if a.dtype != want:
+        if dtype == "f32":
+            a = a.astype(np.float32)
+        else:
+            raise TypeError(f"{dtype} arrays must be passed as {want.__name__} bit patterns")
+    return np.ascontiguousarray(a)
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32_or_none(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+
+
+def default_threads() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:  # pragma: no cover
+        return max(1, os.cpu_count() or 1)
+
+
+def decode(bits: int, dtype: str) -> float:
+    """Exact value of one stored bit pattern."""
+    return float(_load().dresd_oracle_decode(int(bits) & 0xFFFFFFFF, _DTYPE_CODE[dtype]))
+
+
+def preprocess(queries, dtype: str, mean=None, var=None, eps_z: float = 1e-5,
+               W=None, pca_mean=None, eps_n: float = 1e-12) -> np.ndarray:
+    """Eq. 1 -> projection -> Eq. 2.  Returns the unit queries, float64 ``[B][d]``."""
+    q = _store_array(queries, dtype)
+    B, d_in = q.shape
+    mean, var, pca_mean = _f32_or_none(mean), _f32_or_none(var), _f32_or_none(pca_mean)
+    if W is not None:
+        W = _store_array(W, dtype)
+        if W.shape[0] != d_in:
+            raise ValueError("W must be [d_in][d]")
+        d = W.shape[1]
+    else:
+        d = d_in
+    out = np.empty((B, d), dtype=np.float64)
+    rc = _load().dresd_oracle_preprocess(_ptr(q), B, d_in, _DTYPE_CODE[dtype], _ptr(mean),
+                                         _ptr(var), eps_z, _ptr(W), d, _ptr(pca_mean),
+                                         eps_n, _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle preprocess: bad arguments")
+    return out
+
+
+def scores(keys, dtype: str, qhat, threads: int = 1) -> np.ndarray:
+    """Inner product of one float64 unit query with every stored key: ``[N]`` float64."""
+    k = _store_array(keys, dtype)
+    N, d = k.shape
+    qh = np.ascontiguousarray(qhat, dtype=np.float64)
+    if qh.shape != (d,):
+        raise ValueError("qhat must be [d]")
+    s = np.empty(N, dtype=np.float64)
+    rc = _load().dresd_oracle_scores(_ptr(k), N, d, _DTYPE_CODE[dtype], _ptr(qh), _ptr(s), threads)
+    if rc != 0:
+        raise ValueError("oracle scores: bad arguments")
+    return s
+
+
+@dataclass
+class OracleResult:
+    ids: np.ndarray          # int32 [B][top_n]
+    scores: np.ndarray       # float64 [B][top_n]
+    tokens: np.ndarray       # int32 [B][top_n][draft_len]
+    full_scores: np.ndarray | None  # float64 [B][N] when requested
+
+
+def retrieve(keys, next_tokens, dtype: str, queries, top_n: int, draft_len: int,
+             mean=None, var=None, eps_z: float = 1e-5, W=None, pca_mean=None,
+             eps_n: float = 1e-12, want_full_scores: bool = False,
+             threads: int = 1) -> OracleResult:
+    """One whole draft-model call, brute force (see the C file's header)."""
+    k = _store_array(keys, dtype)
+    N, d = k.shape
+    nt = np.ascontiguousarray(next_tokens, dtype=np.int32)
+    if nt.ndim != 2 or nt.shape[0] != N:
+        raise ValueError("next_tokens must be [N][stored_len]")
+    q = _store_array(queries, dtype)
+    B, d_in = q.shape
+    mean, var, pca_mean = _f32_or_none(mean), _f32_or_none(var), _f32_or_none(pca_mean)
+    if W is not None:
+        W = _store_array(W, dtype)
+        if W.shape != (d_in, d):
+            raise ValueError("W must be [d_in][d]")
+    elif d_in != d:
+        raise ValueError("queries must have the key dimension when there is no projection")
+    ids = np.empty((B, top_n), dtype=np.int32)
+    sc = np.empty((B, top_n), dtype=np.float64)
+    tok = np.empty((B, top_n, draft_len), dtype=np.int32)
+    full = np.empty((B, N), dtype=np.float64) if want_full_scores else None
+    rc = _load().dresd_oracle_retrieve(
+        _ptr(k), _ptr(nt), N, d, _DTYPE_CODE[dtype], nt.shape[1],
+        _ptr(q), B, d_in, _ptr(mean), _ptr(var), eps_z, _ptr(W), _ptr(pca_mean), eps_n,
+        top_n, draft_len, _ptr(ids), _ptr(sc), _ptr(tok), _ptr(full), threads)
+    if rc != 0:
+        raise ValueError("oracle retrieve: bad arguments")
+    return OracleResult(ids, sc, tok, full)

@@ -1,0 +1,279 @@
+"""Pins for the CPU oracle: hand cases, closed forms, brute force, invariants.
+
+Everything here runs without a GPU.  The oracle is checked against values
+worked out by hand from the paper's formulas (tests/golden/hand_cases.json),
+against closed forms that the mathematics fixes, against an independent
+float64 numpy formulation on small inputs, and against the invariants of
+exact nearest-neighbour search.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2502_15572_b200 import synth
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+with open(os.path.join(HERE, "golden", "hand_cases.json")) as f:
+    GOLDEN = json.load(f)
+
+
+def _tokens(N, L):
+    return (100 * np.arange(N, dtype=np.int32)[:, None] + np.arange(L, dtype=np.int32)[None, :])
+
+
+# --------------------------------------------------------------------------
+# bit decoders
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("bits,dtype,value", [
+    (0x3C00, "f16", 1.0), (0x0001, "f16", 2.0 ** -24), (0x7BFF, "f16", 65504.0),
+    (0xC000, "f16", -2.0), (0x3555, "f16", 0.333251953125), (0x0400, "f16", 2.0 ** -14),
+    (0x8000, "f16", 0.0),
+    (0x3F80, "bf16", 1.0), (0x4049, "bf16", 3.140625), (0xBF00, "bf16", -0.5),
+    (0x0080, "bf16", 2.0 ** -126), (0x0001, "bf16", 2.0 ** -133),
+    (0x3F800000, "f32", 1.0), (0xC0490FDB, "f32", float(np.float32(-3.14159274))),
+])
+def test_decode_known_patterns(bits, dtype, value):
+    assert oracle.decode(bits, dtype) == value
+
+
+def test_decode_all_16bit_patterns_match_ieee():
+    bits = np.arange(65536, dtype=np.uint32)
+    want16 = bits.astype(np.uint16).view(np.float16).astype(np.float64)
+    wantbf = (bits << np.uint32(16)).view(np.float32).astype(np.float64)
+    for b in range(0, 65536, 1):
+        g16 = oracle.decode(b, "f16")
+        gbf = oracle.decode(b, "bf16")
+        for got, want in ((g16, want16[b]), (gbf, wantbf[b])):
+            if np.isnan(want):
+                assert np.isnan(got)
+            else:
+                assert got == want and np.signbit(got) == np.signbit(want)
+
+
+# --------------------------------------------------------------------------
+# preprocessing: Eq. 1 -> projection -> Eq. 2
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("case", GOLDEN["preprocess"], ids=lambda c: c["cite"])
+def test_preprocess_hand_cases(case):
+    v = np.array([case["v"]], dtype=np.float32)
+    W = None if case["W"] is None else np.array(case["W"], dtype=np.float32)
+    got = oracle.preprocess(v, "f32", mean=case["mean"], var=case["var"], eps_z=case["eps_z"],
+                            W=W, pca_mean=case["pca_mean"])
+    np.testing.assert_allclose(got[0], case["qhat"], atol=1.5e-6, rtol=0)
+
+
+def test_preprocess_closed_forms():
+    rng = np.random.default_rng(5)
+    v = rng.standard_normal((6, 40)).astype(np.float32)
+    q = oracle.preprocess(v, "f32")
+    # unit length
+    np.testing.assert_allclose(np.linalg.norm(q, axis=1), 1.0, atol=1e-14)
+    # scale invariance (powers of two keep the scaled input exactly representable)
+    q4 = oracle.preprocess((4.0 * v).astype(np.float32), "f32")
+    np.testing.assert_allclose(q4, q, atol=1e-15)
+    # direction is preserved
+    v64 = v.astype(np.float64)
+    np.testing.assert_allclose(q, v64 / np.linalg.norm(v64, axis=1, keepdims=True), atol=1e-15)
+    # identity projection changes nothing
+    qi = oracle.preprocess(v, "f32", W=np.eye(40, dtype=np.float32))
+    np.testing.assert_allclose(qi, q, atol=1e-15)
+    # a permutation matrix permutes coordinates
+    perm = rng.permutation(40)
+    P = np.zeros((40, 40), dtype=np.float32)
+    P[perm, np.arange(40)] = 1.0            # (vP)[c] = v[perm[c]]
+    qp = oracle.preprocess(v, "f32", W=P)
+    np.testing.assert_allclose(qp, q[:, perm], atol=1e-15)
+
+
+def test_preprocess_epsilon_guards():
+    z = np.zeros((1, 8), dtype=np.float32)
+    assert np.all(oracle.preprocess(z, "f32") == 0.0)             # 0 / max(0, eps) = 0
+    tiny = np.zeros((1, 4), dtype=np.float32)
+    tiny[0, 0] = 1e-20
+    got = oracle.preprocess(tiny, "f32", eps_n=1e-12)
+    assert got[0, 0] == pytest.approx(float(np.float32(1e-20)) / 1e-12, rel=1e-12)
+    got = oracle.preprocess(tiny, "f32", eps_n=1e-30)
+    assert got[0, 0] == pytest.approx(1.0, rel=1e-12)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+def test_preprocess_matches_numpy_float64(dtype):
+    d_in, d, B = 96, 24, 5
+    mean, var, W = synth.make_preprocess(11, d_in, d, dtype)
+    q = synth.make_hidden_queries(12, B, d_in, dtype)
+    pm = (0.1 * np.arange(d_in)).astype(np.float32)
+    got = oracle.preprocess(q, dtype, mean=mean, var=var, eps_z=1e-5, W=W, pca_mean=pm)
+    q64 = synth.store_to_float32(q, dtype).astype(np.float64)
+    W64 = synth.store_to_float32(W, dtype).astype(np.float64)
+    z = (q64 - mean.astype(np.float64)) / np.sqrt(var.astype(np.float64) + 1e-5)
+    vl = (z - pm.astype(np.float64)) @ W64
+    want = vl / np.maximum(np.linalg.norm(vl, axis=1, keepdims=True), 1e-12)
+    np.testing.assert_allclose(got, want, atol=1e-13)
+
+
+# --------------------------------------------------------------------------
+# scoring + selection + lookup
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("case", GOLDEN["retrieve"], ids=lambda c: c["derivation"][:30])
+def test_retrieve_hand_cases(case):
+    keys = np.array(case["keys"], dtype=np.float32)
+    toks = _tokens(len(keys), 3)
+    r = oracle.retrieve(keys, toks, "f32", np.array([case["query"]], dtype=np.float32),
+                        top_n=case["top_n"], draft_len=2)
+    assert r.ids[0].tolist() == case["ids"]
+    np.testing.assert_allclose(r.scores[0], case["scores"], atol=1.5e-6, rtol=0)
+    assert r.tokens[0].tolist() == [[100 * i, 100 * i + 1] for i in case["ids"]]
+
+
+def test_identity_keys():
+    d = 16
+    keys = np.eye(d, dtype=np.float32)
+    toks = _tokens(d, 4)
+    for j in (0, 5, 15):
+        q = np.zeros((1, d), dtype=np.float32)
+        q[0, j] = 3.0
+        r = oracle.retrieve(keys, toks, "f32", q, top_n=4, draft_len=4)
+        others = [i for i in range(d) if i != j][:3]
+        assert r.ids[0].tolist() == [j] + others
+        assert r.scores[0].tolist() == [1.0, 0.0, 0.0, 0.0]
+        assert r.tokens[0, 0].tolist() == [100 * j + t for t in range(4)]
+
+
+def test_zero_query_returns_lowest_ids():
+    keys, toks = synth.make_store(3, 50, 8, 4, "f32", 3)
+    r = oracle.retrieve(keys, toks, "f32", np.zeros((1, 8), dtype=np.float32), top_n=5, draft_len=3)
+    assert r.ids[0].tolist() == [0, 1, 2, 3, 4]
+    assert np.all(r.scores == 0.0)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+def test_matches_independent_numpy_bruteforce(dtype):
+    N, d, B, n, L = 700, 24, 6, 9, 5
+    keys, toks = synth.make_store(21, N, d, 8, dtype, 7)
+    q, _ = synth.make_queries(22, keys, dtype, B, 0.1)
+    r = oracle.retrieve(keys, toks, dtype, q, top_n=n, draft_len=L, want_full_scores=True)
+    K = synth.store_to_float32(keys, dtype).astype(np.float64)
+    Q = synth.store_to_float32(q, dtype).astype(np.float64)
+    Q = Q / np.linalg.norm(Q, axis=1, keepdims=True)
+    S = Q @ K.T
+    np.testing.assert_allclose(r.full_scores, S, atol=1e-14)
+    for b in range(B):
+        order = np.argsort(-S[b], kind="stable")[:n]
+        assert r.ids[b].tolist() == order.tolist()
+        np.testing.assert_allclose(r.scores[b], S[b, order], atol=1e-14)
+        assert np.array_equal(r.tokens[b], toks[order][:, :L])
+        assert np.all(np.diff(r.scores[b]) <= 0)
+
+
+def test_self_retrieval_and_mrr():
+    # Eq. 4: with exact search over distinct unit keys every key finds itself first.
+    for dtype, tol in (("f32", 1e-6), ("f16", 2.0 ** -10), ("bf16", 2.0 ** -7)):
+        keys, toks = synth.make_store(31, 400, 32, 6, dtype, 4)
+        idx = np.arange(0, 400, 13)
+        r = oracle.retrieve(keys, toks, dtype, keys[idx], top_n=3, draft_len=4,
+                            want_full_scores=True)
+        rr = []
+        for b, i in enumerate(idx):
+            rank = 1 + int(np.sum(r.full_scores[b] > r.full_scores[b, i]))
+            rr.append(1.0 / rank)
+        assert np.mean(rr) == 1.0
+        assert r.ids[:, 0].tolist() == idx.tolist()
+        K = synth.store_to_float32(keys, dtype).astype(np.float64)
+        np.testing.assert_allclose(r.scores[:, 0], np.linalg.norm(K[idx], axis=1), atol=1e-14)
+        np.testing.assert_allclose(r.scores[:, 0], 1.0, atol=tol)
+
+
+def test_cauchy_schwarz_bound():
+    keys, toks = synth.make_store(41, 300, 16, 4, "f16", 2)
+    q, _ = synth.make_queries(42, keys, "f16", 3, 0.3)
+    r = oracle.retrieve(keys, toks, "f16", q, top_n=1, draft_len=1, want_full_scores=True)
+    K = synth.store_to_float32(keys, "f16").astype(np.float64)
+    assert np.all(np.abs(r.full_scores) <= np.linalg.norm(K, axis=1)[None, :] + 1e-14)
+
+
+def test_permutation_invariance():
+    N = 500
+    keys, toks = synth.make_store(51, N, 16, 5, "f32", 6)
+    q, _ = synth.make_queries(52, keys, "f32", 4, 0.1)
+    r0 = oracle.retrieve(keys, toks, "f32", q, top_n=8, draft_len=6)
+    perm = np.random.default_rng(53).permutation(N)     # new row p holds old row perm[p]
+    r1 = oracle.retrieve(keys[perm], toks[perm], "f32", q, top_n=8, draft_len=6)
+    assert np.array_equal(perm[r1.ids], r0.ids)
+    assert np.array_equal(r1.scores, r0.scores)         # per-row arithmetic is position-free
+    assert np.array_equal(r1.tokens, r0.tokens)
+
+
+def test_shard_merge_equals_whole():
+    N, n = 600, 7
+    keys, toks = synth.make_store(61, N, 16, 5, "bf16", 5)
+    q, _ = synth.make_queries(62, keys, "bf16", 3, 0.1)
+    whole = oracle.retrieve(keys, toks, "bf16", q, top_n=n, draft_len=5)
+    cut = 233
+    a = oracle.retrieve(keys[:cut], toks[:cut], "bf16", q, top_n=n, draft_len=5)
+    b = oracle.retrieve(keys[cut:], toks[cut:], "bf16", q, top_n=n, draft_len=5)
+    for i in range(3):
+        ids = np.concatenate([a.ids[i], b.ids[i] + cut])
+        sc = np.concatenate([a.scores[i], b.scores[i]])
+        tk = np.concatenate([a.tokens[i], b.tokens[i]])
+        order = np.lexsort((ids, -sc))[:n]
+        assert np.array_equal(ids[order], whole.ids[i])
+        assert np.array_equal(sc[order], whole.scores[i])
+        assert np.array_equal(tk[order], whole.tokens[i])
+
+
+def test_prefix_properties_and_duplicates():
+    N = 300
+    keys, toks = synth.make_store(71, N, 16, 5, "f32", 8)
+    keys[200] = keys[17]                      # exact duplicate rows: lower id first, adjacent
+    q = keys[17:18].copy()
+    big = oracle.retrieve(keys, toks, "f32", q, top_n=12, draft_len=8)
+    small = oracle.retrieve(keys, toks, "f32", q, top_n=5, draft_len=3)
+    assert np.array_equal(big.ids[:, :5], small.ids)
+    assert np.array_equal(big.tokens[:, :5, :3], small.tokens)
+    assert big.ids[0, :2].tolist() == [17, 200]
+    assert big.scores[0, 0] == big.scores[0, 1]
+
+
+def test_batch_equals_single_queries():
+    keys, toks = synth.make_store(81, 256, 16, 4, "f16", 4)
+    q, _ = synth.make_queries(82, keys, "f16", 5, 0.1)
+    allq = oracle.retrieve(keys, toks, "f16", q, top_n=6, draft_len=4)
+    for b in range(5):
+        one = oracle.retrieve(keys, toks, "f16", q[b:b + 1], top_n=6, draft_len=4)
+        assert np.array_equal(one.ids[0], allq.ids[b])
+        assert np.array_equal(one.scores[0], allq.scores[b])
+
+
+def test_row_threads_do_not_change_scores():
+    keys, _ = synth.make_store(91, 5000, 32, 4, "bf16", 1)
+    qh = oracle.preprocess(keys[:1], "bf16")[0]
+    assert np.array_equal(oracle.scores(keys, "bf16", qh, threads=1),
+                          oracle.scores(keys, "bf16", qh, threads=4))
+
+
+def test_projected_retrieval_end_to_end_matches_two_steps():
+    d_in, d, N = 48, 16, 200
+    keys, toks = synth.make_store(101, N, d, 4, "bf16", 3)
+    mean, var, W = synth.make_preprocess(102, d_in, d, "bf16")
+    q = synth.make_hidden_queries(103, 3, d_in, "bf16")
+    r = oracle.retrieve(keys, toks, "bf16", q, top_n=4, draft_len=3, mean=mean, var=var, W=W,
+                        want_full_scores=True)
+    qh = oracle.preprocess(q, "bf16", mean=mean, var=var, W=W)
+    for b in range(3):
+        assert np.array_equal(r.full_scores[b], oracle.scores(keys, "bf16", qh[b]))
+
+
+def test_bad_arguments_raise():
+    keys, toks = synth.make_store(111, 20, 8, 2, "f32", 4)
+    q = keys[:1]
+    with pytest.raises(ValueError):
+        oracle.retrieve(keys, toks, "f32", q, top_n=21, draft_len=2)
+    with pytest.raises(ValueError):
+        oracle.retrieve(keys, toks, "f32", q, top_n=0, draft_len=2)
+    with pytest.raises(ValueError):
+        oracle.retrieve(keys, toks, "f32", q, top_n=2, draft_len=5)
+    with pytest.raises(ValueError):
+        oracle.retrieve(keys, toks, "f32", q[:, :4], top_n=2, draft_len=2)
