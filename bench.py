@@ -1,0 +1,307 @@
+#!/usr/bin/env python
+"""Benchmark of the DReSD retrieval hot path on B200 (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload NAME] [--rows N]
+
+A *step* is one dresd_retrieve() call -- query preprocessing, scoring of every
+key, top-n selection, merge and continuation gather -- for one decode step of
+the workload (batch 1 on the 10M x 256 fp16 datastore by default).  `value` is
+queries/s with everything resident in HBM; `e2e` is the same through the
+host-buffer entry point, copies included.  With --gpus N > 1 (torchrun) every
+rank serves its own query stream against its own replica of the datastore;
+there is no data-path collective, only the timing barrier.
+
+`--impl reference` times the CPU oracle (plain float64 brute force) on the
+host cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2502_15572_b200 import synth  # noqa: E402
+
+METRIC = "retrieval queries/s at 10M x 256 fp16, batch 1 (exact top-10 + 10-token drafts)"
+N_QUERIES = 1000          # distinct single queries cycled through (config 2: 1,000 sequential queries)
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_decode_b1_f16", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--rows", type=int, default=None, help="override N (debugging; not a bench value)")
+    ap.add_argument("--oracle-queries", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            j = json.load(f)
+        return float(j["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+def metric_name(cfg):
+    if cfg["name"] == "c2_decode_b1_f16" and cfg["N"] == synth.WORKLOADS["c2_decode_b1_f16"]["N"]:
+        return METRIC
+    return (f"retrieval queries/s at {cfg['N']} x {cfg['d']} {cfg['dtype']}, batch {cfg['B']} "
+            f"(exact top-{cfg['top_n']} + {cfg['draft_len']}-token drafts)")
+
+
+def workload_config(cfg):
+    return {"workload": cfg["name"], "N": cfg["N"], "d": cfg["d"], "key_dtype": cfg["dtype"],
+            "batch": cfg["B"], "top_n": cfg["top_n"], "draft_len": cfg["draft_len"],
+            "mixture_components": cfg["C"], "query_noise_sigma": cfg["sigma"], "seed": cfg["seed"],
+            "l2": "keys are %.2f GB per step, far larger than the 126 MB L2: no flush needed"
+                  % (cfg["N"] * cfg["d"] * synth.DTYPE_BYTES[cfg["dtype"]] / 1e9)}
+
+
+def make_inputs(args):
+    cfg = dict(synth.WORKLOADS[args.workload], name=args.workload)
+    if args.rows:
+        cfg["N"] = args.rows
+    if "d_in" in cfg:
+        raise SystemExit("bench.py times stores whose queries arrive at the key dimension")
+    keys, toks = synth.make_store(cfg["seed"], cfg["N"], cfg["d"], cfg["C"], cfg["dtype"], cfg["stored_len"])
+    nq = N_QUERIES if cfg["B"] == 1 else cfg["B"] * 16
+    q, src = synth.make_queries(cfg["seed"] + 100, keys, cfg["dtype"], nq, cfg["sigma"])
+    return cfg, keys, toks, q
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.path = tempfile.mktemp(prefix="dresd_clocks_", suffix=".csv")
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.proc:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1]))
+                    mx.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, p[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm),
+                       reasons=sorted(reasons))
+        return out
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def time_oracle(cfg, keys, toks, q, n_queries):
+    import oracle
+    threads = oracle.dresd_oracle.default_threads()
+    oracle.build()
+    nq = max(1, n_queries) * cfg["B"]
+    t0 = time.perf_counter()
+    r = oracle.retrieve(keys, toks, cfg["dtype"], q[:nq], cfg["top_n"], cfg["draft_len"], threads=threads)
+    dt = time.perf_counter() - t0
+    return nq / dt, threads, nq, dt, r
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, keys, toks, q = make_inputs(args)
+    steps = max(1, min(args.steps, 3))
+    for _ in range(min(args.warmup, 1)):
+        time_oracle(cfg, keys, toks, q, 1)
+    t0 = time.perf_counter()
+    qps, threads, nq, dt, _ = time_oracle(cfg, keys, toks, q, steps)
+    ms = (time.perf_counter() - t0) * 1e3 / steps
+    sample = f"{nq} queries of the workload, whole datastore each (float64 brute force + full sort)"
+    print(json.dumps({
+        "impl": "reference", "metric": metric_name(cfg), "value": qps, "unit": "queries/s",
+        "n_gpus": args.gpus, "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(cfg),
+        "cpu_baseline": {"value": qps, "unit": "queries/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": qps, "unit": "queries/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ----------------------------------------------------------------------------- the CUDA path
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_15572_b200 import binding, build as lib_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the retrieval path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        lib_build.build()
+    if world > 1:
+        dist.barrier()
+
+    cfg, keys, toks, q = make_inputs(args)
+    B, n, L, dtype = cfg["B"], cfg["top_n"], cfg["draft_len"], cfg["dtype"]
+    dkeys = binding.to_device(keys, dtype)
+    dtoks = torch.from_numpy(toks).cuda()
+    dq = binding.to_device(q, dtype)                       # [nq][d] resident in HBM
+    nq = dq.shape[0] // B
+    store = binding.Store(dkeys, dtoks, dtype)
+    out = (torch.empty((B, n), dtype=torch.int32, device="cuda"),
+           torch.empty((B, n), dtype=torch.float32, device="cuda"),
+           torch.empty((B, n, L), dtype=torch.int32, device="cuda"))
+
+    def step(i):
+        j = (i % nq) * B
+        store.retrieve(dq[j:j + B], n, L, out=out)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    store.status()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+
+    # ---- device-resident timed region (CUDA events on the launching stream) ----
+    store.set_option("profile", min(args.steps, 65536))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    launches = store.last_launches() * args.steps
+    passes = store.last_launches() - 3                     # scoring launches per call
+    scan_ms, scan_calls = store.profile_read()
+    store.set_option("profile", 0)
+    store.status()
+
+    # ---- end to end: pinned host buffers in and out through dresd_retrieve_host ----
+    hq = q.view(np.int16) if dtype == "bf16" else q
+    hq = torch.from_numpy(np.ascontiguousarray(hq)).pin_memory()
+    hout = (torch.empty((B, n), dtype=torch.int32).pin_memory(),
+            torch.empty((B, n), dtype=torch.float32).pin_memory(),
+            torch.empty((B, n, L), dtype=torch.int32).pin_memory())
+    for i in range(min(args.warmup, 3)):
+        store.retrieve_host(hq[(i % nq) * B:(i % nq) * B + B], n, L, hout)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        j = ((args.warmup + i) % nq) * B
+        store.retrieve_host(hq[j:j + B], n, L, hout)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+
+    t = torch.tensor([ms_total, e2e_s * 1e3, scan_ms / max(scan_calls, 1)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms_total, scan_ms_avg = (float(x) for x in t.tolist())
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_step = ms_total / args.steps
+    qps = world * B * args.steps / (ms_total * 1e-3)
+    e2e_qps = world * B * args.steps / (e2e_ms_total * 1e-3)
+    eb = synth.DTYPE_BYTES[dtype]
+    key_bytes = cfg["N"] * cfg["d"] * eb                    # algorithmic bytes of one scoring launch
+    peak, peak_src = peaks()
+    achieved = passes * key_bytes / (scan_ms_avg * 1e-3) / 1e9
+    line = {
+        "metric": metric_name(cfg), "value": qps, "unit": "queries/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate over %s keys" % dtype,
+        "data": "synthetic", "config": workload_config(cfg),
+        "e2e": {"value": e2e_qps, "unit": "queries/s",
+                "h2d_bytes_per_step": B * cfg["d"] * eb,
+                "d2h_bytes_per_step": B * n * (8 + 4 * L) + 4},
+        "gpu_launches": launches,
+        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
+        "roofline": {"bound": "hbm", "kernel": "scan (K2+K3: score every key + per-CTA top-n)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": peak_src, "traffic": None,
+                     "bytes_per_launch": key_bytes, "launches_per_step": passes,
+                     "ms_per_launch": scan_ms_avg / passes,
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "non_scan_share_of_step": 1.0 - scan_ms_avg / ms_step},
+        "datastore_gbs_per_step": key_bytes / (ms_step * 1e-3) / 1e9,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        o_qps, threads, o_nq, o_dt, _ = time_oracle(cfg, keys, toks, q, args.oracle_queries)
+        line["cpu_baseline"] = {"value": o_qps, "unit": "queries/s", "cores": threads, "kind": "oracle",
+                                "sample": f"{o_nq} queries of the workload over the whole datastore, {o_dt:.1f} s"}
+    print(json.dumps(line))
+    store.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -1,0 +1,166 @@
+/*
+ * dresd.h -- C ABI of the B200 dense-retrieval draft model of DReSD.
+ *
+ * One call of dresd_retrieve() is steps 4-7 of the paper's Algorithm 1 for a
+ * batch of B decode positions: the query (the LLM's hidden state) is z-scored
+ * (Eq. 1), projected to the datastore dimension (Section 3.3, v_l <- v W_l),
+ * scaled to unit length (Eq. 2), scored by inner product against EVERY key of
+ * the datastore (Eq. 3: cosine similarity, which on unit-length vectors is the
+ * inner product; search is exact, not approximate), the top_n best keys are
+ * selected, and each one's stored continuation -- the value of the key-value
+ * store f_D of Section 3.5 -- is gathered into the n x L draft matrix that
+ * batch verification (Section 3.6) consumes.
+ *
+ * All work runs in CUDA kernels compiled for sm_100a; there is no CPU path.
+ * Pointers are DEVICE pointers unless a parameter says "host".  Every function
+ * returns a dresd_status (never throws, aborts or exits); when validation
+ * fails nothing is enqueued.  dresd_last_error() gives a thread-local message
+ * for the last failing call.
+ */
+#ifndef DRESD_H
+#define DRESD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dresd_store dresd_store; /* opaque handle */
+
+typedef enum { DRESD_F32 = 0, DRESD_F16 = 1, DRESD_BF16 = 2 } dresd_dtype;
+
+typedef enum {
+    DRESD_OK = 0,
+    DRESD_ERR_INVALID = -1,     /* bad pointer / shape / range                        */
+    DRESD_ERR_UNSUPPORTED = -2, /* valid request outside the built kernel range       */
+    DRESD_ERR_ALLOC = -3,       /* workspace allocation failed                        */
+    DRESD_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed                  */
+    DRESD_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (see _status)   */
+} dresd_status;
+
+enum {
+    DRESD_MAX_BATCH = 64,  /* largest B per call                                      */
+    DRESD_MAX_TOP_N = 32,  /* largest top_n                                           */
+    DRESD_MAX_DIM = 4096   /* largest key dimension d                                */
+};
+
+/*
+ * Section 3.5: the datastore is a key-value store; key = (reduced, unit-length)
+ * token embedding, value = the next tokens at that position.
+ *
+ *   keys         device, [N][d] row-major in `dtype`; base 16-byte aligned and
+ *                d * sizeof(dtype) a multiple of 16 (rows are fetched by TMA).
+ *   next_tokens  device, int32 [N][stored_len] row-major.
+ *   N            1 .. 2^31-1 rows;  d: 8 .. DRESD_MAX_DIM.
+ *   stored_len   tokens stored per key (the paper's "next N tokens"), >= 1.
+ *   out_store    host pointer receiving the handle.
+ *
+ * Both arrays are BORROWED (zero copy): the caller keeps them alive and
+ * unmodified until dresd_store_destroy().  The call allocates a workspace of
+ * a few MB on the current device, builds the TMA descriptors and returns; it
+ * launches nothing.  A store is bound to the device that was current here and
+ * may be used from one stream at a time.
+ */
+dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, int64_t N, int d,
+                                dresd_dtype dtype, int stored_len, dresd_store **out_store);
+
+/*
+ * Optional query preprocessing ahead of the unit-length scaling, Algorithm 1
+ * steps 4-5.  Any pointer may be NULL to skip that stage; all are device
+ * pointers, borrowed like the keys.
+ *
+ *   d_in       width of the incoming queries (the LLM hidden size).
+ *   mean, var  fp32 [d_in]: E[V] and Var[V] of Eq. 1 (both or neither).
+ *   eps_z      the epsilon of Eq. 1 (the paper leaves it open; 1e-5 is usual).
+ *   W          [d_in][d] row-major in the store dtype: the first d principal
+ *              components, v_l = v W (Section 3.3).  Without W, d_in must be d.
+ *   pca_mean   fp32 [d_in] subtracted before the projection, or NULL (the
+ *              paper's formula has no centring).
+ *
+ * Without this call queries are [B][d] and only Eq. 2 is applied.
+ */
+dresd_status dresd_store_set_preprocess(dresd_store *store, int d_in, const float *mean,
+                                        const float *var, float eps_z, const void *W,
+                                        const float *pca_mean);
+
+/*
+ * Algorithm 1 steps 4-7 for B queries (Eq. 1, Section 3.3, Eq. 2, Eq. 3,
+ * Section 3.5), asynchronous on `stream` (a cudaStream_t; NULL = legacy
+ * default stream).  No host synchronisation, no allocation.
+ *
+ *   queries     device, [B][d_in] row-major, same dtype as the keys.
+ *   B           0 .. DRESD_MAX_BATCH (0 is a no-op returning DRESD_OK).
+ *   top_n       1 .. min(N, DRESD_MAX_TOP_N) neighbours per query.
+ *   draft_len   1 .. stored_len tokens copied per neighbour.
+ *   out_ids     device, int32 [B][top_n]: row indices, best first; equal
+ *               scores are ordered by ascending row index.
+ *   out_scores  device, fp32 [B][top_n]: inner product of the unit query with
+ *               the stored key (fp32 accumulation).
+ *   out_tokens  device, int32 [B][top_n][draft_len]: the first draft_len
+ *               stored tokens of each neighbour, verbatim.
+ *
+ * Non-finite inputs give unspecified results but neither hang nor fault.
+ */
+dresd_status dresd_retrieve(dresd_store *store, const void *queries, int B, int top_n,
+                            int draft_len, int32_t *out_ids, float *out_scores,
+                            int32_t *out_tokens, void *stream);
+
+/*
+ * The same call for callers whose queries and results live in HOST memory
+ * (ideally pinned): copies the queries to the device, runs dresd_retrieve(),
+ * copies the three results back and waits for `stream`.  The datastore itself
+ * stays on the device.  Returns the device status word as well (see below).
+ */
+dresd_status dresd_retrieve_host(dresd_store *store, const void *queries_host, int B, int top_n,
+                                 int draft_len, int32_t *out_ids_host, float *out_scores_host,
+                                 int32_t *out_tokens_host, void *stream);
+
+/*
+ * Eq. 1 -> Section 3.3 -> Eq. 2 alone: writes the unit-length queries,
+ * fp32 [B][d] (device), exactly as the scoring kernels consume them.
+ */
+dresd_status dresd_preprocess(dresd_store *store, const void *queries, int B, float *out_qhat,
+                              void *stream);
+
+/*
+ * Device-side health: every wait inside the kernels is bounded; a wait that
+ * expires records DRESD_ERR_TIMEOUT in a device word and the kernel returns.
+ * This call synchronises the store's last stream and reports (then clears)
+ * that word: DRESD_OK or DRESD_ERR_TIMEOUT.
+ */
+dresd_status dresd_store_status(dresd_store *store);
+
+/*
+ * Kernel-selection knobs for tests and measurements (set between calls).
+ *   "scan_path"  0 = automatic, 1 = CUDA-core/mma.sync streaming kernel,
+ *                2 = tcgen05 tensor-core kernel (16-bit keys only).
+ *   "grid"       CTAs of the scoring kernel, 0 = one per SM.
+ *   "profile"    > 0: record a CUDA-event pair around the scoring kernel(s) of
+ *                each of the next `value` dresd_retrieve() calls (see
+ *                dresd_store_profile_read); 0 = off (default).
+ * Unknown names return DRESD_ERR_INVALID.
+ */
+dresd_status dresd_store_set_option(dresd_store *store, const char *name, int value);
+
+/*
+ * Waits for the store's last stream, then returns the summed device time (ms)
+ * of the scoring kernel (Eq. 3 over every key, with the fused selection) over
+ * the profiled calls since the last read, and how many calls that covers.
+ * Resets the counter so that profiling continues with fresh slots.
+ */
+dresd_status dresd_store_profile_read(dresd_store *store, double *scan_ms_total, int *calls);
+
+/* Number of kernels dresd_retrieve() enqueued in the store's last call. */
+int dresd_store_last_launches(const dresd_store *store);
+
+/* Message of the calling thread's last failing call ("" if none). */
+const char *dresd_last_error(void);
+
+/* Frees the workspace only, never caller memory.  NULL is allowed. */
+void dresd_store_destroy(dresd_store *store);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DRESD_H */

@@ -1,0 +1,242 @@
+"""Thin ctypes binding of ``libdresd.so`` (see ``include/dresd.h``).
+
+Argument marshalling only: every step of the retrieval path runs in the CUDA
+kernels behind the C ABI.  There is no CPU fallback -- if the library is
+missing or a call fails, a :class:`DresdError` is raised.
+
+Functions carry the C names (``dresd_store_create`` ...); :class:`Store` wraps
+them for torch tensors (used for device memory and streams only).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdresd.so")
+
+DRESD_F32, DRESD_F16, DRESD_BF16 = 0, 1, 2
+DTYPE_CODE = {"f32": DRESD_F32, "f16": DRESD_F16, "bf16": DRESD_BF16}
+DRESD_OK = 0
+STATUS_NAME = {0: "DRESD_OK", -1: "DRESD_ERR_INVALID", -2: "DRESD_ERR_UNSUPPORTED",
+               -3: "DRESD_ERR_ALLOC", -4: "DRESD_ERR_CUDA", -5: "DRESD_ERR_TIMEOUT"}
+MAX_BATCH, MAX_TOP_N, MAX_DIM = 64, 32, 4096
+
+EXPORTS = (
+    "dresd_store_create", "dresd_store_set_preprocess", "dresd_retrieve", "dresd_retrieve_host",
+    "dresd_preprocess", "dresd_store_status", "dresd_store_set_option",
+    "dresd_store_profile_read", "dresd_store_last_launches", "dresd_last_error",
+    "dresd_store_destroy",
+)
+
+
+class DresdError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAME.get(status, status)}: {message}")
+        self.status = status
+        self.message = message
+
+
+_lib = None
+
+
+def load(path: str | None = None) -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise DresdError(-4, f"{p} not found: build it with `python -m paper_2502_15572_b200.build` "
+                             "(there is no CPU fallback)")
+    lib = ctypes.CDLL(p)
+    c = ctypes
+    vp, i32, i64, f32 = c.c_void_p, c.c_int, c.c_int64, c.c_float
+    lib.dresd_store_create.restype = i32
+    lib.dresd_store_create.argtypes = [vp, vp, i64, i32, i32, i32, c.POINTER(vp)]
+    lib.dresd_store_set_preprocess.restype = i32
+    lib.dresd_store_set_preprocess.argtypes = [vp, i32, vp, vp, f32, vp, vp]
+    lib.dresd_retrieve.restype = i32
+    lib.dresd_retrieve.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.dresd_retrieve_host.restype = i32
+    lib.dresd_retrieve_host.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.dresd_preprocess.restype = i32
+    lib.dresd_preprocess.argtypes = [vp, vp, i32, vp, vp]
+    lib.dresd_store_status.restype = i32
+    lib.dresd_store_status.argtypes = [vp]
+    lib.dresd_store_set_option.restype = i32
+    lib.dresd_store_set_option.argtypes = [vp, c.c_char_p, i32]
+    lib.dresd_store_profile_read.restype = i32
+    lib.dresd_store_profile_read.argtypes = [vp, c.POINTER(c.c_double), c.POINTER(c.c_int)]
+    lib.dresd_store_last_launches.restype = i32
+    lib.dresd_store_last_launches.argtypes = [vp]
+    lib.dresd_last_error.restype = c.c_char_p
+    lib.dresd_last_error.argtypes = []
+    lib.dresd_store_destroy.restype = None
+    lib.dresd_store_destroy.argtypes = [vp]
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def dresd_last_error() -> str:
+    return load().dresd_last_error().decode()
+
+
+def _check(status: int) -> None:
+    if status != DRESD_OK:
+        raise DresdError(status, dresd_last_error())
+
+
+# ---- the C calls, by name, on raw addresses -----------------------------------
+def dresd_store_create(keys_ptr: int, next_tokens_ptr: int, N: int, d: int, dtype: int,
+                       stored_len: int) -> int:
+    h = ctypes.c_void_p()
+    _check(load().dresd_store_create(keys_ptr, next_tokens_ptr, N, d, dtype, stored_len, ctypes.byref(h)))
+    return h.value
+
+
+def dresd_store_set_preprocess(store: int, d_in: int, mean_ptr, var_ptr, eps_z: float, W_ptr,
+                               pca_mean_ptr) -> None:
+    _check(load().dresd_store_set_preprocess(store, d_in, mean_ptr, var_ptr, eps_z, W_ptr, pca_mean_ptr))
+
+
+def dresd_retrieve(store: int, queries_ptr: int, B: int, top_n: int, draft_len: int, out_ids_ptr: int,
+                   out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_retrieve(store, queries_ptr, B, top_n, draft_len, out_ids_ptr, out_scores_ptr,
+                                 out_tokens_ptr, stream))
+
+
+def dresd_retrieve_host(store: int, queries_ptr: int, B: int, top_n: int, draft_len: int,
+                        out_ids_ptr: int, out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_retrieve_host(store, queries_ptr, B, top_n, draft_len, out_ids_ptr,
+                                      out_scores_ptr, out_tokens_ptr, stream))
+
+
+def dresd_preprocess(store: int, queries_ptr: int, B: int, out_qhat_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_preprocess(store, queries_ptr, B, out_qhat_ptr, stream))
+
+
+def dresd_store_status(store: int) -> None:
+    _check(load().dresd_store_status(store))
+
+
+def dresd_store_set_option(store: int, name: str, value: int) -> None:
+    _check(load().dresd_store_set_option(store, name.encode(), value))
+
+
+def dresd_store_profile_read(store: int):
+    """Returns ``(scan_ms_total, calls)``."""
+    ms, n = ctypes.c_double(0.0), ctypes.c_int(0)
+    _check(load().dresd_store_profile_read(store, ctypes.byref(ms), ctypes.byref(n)))
+    return ms.value, n.value
+
+
+def dresd_store_last_launches(store: int) -> int:
+    return int(load().dresd_store_last_launches(store))
+
+
+def dresd_store_destroy(store: int) -> None:
+    load().dresd_store_destroy(store)
+
+
+# ---- torch convenience ----------------------------------------------------------
+def _torch():
+    import torch
+    return torch
+
+
+def to_device(array, dtype: str, device="cuda"):
+    """Upload a numpy array holding store-dtype values (bit patterns for 16-bit)."""
+    import numpy as np
+    torch = _torch()
+    a = np.ascontiguousarray(array)
+    if dtype == "bf16":
+        return torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16)
+    if dtype == "f16":
+        return torch.from_numpy(a.view(np.float16)).to(device)
+    return torch.from_numpy(a.astype(np.float32, copy=False)).to(device)
+
+
+class Store:
+    """A datastore on the current CUDA device; tensors passed in are borrowed."""
+
+    def __init__(self, keys, next_tokens, dtype: str):
+        torch = _torch()
+        want = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[dtype]
+        if not keys.is_cuda or not next_tokens.is_cuda:
+            raise DresdError(-1, "keys and next_tokens must be CUDA tensors (there is no CPU path)")
+        if keys.dtype != want or next_tokens.dtype != torch.int32:
+            raise DresdError(-1, f"keys must be {want}, next_tokens int32")
+        if not keys.is_contiguous() or not next_tokens.is_contiguous():
+            raise DresdError(-1, "keys and next_tokens must be contiguous")
+        self.dtype = dtype
+        self.torch_dtype = want
+        self.keys, self.next_tokens = keys, next_tokens       # keep alive
+        self.N, self.d = keys.shape
+        self.stored_len = next_tokens.shape[1]
+        self.d_in = self.d
+        self._pre = None
+        self.handle = dresd_store_create(keys.data_ptr(), next_tokens.data_ptr(), self.N, self.d,
+                                         DTYPE_CODE[dtype], self.stored_len)
+
+    def set_preprocess(self, d_in, mean=None, var=None, eps_z=1e-5, W=None, pca_mean=None):
+        self._pre = (mean, var, W, pca_mean)                  # keep alive
+        ptr = lambda t: None if t is None else t.data_ptr()
+        dresd_store_set_preprocess(self.handle, d_in, ptr(mean), ptr(var), eps_z, ptr(W), ptr(pca_mean))
+        self.d_in = d_in
+
+    def set_option(self, name: str, value: int):
+        dresd_store_set_option(self.handle, name, value)
+
+    def retrieve(self, queries, top_n: int, draft_len: int, out=None, stream=None):
+        """Returns ``(ids [B][n] int32, scores [B][n] f32, tokens [B][n][L] int32)`` on the device."""
+        torch = _torch()
+        B = queries.shape[0]
+        if out is None:
+            dev = queries.device
+            out = (torch.empty((B, top_n), dtype=torch.int32, device=dev),
+                   torch.empty((B, top_n), dtype=torch.float32, device=dev),
+                   torch.empty((B, top_n, draft_len), dtype=torch.int32, device=dev))
+        ids, scores, tokens = out
+        s = (stream or torch.cuda.current_stream()).cuda_stream
+        dresd_retrieve(self.handle, queries.data_ptr(), B, top_n, draft_len, ids.data_ptr(),
+                       scores.data_ptr(), tokens.data_ptr(), s)
+        return ids, scores, tokens
+
+    def retrieve_host(self, queries, top_n: int, draft_len: int, out, stream=None):
+        """Host (pinned) tensors in and out; blocks until the results are on the host."""
+        torch = _torch()
+        ids, scores, tokens = out
+        s = (stream or torch.cuda.current_stream()).cuda_stream
+        dresd_retrieve_host(self.handle, queries.data_ptr(), queries.shape[0], top_n, draft_len,
+                            ids.data_ptr(), scores.data_ptr(), tokens.data_ptr(), s)
+        return ids, scores, tokens
+
+    def preprocess(self, queries, stream=None):
+        torch = _torch()
+        B = queries.shape[0]
+        out = torch.empty((B, self.d), dtype=torch.float32, device=queries.device)
+        s = (stream or torch.cuda.current_stream()).cuda_stream
+        dresd_preprocess(self.handle, queries.data_ptr(), B, out.data_ptr(), s)
+        return out
+
+    def status(self):
+        dresd_store_status(self.handle)
+
+    def profile_read(self):
+        return dresd_store_profile_read(self.handle)
+
+    def last_launches(self) -> int:
+        return dresd_store_last_launches(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            dresd_store_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,487 @@
+// C ABI of the retrieval library: store object, argument validation, TMA
+// descriptors, workspace, and the launch chain K1 -> K2+K3 -> K4 -> K5.
+// See include/dresd.h for the contract of every entry point.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "../../include/dresd.h"
+#include "internal.h"
+
+using namespace dresd;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+dresd_status fail(dresd_status st, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return st;
+}
+dresd_status fail_cuda(cudaError_t e, const char *what)
+{
+    return fail(DRESD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+constexpr uint32_t kMagic = 0xD2E5D001u;
+constexpr float kEpsNorm = 1e-12f;   // epsilon of Eq. 2 (the paper leaves it open)
+
+bool is_device_ptr(const void *p)
+{
+    if (!p) return false;
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+size_t elem_bytes(int dtype) { return dtype == kF32 ? 4 : 2; }
+
+// 2-D map over a row-major [rows][cols] matrix; box = one 128-byte swizzle row
+// wide, box_rows tall; out-of-range elements read as zero.
+bool make_map(CUtensorMap *map, const void *base, int dtype, long long rows, int cols, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const size_t eb = elem_bytes(dtype);
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * eb};
+    cuuint32_t box[2] = {(cuuint32_t)(128 / eb), (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUtensorMapDataType dt = dtype == kF32   ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                             : dtype == kF16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                             : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    CUresult r = fn(map, dt, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct dresd_store {
+    uint32_t magic;
+    int device;
+    int num_sms;
+    // datastore (borrowed)
+    const void *keys;
+    const int32_t *next_tokens;
+    long long N;
+    int d, dpad, dtype, stored_len;
+    // preprocessing (borrowed)
+    int d_in;
+    const float *mean, *var, *pca_mean;
+    const void *W;
+    float eps_z;
+    // workspace (owned)
+    float *qhat;                 // [kMaxBatch][d]
+    void *qsplit;                // [2*kMaxBatch][dpad] 16-bit
+    unsigned long long *cand;    // [max_grid][kMaxBatch][kCandStride]
+    int *status;                 // device status word
+    int max_grid;
+    // staging for dresd_retrieve_host (owned, device)
+    void *q_stage;
+    size_t q_stage_bytes;
+    int32_t *ids_dev;
+    float *scores_dev;
+    int32_t *tokens_dev;
+    size_t tokens_dev_elems;
+    // streaming-kernel geometry
+    CUtensorMap map_stream;
+    int tile_rows, n_tiles;
+    // options / bookkeeping
+    int opt_path, opt_grid;
+    cudaStream_t last_stream;
+    int last_launches;
+    // optional timing of the scoring kernel (option "profile")
+    cudaEvent_t *prof_events;    // [2 * prof_cap]: start/stop pairs
+    int prof_cap, prof_count;
+};
+
+namespace {
+
+bool valid(const dresd_store *s) { return s && s->magic == kMagic; }
+
+void free_store(dresd_store *s)
+{
+    if (!s) return;
+    cudaFree(s->qhat);
+    cudaFree(s->qsplit);
+    cudaFree(s->cand);
+    cudaFree(s->status);
+    cudaFree(s->q_stage);
+    cudaFree(s->ids_dev);
+    cudaFree(s->scores_dev);
+    cudaFree(s->tokens_dev);
+    for (int i = 0; i < 2 * s->prof_cap; ++i) cudaEventDestroy(s->prof_events[i]);
+    delete[] s->prof_events;
+    s->magic = 0;
+    delete s;
+}
+
+dresd_status check_retrieve_args(const dresd_store *s, const void *queries, int B, int top_n,
+                                 int draft_len, const void *ids, const void *scores,
+                                 const void *tokens, bool device_ptrs)
+{
+    if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+    if (B < 0) return fail(DRESD_ERR_INVALID, "B = %d is negative", B);
+    if (top_n < 1 || top_n > s->N) return fail(DRESD_ERR_INVALID, "top_n = %d outside 1..N", top_n);
+    if (draft_len < 1 || draft_len > s->stored_len)
+        return fail(DRESD_ERR_INVALID, "draft_len = %d outside 1..stored_len (%d)", draft_len, s->stored_len);
+    if (B > DRESD_MAX_BATCH) return fail(DRESD_ERR_UNSUPPORTED, "B = %d exceeds DRESD_MAX_BATCH", B);
+    if (top_n > DRESD_MAX_TOP_N) return fail(DRESD_ERR_UNSUPPORTED, "top_n = %d exceeds DRESD_MAX_TOP_N", top_n);
+    if (B == 0) return DRESD_OK;
+    if (!queries || !ids || !scores || !tokens) return fail(DRESD_ERR_INVALID, "NULL buffer");
+    if (device_ptrs && (!is_device_ptr(queries) || !is_device_ptr(ids) || !is_device_ptr(scores) ||
+                        !is_device_ptr(tokens)))
+        return fail(DRESD_ERR_INVALID, "queries/out_* must be device pointers");
+    return DRESD_OK;
+}
+
+// K1 for B queries into the store's workspace.
+dresd_status run_preprocess(dresd_store *s, const void *queries, int B, cudaStream_t stream)
+{
+    PreprocessArgs p{};
+    p.queries = queries;
+    p.mean = s->mean;
+    p.var = s->var;
+    p.W = s->W;
+    p.pca_mean = s->pca_mean;
+    p.eps_z = s->eps_z;
+    p.eps_n = kEpsNorm;
+    p.B = B;
+    p.d_in = s->d_in;
+    p.d = s->d;
+    p.dtype = s->dtype;
+    p.qhat = s->qhat;
+    p.qsplit = s->dtype == kF32 ? nullptr : s->qsplit;
+    p.dpad = s->dpad;
+    p.rows = ((B + 7) / 8) * 8;
+    p.lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
+    cudaError_t e = launch_preprocess(p, stream);
+    if (e != cudaSuccess) return fail_cuda(e, "preprocess launch");
+    s->last_launches += 1;
+    return DRESD_OK;
+}
+
+dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n, int draft_len,
+                          int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream)
+{
+    s->last_stream = stream;
+    s->last_launches = 0;
+    dresd_status st = run_preprocess(s, queries, B, stream);
+    if (st != DRESD_OK) return st;
+
+    int grid = s->opt_grid > 0 ? s->opt_grid : s->num_sms;
+    if (grid > s->max_grid) grid = s->max_grid;
+    if (grid > s->n_tiles) grid = s->n_tiles;
+
+    const bool f32 = s->dtype == kF32;
+    const int qpl = f32 ? scan_f32_queries_per_launch(s->d, B) : scan_mma_queries_per_launch(s->d, B);
+    const float lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
+    const bool prof = s->prof_count < s->prof_cap;
+    if (prof) cudaEventRecord(s->prof_events[2 * s->prof_count], stream);
+    for (int q0 = 0; q0 < B; q0 += qpl) {
+        ScanArgs a{};
+        a.N = s->N;
+        a.d = s->d;
+        a.dpad = s->dpad;
+        a.dtype = s->dtype;
+        a.n_tiles = s->n_tiles;
+        a.B = B - q0 < qpl ? B - q0 : qpl;
+        a.top_n = top_n;
+        a.qhat = s->qhat + (size_t)q0 * s->d;
+        a.qsplit = f32 ? nullptr
+                       : static_cast<const uint8_t *>(s->qsplit) + (size_t)2 * q0 * s->dpad * 2;
+        a.lo_inv_scale = 1.0f / lo_scale;
+        a.cand = s->cand + (size_t)q0 * kCandStride;
+        a.cand_batch = B;
+        a.status = s->status;
+        cudaError_t e = f32 ? launch_scan_f32(s->map_stream, a, grid, stream)
+                            : launch_scan_mma(s->map_stream, a, grid, stream);
+        if (e != cudaSuccess) return fail_cuda(e, "scan launch");
+        s->last_launches += 1;
+    }
+    if (prof) {
+        cudaEventRecord(s->prof_events[2 * s->prof_count + 1], stream);
+        s->prof_count += 1;
+    }
+    cudaError_t e = launch_merge(s->cand, grid, B, top_n, out_ids, out_scores, stream);
+    if (e != cudaSuccess) return fail_cuda(e, "merge launch");
+    e = launch_gather(s->next_tokens, s->stored_len, s->N, out_ids, B, top_n, draft_len, out_tokens, stream);
+    if (e != cudaSuccess) return fail_cuda(e, "gather launch");
+    s->last_launches += 2;
+    return DRESD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, int64_t N, int d,
+                                dresd_dtype dtype, int stored_len, dresd_store **out_store)
+{
+    if (!out_store) return fail(DRESD_ERR_INVALID, "out_store is NULL");
+    *out_store = nullptr;
+    if (dtype != DRESD_F32 && dtype != DRESD_F16 && dtype != DRESD_BF16)
+        return fail(DRESD_ERR_INVALID, "unknown dtype %d", (int)dtype);
+    if (N <= 0 || N > 2147483647LL) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1", (long long)N);
+    if (d <= 0) return fail(DRESD_ERR_INVALID, "d = %d", d);
+    if (stored_len < 1) return fail(DRESD_ERR_INVALID, "stored_len = %d", stored_len);
+    const size_t eb = elem_bytes((int)dtype);
+    if (((size_t)d * eb) % 16 != 0)
+        return fail(DRESD_ERR_INVALID, "row size %zu bytes is not a multiple of 16", (size_t)d * eb);
+    if (!keys || !next_tokens) return fail(DRESD_ERR_INVALID, "keys / next_tokens is NULL");
+    if (reinterpret_cast<uintptr_t>(keys) % 16 != 0) return fail(DRESD_ERR_INVALID, "keys not 16-byte aligned");
+    if (d > DRESD_MAX_DIM) return fail(DRESD_ERR_UNSUPPORTED, "d = %d exceeds DRESD_MAX_DIM", d);
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda(e, "cudaGetDevice");
+    if (!is_device_ptr(keys) || !is_device_ptr(next_tokens))
+        return fail(DRESD_ERR_INVALID, "keys / next_tokens must be device pointers");
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) return fail_cuda(e, "cudaGetDeviceProperties");
+    if (prop.major != 10) return fail(DRESD_ERR_UNSUPPORTED, "device is sm_%d%d; this library is built for sm_100a", prop.major, prop.minor);
+
+    dresd_store *s = new (std::nothrow) dresd_store();
+    if (!s) return fail(DRESD_ERR_ALLOC, "host allocation failed");
+    memset(s, 0, sizeof *s);
+    s->magic = kMagic;
+    s->device = dev;
+    s->num_sms = prop.multiProcessorCount;
+    s->keys = keys;
+    s->next_tokens = next_tokens;
+    s->N = N;
+    s->d = d;
+    s->dpad = ((d + 63) / 64) * 64;
+    s->dtype = (int)dtype;
+    s->stored_len = stored_len;
+    s->d_in = d;
+    s->eps_z = 1e-5f;
+    s->max_grid = 2 * s->num_sms;
+
+    s->tile_rows = dtype == DRESD_F32 ? scan_f32_tile_rows(d) : scan_mma_tile_rows(d);
+    s->n_tiles = (int)((N + s->tile_rows - 1) / s->tile_rows);
+    if (!make_map(&s->map_stream, keys, s->dtype, N, d, s->tile_rows)) {
+        free_store(s);
+        return fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the key matrix");
+    }
+
+    bool ok = cudaMalloc(&s->qhat, sizeof(float) * kMaxBatch * (size_t)d) == cudaSuccess &&
+              cudaMalloc(&s->qsplit, (size_t)2 * 2 * kMaxBatch * s->dpad) == cudaSuccess &&
+              cudaMalloc(&s->cand, sizeof(unsigned long long) * (size_t)s->max_grid * kMaxBatch * kCandStride) == cudaSuccess &&
+              cudaMalloc(&s->status, sizeof(int)) == cudaSuccess &&
+              cudaMalloc(&s->ids_dev, sizeof(int32_t) * kMaxBatch * kMaxTopN) == cudaSuccess &&
+              cudaMalloc(&s->scores_dev, sizeof(float) * kMaxBatch * kMaxTopN) == cudaSuccess;
+    s->tokens_dev_elems = (size_t)kMaxBatch * kMaxTopN * stored_len;
+    ok = ok && cudaMalloc(&s->tokens_dev, sizeof(int32_t) * s->tokens_dev_elems) == cudaSuccess;
+    s->q_stage_bytes = (size_t)kMaxBatch * d * eb;
+    ok = ok && cudaMalloc(&s->q_stage, s->q_stage_bytes) == cudaSuccess;
+    ok = ok && cudaMemset(s->status, 0, sizeof(int)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        free_store(s);
+        return fail(DRESD_ERR_ALLOC, "workspace allocation failed");
+    }
+    *out_store = s;
+    return DRESD_OK;
+}
+
+dresd_status dresd_store_set_preprocess(dresd_store *s, int d_in, const float *mean, const float *var,
+                                        float eps_z, const void *W, const float *pca_mean)
+{
+    if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+    if (d_in <= 0) return fail(DRESD_ERR_INVALID, "d_in = %d", d_in);
+    if ((mean == nullptr) != (var == nullptr)) return fail(DRESD_ERR_INVALID, "mean and var go together");
+    if (!W && d_in != s->d) return fail(DRESD_ERR_INVALID, "without W, d_in must equal d");
+    if (pca_mean && !W) return fail(DRESD_ERR_INVALID, "pca_mean needs W");
+    if (!(eps_z >= 0.f)) return fail(DRESD_ERR_INVALID, "eps_z must be >= 0");
+    if ((mean && !is_device_ptr(mean)) || (var && !is_device_ptr(var)) || (W && !is_device_ptr(W)) ||
+        (pca_mean && !is_device_ptr(pca_mean)))
+        return fail(DRESD_ERR_INVALID, "mean/var/W/pca_mean must be device pointers");
+    if (d_in > 16384) return fail(DRESD_ERR_UNSUPPORTED, "d_in = %d exceeds 16384", d_in);
+    const size_t need = (size_t)kMaxBatch * d_in * elem_bytes(s->dtype);
+    if (need > s->q_stage_bytes) {
+        void *p = nullptr;
+        if (cudaMalloc(&p, need) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(DRESD_ERR_ALLOC, "staging allocation failed");
+        }
+        cudaFree(s->q_stage);
+        s->q_stage = p;
+        s->q_stage_bytes = need;
+    }
+    s->d_in = d_in;
+    s->mean = mean;
+    s->var = var;
+    s->eps_z = eps_z;
+    s->W = W;
+    s->pca_mean = pca_mean;
+    return DRESD_OK;
+}
+
+dresd_status dresd_retrieve(dresd_store *s, const void *queries, int B, int top_n, int draft_len,
+                            int32_t *out_ids, float *out_scores, int32_t *out_tokens, void *stream)
+{
+    dresd_status st = check_retrieve_args(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens, true);
+    if (st != DRESD_OK || B == 0) return st;
+    return run_retrieve(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens,
+                        static_cast<cudaStream_t>(stream));
+}
+
+dresd_status dresd_retrieve_host(dresd_store *s, const void *queries_host, int B, int top_n, int draft_len,
+                                 int32_t *out_ids_host, float *out_scores_host, int32_t *out_tokens_host,
+                                 void *stream_v)
+{
+    dresd_status st = check_retrieve_args(s, queries_host, B, top_n, draft_len, out_ids_host,
+                                          out_scores_host, out_tokens_host, false);
+    if (st != DRESD_OK || B == 0) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t qbytes = (size_t)B * s->d_in * elem_bytes(s->dtype);
+    cudaError_t e = cudaMemcpyAsync(s->q_stage, queries_host, qbytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return fail_cuda(e, "query upload");
+    st = run_retrieve(s, s->q_stage, B, top_n, draft_len, s->ids_dev, s->scores_dev, s->tokens_dev, stream);
+    if (st != DRESD_OK) return st;
+    int dev_status = 0;
+    const size_t n = (size_t)B * top_n;
+    e = cudaMemcpyAsync(out_ids_host, s->ids_dev, n * sizeof(int32_t), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(out_scores_host, s->scores_dev, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(out_tokens_host, s->tokens_dev, n * draft_len * sizeof(int32_t),
+                            cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&dev_status, s->status, sizeof(int), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return fail_cuda(e, "result download");
+    if (dev_status != 0) {
+        cudaMemsetAsync(s->status, 0, sizeof(int), stream);
+        return fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
+    }
+    return DRESD_OK;
+}
+
+dresd_status dresd_preprocess(dresd_store *s, const void *queries, int B, float *out_qhat, void *stream_v)
+{
+    if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+    if (B < 0) return fail(DRESD_ERR_INVALID, "B = %d is negative", B);
+    if (B > DRESD_MAX_BATCH) return fail(DRESD_ERR_UNSUPPORTED, "B = %d exceeds DRESD_MAX_BATCH", B);
+    if (B == 0) return DRESD_OK;
+    if (!is_device_ptr(queries) || !is_device_ptr(out_qhat))
+        return fail(DRESD_ERR_INVALID, "queries/out_qhat must be device pointers");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    s->last_stream = stream;
+    s->last_launches = 0;
+    dresd_status st = run_preprocess(s, queries, B, stream);
+    if (st != DRESD_OK) return st;
+    cudaError_t e = cudaMemcpyAsync(out_qhat, s->qhat, sizeof(float) * (size_t)B * s->d,
+                                    cudaMemcpyDeviceToDevice, stream);
+    if (e != cudaSuccess) return fail_cuda(e, "qhat copy");
+    return DRESD_OK;
+}
+
+dresd_status dresd_store_status(dresd_store *s)
+{
+    if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+    cudaError_t e = cudaStreamSynchronize(s->last_stream);
+    if (e != cudaSuccess) return fail_cuda(e, "stream synchronize");
+    int word = 0;
+    e = cudaMemcpy(&word, s->status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail_cuda(e, "status read");
+    if (word != 0) {
+        cudaMemset(s->status, 0, sizeof(int));
+        return fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
+    }
+    return DRESD_OK;
+}
+
+dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
+{
+    if (!valid(s) || !name) return fail(DRESD_ERR_INVALID, "store handle or name is NULL");
+    if (strcmp(name, "scan_path") == 0) {
+        if (value < 0 || value > 2) return fail(DRESD_ERR_INVALID, "scan_path = %d outside 0..2", value);
+        s->opt_path = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "grid") == 0) {
+        if (value < 0 || value > s->max_grid) return fail(DRESD_ERR_INVALID, "grid = %d outside 0..%d", value, s->max_grid);
+        s->opt_grid = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "profile") == 0) {
+        if (value < 0 || value > 65536) return fail(DRESD_ERR_INVALID, "profile = %d outside 0..65536", value);
+        for (int i = 0; i < 2 * s->prof_cap; ++i) cudaEventDestroy(s->prof_events[i]);
+        delete[] s->prof_events;
+        s->prof_events = nullptr;
+        s->prof_cap = s->prof_count = 0;
+        if (value > 0) {
+            s->prof_events = new (std::nothrow) cudaEvent_t[2 * (size_t)value];
+            if (!s->prof_events) return fail(DRESD_ERR_ALLOC, "host allocation failed");
+            for (int i = 0; i < 2 * value; ++i)
+                if (cudaEventCreate(&s->prof_events[i]) != cudaSuccess) {
+                    for (int j = 0; j < i; ++j) cudaEventDestroy(s->prof_events[j]);
+                    delete[] s->prof_events;
+                    s->prof_events = nullptr;
+                    return fail(DRESD_ERR_CUDA, "cudaEventCreate failed");
+                }
+            s->prof_cap = value;
+        }
+        return DRESD_OK;
+    }
+    return fail(DRESD_ERR_INVALID, "unknown option '%s'", name);
+}
+
+dresd_status dresd_store_profile_read(dresd_store *s, double *scan_ms_total, int *calls)
+{
+    if (!valid(s) || !scan_ms_total || !calls) return fail(DRESD_ERR_INVALID, "NULL argument");
+    cudaError_t e = cudaStreamSynchronize(s->last_stream);
+    if (e != cudaSuccess) return fail_cuda(e, "stream synchronize");
+    double total = 0.0;
+    for (int i = 0; i < s->prof_count; ++i) {
+        float ms = 0.f;
+        e = cudaEventElapsedTime(&ms, s->prof_events[2 * i], s->prof_events[2 * i + 1]);
+        if (e != cudaSuccess) return fail_cuda(e, "cudaEventElapsedTime");
+        total += ms;
+    }
+    *scan_ms_total = total;
+    *calls = s->prof_count;
+    s->prof_count = 0;
+    return DRESD_OK;
+}
+
+int dresd_store_last_launches(const dresd_store *s) { return valid(s) ? s->last_launches : 0; }
+
+const char *dresd_last_error(void) { return g_err; }
+
+void dresd_store_destroy(dresd_store *s)
+{
+    if (valid(s)) free_store(s);
+}
+
+}  // extern "C"

@@ -1,0 +1,225 @@
+// Device-side building blocks shared by the retrieval kernels (sm_100a).
+//
+//  * candidate packing: (score, id) -> one u64 whose unsigned order is
+//    "score descending, then id ascending" (Eq. 3's arg max extended to the
+//    n best, ties to the lower row index);
+//  * warp-wide bitonic sort / merge of such words held one per lane;
+//  * WarpTopN: a warp-private running top-n list with a candidate queue;
+//  * mbarrier + TMA (cp.async.bulk.tensor) wrappers with BOUNDED waits.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dresd {
+
+constexpr int kListLen = 32;            // lanes of one warp-held list (>= top_n)
+constexpr int kQueueCap = 32;           // pending candidates per (warp, query)
+constexpr int kMergeLevel = 16;         // merge the queue once it holds this many
+constexpr int kStatusTimeout = -5;      // value of DRESD_ERR_TIMEOUT
+constexpr long long kWaitCycles = 4000000000LL;  // ~2-3 s at B200 clocks
+
+// ---------------------------------------------------------------------------
+// (score, id) <-> orderable u64.  0 is "empty" and sorts below every candidate.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long pack_candidate(float score, uint32_t id)
+{
+    score += 0.0f;                                   // -0.0 -> +0.0: one zero
+    uint32_t u = __float_as_uint(score);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // monotone float -> uint
+    return (static_cast<unsigned long long>(u) << 32) | (0xFFFFFFFFu - id);
+}
+__device__ __forceinline__ float candidate_score(unsigned long long p)
+{
+    uint32_t u = static_cast<uint32_t>(p >> 32);
+    u = (u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u;
+    return __uint_as_float(u);
+}
+__device__ __forceinline__ uint32_t candidate_id(unsigned long long p)
+{
+    return 0xFFFFFFFFu - static_cast<uint32_t>(p);
+}
+
+__device__ __forceinline__ unsigned long long shfl_xor_u64(unsigned long long v, int m)
+{
+    return __shfl_xor_sync(0xFFFFFFFFu, v, m);
+}
+__device__ __forceinline__ unsigned long long shfl_u64(unsigned long long v, int src)
+{
+    return __shfl_sync(0xFFFFFFFFu, v, src);
+}
+__device__ __forceinline__ unsigned long long umax64(unsigned long long a, unsigned long long b)
+{
+    return a > b ? a : b;
+}
+__device__ __forceinline__ unsigned long long umin64(unsigned long long a, unsigned long long b)
+{
+    return a < b ? a : b;
+}
+
+// Sort 32 words (one per lane) so that lane 0 holds the largest.
+__device__ __forceinline__ unsigned long long warp_sort_desc(unsigned long long x, int lane)
+{
+#pragma unroll
+    for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            unsigned long long o = shfl_xor_u64(x, j);
+            bool desc_block = (lane & k) == 0;       // k == 32: always true
+            bool lower = (lane & j) == 0;
+            x = (lower == desc_block) ? umax64(x, o) : umin64(x, o);
+        }
+    }
+    return x;
+}
+// Turn a bitonic sequence (one word per lane) into descending order.
+__device__ __forceinline__ unsigned long long warp_bitonic_merge_desc(unsigned long long x, int lane)
+{
+#pragma unroll
+    for (int j = 16; j > 0; j >>= 1) {
+        unsigned long long o = shfl_xor_u64(x, j);
+        x = ((lane & j) == 0) ? umax64(x, o) : umin64(x, o);
+    }
+    return x;
+}
+// Top 32 of the union of two descending lists a, b (one word per lane each).
+__device__ __forceinline__ unsigned long long warp_merge_top32(unsigned long long a,
+                                                               unsigned long long b, int lane)
+{
+    unsigned long long rb = shfl_u64(b, 31 - lane);  // ascending copy of b
+    return warp_bitonic_merge_desc(umax64(a, rb), lane);
+}
+
+// ---------------------------------------------------------------------------
+// WarpTopN: running top-n of one (warp, query) pair.  All state is in shared
+// memory owned by ONE warp, so no CTA-wide synchronisation is ever needed in
+// the streaming loop.  Candidates that pass the cheap score filter are queued;
+// the queue is folded into the sorted list kMergeLevel at a time.
+// ---------------------------------------------------------------------------
+struct WarpTopN {
+    unsigned long long list[kListLen];   // sorted descending; slots >= n are 0
+    unsigned long long queue[kQueueCap];
+    int count;                           // entries waiting in queue
+    float tau;                           // filter: score of the n-th best so far
+};
+
+__device__ __forceinline__ void warp_topn_init(WarpTopN *s, int lane)
+{
+    s->list[lane] = 0ull;
+    if (lane == 0) {
+        s->count = 0;
+        s->tau = -INFINITY;
+    }
+    __syncwarp();
+}
+
+// Fold the queue into the sorted list and tighten the filter score (-inf while
+// fewer than n candidates are known).  Call with all 32 lanes.
+static __device__ __noinline__ void warp_topn_merge(WarpTopN *s, int n, int lane)
+{
+    int count = s->count;
+    unsigned long long x = lane < count ? s->queue[lane] : 0ull;
+    x = warp_sort_desc(x, lane);
+    unsigned long long m = warp_merge_top32(s->list[lane], x, lane);
+    if (lane >= n) m = 0ull;
+    unsigned long long nth = shfl_u64(m, n - 1);
+    __syncwarp();
+    s->list[lane] = m;
+    if (lane == 0) {
+        s->count = 0;
+        s->tau = nth ? candidate_score(nth) : -INFINITY;
+    }
+    __syncwarp();
+}
+
+// Append this lane's candidate (if `take`) to the queue of one (warp, query).
+// Call with all 32 lanes.  Overflow is handled by merging first; the queue is
+// merged again once it reaches kMergeLevel so the filter stays tight.
+static __device__ __noinline__ void warp_topn_push(WarpTopN *s, int n, int lane, bool take, float score,
+                                            uint32_t id)
+{
+    unsigned m = __ballot_sync(0xFFFFFFFFu, take);
+    if (m == 0) return;
+    int incoming = __popc(m);
+    if (s->count + incoming > kQueueCap) warp_topn_merge(s, n, lane);
+    int count = s->count;
+    if (take) s->queue[count + __popc(m & ((1u << lane) - 1u))] = pack_candidate(score, id);
+    __syncwarp();
+    if (lane == 0) s->count = count + incoming;
+    __syncwarp();
+    if (count + incoming >= kMergeLevel) warp_topn_merge(s, n, lane);
+}
+
+// ---------------------------------------------------------------------------
+// mbarrier / TMA wrappers.  Every wait is bounded: after kWaitCycles the
+// caller gets `false`, records a timeout and leaves its loop.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_fence_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; false = gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+    return true;
+}
+// 2-D tiled TMA load global -> shared, completion on `bar`.  x is the
+// innermost (element) coordinate and must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y,
+                                            uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3}], [%4];" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void report_timeout(int *status_word)
+{
+    atomicExch(status_word, kStatusTimeout);
+}
+
+}  // namespace dresd

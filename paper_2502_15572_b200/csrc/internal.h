@@ -1,0 +1,71 @@
+// Host-side declarations shared by the kernel files and the C ABI (api.cu).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dresd {
+
+enum { kF32 = 0, kF16 = 1, kBF16 = 2 };
+
+constexpr int kMaxBatch = 64;
+constexpr int kMaxTopN = 32;
+constexpr int kCandStride = 32;          // u64 slots per (CTA, query) in the workspace
+constexpr float kHiLoScaleF16 = 2048.f;  // low half of an fp16-split query is stored x 2^11
+constexpr float kHiLoScaleBF16 = 256.f;  // low half of a bf16-split query is stored x 2^8
+
+// ---- K1: Eq. 1 -> v W -> Eq. 2 -------------------------------------------
+struct PreprocessArgs {
+    const void *queries;    // [B][d_in] store dtype
+    const float *mean;      // [d_in] or null
+    const float *var;       // [d_in] or null
+    const void *W;          // [d_in][d] store dtype or null
+    const float *pca_mean;  // [d_in] or null
+    float eps_z, eps_n;
+    int B, d_in, d, dtype;
+    float *qhat;            // [rows][d] fp32 unit queries (rows >= B zero)
+    void *qsplit;           // 16-bit keys: [2*rows][dpad] hi/lo operand rows, else null
+    int dpad;               // d rounded up to 64
+    int rows;               // CTAs launched: B rounded up to the operand row count
+    float lo_scale;
+};
+cudaError_t launch_preprocess(const PreprocessArgs &a, cudaStream_t stream);
+
+// ---- K2+K3: score every key, keep a per-CTA top-n per query ----------------
+struct ScanArgs {
+    long long N;            // rows
+    int d;                  // key dimension
+    int dpad;               // row length of qsplit (multiple of 64)
+    int dtype;
+    int n_tiles;            // row tiles of the kernel's tile height
+    int B;                  // queries handled by this launch
+    int top_n;
+    const float *qhat;      // fp32 unit queries of this launch, [B][d]
+    const void *qsplit;     // hi/lo operand rows of this launch, [2*Bpad][dpad]
+    float lo_inv_scale;     // 1 / lo_scale
+    unsigned long long *cand;  // [grid][cand_batch][kCandStride], at this launch's first query
+    int cand_batch;         // query stride of `cand` (the call's B)
+    int *status;            // device status word
+    int stages;             // pipeline depth
+};
+// Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.
+int scan_mma_tile_rows(int d);
+int scan_mma_queries_per_launch(int d, int B);
+size_t scan_mma_smem_bytes(int d, int B, int *stages_out);
+cudaError_t launch_scan_mma(const CUtensorMap &keys_map, const ScanArgs &a, int grid,
+                            cudaStream_t stream);
+
+int scan_f32_tile_rows(int d);
+int scan_f32_queries_per_launch(int d, int B);
+cudaError_t launch_scan_f32(const CUtensorMap &keys_map, const ScanArgs &a, int grid,
+                            cudaStream_t stream);
+
+// ---- K4: merge the per-CTA lists;  K5: gather continuations ----------------
+cudaError_t launch_merge(const unsigned long long *cand, int grid_lists, int B, int top_n,
+                         int32_t *out_ids, float *out_scores, cudaStream_t stream);
+cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long N,
+                          const int32_t *ids, int B, int top_n, int draft_len,
+                          int32_t *out_tokens, cudaStream_t stream);
+
+}  // namespace dresd

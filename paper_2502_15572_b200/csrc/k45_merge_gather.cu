@@ -1,0 +1,81 @@
+// K4 -- grid-level merge: the per-CTA sorted candidate lists of one query are
+// folded into the final top-n (Eq. 3's arg max over the whole datastore,
+// extended to the n best; ties to the lower row index).
+// K5 -- value lookup f_D of Section 3.5: copy the first draft_len stored
+// continuation tokens of every selected key into the n x L draft matrix.
+#include "common.cuh"
+#include "internal.h"
+
+namespace dresd {
+namespace {
+
+constexpr int kMergeWarps = 8;
+
+__global__ void __launch_bounds__(kMergeWarps * 32)
+merge_kernel(const unsigned long long *__restrict__ cand, int lists, int B, int top_n,
+             int32_t *__restrict__ out_ids, float *__restrict__ out_scores)
+{
+    __shared__ unsigned long long part[kMergeWarps][kListLen];
+    const int b = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    unsigned long long m = 0ull;
+    int g = warp;
+    // Four loads in flight per lane before the dependent merge chain starts.
+    for (; g + 3 * kMergeWarps < lists; g += 4 * kMergeWarps) {
+        unsigned long long l0 = cand[((size_t)(g + 0 * kMergeWarps) * B + b) * kCandStride + lane];
+        unsigned long long l1 = cand[((size_t)(g + 1 * kMergeWarps) * B + b) * kCandStride + lane];
+        unsigned long long l2 = cand[((size_t)(g + 2 * kMergeWarps) * B + b) * kCandStride + lane];
+        unsigned long long l3 = cand[((size_t)(g + 3 * kMergeWarps) * B + b) * kCandStride + lane];
+        m = warp_merge_top32(m, l0, lane);
+        m = warp_merge_top32(m, l1, lane);
+        m = warp_merge_top32(m, l2, lane);
+        m = warp_merge_top32(m, l3, lane);
+    }
+    for (; g < lists; g += kMergeWarps)
+        m = warp_merge_top32(m, cand[((size_t)g * B + b) * kCandStride + lane], lane);
+    part[warp][lane] = m;
+    __syncthreads();
+    if (warp == 0) {
+        m = part[0][lane];
+        for (int w = 1; w < kMergeWarps; ++w) m = warp_merge_top32(m, part[w][lane], lane);
+        if (lane < top_n) {
+            out_ids[(size_t)b * top_n + lane] = m ? (int32_t)candidate_id(m) : -1;
+            out_scores[(size_t)b * top_n + lane] = m ? candidate_score(m) : -INFINITY;
+        }
+    }
+}
+
+__global__ void gather_kernel(const int32_t *__restrict__ next_tokens, int stored_len, long long N,
+                              const int32_t *__restrict__ ids, int top_n, int draft_len,
+                              int32_t *__restrict__ out_tokens)
+{
+    const int b = blockIdx.x;
+    const int total = top_n * draft_len;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        const int r = i / draft_len, t = i - r * draft_len;
+        const long long id = ids[(size_t)b * top_n + r];
+        out_tokens[(size_t)b * total + i] =
+            (id >= 0 && id < N) ? next_tokens[(size_t)id * stored_len + t] : -1;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_merge(const unsigned long long *cand, int lists, int B, int top_n,
+                         int32_t *out_ids, float *out_scores, cudaStream_t stream)
+{
+    merge_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, out_ids, out_scores);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long N, const int32_t *ids,
+                          int B, int top_n, int draft_len, int32_t *out_tokens, cudaStream_t stream)
+{
+    int threads = top_n * draft_len;
+    threads = threads < 32 ? 32 : threads > 512 ? 512 : ((threads + 31) / 32) * 32;
+    gather_kernel<<<B, threads, 0, stream>>>(next_tokens, stored_len, N, ids, top_n, draft_len, out_tokens);
+    return cudaGetLastError();
+}
+
+}  // namespace dresd

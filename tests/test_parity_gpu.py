@@ -1,0 +1,252 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2502_15572_b200 import binding, synth
+from tests import checker
+from tests.gpu_util import gpu_retrieve, gpu_store, run_both
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(keys, toks, dtype, q, n, L, pre=None, options=None):
+    ids, sc, tok, o = run_both(keys, toks, dtype, q, n, L, pre=pre, options=options)
+    return checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids)
+
+
+# Sizes span several tiles per CTA of a 148-CTA grid plus a ragged tail.
+@pytest.mark.parametrize("dtype,d,B,n,L,N", [
+    ("f16", 256, 1, 10, 10, 148 * 64 * 3 + 37),
+    ("bf16", 256, 4, 10, 10, 148 * 64 * 2 + 5),
+    ("f16", 256, 8, 32, 16, 30011),
+    ("bf16", 256, 7, 5, 3, 9001),
+    ("f16", 128, 3, 10, 10, 148 * 128 * 2 + 77),
+    ("bf16", 128, 8, 32, 4, 40009),
+    ("f16", 64, 2, 10, 10, 148 * 256 + 300),
+    ("bf16", 64, 5, 17, 10, 50021),
+    ("f16", 72, 2, 10, 6, 20011),          # row = 144 bytes: not a multiple of the 128-byte slab
+    ("bf16", 200, 3, 10, 6, 20011),
+    ("f16", 512, 2, 10, 6, 20011),         # long rows: k-chunked kernel
+    ("bf16", 1024, 4, 10, 6, 9973),
+    ("bf16", 320, 5, 8, 6, 9973),
+    ("f32", 128, 8, 10, 10, 148 * 128 * 2 + 19),
+    ("f32", 64, 3, 32, 10, 20011),
+    ("f32", 200, 9, 10, 5, 10007),
+    ("f32", 1100, 2, 10, 5, 5003),
+    ("f16", 256, 9, 10, 10, 20011),        # more queries than one launch holds
+    ("bf16", 256, 64, 32, 16, 20011),
+    ("f32", 128, 20, 10, 10, 20011),
+])
+def test_parity_shapes(dtype, d, B, n, L, N):
+    keys, toks = synth.make_store(7000 + d + B, N, d, 32, dtype, L + 2)
+    q, _ = synth.make_queries(7100 + d + B, keys, dtype, B, 0.1)
+    _check(keys, toks, dtype, q, n, L)
+
+
+def test_config1_tiny_exact_knn_full():
+    w = synth.make_workload("c1_tiny_f32")
+    rate = _check(w["keys"], w["next_tokens"], "f32", w["queries"], w["top_n"], w["draft_len"])
+    assert rate >= 0.95
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+def test_preprocess_matches_oracle(dtype):
+    import torch
+    d_in, d, B = 1024, 256, 5
+    keys, toks = synth.make_store(7301, 4096, d, 8, dtype, 4)
+    mean, var, W = synth.make_preprocess(7302, d_in, d, dtype)
+    pm = (0.01 * np.arange(d_in)).astype(np.float32)
+    q = synth.make_hidden_queries(7303, B, d_in, dtype)
+    st = gpu_store(keys, toks, dtype)
+    try:
+        cases = [
+            dict(),                                          # Eq. 2 only (needs d_in == d)
+            dict(mean=mean, var=var, W=W),
+            dict(W=W),
+            dict(mean=mean, var=var, W=W, pca_mean=pm),
+        ]
+        for c in cases:
+            qq = q if c else synth.make_hidden_queries(7304, B, d, dtype)
+            dev = {k: (binding.to_device(v, dtype) if k == "W" else torch.from_numpy(v).cuda())
+                   for k, v in c.items()}
+            st.set_preprocess(qq.shape[1], dev.get("mean"), dev.get("var"), 1e-5, dev.get("W"),
+                              dev.get("pca_mean"))
+            got = st.preprocess(binding.to_device(qq, dtype)).cpu().numpy()
+            want = oracle.preprocess(qq, dtype, mean=c.get("mean"), var=c.get("var"), eps_z=1e-5,
+                                     W=c.get("W"), pca_mean=c.get("pca_mean"))
+            # fp32 arithmetic over d_in terms: a few 1e-7 relative to a unit vector
+            np.testing.assert_allclose(got, want, atol=2e-6, rtol=0)
+            np.testing.assert_allclose(np.linalg.norm(got.astype(np.float64), axis=1), 1.0, atol=1e-6)
+    finally:
+        st.close()
+
+
+def test_zscore_only_without_projection():
+    d = 256
+    keys, toks = synth.make_store(7401, 20011, d, 8, "f16", 4)
+    mean, var, _ = synth.make_preprocess(7402, d, d, "f16")
+    q = synth.make_hidden_queries(7403, 3, d, "f16")
+    _check(keys, toks, "f16", q, 10, 4, pre=dict(mean=mean, var=var, eps_z=1e-3))
+
+
+@pytest.mark.parametrize("dtype,d_in,d,B", [("bf16", 4096, 256, 16), ("f16", 768, 64, 3), ("f32", 512, 128, 4)])
+def test_projected_retrieval(dtype, d_in, d, B):
+    keys, toks = synth.make_store(7501, 30011, d, 16, dtype, 10)
+    mean, var, W = synth.make_preprocess(7502, d_in, d, dtype)
+    q = synth.make_hidden_queries(7503, B, d_in, dtype)
+    _check(keys, toks, dtype, q, 10, 10, pre=dict(mean=mean, var=var, W=W))
+
+
+# ---------------------------------------------------------------------------- edge cases
+@pytest.mark.parametrize("dtype", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("N,n", [(1, 1), (5, 5), (33, 32), (64, 10), (257, 32)])
+def test_tiny_stores(dtype, N, n):
+    keys, toks = synth.make_store(7600 + N, N, 64, 3, dtype, 3)
+    q, _ = synth.make_queries(7601, keys, dtype, 3, 0.2)
+    _check(keys, toks, dtype, q, n, 3)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16"])
+def test_scores_ascending_in_memory(dtype):
+    # Worst case for a running-threshold filter: every key beats all before it.
+    N, d = 20000, 64
+    keys, toks = synth.make_store(7701, N, d, 4, dtype, 2)
+    q, _ = synth.make_queries(7702, keys, dtype, 2, 0.1)
+    s = oracle.scores(keys, dtype, oracle.preprocess(q[:1], dtype)[0])
+    order = np.argsort(s, kind="stable")
+    _check(keys[order], toks[order], dtype, q, 10, 2)
+    _check(keys[order[::-1]], toks[order[::-1]], dtype, q, 10, 2)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_all_keys_identical_gives_lowest_ids(dtype):
+    N, d = 5000, 64
+    keys, toks = synth.make_store(7801, N, d, 2, dtype, 2)
+    keys[:] = keys[0]
+    q, _ = synth.make_queries(7802, keys, dtype, 2, 0.1)
+    ids, sc, tok, o = run_both(keys, toks, dtype, q, 12, 2)
+    assert np.array_equal(ids, np.tile(np.arange(12), (2, 1)))
+    assert np.array_equal(o.ids, ids)
+    assert np.array_equal(tok, toks[ids][:, :, :2])
+
+
+def test_duplicates_and_zero_query():
+    N, d = 9000, 128
+    keys, toks = synth.make_store(7901, N, d, 8, "f16", 4)
+    keys[8000] = keys[123]
+    keys[4000] = keys[123]
+    q = np.concatenate([keys[123:124], np.zeros((1, d), dtype=np.float16)])
+    ids, sc, tok, o = run_both(keys, toks, "f16", q, 6, 4)
+    assert ids[0, :3].tolist() == [123, 4000, 8000]
+    assert sc[0, 0] == sc[0, 1] == sc[0, 2]
+    assert ids[1].tolist() == [0, 1, 2, 3, 4, 5] and np.all(sc[1] == 0.0)
+    checker.check_batch(o.full_scores, toks, ids, sc, tok, "f16", 6, 4, oracle_ids=o.ids)
+
+
+# ---------------------------------------------------------------------------- invariants on the GPU
+def test_invariants_permutation_shards_prefix_repeat():
+    N, d, dtype = 30011, 256, "f16"
+    keys, toks = synth.make_store(8001, N, d, 16, dtype, 10)
+    q, _ = synth.make_queries(8002, keys, dtype, 4, 0.1)
+    st = gpu_store(keys, toks, dtype)
+    ids, sc, tok = gpu_retrieve(st, q, 10, 10)
+    ids2, sc2, tok2 = gpu_retrieve(st, q, 10, 10)
+    assert np.array_equal(ids, ids2) and np.array_equal(sc, sc2) and np.array_equal(tok, tok2)
+    # prefixes
+    ids5, sc5, tok5 = gpu_retrieve(st, q, 5, 4)
+    assert np.array_equal(ids5, ids[:, :5]) and np.array_equal(sc5, sc[:, :5])
+    assert np.array_equal(tok5, tok[:, :5, :4])
+    # batch of B equals B single-query calls (different kernel instantiations)
+    for b in range(4):
+        i1, s1, t1 = gpu_retrieve(st, q[b:b + 1], 10, 10)
+        assert np.array_equal(i1[0], ids[b])
+        np.testing.assert_allclose(s1[0], sc[b], atol=1e-6)
+    st.close()
+    # permutation of the rows: ids map through the permutation, scores are bit-identical
+    perm = np.random.default_rng(8003).permutation(N)
+    stp = gpu_store(keys[perm], toks[perm], dtype)
+    idp, scp, tokp = gpu_retrieve(stp, q, 10, 10)
+    stp.close()
+    assert np.array_equal(perm[idp], ids) and np.array_equal(scp, sc) and np.array_equal(tokp, tok)
+    # shard merge: top-n of the whole = merge of the shards' top-n
+    cut = 12345
+    sa = gpu_store(keys[:cut], toks[:cut], dtype)
+    sb = gpu_store(keys[cut:], toks[cut:], dtype)
+    ia, sca, ta = gpu_retrieve(sa, q, 10, 10)
+    ib, scb, tb = gpu_retrieve(sb, q, 10, 10)
+    sa.close()
+    sb.close()
+    for b in range(4):
+        mi = np.concatenate([ia[b], ib[b] + cut])
+        ms = np.concatenate([sca[b], scb[b]])
+        mt = np.concatenate([ta[b], tb[b]])
+        order = np.lexsort((mi, -ms.astype(np.float64)))[:10]
+        assert np.array_equal(mi[order], ids[b]) and np.array_equal(ms[order], sc[b])
+        assert np.array_equal(mt[order], tok[b])
+
+
+def test_self_retrieval_mrr_is_one():
+    N, d, dtype = 40000, 128, "bf16"
+    keys, toks = synth.make_store(8101, N, d, 64, dtype, 2)
+    idx = np.random.default_rng(8102).integers(0, N, size=64)
+    st = gpu_store(keys, toks, dtype)
+    ids, sc, _ = gpu_retrieve(st, keys[idx], 1, 1)
+    st.close()
+    # Eq. 4: reciprocal rank of the correct item; exact search finds every key first
+    assert np.mean(1.0 / (1 + (ids[:, 0] != idx))) == 1.0
+    np.testing.assert_allclose(sc[:, 0], 1.0, atol=2.0 ** -7)
+
+
+def test_grid_option_and_host_call():
+    import torch
+    N, d, dtype = 30011, 256, "f16"
+    keys, toks = synth.make_store(8201, N, d, 16, dtype, 10)
+    q, _ = synth.make_queries(8202, keys, dtype, 2, 0.1)
+    st = gpu_store(keys, toks, dtype)
+    ref = gpu_retrieve(st, q, 10, 10)
+    for grid in (1, 7, 296):
+        st.set_option("grid", grid)
+        got = gpu_retrieve(st, q, 10, 10)
+        assert all(np.array_equal(a, b) for a, b in zip(ref, got))
+    st.set_option("grid", 0)
+    qh = torch.from_numpy(q.view(np.float16)).pin_memory()
+    out = (torch.empty((2, 10), dtype=torch.int32).pin_memory(),
+           torch.empty((2, 10), dtype=torch.float32).pin_memory(),
+           torch.empty((2, 10, 10), dtype=torch.int32).pin_memory())
+    st.retrieve_host(qh, 10, 10, out)
+    assert all(np.array_equal(a, b.numpy()) for a, b in zip(ref, out))
+    assert st.last_launches() == 4
+    st.close()
+
+
+def test_argument_errors_on_device():
+    import torch
+    keys, toks = synth.make_store(8301, 1000, 64, 4, "f16", 4)
+    st = gpu_store(keys, toks, "f16")
+    q = binding.to_device(keys[:2], "f16")
+    with pytest.raises(binding.DresdError) as e:
+        st.retrieve(q, 0, 2)
+    assert e.value.status == -1
+    with pytest.raises(binding.DresdError) as e:
+        st.retrieve(q, 2, 5)
+    assert e.value.status == -1
+    with pytest.raises(binding.DresdError) as e:
+        st.retrieve(q, 33, 2)
+    assert e.value.status == -2
+    big = torch.zeros((65, 64), dtype=torch.float16, device="cuda")
+    with pytest.raises(binding.DresdError) as e:
+        st.retrieve(big, 2, 2)
+    assert e.value.status == -2
+    with pytest.raises(binding.DresdError) as e:      # host pointer where a device pointer is required
+        binding.dresd_retrieve(st.handle, keys.ctypes.data, 1, 1, 1, keys.ctypes.data, keys.ctypes.data,
+                               keys.ctypes.data, 0)
+    assert e.value.status == -1
+    ids, sc, tok = st.retrieve(q[:0], 2, 2)          # B == 0 is a no-op
+    st.close()
+    with pytest.raises(binding.DresdError):
+        binding.dresd_store_create(0, 0, 10, 64, 1, 4)
+    k = torch.zeros((8, 12), dtype=torch.float16, device="cuda")   # 24-byte rows
+    with pytest.raises(binding.DresdError) as e:
+        binding.Store(k, torch.zeros((8, 2), dtype=torch.int32, device="cuda"), "f16")
+    assert e.value.status == -1
