@@ -157,6 +157,44 @@ int dresd_store_last_launches(const dresd_store *store);
 /* Message of the calling thread's last failing call ("" if none). */
 const char *dresd_last_error(void);
 
+/*
+ * (No counterpart in the paper: a deployment variant of dresd_retrieve().)
+ *
+ * Retrieval for callers that cannot allocate device memory when they need a
+ * draft -- a serving runtime that gave all device memory to its own pool and
+ * forbids cudaMalloc afterwards, a plug-in living inside another program's
+ * memory budget, a latency-critical path that cannot afford the device-wide
+ * synchronisation an allocation implies.  dresd_store_create() needs cudaMalloc
+ * for its workspace; this call needs no store: its workspace (unit queries,
+ * their 16-bit split, per-CTA candidate lists, status word) is a fixed
+ * ~576 KB array inside the library image, held by every GPU that loads the
+ * library until the process exits.  It calls no cudaMalloc/cudaFree and no
+ * allocating library routine; it computes exactly what dresd_retrieve() does
+ * on a store without z-scoring or projection (Eq. 2, Eq. 3, Section 3.5),
+ * with the same kernels, so results are identical.
+ *
+ *   keys, next_tokens, N, d, dtype, stored_len   as for dresd_store_create();
+ *   queries [B][d], B, top_n, draft_len, out_*   as for dresd_retrieve()
+ *   (all device pointers; the caller owns inputs and outputs).
+ *
+ * Limits: B <= DRESD_NOALLOC_MAX_BATCH (8); larger B returns
+ * DRESD_ERR_UNSUPPORTED with a message, as do top_n > DRESD_MAX_TOP_N and
+ * d > DRESD_MAX_DIM.  Pointers are checked for NULL and alignment only.
+ *
+ * The first call on each device resolves the workspace's device address
+ * (with that device current); make that first call outside any stream
+ * capture.  The workspace is ONE per device and keeps the previous call's
+ * contents (the call clears the one word that must start at zero): two calls
+ * whose kernels overlap on the GPU -- different streams, or threads -- race
+ * on it and return garbage.  Serialise them on one stream.  Asynchronous on
+ * `stream` like dresd_retrieve(); device-side timeouts are not reported here.
+ */
+enum { DRESD_NOALLOC_MAX_BATCH = 8 };
+dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *next_tokens, int64_t N, int d,
+                                    dresd_dtype dtype, int stored_len, const void *queries, int B,
+                                    int top_n, int draft_len, int32_t *out_ids, float *out_scores,
+                                    int32_t *out_tokens, void *stream);
+
 /* Frees the workspace only, never caller memory.  NULL is allowed. */
 void dresd_store_destroy(dresd_store *store);
 

@@ -26,7 +26,7 @@ EXPORTS = (
     "dresd_store_create", "dresd_store_set_preprocess", "dresd_retrieve", "dresd_retrieve_host",
     "dresd_preprocess", "dresd_store_status", "dresd_store_set_option",
     "dresd_store_profile_read", "dresd_store_last_launches", "dresd_last_error",
-    "dresd_store_destroy",
+    "dresd_store_destroy", "dresd_retrieve_noalloc",
 )
 
 
@@ -74,6 +74,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_last_error.argtypes = []
     lib.dresd_store_destroy.restype = None
     lib.dresd_store_destroy.argtypes = [vp]
+    lib.dresd_retrieve_noalloc.restype = i32
+    lib.dresd_retrieve_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
     if path is None:
         _lib = lib
     return lib
@@ -138,6 +140,19 @@ def dresd_store_last_launches(store: int) -> int:
 
 def dresd_store_destroy(store: int) -> None:
     load().dresd_store_destroy(store)
+
+
+def dresd_retrieve_noalloc(keys_ptr: int, next_tokens_ptr: int, N: int, d: int, dtype: int,
+                           stored_len: int, queries_ptr: int, B: int, top_n: int, draft_len: int,
+                           out_ids_ptr: int, out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
+    """Retrieval without any device allocation (static in-library workspace, B <= 8).
+
+    For hosts that may not call cudaMalloc when a draft is needed; see the
+    header for the limits and the rule that calls must not overlap on the GPU.
+    """
+    _check(load().dresd_retrieve_noalloc(keys_ptr, next_tokens_ptr, N, d, dtype, stored_len, queries_ptr,
+                                         B, top_n, draft_len, out_ids_ptr, out_scores_ptr, out_tokens_ptr,
+                                         stream))
 
 
 # ---- torch convenience ----------------------------------------------------------

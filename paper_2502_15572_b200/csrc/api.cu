@@ -84,6 +84,8 @@ bool make_map(CUtensorMap *map, const void *base, int dtype, long long rows, int
 
 }  // namespace
 
+void dresd::set_last_error(const char *msg) { snprintf(g_err, sizeof g_err, "%s", msg ? msg : ""); }
+
 struct dresd_store {
     uint32_t magic;
     int device;

@@ -68,4 +68,7 @@ cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long 
                           const int32_t *ids, int B, int top_n, int draft_len,
                           int32_t *out_tokens, cudaStream_t stream);
 
+// Stores `msg` as the calling thread's dresd_last_error() text.
+void set_last_error(const char *msg);
+
 }  // namespace dresd
