@@ -116,6 +116,10 @@ struct dresd_store {
     // streaming-kernel geometry
     CUtensorMap map_stream;
     int tile_rows, n_tiles;
+    // tensor-core kernel geometry (16-bit keys): 128-row key tiles, query operand maps
+    CUtensorMap map_umma;
+    CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
+    int n_tiles_umma;
     // options / bookkeeping
     int opt_path, opt_grid;
     cudaStream_t last_stream;
@@ -166,7 +170,7 @@ dresd_status check_retrieve_args(const dresd_store *s, const void *queries, int 
 }
 
 // K1 for B queries into the store's workspace.
-dresd_status run_preprocess(dresd_store *s, const void *queries, int B, cudaStream_t stream)
+dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows, cudaStream_t stream)
 {
     PreprocessArgs p{};
     p.queries = queries;
@@ -183,7 +187,7 @@ dresd_status run_preprocess(dresd_store *s, const void *queries, int B, cudaStre
     p.qhat = s->qhat;
     p.qsplit = s->dtype == kF32 ? nullptr : s->qsplit;
     p.dpad = s->dpad;
-    p.rows = ((B + 7) / 8) * 8;
+    p.rows = rows;                   // operand rows beyond B are written as zeros
     p.lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
     cudaError_t e = launch_preprocess(p, stream);
     if (e != cudaSuccess) return fail_cuda(e, "preprocess launch");
@@ -196,19 +200,42 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
 {
     s->last_stream = stream;
     s->last_launches = 0;
-    dresd_status st = run_preprocess(s, queries, B, stream);
+    const bool f32 = s->dtype == kF32;
+    // 16-bit keys: the streaming mma.sync kernel serves up to 8 queries per pass over
+    // the keys; beyond that the tcgen05 kernel serves all of them in one pass.
+    const bool umma = !f32 && (s->opt_path == 2 || (s->opt_path == 0 && B > 8));
+    const int op_rows = umma ? scan_umma_operand_rows(B) : 0;
+    dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream);
     if (st != DRESD_OK) return st;
 
+    const int n_tiles = umma ? s->n_tiles_umma : s->n_tiles;
     int grid = s->opt_grid > 0 ? s->opt_grid : s->num_sms;
     if (grid > s->max_grid) grid = s->max_grid;
-    if (grid > s->n_tiles) grid = s->n_tiles;
+    if (grid > n_tiles) grid = n_tiles;
 
-    const bool f32 = s->dtype == kF32;
-    const int qpl = f32 ? scan_f32_queries_per_launch(s->d, B) : scan_mma_queries_per_launch(s->d, B);
+    const int qpl = umma ? B : f32 ? scan_f32_queries_per_launch(s->d, B) : scan_mma_queries_per_launch(s->d, B);
     const float lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
     const bool prof = s->prof_count < s->prof_cap;
     if (prof) cudaEventRecord(s->prof_events[2 * s->prof_count], stream);
-    for (int q0 = 0; q0 < B; q0 += qpl) {
+    if (umma) {
+        ScanArgs a{};
+        a.N = s->N;
+        a.d = s->d;
+        a.dpad = s->dpad;
+        a.dtype = s->dtype;
+        a.n_tiles = n_tiles;
+        a.B = B;
+        a.top_n = top_n;
+        a.lo_inv_scale = 1.0f / lo_scale;
+        a.cand = s->cand;
+        a.cand_batch = B;
+        a.status = s->status;
+        const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
+        cudaError_t e = launch_scan_umma(s->map_umma, s->map_q[mi], a, grid, stream);
+        if (e != cudaSuccess) return fail_cuda(e, "scan launch");
+        s->last_launches += 1;
+    }
+    for (int q0 = 0; q0 < B && !umma; q0 += qpl) {
         ScanArgs a{};
         a.N = s->N;
         a.d = s->d;
@@ -304,6 +331,16 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
               cudaMalloc(&s->scores_dev, sizeof(float) * kMaxBatch * kMaxTopN) == cudaSuccess;
     s->tokens_dev_elems = (size_t)kMaxBatch * kMaxTopN * stored_len;
     ok = ok && cudaMalloc(&s->tokens_dev, sizeof(int32_t) * s->tokens_dev_elems) == cudaSuccess;
+    if (ok && dtype != DRESD_F32) {
+        s->n_tiles_umma = (int)((N + scan_umma_tile_rows() - 1) / scan_umma_tile_rows());
+        bool mok = make_map(&s->map_umma, keys, s->dtype, N, d, scan_umma_tile_rows());
+        for (int i = 0; i < 4; ++i)
+            mok = mok && make_map(&s->map_q[i], s->qsplit, s->dtype, 2 * kMaxBatch, s->dpad, 16 << i);
+        if (!mok) {
+            free_store(s);
+            return fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the tensor-core path");
+        }
+    }
     s->q_stage_bytes = (size_t)kMaxBatch * d * eb;
     ok = ok && cudaMalloc(&s->q_stage, s->q_stage_bytes) == cudaSuccess;
     ok = ok && cudaMemset(s->status, 0, sizeof(int)) == cudaSuccess;
@@ -400,7 +437,7 @@ dresd_status dresd_preprocess(dresd_store *s, const void *queries, int B, float 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     s->last_stream = stream;
     s->last_launches = 0;
-    dresd_status st = run_preprocess(s, queries, B, stream);
+    dresd_status st = run_preprocess(s, queries, B, ((B + 7) / 8) * 8, stream);
     if (st != DRESD_OK) return st;
     cudaError_t e = cudaMemcpyAsync(out_qhat, s->qhat, sizeof(float) * (size_t)B * s->d,
                                     cudaMemcpyDeviceToDevice, stream);

@@ -56,6 +56,13 @@ size_t scan_mma_smem_bytes(int d, int B, int *stages_out);
 cudaError_t launch_scan_mma(const CUtensorMap &keys_map, const ScanArgs &a, int grid,
                             cudaStream_t stream);
 
+// Batched tensor-core kernel (tcgen05/TMEM, 16-bit keys): 128-row tiles; the query
+// operand holds 2 rows per query, padded to 16/32/64/128 rows.
+int scan_umma_tile_rows();
+int scan_umma_operand_rows(int B);
+cudaError_t launch_scan_umma(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
+                             int grid, cudaStream_t stream);
+
 int scan_f32_tile_rows(int d);
 int scan_f32_queries_per_launch(int d, int B);
 cudaError_t launch_scan_f32(const CUtensorMap &keys_map, const ScanArgs &a, int grid,

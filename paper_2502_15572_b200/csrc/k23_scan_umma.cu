@@ -1,0 +1,375 @@
+// K2+K3 (batched path, 16-bit keys) -- Eq. 3 of the paper for every key and
+// up to 64 queries at once on the 5th-generation tensor cores, fused with the
+// per-CTA top-n selection.  Still HBM-bound (B flop/byte is far left of the
+// ridge): tensor cores are used so that the arithmetic of B queries hides
+// under ONE pass over the keys.
+//
+// One persistent CTA per SM, six warps:
+//   warp 0    producer: one thread streams 128-row x 64-column key slabs
+//             (16 KB, 128-byte swizzle) with TMA through an mbarrier ring and,
+//             when the query operand is too large to stay resident, the
+//             matching query slab next to each key slab;
+//   warp 1    allocates TMEM; one thread issues tcgen05.mma (M = 128 key rows,
+//             N = 2 columns per query: q = hi + lo/scale, K = 16 per
+//             instruction, fp32 accumulators in TMEM, two accumulator buffers
+//             so that the epilogue of tile t overlaps the MMAs of tile t+1);
+//             tcgen05.commit releases shared-memory stages and publishes
+//             finished accumulators;
+//   warps 2-5 epilogue: each thread owns one key row of the tile, reads its
+//             N accumulator columns with tcgen05.ld, combines hi and lo,
+//             filters against the CTA's running n-th best per query and
+//             queues survivors; queues are folded into sorted 32-lane lists
+//             with shuffle-based bitonic merges.
+// Every wait is bounded; TMEM is freed on every path.
+#include <type_traits>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace dresd {
+namespace {
+
+constexpr int kThreads = 6 * 32;
+constexpr int kEpiThreads = 128;
+constexpr int kTileRows = 128;
+constexpr int kSlabBytes = 128;
+constexpr int kSlabElems = 64;
+constexpr int kKeyStageBytes = kTileRows * kSlabBytes;     // 16 KB
+constexpr int kMaxStages = 12;
+constexpr int kResidentLimit = 64 * 1024;                  // query operand kept in smem up to this size
+
+// ------------------------------- tcgen05 wrappers -------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t *smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]; fp16/bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// K-major operand, 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr)
+{
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+struct EpiFlags {
+    int need_merge;
+    int overflow;
+};
+
+template <typename T, int NCOLS>
+__global__ void __launch_bounds__(kThreads, 1)
+scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_constant__ CUtensorMap q_map,
+                 const ScanArgs a, const int q_resident)
+{
+    constexpr int NQ = NCOLS / 2;                           // queries (padded)
+    constexpr int kTmemCols = 2 * NCOLS < 32 ? 32 : 2 * NCOLS;
+    constexpr int kQSlabBytes = NCOLS * kSlabBytes;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *base = reinterpret_cast<uint8_t *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int n_stages = a.stages;
+    const int dslabs = (a.d + kSlabElems - 1) / kSlabElems;
+    const int stage_bytes = kKeyStageBytes + (q_resident ? 0 : kQSlabBytes);
+    uint8_t *stages = base;
+    uint8_t *qres = stages + (size_t)n_stages * stage_bytes;                 // resident query operand
+    WarpTopN *sel = reinterpret_cast<WarpTopN *>(qres + (q_resident ? (size_t)dslabs * kQSlabBytes : 0));
+    float *tau = reinterpret_cast<float *>(sel + NQ);
+    uint64_t *full = reinterpret_cast<uint64_t *>(tau + NQ);
+    uint64_t *empty = full + kMaxStages;
+    uint64_t *tfull = empty + kMaxStages;                   // [2] accumulator ready
+    uint64_t *tempty = tfull + 2;                           // [2] accumulator drained
+    uint64_t *qbar = tempty + 2;                            // resident query operand landed
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(qbar + 1);
+    EpiFlags *flags = reinterpret_cast<EpiFlags *>(tmem_slot + 2);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x, G = gridDim.x;
+    const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
+    const int n_it = my_tiles * dslabs;
+
+    if (tid == 0) {
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&tfull[b], 1);
+            mbar_init(&tempty[b], 4);
+        }
+        mbar_init(qbar, 1);
+        for (int i = 0; i < 3; ++i) {
+            flags[i].need_merge = 0;
+            flags[i].overflow = 0;
+        }
+        mbar_fence_init();
+    }
+    if (warp >= 2) {
+        for (int q = warp - 2; q < NQ; q += 4) {
+            warp_topn_init(&sel[q], lane);
+            if (lane == 0) tau[q] = -INFINITY;
+        }
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------------------------- producer ----------------------------------
+        if (lane == 0) {
+            tma_prefetch_desc(&keys_map);
+            tma_prefetch_desc(&q_map);
+            if (q_resident) {
+                mbar_arrive_expect_tx(qbar, (uint32_t)(dslabs * kQSlabBytes));
+                for (int s = 0; s < dslabs; ++s)
+                    tma_load_2d(qres + (size_t)s * kQSlabBytes, &q_map, s * kSlabElems, 0, qbar);
+            }
+            int issued = 0;
+            for (int it = 0; it < n_it; ++it) {
+                const int s = it % n_stages;
+                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
+                    report_timeout(a.status);
+                    break;
+                }
+                const int tile = cta + (it / dslabs) * G;
+                const int sl = it % dslabs;
+                uint8_t *dst = stages + (size_t)s * stage_bytes;
+                mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
+                tma_load_2d(dst, &keys_map, sl * kSlabElems, tile * kTileRows, &full[s]);
+                if (!q_resident) tma_load_2d(dst + kKeyStageBytes, &q_map, sl * kSlabElems, 0, &full[s]);
+                issued = it + 1;
+            }
+            for (int it = max(0, issued - n_stages); it < issued; ++it)
+                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1)) {
+                    report_timeout(a.status);
+                    break;
+                }
+            if (q_resident && !mbar_wait(qbar, 0)) report_timeout(a.status);
+        }
+    } else if (warp == 1) {
+        // ---------------------------------- MMA issuer ----------------------------------
+        if (lane == 0) {
+            constexpr uint32_t kFmt = sizeof(T) == 2 && std::is_same<T, __nv_bfloat16>::value ? 1u : 0u;
+            constexpr uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(NCOLS >> 3) << 17) |
+                                       ((uint32_t)(kTileRows >> 4) << 24);
+            bool ok = true;
+            if (q_resident && my_tiles > 0) ok = mbar_wait(qbar, 0);
+            for (int tl = 0; tl < my_tiles && ok; ++tl) {
+                const int acc = tl & 1, use = tl >> 1;
+                if (use >= 1 && !mbar_wait(&tempty[acc], (use - 1) & 1)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * NCOLS);
+                for (int sl = 0; sl < dslabs; ++sl) {
+                    const int it = tl * dslabs + sl;
+                    const int s = it % n_stages;
+                    if (!mbar_wait(&full[s], (it / n_stages) & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(stages + (size_t)s * stage_bytes);
+                    const uint32_t b_addr = q_resident ? smem_u32(qres + (size_t)sl * kQSlabBytes)
+                                                       : a_addr + kKeyStageBytes;
+                    const uint64_t a_desc = make_desc(a_addr), b_desc = make_desc(b_addr);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)     // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
+                        umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl | k) != 0);
+                    tc_commit(&empty[s]);           // stage reusable once these MMAs have read it
+                }
+                if (!ok) break;
+                tc_commit(&tfull[acc]);             // accumulator complete
+            }
+            if (!ok) report_timeout(a.status);
+        }
+    } else {
+        // ---------------------------------- epilogue ----------------------------------
+        const int ew = warp - 2;                            // 0..3
+        const int lane_grp = warp & 3;                      // TMEM lanes this warp may read
+        const int et = ew * 32 + lane;                      // 0..127 among epilogue threads
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
+        // A warp whose wait expired goes "dead": it does no more work and no more
+        // waits, but keeps taking part in every barrier so that nobody is left behind.
+        bool dead = false;
+        int round = 0;                                      // barrier-A count: selects the flag slot
+        EpiFlags *fl = &flags[0];
+        for (int tl = 0; tl < my_tiles; ++tl) {
+            const int acc = tl & 1, use = tl >> 1;
+            if (!dead && !mbar_wait(&tfull[acc], use & 1)) {
+                report_timeout(a.status);
+                dead = true;
+            }
+            dead = __any_sync(0xFFFFFFFFu, dead);
+            tc_fence_after();
+            const long long row = (long long)(cta + tl * G) * kTileRows + lane_grp * 32 + lane;
+            const bool row_ok = !dead && row < a.N;
+            unsigned long long pending = 0ull;              // queries whose candidate found the queue full
+            bool first = true;
+            while (true) {
+#pragma unroll
+                for (int c = 0; c < NCOLS / 16; ++c) {
+                    // warp-uniform decision: tcgen05.ld needs the whole warp
+                    if (dead || (!first && !__any_sync(0xFFFFFFFFu, ((pending >> (c * 8)) & 0xFFull) != 0))) continue;
+                    uint32_t r[16];
+                    tmem_ld16(lane_addr + (uint32_t)(acc * NCOLS + c * 16), r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int q = c * 8 + j;
+                        const float s = __uint_as_float(r[2 * j]) + __uint_as_float(r[2 * j + 1]) * a.lo_inv_scale;
+                        bool want = first ? (row_ok && q < a.B) : ((pending >> q) & 1ull) != 0;
+                        if (want && s >= tau[q]) {
+                            const int slot = atomicAdd(&sel[q].count, 1);
+                            if (slot < kQueueCap) {
+                                sel[q].queue[slot] = pack_candidate(s, (uint32_t)row);
+                                pending &= ~(1ull << q);
+                                if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
+                            } else {
+                                pending |= 1ull << q;
+                                fl->overflow = 1;
+                            }
+                        } else {
+                            pending &= ~(1ull << q);
+                        }
+                    }
+                }
+                first = false;
+                epi_bar();                                   // A: every push of this round is visible
+                const int need = fl->need_merge, over = fl->overflow;
+                // Flags rotate over three slots: the slot of the previous round was read by
+                // everyone before arriving at A and is not written again before the next A.
+                if (et == 0) {
+                    EpiFlags *prev = &flags[(round + 2) % 3];
+                    prev->need_merge = 0;
+                    prev->overflow = 0;
+                }
+                round += 1;
+                fl = &flags[round % 3];
+                if (!(need | over)) break;
+                for (int q = ew; q < NQ; q += 4) {
+                    if (sel[q].count > 0) {
+                        warp_topn_merge(&sel[q], a.top_n, lane);
+                        if (lane == 0) tau[q] = sel[q].tau;
+                    }
+                }
+                epi_bar();                                   // C: lists, counts and tau are settled
+                if (!over) break;
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty[acc]);
+        }
+        // flush and publish this CTA's lists
+        epi_bar();
+        for (int q = ew; q < NQ; q += 4) {
+            if (sel[q].count > 0) warp_topn_merge(&sel[q], a.top_n, lane);
+            if (q < a.B) {
+                unsigned long long m = sel[q].list[lane];
+                if (lane >= a.top_n) m = 0ull;
+                a.cand[((size_t)cta * a.cand_batch + q) * kCandStride + lane] = m;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+struct Plan {
+    int ncols, stages, q_resident;
+    size_t smem;
+};
+
+Plan make_plan(int d, int B)
+{
+    Plan p{};
+    p.ncols = B <= 8 ? 16 : B <= 16 ? 32 : B <= 32 ? 64 : 128;
+    const int dslabs = (d + kSlabElems - 1) / kSlabElems;
+    const size_t qbytes = (size_t)dslabs * p.ncols * kSlabBytes;
+    p.q_resident = qbytes <= (size_t)kResidentLimit;
+    const size_t fixed = 1024 + (p.q_resident ? qbytes : 0) + sizeof(WarpTopN) * (p.ncols / 2) +
+                         sizeof(float) * (p.ncols / 2) + sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
+    const size_t stage = kKeyStageBytes + (p.q_resident ? 0 : (size_t)p.ncols * kSlabBytes);
+    long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)stage;
+    p.stages = (int)(s > kMaxStages ? kMaxStages : s);
+    p.smem = fixed + (size_t)(p.stages > 0 ? p.stages : 0) * stage;
+    return p;
+}
+
+template <typename T, int NCOLS>
+cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a, const Plan &p,
+                       int grid, cudaStream_t stream)
+{
+    auto kernel = scan_umma_kernel<T, NCOLS>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
+    if (e != cudaSuccess) return e;
+    kernel<<<grid, kThreads, p.smem, stream>>>(kmap, qmap, a, p.q_resident);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int scan_umma_tile_rows() { return kTileRows; }
+int scan_umma_operand_rows(int B) { return B <= 8 ? 16 : B <= 16 ? 32 : B <= 32 ? 64 : 128; }
+
+cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a_in, int grid,
+                             cudaStream_t stream)
+{
+    ScanArgs a = a_in;
+    const Plan p = make_plan(a.d, a.B);
+    if (p.stages < 2) return cudaErrorInvalidValue;
+    a.stages = p.stages;
+    const bool h = a.dtype == kF16;
+#define DRESD_GO(N_)                                                                          \
+    return h ? launch_one<__half, N_>(kmap, qmap, a, p, grid, stream)                         \
+             : launch_one<__nv_bfloat16, N_>(kmap, qmap, a, p, grid, stream)
+    switch (p.ncols) {
+    case 16: DRESD_GO(16);
+    case 32: DRESD_GO(32);
+    case 64: DRESD_GO(64);
+    default: DRESD_GO(128);
+    }
+#undef DRESD_GO
+}
+
+}  // namespace dresd

@@ -44,6 +44,39 @@ def test_parity_shapes(dtype, d, B, n, L, N):
     _check(keys, toks, dtype, q, n, L)
 
 
+# Both 16-bit scoring kernels at every batch size: path 1 = streaming mma.sync kernel
+# (several passes when B > 8), path 2 = tcgen05/TMEM kernel (one pass, operand padded).
+@pytest.mark.parametrize("path", [1, 2])
+@pytest.mark.parametrize("dtype,d,B,n,L,N", [
+    ("f16", 256, 1, 10, 10, 148 * 128 * 2 + 37),
+    ("bf16", 256, 8, 32, 4, 30011),
+    ("f16", 256, 16, 10, 10, 30011),
+    ("bf16", 256, 33, 32, 16, 148 * 128 + 77),
+    ("bf16", 256, 64, 32, 16, 30011),
+    ("f16", 64, 20, 10, 3, 40009),
+    ("bf16", 128, 12, 10, 3, 40009),
+    ("f16", 72, 5, 10, 3, 20011),
+    ("bf16", 512, 16, 10, 3, 20011),
+    ("bf16", 4096, 16, 10, 3, 2003),       # query operand too large to stay in shared memory
+    ("f16", 2048, 40, 7, 3, 1501),
+])
+def test_parity_both_16bit_paths(path, dtype, d, B, n, L, N):
+    keys, toks = synth.make_store(7200 + d + B, N, d, 32, dtype, L + 1)
+    q, _ = synth.make_queries(7250 + d + B, keys, dtype, B, 0.1)
+    _check(keys, toks, dtype, q, n, L, options={"scan_path": path})
+
+
+@pytest.mark.parametrize("path", [1, 2])
+def test_adversarial_order_both_paths(path):
+    # ascending scores in memory: every row beats all rows before it (queue overflow path)
+    N, d, dtype = 12000, 64, "bf16"
+    keys, toks = synth.make_store(7270, N, d, 4, dtype, 2)
+    q, _ = synth.make_queries(7271, keys, dtype, 12, 0.1)
+    s = oracle.scores(keys, dtype, oracle.preprocess(q[:1], dtype)[0])
+    order = np.argsort(s, kind="stable")
+    _check(keys[order], toks[order], dtype, q, 10, 2, options={"scan_path": path})
+
+
 def test_config1_tiny_exact_knn_full():
     w = synth.make_workload("c1_tiny_f32")
     rate = _check(w["keys"], w["next_tokens"], "f32", w["queries"], w["top_n"], w["draft_len"])
