@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--rows", type=int, default=None, help="override N (debugging; not a bench value)")
     ap.add_argument("--oracle-queries", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scan-path", type=int, default=0, choices=[0, 1, 2],
+                    help="0 auto, 1 streaming mma.sync kernel, 2 tcgen05 kernel (16-bit keys)")
     return ap.parse_args()
 
 
@@ -66,7 +68,8 @@ def metric_name(cfg):
 
 
 def workload_config(cfg):
-    return {"workload": cfg["name"], "N": cfg["N"], "d": cfg["d"], "key_dtype": cfg["dtype"],
+    return {"workload": cfg["name"], "N": cfg["N"], "d": cfg["d"], "d_in": cfg.get("d_in", cfg["d"]),
+            "key_dtype": cfg["dtype"],
             "batch": cfg["B"], "top_n": cfg["top_n"], "draft_len": cfg["draft_len"],
             "mixture_components": cfg["C"], "query_noise_sigma": cfg["sigma"], "seed": cfg["seed"],
             "l2": "keys are %.2f GB per step, far larger than the 126 MB L2: no flush needed"
@@ -77,11 +80,14 @@ def make_inputs(args):
     cfg = dict(synth.WORKLOADS[args.workload], name=args.workload)
     if args.rows:
         cfg["N"] = args.rows
-    if "d_in" in cfg:
-        raise SystemExit("bench.py times stores whose queries arrive at the key dimension")
     keys, toks = synth.make_store(cfg["seed"], cfg["N"], cfg["d"], cfg["C"], cfg["dtype"], cfg["stored_len"])
     nq = N_QUERIES if cfg["B"] == 1 else cfg["B"] * 16
-    q, src = synth.make_queries(cfg["seed"] + 100, keys, cfg["dtype"], nq, cfg["sigma"])
+    if "d_in" in cfg:       # queries arrive at the LLM's hidden width and are projected (Section 3.3)
+        _, _, W = synth.make_preprocess(cfg["proj_seed"], cfg["d_in"], cfg["d"], cfg["dtype"])
+        cfg["W"] = W
+        q = synth.make_hidden_queries(cfg["seed"] + 100, nq, cfg["d_in"], cfg["dtype"], scale=1.0, offset=0.0)
+    else:
+        q, _ = synth.make_queries(cfg["seed"] + 100, keys, cfg["dtype"], nq, cfg["sigma"])
     return cfg, keys, toks, q
 
 
@@ -142,9 +148,10 @@ def time_oracle(cfg, keys, toks, q, n_queries):
     import oracle
     threads = oracle.dresd_oracle.default_threads()
     oracle.build()
-    nq = max(1, n_queries) * cfg["B"]
+    nq = max(1, n_queries)
     t0 = time.perf_counter()
-    r = oracle.retrieve(keys, toks, cfg["dtype"], q[:nq], cfg["top_n"], cfg["draft_len"], threads=threads)
+    r = oracle.retrieve(keys, toks, cfg["dtype"], q[:nq], cfg["top_n"], cfg["draft_len"], W=cfg.get("W"),
+                        threads=threads)
     dt = time.perf_counter() - t0
     return nq / dt, threads, nq, dt, r
 
@@ -197,6 +204,10 @@ def run_ours(args):
     dq = binding.to_device(q, dtype)                       # [nq][d] resident in HBM
     nq = dq.shape[0] // B
     store = binding.Store(dkeys, dtoks, dtype)
+    if "W" in cfg:
+        dW = binding.to_device(cfg["W"], dtype)
+        store.set_preprocess(cfg["d_in"], W=dW)
+    store.set_option("scan_path", args.scan_path)
     out = (torch.empty((B, n), dtype=torch.int32, device="cuda"),
            torch.empty((B, n), dtype=torch.float32, device="cuda"),
            torch.empty((B, n, L), dtype=torch.int32, device="cuda"))
@@ -276,7 +287,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate over %s keys" % dtype,
         "data": "synthetic", "config": workload_config(cfg),
         "e2e": {"value": e2e_qps, "unit": "queries/s",
-                "h2d_bytes_per_step": B * cfg["d"] * eb,
+                "h2d_bytes_per_step": B * cfg.get("d_in", cfg["d"]) * eb,
                 "d2h_bytes_per_step": B * n * (8 + 4 * L) + 4},
         "gpu_launches": launches,
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},

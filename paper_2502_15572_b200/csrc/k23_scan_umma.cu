@@ -4,7 +4,7 @@
 // ridge): tensor cores are used so that the arithmetic of B queries hides
 // under ONE pass over the keys.
 //
-// One persistent CTA per SM, six warps:
+// One persistent CTA per SM, ten warps:
 //   warp 0    producer: one thread streams 128-row x 64-column key slabs
 //             (16 KB, 128-byte swizzle) with TMA through an mbarrier ring and,
 //             when the query operand is too large to stay resident, the
@@ -15,11 +15,12 @@
 //             so that the epilogue of tile t overlaps the MMAs of tile t+1);
 //             tcgen05.commit releases shared-memory stages and publishes
 //             finished accumulators;
-//   warps 2-5 epilogue: each thread owns one key row of the tile, reads its
-//             N accumulator columns with tcgen05.ld, combines hi and lo,
-//             filters against the CTA's running n-th best per query and
-//             queues survivors; queues are folded into sorted 32-lane lists
-//             with shuffle-based bitonic merges.
+//   warps 2-9 epilogue: each thread owns one key row of the tile and half of
+//             its N accumulator columns (two warps share a TMEM lane group),
+//             reads them with tcgen05.ld, combines hi and lo, filters against
+//             the CTA's running n-th best per query and queues survivors;
+//             queues are folded into sorted 32-lane lists with shuffle-based
+//             bitonic merges.
 // Every wait is bounded; TMEM is freed on every path.
 #include <type_traits>
 
@@ -29,8 +30,9 @@
 namespace dresd {
 namespace {
 
-constexpr int kThreads = 6 * 32;
-constexpr int kEpiThreads = 128;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = (2 + kEpiWarps) * 32;
+constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kTileRows = 128;
 constexpr int kSlabBytes = 128;
 constexpr int kSlabElems = 64;
@@ -86,7 +88,31 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
         : "r"(taddr));
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t *r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld16p(uint32_t taddr, uint32_t *r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+}
+// CW consecutive accumulator columns of this thread's TMEM lane -> registers.
+template <int CW> __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[CW])
+{
+    if constexpr (CW == 8) {
+        tmem_ld8(taddr, r);
+    } else {
+#pragma unroll
+        for (int c = 0; c < CW / 16; ++c) tmem_ld16p(taddr + 16 * c, r + 16 * c);
+    }
+}
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 struct EpiFlags {
     int need_merge;
@@ -96,7 +122,7 @@ struct EpiFlags {
 template <typename T, int NCOLS>
 __global__ void __launch_bounds__(kThreads, 1)
 scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_constant__ CUtensorMap q_map,
-                 const ScanArgs a, const int q_resident)
+                 const ScanArgs a, const int q_resident, const int gs)
 {
     constexpr int NQ = NCOLS / 2;                           // queries (padded)
     constexpr int kTmemCols = 2 * NCOLS < 32 ? 32 : 2 * NCOLS;
@@ -104,9 +130,13 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    // A pipeline stage holds a GROUP of `gs` consecutive 64-column slabs of one
+    // 128-row tile (one full/empty barrier pair, one wait and one commit per group).
     const int n_stages = a.stages;
     const int dslabs = (a.d + kSlabElems - 1) / kSlabElems;
-    const int stage_bytes = kKeyStageBytes + (q_resident ? 0 : kQSlabBytes);
+    const int gpt = (dslabs + gs - 1) / gs;                 // groups per tile
+    const int slab_bytes = kKeyStageBytes + (q_resident ? 0 : kQSlabBytes);
+    const int stage_bytes = gs * slab_bytes;
     uint8_t *stages = base;
     uint8_t *qres = stages + (size_t)n_stages * stage_bytes;                 // resident query operand
     WarpTopN *sel = reinterpret_cast<WarpTopN *>(qres + (q_resident ? (size_t)dslabs * kQSlabBytes : 0));
@@ -122,7 +152,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
     const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
-    const int n_it = my_tiles * dslabs;
+    const int n_it = my_tiles * gpt;
 
     if (tid == 0) {
         for (int s = 0; s < n_stages; ++s) {
@@ -131,7 +161,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&tfull[b], 1);
-            mbar_init(&tempty[b], 4);
+            mbar_init(&tempty[b], kEpiWarps);
         }
         mbar_init(qbar, 1);
         for (int i = 0; i < 3; ++i) {
@@ -141,9 +171,9 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         mbar_fence_init();
     }
     if (warp >= 2) {
-        for (int q = warp - 2; q < NQ; q += 4) {
+        for (int q = warp - 2; q < NQ; q += kEpiWarps) {
             warp_topn_init(&sel[q], lane);
-            if (lane == 0) tau[q] = -INFINITY;
+            if (lane == 0) tau[q] = q < a.B ? -INFINITY : INFINITY;     // padding columns never pass
         }
     }
     if (warp == 1) {
@@ -172,14 +202,21 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     report_timeout(a.status);
                     break;
                 }
-                const int tile = cta + (it / dslabs) * G;
-                const int sl = it % dslabs;
+                const int tile = cta + (it / gpt) * G;
+                const int sl0 = (it % gpt) * gs;
+                const int nsl = min(gs, dslabs - sl0);
                 uint8_t *dst = stages + (size_t)s * stage_bytes;
-                mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
-                tma_load_2d(dst, &keys_map, sl * kSlabElems, tile * kTileRows, &full[s]);
-                if (!q_resident) tma_load_2d(dst + kKeyStageBytes, &q_map, sl * kSlabElems, 0, &full[s]);
+                mbar_arrive_expect_tx(&full[s], (uint32_t)(nsl * slab_bytes));
+                for (int j = 0; j < nsl; ++j) {
+                    tma_load_2d(dst + (size_t)j * slab_bytes, &keys_map, (sl0 + j) * kSlabElems,
+                                tile * kTileRows, &full[s]);
+                    if (!q_resident)
+                        tma_load_2d(dst + (size_t)j * slab_bytes + kKeyStageBytes, &q_map,
+                                    (sl0 + j) * kSlabElems, 0, &full[s]);
+                }
                 issued = it + 1;
             }
+            // Do not leave while copies into this CTA's shared memory are in flight.
             for (int it = max(0, issued - n_stages); it < issued; ++it)
                 if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1)) {
                     report_timeout(a.status);
@@ -190,7 +227,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     } else if (warp == 1) {
         // ---------------------------------- MMA issuer ----------------------------------
         if (lane == 0) {
-            constexpr uint32_t kFmt = sizeof(T) == 2 && std::is_same<T, __nv_bfloat16>::value ? 1u : 0u;
+            constexpr uint32_t kFmt = std::is_same<T, __nv_bfloat16>::value ? 1u : 0u;
             constexpr uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(NCOLS >> 3) << 17) |
                                        ((uint32_t)(kTileRows >> 4) << 24);
             bool ok = true;
@@ -200,31 +237,43 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 if (use >= 1 && !mbar_wait(&tempty[acc], (use - 1) & 1)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * NCOLS);
-                for (int sl = 0; sl < dslabs; ++sl) {
-                    const int it = tl * dslabs + sl;
+                for (int g = 0; g < gpt; ++g) {
+                    const int it = tl * gpt + g;
                     const int s = it % n_stages;
                     if (!mbar_wait(&full[s], (it / n_stages) & 1)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(stages + (size_t)s * stage_bytes);
-                    const uint32_t b_addr = q_resident ? smem_u32(qres + (size_t)sl * kQSlabBytes)
-                                                       : a_addr + kKeyStageBytes;
-                    const uint64_t a_desc = make_desc(a_addr), b_desc = make_desc(b_addr);
+                    const int sl0 = g * gs;
+                    const int nsl = min(gs, dslabs - sl0);
+                    const uint32_t st_addr = smem_u32(stages + (size_t)s * stage_bytes);
+                    for (int j = 0; j < nsl; ++j) {
+                        const uint32_t a_addr = st_addr + (uint32_t)(j * slab_bytes);
+                        const uint32_t b_addr = q_resident ? smem_u32(qres + (size_t)(sl0 + j) * kQSlabBytes)
+                                                           : a_addr + kKeyStageBytes;
+                        const uint64_t a_desc = make_desc(a_addr), b_desc = make_desc(b_addr);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)     // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
-                        umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl | k) != 0);
-                    tc_commit(&empty[s]);           // stage reusable once these MMAs have read it
+                        for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
+                            umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
+                    }
+                    tc_commit(&empty[s]);             // group reusable once these MMAs have read it
                 }
                 if (!ok) break;
-                tc_commit(&tfull[acc]);             // accumulator complete
+                tc_commit(&tfull[acc]);               // accumulator complete
             }
             if (!ok) report_timeout(a.status);
         }
     } else {
         // ---------------------------------- epilogue ----------------------------------
-        const int ew = warp - 2;                            // 0..3
-        const int lane_grp = warp & 3;                      // TMEM lanes this warp may read
-        const int et = ew * 32 + lane;                      // 0..127 among epilogue threads
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16);
+        // Eight warps: warp w may read TMEM lanes 32*(w&3)..+31 (one key row per thread);
+        // the two warps that share a lane group split the accumulator columns in halves.
+        constexpr int CW = NCOLS / 2;                       // columns per warp
+        constexpr int QW = CW / 2;                          // queries per warp
+        const int ew = warp - 2;                            // 0..7
+        const int lane_grp = warp & 3;
+        const int half = ew >> 2;
+        const int et = ew * 32 + lane;
+        const int qbase = half * QW;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(half * CW);
+        const float inv = a.lo_inv_scale;
         // A warp whose wait expired goes "dead": it does no more work and no more
         // waits, but keeps taking part in every barrier so that nobody is left behind.
         bool dead = false;
@@ -240,33 +289,37 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             tc_fence_after();
             const long long row = (long long)(cta + tl * G) * kTileRows + lane_grp * 32 + lane;
             const bool row_ok = !dead && row < a.N;
-            unsigned long long pending = 0ull;              // queries whose candidate found the queue full
+            uint32_t pending = 0u;                          // queries whose candidate found the queue full
             bool first = true;
             while (true) {
-#pragma unroll
-                for (int c = 0; c < NCOLS / 16; ++c) {
-                    // warp-uniform decision: tcgen05.ld needs the whole warp
-                    if (dead || (!first && !__any_sync(0xFFFFFFFFu, ((pending >> (c * 8)) & 0xFFull) != 0))) continue;
-                    uint32_t r[16];
-                    tmem_ld16(lane_addr + (uint32_t)(acc * NCOLS + c * 16), r);
+                // warp-uniform decision: tcgen05.ld needs the whole warp
+                if (!dead && (first || __any_sync(0xFFFFFFFFu, pending != 0u))) {
+                    uint32_t r[CW];
+                    tmem_ld_cols<CW>(lane_addr + (uint32_t)(acc * NCOLS), r);
                     tmem_ld_wait();
+                    const uint32_t todo = first ? (row_ok ? 0xFFFFFFFFu : 0u) : pending;
+                    pending = 0u;
+                    if (todo) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int q = c * 8 + j;
-                        const float s = __uint_as_float(r[2 * j]) + __uint_as_float(r[2 * j + 1]) * a.lo_inv_scale;
-                        bool want = first ? (row_ok && q < a.B) : ((pending >> q) & 1ull) != 0;
-                        if (want && s >= tau[q]) {
-                            const int slot = atomicAdd(&sel[q].count, 1);
-                            if (slot < kQueueCap) {
-                                sel[q].queue[slot] = pack_candidate(s, (uint32_t)row);
-                                pending &= ~(1ull << q);
-                                if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
-                            } else {
-                                pending |= 1ull << q;
-                                fl->overflow = 1;
+                        for (int j4 = 0; j4 < QW / 4; ++j4) {
+                            const float4 t = *reinterpret_cast<const float4 *>(tau + qbase + 4 * j4);
+                            const float tt[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int j = 4 * j4 + i;
+                                const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
+                                if (s >= tt[i] && ((todo >> j) & 1u)) {      // rare: a survivor
+                                    const int q = qbase + j;
+                                    const int slot = atomicAdd(&sel[q].count, 1);
+                                    if (slot < kQueueCap) {
+                                        sel[q].queue[slot] = pack_candidate(s, (uint32_t)row);
+                                        if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
+                                    } else {
+                                        pending |= 1u << j;
+                                        fl->overflow = 1;
+                                    }
+                                }
                             }
-                        } else {
-                            pending &= ~(1ull << q);
                         }
                     }
                 }
@@ -283,10 +336,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 round += 1;
                 fl = &flags[round % 3];
                 if (!(need | over)) break;
-                for (int q = ew; q < NQ; q += 4) {
+                for (int q = ew; q < NQ; q += kEpiWarps) {
                     if (sel[q].count > 0) {
                         warp_topn_merge(&sel[q], a.top_n, lane);
-                        if (lane == 0) tau[q] = sel[q].tau;
+                        if (lane == 0 && q < a.B) tau[q] = sel[q].tau;
                     }
                 }
                 epi_bar();                                   // C: lists, counts and tau are settled
@@ -298,7 +351,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         }
         // flush and publish this CTA's lists
         epi_bar();
-        for (int q = ew; q < NQ; q += 4) {
+        for (int q = ew; q < NQ; q += kEpiWarps) {
             if (sel[q].count > 0) warp_topn_merge(&sel[q], a.top_n, lane);
             if (q < a.B) {
                 unsigned long long m = sel[q].list[lane];
@@ -316,7 +369,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
 }
 
 struct Plan {
-    int ncols, stages, q_resident;
+    int ncols, stages, q_resident, gs;
     size_t smem;
 };
 
@@ -329,10 +382,18 @@ Plan make_plan(int d, int B)
     p.q_resident = qbytes <= (size_t)kResidentLimit;
     const size_t fixed = 1024 + (p.q_resident ? qbytes : 0) + sizeof(WarpTopN) * (p.ncols / 2) +
                          sizeof(float) * (p.ncols / 2) + sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
-    const size_t stage = kKeyStageBytes + (p.q_resident ? 0 : (size_t)p.ncols * kSlabBytes);
-    long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)stage;
-    p.stages = (int)(s > kMaxStages ? kMaxStages : s);
-    p.smem = fixed + (size_t)(p.stages > 0 ? p.stages : 0) * stage;
+    const size_t slab = kKeyStageBytes + (p.q_resident ? 0 : (size_t)p.ncols * kSlabBytes);
+    // Largest slab group (fewest barrier round trips per tile) that still leaves
+    // at least three groups in flight.
+    for (int gs = 4; gs >= 1; gs >>= 1) {
+        if (gs > dslabs && gs > 1) continue;
+        long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)(gs * slab);
+        if (s > kMaxStages) s = kMaxStages;
+        p.gs = gs;
+        p.stages = (int)s;
+        if (s >= 3) break;
+    }
+    p.smem = fixed + (size_t)(p.stages > 0 ? p.stages : 0) * p.gs * slab;
     return p;
 }
 
@@ -343,7 +404,7 @@ cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const S
     auto kernel = scan_umma_kernel<T, NCOLS>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
     if (e != cudaSuccess) return e;
-    kernel<<<grid, kThreads, p.smem, stream>>>(kmap, qmap, a, p.q_resident);
+    kernel<<<grid, kThreads, p.smem, stream>>>(kmap, qmap, a, p.q_resident, p.gs);
     return cudaGetLastError();
 }
 
