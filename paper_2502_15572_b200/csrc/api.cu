@@ -105,6 +105,7 @@ struct dresd_store {
     void *qsplit;                // [2*kMaxBatch][dpad] 16-bit
     unsigned long long *cand;    // [max_grid][kMaxBatch][kCandStride]
     int *status;                 // device status word
+    unsigned int *gtau;          // [kMaxBatch] grid-wide filter words
     int max_grid;
     // staging for dresd_retrieve_host (owned, device)
     void *q_stage;
@@ -140,6 +141,7 @@ void free_store(dresd_store *s)
     cudaFree(s->qsplit);
     cudaFree(s->cand);
     cudaFree(s->status);
+    cudaFree(s->gtau);
     cudaFree(s->q_stage);
     cudaFree(s->ids_dev);
     cudaFree(s->scores_dev);
@@ -189,6 +191,7 @@ dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows
     p.dpad = s->dpad;
     p.rows = rows;                   // operand rows beyond B are written as zeros
     p.lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
+    p.gtau = s->gtau;
     cudaError_t e = launch_preprocess(p, stream);
     if (e != cudaSuccess) return fail_cuda(e, "preprocess launch");
     s->last_launches += 1;
@@ -230,6 +233,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.cand = s->cand;
         a.cand_batch = B;
         a.status = s->status;
+        a.gtau = s->gtau;
         const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
         cudaError_t e = launch_scan_umma(s->map_umma, s->map_q[mi], a, grid, stream);
         if (e != cudaSuccess) return fail_cuda(e, "scan launch");
@@ -251,6 +255,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.cand = s->cand + (size_t)q0 * kCandStride;
         a.cand_batch = B;
         a.status = s->status;
+        a.gtau = s->gtau + q0;
         cudaError_t e = f32 ? launch_scan_f32(s->map_stream, a, grid, stream)
                             : launch_scan_mma(s->map_stream, a, grid, stream);
         if (e != cudaSuccess) return fail_cuda(e, "scan launch");
@@ -327,6 +332,7 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
               cudaMalloc(&s->qsplit, (size_t)2 * 2 * kMaxBatch * s->dpad) == cudaSuccess &&
               cudaMalloc(&s->cand, sizeof(unsigned long long) * (size_t)s->max_grid * kMaxBatch * kCandStride) == cudaSuccess &&
               cudaMalloc(&s->status, sizeof(int)) == cudaSuccess &&
+              cudaMalloc(&s->gtau, sizeof(unsigned int) * kMaxBatch) == cudaSuccess &&
               cudaMalloc(&s->ids_dev, sizeof(int32_t) * kMaxBatch * kMaxTopN) == cudaSuccess &&
               cudaMalloc(&s->scores_dev, sizeof(float) * kMaxBatch * kMaxTopN) == cudaSuccess;
     s->tokens_dev_elems = (size_t)kMaxBatch * kMaxTopN * stored_len;

@@ -25,18 +25,45 @@ constexpr long long kWaitCycles = 4000000000LL;  // ~2-3 s at B200 clocks
 // ---------------------------------------------------------------------------
 // (score, id) <-> orderable u64.  0 is "empty" and sorts below every candidate.
 // ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t float_to_ordered(float f)      // monotone float -> uint, never 0
+{
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float ordered_to_float(uint32_t u)
+{
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u);
+}
 __device__ __forceinline__ unsigned long long pack_candidate(float score, uint32_t id)
 {
     score += 0.0f;                                   // -0.0 -> +0.0: one zero
-    uint32_t u = __float_as_uint(score);
-    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // monotone float -> uint
-    return (static_cast<unsigned long long>(u) << 32) | (0xFFFFFFFFu - id);
+    return (static_cast<unsigned long long>(float_to_ordered(score)) << 32) | (0xFFFFFFFFu - id);
 }
 __device__ __forceinline__ float candidate_score(unsigned long long p)
 {
-    uint32_t u = static_cast<uint32_t>(p >> 32);
-    u = (u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u;
-    return __uint_as_float(u);
+    return ordered_to_float(static_cast<uint32_t>(p >> 32));
+}
+
+// Grid-wide filter: every CTA's n-th best score is a lower bound of the final n-th
+// best, so the maximum over CTAs (kept per query in global memory, ordered-uint
+// encoded, 0 = nothing known) may be used by all of them to reject rows early.
+// The filter only rejects rows that cannot be in the result, so the result does not
+// depend on when a CTA sees an update.
+__device__ __forceinline__ float share_tau(unsigned int *gtau, float local)
+{
+    if (!(local > -INFINITY)) {
+        const unsigned int g = *reinterpret_cast<volatile unsigned int *>(gtau);
+        return g ? ordered_to_float(g) : local;
+    }
+    const unsigned int mine = float_to_ordered(local);
+    const unsigned int old = atomicMax(gtau, mine);
+    return old > mine ? ordered_to_float(old) : local;
+}
+__device__ __forceinline__ float peek_tau(const unsigned int *gtau, float current)
+{
+    const unsigned int g = *reinterpret_cast<const volatile unsigned int *>(gtau);
+    const float t = g ? ordered_to_float(g) : -INFINITY;
+    return t > current ? t : current;
 }
 __device__ __forceinline__ uint32_t candidate_id(unsigned long long p)
 {

@@ -29,6 +29,7 @@ struct PreprocessArgs {
     int dpad;               // d rounded up to 64
     int rows;               // CTAs launched: B rounded up to the operand row count
     float lo_scale;
+    unsigned int *gtau;     // [rows] grid-wide filter words, reset to 0 ("nothing known") here
 };
 cudaError_t launch_preprocess(const PreprocessArgs &a, cudaStream_t stream);
 
@@ -47,6 +48,7 @@ struct ScanArgs {
     unsigned long long *cand;  // [grid][cand_batch][kCandStride], at this launch's first query
     int cand_batch;         // query stride of `cand` (the call's B)
     int *status;            // device status word
+    unsigned int *gtau;     // grid-wide filter words of this launch's queries (see share_tau)
     int stages;             // pipeline depth
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.

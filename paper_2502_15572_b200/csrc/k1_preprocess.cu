@@ -58,6 +58,7 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
     T *split_hi = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)(2 * b) * a.dpad : nullptr;
     T *split_lo = split_hi ? split_hi + a.dpad : nullptr;
     float *qrow = a.qhat + (size_t)b * a.d;
+    if (tid == 0 && a.gtau) a.gtau[b] = 0u;          // fresh grid-wide filter for this call
 
     if (b >= a.B) {                       // padding rows of the operand: zeros
         for (int c = tid; c < a.d; c += blockDim.x) qrow[c] = 0.f;

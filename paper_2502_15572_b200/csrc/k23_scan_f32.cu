@@ -140,9 +140,14 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 any |= take[q];
             }
             if (__any_sync(0xFFFFFFFFu, any)) {
+                // Rare path: pull the grid-wide filter, re-test, queue, publish ours.
+                if (lane < QB && lane < a.B) my_sel[lane].tau = peek_tau(&a.gtau[lane], my_sel[lane].tau);
+                __syncwarp();
 #pragma unroll
                 for (int q = 0; q < QB; ++q)
-                    warp_topn_push(&my_sel[q], a.top_n, lane, take[q], sc[q], (uint32_t)row);
+                    warp_topn_push(&my_sel[q], a.top_n, lane, take[q] && sc[q] >= my_sel[q].tau, sc[q], (uint32_t)row);
+                if (lane < QB && lane < a.B) my_sel[lane].tau = share_tau(&a.gtau[lane], my_sel[lane].tau);
+                __syncwarp();
             }
         }
         for (int q = 0; q < QB; ++q)

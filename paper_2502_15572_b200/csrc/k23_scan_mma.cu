@@ -261,6 +261,16 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                     any |= pa[grp] | pb[grp];
                 }
                 if (__any_sync(0xFFFFFFFFu, any)) {
+                    // Rare path.  First pull the grid-wide filter (other CTAs may know a
+                    // better n-th best), re-test, queue what survives, publish our filter.
+                    if (lane < NQ && lane < a.B) my_sel[lane].tau = peek_tau(&a.gtau[lane], my_sel[lane].tau);
+                    __syncwarp();
+#pragma unroll
+                    for (int grp = 0; grp < NG; ++grp) {
+                        const float tau = my_sel[grp * 4 + t].tau;
+                        pa[grp] = pa[grp] && sa[grp] >= tau;
+                        pb[grp] = pb[grp] && sb[grp] >= tau;
+                    }
 #pragma unroll
                     for (int grp = 0; grp < NG; ++grp)
 #pragma unroll
@@ -269,6 +279,8 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                             warp_topn_push(sq, a.top_n, lane, pa[grp] && t == tq, sa[grp], (uint32_t)row_a);
                             warp_topn_push(sq, a.top_n, lane, pb[grp] && t == tq, sb[grp], (uint32_t)row_b);
                         }
+                    if (lane < NQ && lane < a.B) my_sel[lane].tau = share_tau(&a.gtau[lane], my_sel[lane].tau);
+                    __syncwarp();
                 }
             }
         }

@@ -287,6 +287,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             }
             dead = __any_sync(0xFFFFFFFFu, dead);
             tc_fence_after();
+            // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
+            if ((tl & 3) == 0 && et < a.B) tau[et] = peek_tau(&a.gtau[et], tau[et]);
             const long long row = (long long)(cta + tl * G) * kTileRows + lane_grp * 32 + lane;
             const bool row_ok = !dead && row < a.N;
             uint32_t pending = 0u;                          // queries whose candidate found the queue full
@@ -339,7 +341,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 for (int q = ew; q < NQ; q += kEpiWarps) {
                     if (sel[q].count > 0) {
                         warp_topn_merge(&sel[q], a.top_n, lane);
-                        if (lane == 0 && q < a.B) tau[q] = sel[q].tau;
+                        if (lane == 0 && q < a.B) tau[q] = share_tau(&a.gtau[q], sel[q].tau);
                     }
                 }
                 epi_bar();                                   // C: lists, counts and tau are settled

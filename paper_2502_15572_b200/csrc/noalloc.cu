@@ -139,6 +139,7 @@ extern "C" dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     int *status = reinterpret_cast<int *>(scratch + kOffStatus);
+    unsigned int *gtau = reinterpret_cast<unsigned int *>(scratch + kOffStatus + 128);   // 8 words
     float *qhat = reinterpret_cast<float *>(scratch + kOffQhat);
     void *qsplit = scratch + kOffQsplit;
     unsigned long long *cand = reinterpret_cast<unsigned long long *>(scratch + kOffCand);
@@ -170,6 +171,7 @@ extern "C" dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *
     p.dpad = dpad;
     p.rows = kNaMaxBatch;
     p.lo_scale = lo_scale;
+    p.gtau = gtau;
     if (launch_preprocess(p, stream) != cudaSuccess) return na_fail(DRESD_ERR_CUDA, "preprocess launch failed");
 
     int grid = sms < kNaMaxGrid ? sms : kNaMaxGrid;
@@ -190,6 +192,7 @@ extern "C" dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *
         a.cand = cand + (size_t)q0 * kCandStride;
         a.cand_batch = B;
         a.status = status;
+        a.gtau = gtau + q0;
         cudaError_t e = f32 ? launch_scan_f32(map, a, grid, stream) : launch_scan_mma(map, a, grid, stream);
         if (e != cudaSuccess) return na_fail(DRESD_ERR_CUDA, "scan launch failed");
     }
