@@ -136,6 +136,9 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "scan_path"  0 = automatic, 1 = CUDA-core/mma.sync streaming kernel,
  *                2 = tcgen05 tensor-core kernel (16-bit keys only).
  *   "grid"       CTAs of the scoring kernel, 0 = one per SM.
+ *   "probe"      large batches on large stores first run a probe pass over every
+ *                value-th key tile to seed the selection filter; 0 = never,
+ *                1 = default stride (256).
  *   "profile"    > 0: record a CUDA-event pair around the scoring kernel(s) of
  *                each of the next `value` dresd_retrieve() calls (see
  *                dresd_store_profile_read); 0 = off (default).
@@ -153,6 +156,10 @@ dresd_status dresd_store_profile_read(dresd_store *store, double *scan_ms_total,
 
 /* Number of kernels dresd_retrieve() enqueued in the store's last call. */
 int dresd_store_last_launches(const dresd_store *store);
+
+/* Passes over the key matrix made by the store's last dresd_retrieve(): 1 per scoring
+ * launch over all keys, plus 1/stride when the probe pass ran. */
+double dresd_store_last_key_passes(const dresd_store *store);
 
 /* Message of the calling thread's last failing call ("" if none). */
 const char *dresd_last_error(void);

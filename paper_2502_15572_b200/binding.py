@@ -25,7 +25,8 @@ MAX_BATCH, MAX_TOP_N, MAX_DIM = 64, 32, 4096
 EXPORTS = (
     "dresd_store_create", "dresd_store_set_preprocess", "dresd_retrieve", "dresd_retrieve_host",
     "dresd_preprocess", "dresd_store_status", "dresd_store_set_option",
-    "dresd_store_profile_read", "dresd_store_last_launches", "dresd_last_error",
+    "dresd_store_profile_read", "dresd_store_last_launches", "dresd_store_last_key_passes",
+    "dresd_last_error",
     "dresd_store_destroy", "dresd_retrieve_noalloc",
 )
 
@@ -70,6 +71,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_store_profile_read.argtypes = [vp, c.POINTER(c.c_double), c.POINTER(c.c_int)]
     lib.dresd_store_last_launches.restype = i32
     lib.dresd_store_last_launches.argtypes = [vp]
+    lib.dresd_store_last_key_passes.restype = c.c_double
+    lib.dresd_store_last_key_passes.argtypes = [vp]
     lib.dresd_last_error.restype = c.c_char_p
     lib.dresd_last_error.argtypes = []
     lib.dresd_store_destroy.restype = None
@@ -136,6 +139,10 @@ def dresd_store_profile_read(store: int):
 
 def dresd_store_last_launches(store: int) -> int:
     return int(load().dresd_store_last_launches(store))
+
+
+def dresd_store_last_key_passes(store: int) -> float:
+    return float(load().dresd_store_last_key_passes(store))
 
 
 def dresd_store_destroy(store: int) -> None:
@@ -241,6 +248,9 @@ class Store:
 
     def profile_read(self):
         return dresd_store_profile_read(self.handle)
+
+    def last_key_passes(self) -> float:
+        return dresd_store_last_key_passes(self.handle)
 
     def last_launches(self) -> int:
         return dresd_store_last_launches(self.handle)

@@ -29,6 +29,7 @@ dresd_status fail_cuda(cudaError_t e, const char *what)
 }
 
 constexpr uint32_t kMagic = 0xD2E5D001u;
+constexpr int kProbeStride = 256;    // default: the probe pass visits every 256th tile
 constexpr float kEpsNorm = 1e-12f;   // epsilon of Eq. 2 (the paper leaves it open)
 
 bool is_device_ptr(const void *p)
@@ -122,7 +123,8 @@ struct dresd_store {
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     int n_tiles_umma;
     // options / bookkeeping
-    int opt_path, opt_grid;
+    int opt_path, opt_grid, opt_probe;
+    double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
     cudaStream_t last_stream;
     int last_launches;
     // optional timing of the scoring kernel (option "profile")
@@ -203,6 +205,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
 {
     s->last_stream = stream;
     s->last_launches = 0;
+    s->last_key_passes = 0.0;
     const bool f32 = s->dtype == kF32;
     // 16-bit keys: the streaming mma.sync kernel serves up to 8 queries per pass over
     // the keys; beyond that the tcgen05 kernel serves all of them in one pass.
@@ -235,9 +238,27 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.status = s->status;
         a.gtau = s->gtau;
         const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
-        cudaError_t e = launch_scan_umma(s->map_umma, s->map_q[mi], a, grid, stream);
+        cudaError_t e = cudaSuccess;
+        // Large batches on large stores: a probe pass over every 64th tile first.  Its
+        // n-th best score per query seeds the grid-wide filter, so that the full pass
+        // queues ~64 n survivors per query GPU-wide instead of ~n ln(rows/n) per CTA.
+        // The filter only rejects rows that cannot be in the result.
+        const int pstride = s->opt_probe;
+        if (pstride > 1 && B * top_n >= 256 && n_tiles >= pstride * grid) {
+            ScanArgs pa = a;
+            pa.tile_stride = pstride;
+            pa.n_tiles = (n_tiles + pstride - 1) / pstride;
+            int pgrid = grid < pa.n_tiles ? grid : pa.n_tiles;
+            e = launch_scan_umma(s->map_umma, s->map_q[mi], pa, pgrid, stream);
+            if (e == cudaSuccess) e = launch_merge_tau(s->cand, pgrid, B, top_n, s->gtau, stream);
+            if (e != cudaSuccess) return fail_cuda(e, "probe launch");
+            s->last_launches += 2;
+            s->last_key_passes += 1.0 / pstride;
+        }
+        e = launch_scan_umma(s->map_umma, s->map_q[mi], a, grid, stream);
         if (e != cudaSuccess) return fail_cuda(e, "scan launch");
         s->last_launches += 1;
+        s->last_key_passes += 1.0;
     }
     for (int q0 = 0; q0 < B && !umma; q0 += qpl) {
         ScanArgs a{};
@@ -260,6 +281,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
                             : launch_scan_mma(s->map_stream, a, grid, stream);
         if (e != cudaSuccess) return fail_cuda(e, "scan launch");
         s->last_launches += 1;
+        s->last_key_passes += 1.0;
     }
     if (prof) {
         cudaEventRecord(s->prof_events[2 * s->prof_count + 1], stream);
@@ -320,6 +342,7 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
     s->d_in = d;
     s->eps_z = 1e-5f;
     s->max_grid = 2 * s->num_sms;
+    s->opt_probe = kProbeStride;
 
     s->tile_rows = dtype == DRESD_F32 ? scan_f32_tile_rows(d) : scan_mma_tile_rows(d);
     s->n_tiles = (int)((N + s->tile_rows - 1) / s->tile_rows);
@@ -474,6 +497,11 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
         s->opt_path = value;
         return DRESD_OK;
     }
+    if (strcmp(name, "probe") == 0) {
+        if (value < 0 || value > 65536) return fail(DRESD_ERR_INVALID, "probe = %d outside 0..65536", value);
+        s->opt_probe = value == 1 ? kProbeStride : value;
+        return DRESD_OK;
+    }
     if (strcmp(name, "grid") == 0) {
         if (value < 0 || value > s->max_grid) return fail(DRESD_ERR_INVALID, "grid = %d outside 0..%d", value, s->max_grid);
         s->opt_grid = value;
@@ -521,6 +549,8 @@ dresd_status dresd_store_profile_read(dresd_store *s, double *scan_ms_total, int
 }
 
 int dresd_store_last_launches(const dresd_store *s) { return valid(s) ? s->last_launches : 0; }
+
+double dresd_store_last_key_passes(const dresd_store *s) { return valid(s) ? s->last_key_passes : 0.0; }
 
 const char *dresd_last_error(void) { return g_err; }
 

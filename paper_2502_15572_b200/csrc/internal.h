@@ -50,6 +50,7 @@ struct ScanArgs {
     int *status;            // device status word
     unsigned int *gtau;     // grid-wide filter words of this launch's queries (see share_tau)
     int stages;             // pipeline depth
+    int tile_stride;        // tcgen05 kernel: visit every tile_stride-th tile (probe pass), default 1
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.
 int scan_mma_tile_rows(int d);
@@ -73,6 +74,10 @@ cudaError_t launch_scan_f32(const CUtensorMap &keys_map, const ScanArgs &a, int 
 // ---- K4: merge the per-CTA lists;  K5: gather continuations ----------------
 cudaError_t launch_merge(const unsigned long long *cand, int grid_lists, int B, int top_n,
                          int32_t *out_ids, float *out_scores, cudaStream_t stream);
+// Same merge, but only the n-th best score of each query is kept, as a grid-wide
+// filter word (see share_tau); 0 when fewer than top_n candidates exist.
+cudaError_t launch_merge_tau(const unsigned long long *cand, int grid_lists, int B, int top_n,
+                             unsigned int *gtau, cudaStream_t stream);
 cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long N,
                           const int32_t *ids, int B, int top_n, int draft_len,
                           int32_t *out_tokens, cudaStream_t stream);

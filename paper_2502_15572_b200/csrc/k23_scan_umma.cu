@@ -102,6 +102,10 @@ __device__ __forceinline__ void tmem_ld16p(uint32_t taddr, uint32_t *r)
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
 }
+__device__ __forceinline__ void tmem_ld2(uint32_t taddr, uint32_t &v0, uint32_t &v1)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(v0), "=r"(v1) : "r"(taddr));
+}
 // CW consecutive accumulator columns of this thread's TMEM lane -> registers.
 template <int CW> __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[CW])
 {
@@ -173,7 +177,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     if (warp >= 2) {
         for (int q = warp - 2; q < NQ; q += kEpiWarps) {
             warp_topn_init(&sel[q], lane);
-            if (lane == 0) tau[q] = q < a.B ? -INFINITY : INFINITY;     // padding columns never pass
+            // start from whatever the grid already knows; padding columns never pass
+            if (lane == 0) tau[q] = q < a.B ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
         }
     }
     if (warp == 1) {
@@ -202,7 +207,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     report_timeout(a.status);
                     break;
                 }
-                const int tile = cta + (it / gpt) * G;
+                const int tile = (cta + (it / gpt) * G) * a.tile_stride;
                 const int sl0 = (it % gpt) * gs;
                 const int nsl = min(gs, dslabs - sl0);
                 uint8_t *dst = stages + (size_t)s * stage_bytes;
@@ -274,6 +279,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         const int qbase = half * QW;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(half * CW);
         const float inv = a.lo_inv_scale;
+        const float4 *tau4 = reinterpret_cast<const float4 *>(tau + qbase);
         // A warp whose wait expired goes "dead": it does no more work and no more
         // waits, but keeps taking part in every barrier so that nobody is left behind.
         bool dead = false;
@@ -289,7 +295,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             tc_fence_after();
             // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
             if ((tl & 3) == 0 && et < a.B) tau[et] = peek_tau(&a.gtau[et], tau[et]);
-            const long long row = (long long)(cta + tl * G) * kTileRows + lane_grp * 32 + lane;
+            const long long row =
+                (long long)(cta + tl * G) * a.tile_stride * kTileRows + lane_grp * 32 + lane;
             const bool row_ok = !dead && row < a.N;
             uint32_t pending = 0u;                          // queries whose candidate found the queue full
             bool first = true;
@@ -299,28 +306,42 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     uint32_t r[CW];
                     tmem_ld_cols<CW>(lane_addr + (uint32_t)(acc * NCOLS), r);
                     tmem_ld_wait();
-                    const uint32_t todo = first ? (row_ok ? 0xFFFFFFFFu : 0u) : pending;
+                    // Hot part, branch-free and compact: one bit per query whose score
+                    // reaches the filter.
+                    uint32_t mask = 0u;
+#pragma unroll
+                    for (int j4 = 0; j4 < QW / 4; ++j4) {
+                        const float4 t = tau4[j4];
+                        const float tt[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int j = 4 * j4 + i;
+                            const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
+                            mask |= (s >= tt[i]) ? (1u << j) : 0u;
+                        }
+                    }
+                    mask &= first ? (row_ok ? 0xFFFFFFFFu : 0u) : pending;
                     pending = 0u;
-                    if (todo) {
-#pragma unroll
-                        for (int j4 = 0; j4 < QW / 4; ++j4) {
-                            const float4 t = *reinterpret_cast<const float4 *>(tau + qbase + 4 * j4);
-                            const float tt[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int j = 4 * j4 + i;
-                                const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
-                                if (s >= tt[i] && ((todo >> j) & 1u)) {      // rare: a survivor
-                                    const int q = qbase + j;
-                                    const int slot = atomicAdd(&sel[q].count, 1);
-                                    if (slot < kQueueCap) {
-                                        sel[q].queue[slot] = pack_candidate(s, (uint32_t)row);
-                                        if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
-                                    } else {
-                                        pending |= 1u << j;
-                                        fl->overflow = 1;
-                                    }
-                                }
+                    // Cold part (rare once the filter is warm), kept out of the hot code:
+                    // a warp-uniform loop over the queries that have a survivor in some
+                    // lane; the two accumulator columns are re-read from TMEM.
+                    uint32_t wm = __reduce_or_sync(0xFFFFFFFFu, mask);
+                    while (wm) {
+                        const int j = __ffs(wm) - 1;
+                        wm &= wm - 1;
+                        uint32_t v0, v1;
+                        tmem_ld2(lane_addr + (uint32_t)(acc * NCOLS + 2 * j), v0, v1);
+                        tmem_ld_wait();
+                        if ((mask >> j) & 1u) {
+                            const float s = fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
+                            const int q = qbase + j;
+                            const int slot = atomicAdd(&sel[q].count, 1);
+                            if (slot < kQueueCap) {
+                                sel[q].queue[slot] = pack_candidate(s, (uint32_t)row);
+                                if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
+                            } else {
+                                pending |= 1u << j;
+                                fl->overflow = 1;
                             }
                         }
                     }
@@ -419,6 +440,7 @@ cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, c
                              cudaStream_t stream)
 {
     ScanArgs a = a_in;
+    if (a.tile_stride < 1) a.tile_stride = 1;
     const Plan p = make_plan(a.d, a.B);
     if (p.stages < 2) return cudaErrorInvalidValue;
     a.stages = p.stages;

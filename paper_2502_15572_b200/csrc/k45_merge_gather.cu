@@ -13,7 +13,7 @@ constexpr int kMergeWarps = 8;
 
 __global__ void __launch_bounds__(kMergeWarps * 32)
 merge_kernel(const unsigned long long *__restrict__ cand, int lists, int B, int top_n,
-             int32_t *__restrict__ out_ids, float *__restrict__ out_scores)
+             int32_t *__restrict__ out_ids, float *__restrict__ out_scores, unsigned int *__restrict__ gtau)
 {
     __shared__ unsigned long long part[kMergeWarps][kListLen];
     const int b = blockIdx.x;
@@ -39,7 +39,9 @@ merge_kernel(const unsigned long long *__restrict__ cand, int lists, int B, int 
     if (warp == 0) {
         m = part[0][lane];
         for (int w = 1; w < kMergeWarps; ++w) m = warp_merge_top32(m, part[w][lane], lane);
-        if (lane < top_n) {
+        if (gtau) {                       // probe pass: publish the n-th best as the filter
+            if (lane == top_n - 1) gtau[b] = m ? float_to_ordered(candidate_score(m)) : 0u;
+        } else if (lane < top_n) {
             out_ids[(size_t)b * top_n + lane] = m ? (int32_t)candidate_id(m) : -1;
             out_scores[(size_t)b * top_n + lane] = m ? candidate_score(m) : -INFINITY;
         }
@@ -65,7 +67,14 @@ __global__ void gather_kernel(const int32_t *__restrict__ next_tokens, int store
 cudaError_t launch_merge(const unsigned long long *cand, int lists, int B, int top_n,
                          int32_t *out_ids, float *out_scores, cudaStream_t stream)
 {
-    merge_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, out_ids, out_scores);
+    merge_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, out_ids, out_scores, nullptr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_merge_tau(const unsigned long long *cand, int lists, int B, int top_n, unsigned int *gtau,
+                             cudaStream_t stream)
+{
+    merge_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, nullptr, nullptr, gtau);
     return cudaGetLastError();
 }
 

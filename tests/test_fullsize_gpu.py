@@ -1,0 +1,94 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle needs several seconds per query on a 10M-row datastore, so full-size
+runs are checked on a SAMPLE of the queries element by element (the same checker
+as the small cases), and on ALL queries via properties that hold at any size:
+ids distinct and in range, scores non-increasing, tokens equal to the stored
+continuation of the returned id, and every returned score equal to the oracle's
+score of that row (computed row by row for the returned ids only).
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2502_15572_b200 import binding, synth
+from tests import checker
+from tests.gpu_util import gpu_store
+
+pytestmark = pytest.mark.gpu
+
+
+def _row_scores(keys, dtype, qhat, ids):
+    """Oracle scores of selected rows only (float64, exact decode)."""
+    return oracle.scores(keys[ids], dtype, qhat)
+
+
+def _properties(keys, toks, dtype, q, ids, sc, tok, n, L):
+    N = keys.shape[0]
+    tol = checker.TOL[dtype]
+    qh = oracle.preprocess(q, dtype)
+    for b in range(q.shape[0]):
+        assert np.all((ids[b] >= 0) & (ids[b] < N)) and len(set(ids[b].tolist())) == n
+        assert np.all(np.diff(sc[b]) <= 0)
+        assert np.array_equal(tok[b], toks[ids[b]][:, :L])
+        want = _row_scores(keys, dtype, qh[b], ids[b])
+        assert np.max(np.abs(want - sc[b])) <= tol
+
+
+def _sampled_parity(w, sample, q=None):
+    import torch
+    keys, toks, dtype = w["keys"], w["next_tokens"], w["dtype"]
+    n, L, B = w["top_n"], w["draft_len"], w["B"]
+    q = w["queries"] if q is None else q
+    st = gpu_store(keys, toks, dtype)
+    dq = binding.to_device(q, dtype)
+    outs = []
+    for j in range(0, q.shape[0], B):                      # batches exactly as bench.py issues them
+        ids, sc, tok = st.retrieve(dq[j:j + B], n, L)
+        outs.append((ids.cpu().numpy(), sc.cpu().numpy(), tok.cpu().numpy()))
+    torch.cuda.synchronize()
+    st.status()
+    st.close()
+    ids = np.concatenate([o[0] for o in outs])
+    sc = np.concatenate([o[1] for o in outs])
+    tok = np.concatenate([o[2] for o in outs])
+    _properties(keys, toks, dtype, q, ids, sc, tok, n, L)
+    o = oracle.retrieve(keys, toks, dtype, q[sample], n, L, want_full_scores=True,
+                        threads=oracle.dresd_oracle.default_threads())
+    rate = checker.check_batch(o.full_scores, toks, ids[sample], sc[sample], tok[sample], dtype, n, L,
+                               oracle_ids=o.ids)
+    return rate
+
+
+def test_config2_decode_batch1_full_size():
+    """10M x 256 fp16, single queries: 64 calls checked by properties, 3 against the oracle."""
+    w = synth.make_workload("c2_decode_b1_f16")
+    q, _ = synth.make_queries(w["seed"] + 100, w["keys"], "f16", 64, w["sigma"])
+    rate = _sampled_parity(w, sample=[0, 17, 63], q=q)
+    assert rate >= 0.9
+
+
+def test_config3_batched_full_size():
+    """10M x 256 bf16, one batch of 64 (tensor-core kernel with its probe pass): 3 queries against the oracle."""
+    w = synth.make_workload("c3_batched_bf16")
+    rate = _sampled_parity(w, sample=[0, 31, 63])
+    assert rate >= 0.9
+
+
+def test_config5b_projected_full_size():
+    """4M x 256 bf16 with the 4096 -> 256 projection, batch 16: all 16 queries against the oracle."""
+    import torch
+    w = synth.make_workload("c5b_projected_bf16")
+    keys, toks, dtype, n, L = w["keys"], w["next_tokens"], w["dtype"], w["top_n"], w["draft_len"]
+    st = gpu_store(keys, toks, dtype)
+    dW = binding.to_device(w["W"], dtype)
+    st.set_preprocess(w["d_in"], W=dW)
+    ids, sc, tok = st.retrieve(binding.to_device(w["queries"], dtype), n, L)
+    torch.cuda.synchronize()
+    st.status()
+    ids, sc, tok = ids.cpu().numpy(), sc.cpu().numpy(), tok.cpu().numpy()
+    st.close()
+    o = oracle.retrieve(keys, toks, dtype, w["queries"], n, L, W=w["W"], want_full_scores=True,
+                        threads=oracle.dresd_oracle.default_threads())
+    rate = checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids)
+    assert rate >= 0.9
