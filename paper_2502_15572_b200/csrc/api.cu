@@ -207,9 +207,11 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     s->last_launches = 0;
     s->last_key_passes = 0.0;
     const bool f32 = s->dtype == kF32;
-    // 16-bit keys: the streaming mma.sync kernel serves up to 8 queries per pass over
-    // the keys; beyond that the tcgen05 kernel serves all of them in one pass.
-    const bool umma = !f32 && (s->opt_path == 2 || (s->opt_path == 0 && B > 8));
+    // 16-bit keys: the tcgen05 kernel serves any batch in one pass over the keys and is
+    // also the fastest for rows of at least four 64-element slabs (7.1 vs 6.8 TB/s at
+    // d = 256); for narrow rows and up to 8 queries the streaming mma.sync kernel wins
+    // (6.8 vs 6.0 TB/s at d = 128) because its per-tile cost is lower.
+    const bool umma = !f32 && (s->opt_path == 2 || (s->opt_path == 0 && (B > 8 || s->d > 192)));
     const int op_rows = umma ? scan_umma_operand_rows(B) : 0;
     dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream);
     if (st != DRESD_OK) return st;
