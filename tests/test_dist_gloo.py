@@ -1,0 +1,63 @@
+"""World-size-2 checks of the multi-GPU plumbing on CPU (gloo): the path shards by
+query stream with no data-path collective, so what is covered is the partition of
+the stream and the barrier / max-over-ranks timing protocol of the benchmark."""
+import os
+import socket
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2502_15572_b200 import dist_util
+
+
+def test_query_slices_partition_the_stream():
+    for n in (0, 1, 7, 1000, 1001):
+        for world in (1, 2, 3, 8):
+            seen = []
+            for r in range(world):
+                sl = dist_util.query_slice(n, r, world)
+                seen.extend(sl)
+                assert abs(len(sl) - n / world) < 1
+            assert seen == list(range(n))
+    with pytest.raises(ValueError):
+        dist_util.query_slice(10, 2, 2)
+
+
+def test_aggregate_throughput():
+    assert dist_util.aggregate_throughput(1, 1000, 1, 800.0) == pytest.approx(1250.0)
+    assert dist_util.aggregate_throughput(64, 100, 8, 100.0) == pytest.approx(512000.0)
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      LOCAL_RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        assert dist_util.rank_info() == (rank, rank, world)
+        sl = dist_util.query_slice(1001, rank, world)
+        dist.barrier()
+        mine = [10.0 + rank, 5.0 - rank, float(len(sl))]
+        got = dist_util.max_over_ranks(mine)
+        dist.barrier()
+        out.put((rank, got, (sl.start, sl.stop)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_gloo_max_and_partition():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res[0][1] == res[1][1] == [11.0, 5.0, 501.0]          # element-wise max over both ranks
+    assert res[0][2] == (0, 501) and res[1][2] == (501, 1001)    # disjoint, covering
