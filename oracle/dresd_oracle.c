@@ -22,7 +22,12 @@
  *   - keys are used as stored (they are unit length by construction), so the
  *     similarity is the inner product of the unit query with the stored key;
  *   - no PCA centring unless a pca_mean vector is supplied;
- *   - the value lookup copies the first draft_len stored tokens verbatim.
+ *   - the value lookup copies the first draft_len stored tokens verbatim;
+ *   - the first-token filter of Sections 3.1 / 3.5 (the LLM's own next token
+ *     x_{t+1} rules out drafts that do not start with it) is applied BEFORE
+ *     the selection: only keys whose first stored token equals first_token[b]
+ *     are candidates; when fewer than n exist the tail is id -1, score
+ *     -infinity, tokens -1.  first_token NULL or -1 = no filter.
  *
  * Pins (tests/test_oracle_*.py): hand-computed cases, closed forms
  * (unit norm, scale invariance, identity keys), brute-force cross-check
@@ -171,7 +176,7 @@ int dresd_oracle_retrieve(const void *keys, const int32_t *next_tokens, int64_t 
                           const void *queries, int B, int d_in,
                           const float *mean, const float *var, double eps_z,
                           const void *W, const float *pca_mean, double eps_n,
-                          int top_n, int draft_len,
+                          int top_n, int draft_len, const int32_t *first_token,
                           int32_t *out_ids, double *out_scores, int32_t *out_tokens,
                           double *full_scores, int threads)
 {
@@ -188,9 +193,21 @@ int dresd_oracle_retrieve(const void *keys, const int32_t *next_tokens, int64_t 
         goto done;
     for (int b = 0; b < B; ++b) {
         dresd_oracle_scores(keys, N, d, dtype, qhat + (size_t)b * d, s, threads);
-        for (int64_t i = 0; i < N; ++i) order[i] = i;
-        qsort_r(order, (size_t)N, sizeof(int64_t), by_score_then_id, s);
+        /* candidates: every key, or (Sections 3.1, 3.5) only the keys whose stored
+           continuation starts with the LLM's own next token */
+        int64_t n_cand = 0;
+        for (int64_t i = 0; i < N; ++i)
+            if (!first_token || first_token[b] < 0 || next_tokens[i * stored_len] == first_token[b])
+                order[n_cand++] = i;
+        qsort_r(order, (size_t)n_cand, sizeof(int64_t), by_score_then_id, s);
         for (int r = 0; r < top_n; ++r) {
+            if (r >= n_cand) {
+                out_ids[(size_t)b * top_n + r] = -1;
+                out_scores[(size_t)b * top_n + r] = -INFINITY;
+                for (int t = 0; t < draft_len; ++t)
+                    out_tokens[((size_t)b * top_n + r) * draft_len + t] = -1;
+                continue;
+            }
             int64_t id = order[r];
             out_ids[(size_t)b * top_n + r] = (int32_t)id;
             out_scores[(size_t)b * top_n + r] = s[id];

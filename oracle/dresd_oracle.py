@@ -50,7 +50,7 @@ def _load():
             c.c_void_p, c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_int,
             c.c_void_p, c.c_int, c.c_int,
             c.c_void_p, c.c_void_p, c.c_double, c.c_void_p, c.c_void_p, c.c_double,
-            c.c_int, c.c_int,
+            c.c_int, c.c_int, c.c_void_p,
             c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_int]
         _lib = lib
     return _lib
@@ -134,8 +134,13 @@ class OracleResult:
 def retrieve(keys, next_tokens, dtype: str, queries, top_n: int, draft_len: int,
              mean=None, var=None, eps_z: float = 1e-5, W=None, pca_mean=None,
              eps_n: float = 1e-12, want_full_scores: bool = False,
-             threads: int = 1) -> OracleResult:
-    """One whole draft-model call, brute force (see the C file's header)."""
+             threads: int = 1, first_token=None) -> OracleResult:
+    """One whole draft-model call, brute force (see the C file's header).
+
+    ``first_token``: optional int32 ``[B]``; query b only considers keys whose first
+    stored token equals ``first_token[b]`` (-1 = no filter).  Missing neighbours come
+    back as id -1, score -inf, tokens -1.
+    """
     k = _store_array(keys, dtype)
     N, d = k.shape
     nt = np.ascontiguousarray(next_tokens, dtype=np.int32)
@@ -154,10 +159,15 @@ def retrieve(keys, next_tokens, dtype: str, queries, top_n: int, draft_len: int,
     sc = np.empty((B, top_n), dtype=np.float64)
     tok = np.empty((B, top_n, draft_len), dtype=np.int32)
     full = np.empty((B, N), dtype=np.float64) if want_full_scores else None
+    ft = None
+    if first_token is not None:
+        ft = np.ascontiguousarray(first_token, dtype=np.int32)
+        if ft.shape != (B,):
+            raise ValueError("first_token must be [B]")
     rc = _load().dresd_oracle_retrieve(
         _ptr(k), _ptr(nt), N, d, _DTYPE_CODE[dtype], nt.shape[1],
         _ptr(q), B, d_in, _ptr(mean), _ptr(var), eps_z, _ptr(W), _ptr(pca_mean), eps_n,
-        top_n, draft_len, _ptr(ids), _ptr(sc), _ptr(tok), _ptr(full), threads)
+        top_n, draft_len, _ptr(ft), _ptr(ids), _ptr(sc), _ptr(tok), _ptr(full), threads)
     if rc != 0:
         raise ValueError("oracle retrieve: bad arguments")
     return OracleResult(ids, sc, tok, full)

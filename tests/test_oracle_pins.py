@@ -277,3 +277,41 @@ def test_bad_arguments_raise():
         oracle.retrieve(keys, toks, "f32", q, top_n=2, draft_len=5)
     with pytest.raises(ValueError):
         oracle.retrieve(keys, toks, "f32", q[:, :4], top_n=2, draft_len=2)
+
+
+# --------------------------------------------------------------------------
+# first-token filter (Sections 3.1 / 3.5)
+# --------------------------------------------------------------------------
+def test_first_token_filter_hand_case():
+    # keys k0..k3 as in the golden cases; unit query (1,0) scores (1, 0, 0.6, -1).
+    keys = np.array([[1.0, 0.0], [0.0, 1.0], [0.6, 0.8], [-1.0, 0.0]], dtype=np.float32)
+    toks = np.array([[7, 1], [5, 2], [5, 3], [5, 4]], dtype=np.int32)
+    q = np.array([[2.0, 0.0]], dtype=np.float32)
+    r = oracle.retrieve(keys, toks, "f32", q, top_n=3, draft_len=2, first_token=[5])
+    assert r.ids[0].tolist() == [2, 1, 3]                       # k0 starts with 7: ruled out
+    np.testing.assert_allclose(r.scores[0], [0.6, 0.0, -1.0], atol=1e-7)
+    assert r.tokens[0].tolist() == [[5, 3], [5, 2], [5, 4]]
+    r = oracle.retrieve(keys, toks, "f32", q, top_n=3, draft_len=2, first_token=[7])
+    assert r.ids[0].tolist() == [0, -1, -1]                     # one match only: padded
+    assert r.scores[0, 0] == 1.0 and np.all(np.isneginf(r.scores[0, 1:]))
+    assert r.tokens[0].tolist() == [[7, 1], [-1, -1], [-1, -1]]
+    r = oracle.retrieve(keys, toks, "f32", q, top_n=3, draft_len=2, first_token=[-1])
+    assert r.ids[0].tolist() == [0, 2, 1]                       # -1 = no filter
+
+
+def test_first_token_filter_equals_search_of_the_matching_subset():
+    N, d, B, n = 800, 16, 5, 6
+    keys, toks = synth.make_store(131, N, d, 6, "f16", 4, vocab=7)
+    q, _ = synth.make_queries(132, keys, "f16", B, 0.1)
+    ft = np.array([0, 1, 2, 6, -1], dtype=np.int32)
+    got = oracle.retrieve(keys, toks, "f16", q, top_n=n, draft_len=4, first_token=ft)
+    for b in range(B):
+        rows = np.arange(N) if ft[b] < 0 else np.nonzero(toks[:, 0] == ft[b])[0]
+        k = min(n, len(rows))
+        sub = oracle.retrieve(keys[rows], toks[rows], "f16", q[b:b + 1], top_n=k, draft_len=4)
+        assert np.array_equal(got.ids[b, :k], rows[sub.ids[0]])
+        assert np.array_equal(got.scores[b, :k], sub.scores[0])
+        assert np.array_equal(got.tokens[b, :k], sub.tokens[0])
+        assert np.all(got.ids[b, k:] == -1) and np.all(np.isneginf(got.scores[b, k:]))
+        if ft[b] >= 0:
+            assert np.all(got.tokens[b, :k, 0] == ft[b])
