@@ -107,6 +107,27 @@ dresd_status dresd_retrieve(dresd_store *store, const void *queries, int B, int 
                             int32_t *out_tokens, void *stream);
 
 /*
+ * First-token filter, Sections 3.1 and 3.5: the LLM's own next token x_{t+1}
+ * rules out every draft that does not start with it.  The filter is applied
+ * BEFORE the selection: query b only considers keys whose first stored token
+ * equals first_tokens[b], and returns the top_n best of those.
+ *
+ * dresd_store_enable_first_token_filter() builds, once per store, a compact
+ * int32 [N] copy of next_tokens[.][0] (4 N bytes of device memory, one kernel on
+ * `stream`); the scoring kernels read it beside the keys (+4 bytes per row).
+ *
+ * dresd_retrieve_filtered() is dresd_retrieve() with
+ *   first_tokens  device, int32 [B]; a negative entry disables the filter for
+ *                 that query; NULL disables it for the call.
+ * When fewer than top_n keys match, the missing neighbours are reported as
+ * id -1, score -infinity, tokens -1.
+ */
+dresd_status dresd_store_enable_first_token_filter(dresd_store *store, void *stream);
+dresd_status dresd_retrieve_filtered(dresd_store *store, const void *queries, const int32_t *first_tokens,
+                                     int B, int top_n, int draft_len, int32_t *out_ids, float *out_scores,
+                                     int32_t *out_tokens, void *stream);
+
+/*
  * The same call for callers whose queries and results live in HOST memory
  * (ideally pinned): copies the queries to the device, runs dresd_retrieve(),
  * copies the three results back and waits for `stream`.  The datastore itself

@@ -27,7 +27,8 @@ EXPORTS = (
     "dresd_preprocess", "dresd_store_status", "dresd_store_set_option",
     "dresd_store_profile_read", "dresd_store_last_launches", "dresd_store_last_key_passes",
     "dresd_last_error",
-    "dresd_store_destroy", "dresd_retrieve_noalloc",
+    "dresd_store_destroy", "dresd_retrieve_noalloc", "dresd_store_enable_first_token_filter",
+    "dresd_retrieve_filtered",
 )
 
 
@@ -77,6 +78,10 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_last_error.argtypes = []
     lib.dresd_store_destroy.restype = None
     lib.dresd_store_destroy.argtypes = [vp]
+    lib.dresd_store_enable_first_token_filter.restype = i32
+    lib.dresd_store_enable_first_token_filter.argtypes = [vp, vp]
+    lib.dresd_retrieve_filtered.restype = i32
+    lib.dresd_retrieve_filtered.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_retrieve_noalloc.restype = i32
     lib.dresd_retrieve_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
     if path is None:
@@ -110,6 +115,16 @@ def dresd_retrieve(store: int, queries_ptr: int, B: int, top_n: int, draft_len: 
                    out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
     _check(load().dresd_retrieve(store, queries_ptr, B, top_n, draft_len, out_ids_ptr, out_scores_ptr,
                                  out_tokens_ptr, stream))
+
+
+def dresd_store_enable_first_token_filter(store: int, stream: int = 0) -> None:
+    _check(load().dresd_store_enable_first_token_filter(store, stream))
+
+
+def dresd_retrieve_filtered(store: int, queries_ptr: int, first_tokens_ptr, B: int, top_n: int, draft_len: int,
+                            out_ids_ptr: int, out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_retrieve_filtered(store, queries_ptr, first_tokens_ptr, B, top_n, draft_len,
+                                          out_ids_ptr, out_scores_ptr, out_tokens_ptr, stream))
 
 
 def dresd_retrieve_host(store: int, queries_ptr: int, B: int, top_n: int, draft_len: int,
@@ -224,6 +239,26 @@ class Store:
         s = (stream or torch.cuda.current_stream()).cuda_stream
         dresd_retrieve(self.handle, queries.data_ptr(), B, top_n, draft_len, ids.data_ptr(),
                        scores.data_ptr(), tokens.data_ptr(), s)
+        return ids, scores, tokens
+
+    def enable_first_token_filter(self, stream=None):
+        s = (stream or _torch().cuda.current_stream()).cuda_stream
+        dresd_store_enable_first_token_filter(self.handle, s)
+
+    def retrieve_filtered(self, queries, first_tokens, top_n: int, draft_len: int, out=None, stream=None):
+        """Like retrieve(), restricted per query to keys whose first stored token is first_tokens[b]."""
+        torch = _torch()
+        B = queries.shape[0]
+        if out is None:
+            dev = queries.device
+            out = (torch.empty((B, top_n), dtype=torch.int32, device=dev),
+                   torch.empty((B, top_n), dtype=torch.float32, device=dev),
+                   torch.empty((B, top_n, draft_len), dtype=torch.int32, device=dev))
+        ids, scores, tokens = out
+        s = (stream or torch.cuda.current_stream()).cuda_stream
+        dresd_retrieve_filtered(self.handle, queries.data_ptr(),
+                                None if first_tokens is None else first_tokens.data_ptr(), B, top_n, draft_len,
+                                ids.data_ptr(), scores.data_ptr(), tokens.data_ptr(), s)
         return ids, scores, tokens
 
     def retrieve_host(self, queries, top_n: int, draft_len: int, out, stream=None):

@@ -107,6 +107,7 @@ struct dresd_store {
     unsigned long long *cand;    // [max_grid][kMaxBatch][kCandStride]
     int *status;                 // device status word
     unsigned int *gtau;          // [kMaxBatch] grid-wide filter words
+    int32_t *first_col;          // [N] first stored token of every key; allocated on request
     int max_grid;
     // staging for dresd_retrieve_host (owned, device)
     void *q_stage;
@@ -144,6 +145,7 @@ void free_store(dresd_store *s)
     cudaFree(s->cand);
     cudaFree(s->status);
     cudaFree(s->gtau);
+    cudaFree(s->first_col);
     cudaFree(s->q_stage);
     cudaFree(s->ids_dev);
     cudaFree(s->scores_dev);
@@ -201,7 +203,8 @@ dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows
 }
 
 dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n, int draft_len,
-                          int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream)
+                          int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream,
+                          const int32_t *first_tokens = nullptr)
 {
     s->last_stream = stream;
     s->last_launches = 0;
@@ -239,6 +242,8 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.cand_batch = B;
         a.status = s->status;
         a.gtau = s->gtau;
+        a.first_col = first_tokens ? s->first_col : nullptr;
+        a.want_first = first_tokens;
         const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
         cudaError_t e = cudaSuccess;
         // Large batches on large stores: a probe pass over every 64th tile first.  Its
@@ -279,6 +284,8 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.cand_batch = B;
         a.status = s->status;
         a.gtau = s->gtau + q0;
+        a.first_col = first_tokens ? s->first_col : nullptr;
+        a.want_first = first_tokens ? first_tokens + q0 : nullptr;
         cudaError_t e = f32 ? launch_scan_f32(s->map_stream, a, grid, stream)
                             : launch_scan_mma(s->map_stream, a, grid, stream);
         if (e != cudaSuccess) return fail_cuda(e, "scan launch");
@@ -455,6 +462,40 @@ dresd_status dresd_retrieve_host(dresd_store *s, const void *queries_host, int B
         return fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
     }
     return DRESD_OK;
+}
+
+dresd_status dresd_store_enable_first_token_filter(dresd_store *s, void *stream_v)
+{
+    if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+    if (s->first_col) return DRESD_OK;
+    int32_t *col = nullptr;
+    if (cudaMalloc(&col, sizeof(int32_t) * (size_t)s->N) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(DRESD_ERR_ALLOC, "allocation of the first-token column (%lld bytes) failed", 4LL * s->N);
+    }
+    cudaError_t e = launch_extract_first(s->next_tokens, s->stored_len, s->N, col, static_cast<cudaStream_t>(stream_v));
+    if (e != cudaSuccess) {
+        cudaFree(col);
+        return fail_cuda(e, "first-token column launch");
+    }
+    s->first_col = col;
+    return DRESD_OK;
+}
+
+dresd_status dresd_retrieve_filtered(dresd_store *s, const void *queries, const int32_t *first_tokens, int B,
+                                     int top_n, int draft_len, int32_t *out_ids, float *out_scores,
+                                     int32_t *out_tokens, void *stream)
+{
+    dresd_status st = check_retrieve_args(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens, true);
+    if (st != DRESD_OK || B == 0) return st;
+    if (!first_tokens)
+        return run_retrieve(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens,
+                            static_cast<cudaStream_t>(stream));
+    if (!is_device_ptr(first_tokens)) return fail(DRESD_ERR_INVALID, "first_tokens must be a device pointer");
+    if (!s->first_col)
+        return fail(DRESD_ERR_INVALID, "call dresd_store_enable_first_token_filter() on this store first");
+    return run_retrieve(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens,
+                        static_cast<cudaStream_t>(stream), first_tokens);
 }
 
 dresd_status dresd_preprocess(dresd_store *s, const void *queries, int B, float *out_qhat, void *stream_v)

@@ -49,6 +49,10 @@ struct ScanArgs {
     int cand_batch;         // query stride of `cand` (the call's B)
     int *status;            // device status word
     unsigned int *gtau;     // grid-wide filter words of this launch's queries (see share_tau)
+    // First-token filter (Section 3.5): when both are set, query q only accepts rows
+    // with first_col[row] == want_first[q]; want_first[q] < 0 disables it for that query.
+    const int32_t *first_col;   // [N] first stored token of every key (compact copy)
+    const int32_t *want_first;  // [B] of this launch
     int stages;             // pipeline depth
     int tile_stride;        // tcgen05 kernel: visit every tile_stride-th tile (probe pass), default 1
 };
@@ -81,6 +85,10 @@ cudaError_t launch_merge_tau(const unsigned long long *cand, int grid_lists, int
 cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long N,
                           const int32_t *ids, int B, int top_n, int draft_len,
                           int32_t *out_tokens, cudaStream_t stream);
+
+// first_col[i] = next_tokens[i][0]: the compact column the first-token filter reads.
+cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, long long N,
+                                 int32_t *first_col, cudaStream_t stream);
 
 // Stores `msg` as the calling thread's dresd_last_error() text.
 void set_last_error(const char *msg);

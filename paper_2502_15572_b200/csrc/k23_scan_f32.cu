@@ -92,7 +92,13 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
         const int row_in_tile = tid;                  // 0..127
         const uint32_t swz = (uint32_t)(row_in_tile & 7);
         bool dead = false;
+        int want[QB];                                  // first-token filter, -1 = off
+#pragma unroll
+        for (int q = 0; q < QB; ++q) want[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
         for (int tl = 0; tl < my_tiles && !dead; ++tl) {
+            // this row's first stored token, requested before the tile is waited for
+            const long long row_pre = (long long)(cta + tl * G) * kRows + row_in_tile;
+            const int tok = (a.first_col && row_pre < a.N) ? a.first_col[row_pre] : 0;
             float acc[QB][4];
 #pragma unroll
             for (int q = 0; q < QB; ++q)
@@ -136,7 +142,7 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
 #pragma unroll
             for (int q = 0; q < QB; ++q) {
                 sc[q] = (acc[q][0] + acc[q][1]) + (acc[q][2] + acc[q][3]);
-                take[q] = q < a.B && row < a.N && sc[q] >= my_sel[q].tau;
+                take[q] = q < a.B && row < a.N && sc[q] >= my_sel[q].tau && (want[q] < 0 || tok == want[q]);
                 any |= take[q];
             }
             if (__any_sync(0xFFFFFFFFu, any)) {

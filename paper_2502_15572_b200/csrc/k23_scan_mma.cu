@@ -174,8 +174,12 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 }
         }
         bool q_valid[NG];
+        int want[NG];                                  // first-token filter of this thread's queries, -1 = off
 #pragma unroll
-        for (int grp = 0; grp < NG; ++grp) q_valid[grp] = grp * 4 + t < a.B;
+        for (int grp = 0; grp < NG; ++grp) {
+            q_valid[grp] = grp * 4 + t < a.B;
+            want[grp] = (a.first_col && q_valid[grp]) ? a.want_first[grp * 4 + t] : -1;
+        }
 
         const uint32_t swz = (uint32_t)g;          // (row & 7) of both of this thread's rows
         const uint32_t off0 = (uint32_t)(((2 * t) ^ swz) << 4);
@@ -183,6 +187,14 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
 
         for (int tl = group; tl < my_tiles && !dead; tl += 2) {
             const long long tile_row0 = (long long)(cta + tl * G) * S::kRows;
+            // first stored tokens of this thread's rows, requested before the tile is waited for
+            int tok_a[S::kBlocksPerWarp], tok_b[S::kBlocksPerWarp];
+#pragma unroll
+            for (int bi = 0; bi < S::kBlocksPerWarp; ++bi) {
+                const long long ra = tile_row0 + (wg * S::kBlocksPerWarp + bi) * 16 + g;
+                tok_a[bi] = (a.first_col && ra < a.N) ? a.first_col[ra] : 0;
+                tok_b[bi] = (a.first_col && ra + 8 < a.N) ? a.first_col[ra + 8] : 0;
+            }
             float acc[S::kBlocksPerWarp][NG][2][4];
 #pragma unroll
             for (int bi = 0; bi < S::kBlocksPerWarp; ++bi)
@@ -256,8 +268,8 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                     sa[grp] = (c0[0] + c1[0]) + (c0[1] + c1[1]) * a.lo_inv_scale;
                     sb[grp] = (c0[2] + c1[2]) + (c0[3] + c1[3]) * a.lo_inv_scale;
                     const float tau = my_sel[grp * 4 + t].tau;
-                    pa[grp] = q_valid[grp] && row_a < a.N && sa[grp] >= tau;
-                    pb[grp] = q_valid[grp] && row_b < a.N && sb[grp] >= tau;
+                    pa[grp] = q_valid[grp] && row_a < a.N && sa[grp] >= tau && (want[grp] < 0 || tok_a[bi] == want[grp]);
+                    pb[grp] = q_valid[grp] && row_b < a.N && sb[grp] >= tau && (want[grp] < 0 || tok_b[bi] == want[grp]);
                     any |= pa[grp] | pb[grp];
                 }
                 if (__any_sync(0xFFFFFFFFu, any)) {

@@ -145,7 +145,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     uint8_t *qres = stages + (size_t)n_stages * stage_bytes;                 // resident query operand
     WarpTopN *sel = reinterpret_cast<WarpTopN *>(qres + (q_resident ? (size_t)dslabs * kQSlabBytes : 0));
     float *tau = reinterpret_cast<float *>(sel + NQ);
-    uint64_t *full = reinterpret_cast<uint64_t *>(tau + NQ);
+    int *want_s = reinterpret_cast<int *>(tau + NQ);        // first-token filter per query, -1 = off
+    uint64_t *full = reinterpret_cast<uint64_t *>(want_s + NQ);
     uint64_t *empty = full + kMaxStages;
     uint64_t *tfull = empty + kMaxStages;                   // [2] accumulator ready
     uint64_t *tempty = tfull + 2;                           // [2] accumulator drained
@@ -178,7 +179,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         for (int q = warp - 2; q < NQ; q += kEpiWarps) {
             warp_topn_init(&sel[q], lane);
             // start from whatever the grid already knows; padding columns never pass
-            if (lane == 0) tau[q] = q < a.B ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
+            if (lane == 0) {
+                tau[q] = q < a.B ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
+                want_s[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
+            }
         }
     }
     if (warp == 1) {
@@ -280,6 +284,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(half * CW);
         const float inv = a.lo_inv_scale;
         const float4 *tau4 = reinterpret_cast<const float4 *>(tau + qbase);
+        const int4 *want4 = reinterpret_cast<const int4 *>(want_s + qbase);
+        const bool filtered = a.first_col != nullptr;
+        uint32_t wild = 0u;                                 // this warp's queries without a token filter
+        for (int j = 0; j < QW; ++j) wild |= (want_s[qbase + j] < 0) ? (1u << j) : 0u;
         // A warp whose wait expired goes "dead": it does no more work and no more
         // waits, but keeps taking part in every barrier so that nobody is left behind.
         bool dead = false;
@@ -287,6 +295,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         EpiFlags *fl = &flags[0];
         for (int tl = 0; tl < my_tiles; ++tl) {
             const int acc = tl & 1, use = tl >> 1;
+            // this row's first stored token (filtered calls), requested before the wait
+            const long long row_pre =
+                (long long)(cta + tl * G) * a.tile_stride * kTileRows + lane_grp * 32 + lane;
+            const int tok = (filtered && row_pre < a.N) ? a.first_col[row_pre] : 0;
             if (!dead && !mbar_wait(&tfull[acc], use & 1)) {
                 report_timeout(a.status);
                 dead = true;
@@ -319,6 +331,16 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                             const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
                             mask |= (s >= tt[i]) ? (1u << j) : 0u;
                         }
+                    }
+                    if (filtered) {                         // Section 3.5: drafts must start with x_{t+1}
+                        uint32_t match = wild;
+#pragma unroll
+                        for (int j4 = 0; j4 < QW / 4; ++j4) {
+                            const int4 w = want4[j4];
+                            match |= (tok == w.x ? 1u : 0u) << (4 * j4) | (tok == w.y ? 2u : 0u) << (4 * j4) |
+                                     (tok == w.z ? 4u : 0u) << (4 * j4) | (tok == w.w ? 8u : 0u) << (4 * j4);
+                        }
+                        mask &= match;
                     }
                     mask &= first ? (row_ok ? 0xFFFFFFFFu : 0u) : pending;
                     pending = 0u;
@@ -404,7 +426,7 @@ Plan make_plan(int d, int B)
     const size_t qbytes = (size_t)dslabs * p.ncols * kSlabBytes;
     p.q_resident = qbytes <= (size_t)kResidentLimit;
     const size_t fixed = 1024 + (p.q_resident ? qbytes : 0) + sizeof(WarpTopN) * (p.ncols / 2) +
-                         sizeof(float) * (p.ncols / 2) + sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
+                         (sizeof(float) + sizeof(int)) * (p.ncols / 2) + sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
     const size_t slab = kKeyStageBytes + (p.q_resident ? 0 : (size_t)p.ncols * kSlabBytes);
     // Largest slab group (fewest barrier round trips per tile) that still leaves
     // at least three groups in flight.

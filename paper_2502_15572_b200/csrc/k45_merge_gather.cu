@@ -62,7 +62,27 @@ __global__ void gather_kernel(const int32_t *__restrict__ next_tokens, int store
     }
 }
 
+// Compact copy of the first stored token of every key (the column the first-token
+// filter of Section 3.5 tests), so that the scan reads 4 bytes per row for it.
+__global__ void extract_first_kernel(const int32_t *__restrict__ next_tokens, int stored_len, long long N,
+                                     int32_t *__restrict__ first_col)
+{
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < N;
+         i += (long long)gridDim.x * blockDim.x)
+        first_col[i] = next_tokens[i * stored_len];
+}
+
 }  // namespace
+
+cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, long long N, int32_t *first_col,
+                                 cudaStream_t stream)
+{
+    const int threads = 256;
+    long long blocks = (N + threads - 1) / threads;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    extract_first_kernel<<<(int)blocks, threads, 0, stream>>>(next_tokens, stored_len, N, first_col);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_merge(const unsigned long long *cand, int lists, int B, int top_n,
                          int32_t *out_ids, float *out_scores, cudaStream_t stream)

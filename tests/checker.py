@@ -105,3 +105,20 @@ def check_batch(full_scores, next_tokens, ids, scores, tokens, dtype, top_n, dra
         except AssertionError as e:
             raise AssertionError(f"query {b}: {e}") from None
     return exact / float(B * top_n)
+
+
+def check_query_filtered(s, next_tokens, g_ids, g_scores, g_tokens, dtype, top_n, draft_len, first_token):
+    """First-token filter: the result must be the top-n of the rows whose first stored
+    token is `first_token` (all rows when it is negative), padded with id -1 / -inf / -1."""
+    g_ids = np.asarray(g_ids).astype(np.int64)
+    rows = np.arange(s.shape[0]) if first_token < 0 else np.nonzero(next_tokens[:, 0] == first_token)[0]
+    k = min(top_n, len(rows))
+    assert np.all(g_ids[k:] == -1), f"expected {top_n - k} padding ids, got {g_ids[k:]}"
+    assert np.all(np.isneginf(np.asarray(g_scores)[k:])) and np.all(np.asarray(g_tokens)[k:] == -1)
+    if k == 0:
+        return 0
+    pos = np.searchsorted(rows, g_ids[:k])
+    assert np.all(pos < len(rows)) and np.all(rows[np.minimum(pos, len(rows) - 1)] == g_ids[:k]), \
+        f"a returned row does not start with token {first_token}: {g_ids[:k]}"
+    return check_query(s[rows], next_tokens[rows], pos, np.asarray(g_scores)[:k], np.asarray(g_tokens)[:k],
+                       dtype, k, draft_len)
