@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--rows", type=int, default=None, help="override N (debugging; not a bench value)")
     ap.add_argument("--oracle-queries", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--first-token-filter", action="store_true",
+                    help="time dresd_retrieve_filtered: each query wants the first stored token of its source row")
     ap.add_argument("--probe", type=int, default=1, help="probe-pass tile stride (0 off, 1 default)")
     ap.add_argument("--scan-path", type=int, default=0, choices=[0, 1, 2],
                     help="0 auto, 1 streaming mma.sync kernel, 2 tcgen05 kernel (16-bit keys)")
@@ -73,6 +75,7 @@ def workload_config(cfg):
     return {"workload": cfg["name"], "N": cfg["N"], "d": cfg["d"], "d_in": cfg.get("d_in", cfg["d"]),
             "key_dtype": cfg["dtype"],
             "batch": cfg["B"], "top_n": cfg["top_n"], "draft_len": cfg["draft_len"],
+            "first_token_filter": bool(cfg.get("filter_on", False)),
             "mixture_components": cfg["C"], "query_noise_sigma": cfg["sigma"], "seed": cfg["seed"],
             "l2": "keys are %.2f GB per step, far larger than the 126 MB L2: no flush needed"
                   % (cfg["N"] * cfg["d"] * synth.DTYPE_BYTES[cfg["dtype"]] / 1e9)}
@@ -89,7 +92,8 @@ def make_inputs(args):
         cfg["W"] = W
         q = synth.make_hidden_queries(cfg["seed"] + 100, nq, cfg["d_in"], cfg["dtype"], scale=1.0, offset=0.0)
     else:
-        q, _ = synth.make_queries(cfg["seed"] + 100, keys, cfg["dtype"], nq, cfg["sigma"])
+        q, src = synth.make_queries(cfg["seed"] + 100, keys, cfg["dtype"], nq, cfg["sigma"])
+        cfg["first_tokens"] = np.ascontiguousarray(toks[src, 0])      # the token the LLM would have produced
     return cfg, keys, toks, q
 
 
@@ -199,6 +203,7 @@ def run_ours(args):
         dist.barrier()
 
     cfg, keys, toks, q = make_inputs(args)
+    cfg["filter_on"] = args.first_token_filter
     B, n, L, dtype = cfg["B"], cfg["top_n"], cfg["draft_len"], cfg["dtype"]
     dkeys = binding.to_device(keys, dtype)
     dtoks = torch.from_numpy(toks).cuda()
@@ -212,13 +217,22 @@ def run_ours(args):
         store.set_preprocess(cfg["d_in"], W=dW)
     store.set_option("scan_path", args.scan_path)
     store.set_option("probe", args.probe)
+    dft = None
+    if args.first_token_filter:
+        if "first_tokens" not in cfg:
+            raise SystemExit("--first-token-filter needs a workload whose queries have source rows")
+        store.enable_first_token_filter()
+        dft = torch.from_numpy(cfg["first_tokens"]).cuda()
     out = (torch.empty((B, n), dtype=torch.int32, device="cuda"),
            torch.empty((B, n), dtype=torch.float32, device="cuda"),
            torch.empty((B, n, L), dtype=torch.int32, device="cuda"))
 
     def step(i):
         j = (q_first + i % nq) * B
-        store.retrieve(dq[j:j + B], n, L, out=out)
+        if dft is None:
+            store.retrieve(dq[j:j + B], n, L, out=out)
+        else:
+            store.retrieve_filtered(dq[j:j + B], dft[j:j + B], n, L, out=out)
 
     def barrier():
         if world > 1:
