@@ -160,6 +160,12 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "probe"      large batches on large stores first run a probe pass over every
  *                value-th key tile to seed the selection filter; 0 = never,
  *                1 = default stride (256).
+ *   "wait_ms"    bound of the device-side waits of the streaming kernels in
+ *                milliseconds (0 = default, about 2 s).
+ *   "debug_lose_stage"  test hook: in the next calls the streaming 16-bit kernel's
+ *                first CTA never receives the copies of pipeline stage (value-1),
+ *                so its waits run out: the kernel returns in an orderly way and
+ *                dresd_store_status() reports DRESD_ERR_TIMEOUT.  0 = off.
  *   "profile"    > 0: record a CUDA-event pair around the scoring kernel(s) of
  *                each of the next `value` dresd_retrieve() calls (see
  *                dresd_store_profile_read); 0 = off (default).

@@ -124,7 +124,7 @@ struct dresd_store {
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     int n_tiles_umma;
     // options / bookkeeping
-    int opt_path, opt_grid, opt_probe;
+    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage;
     double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
     cudaStream_t last_stream;
     int last_launches;
@@ -284,6 +284,8 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.cand_batch = B;
         a.status = s->status;
         a.gtau = s->gtau + q0;
+        a.wait_cycles = (long long)s->opt_wait_ms * 2000000LL;     // ~2 GHz
+        a.debug_lose_stage = s->opt_lose_stage;
         a.first_col = first_tokens ? s->first_col : nullptr;
         a.want_first = first_tokens ? first_tokens + q0 : nullptr;
         cudaError_t e = f32 ? launch_scan_f32(s->map_stream, a, grid, stream)
@@ -538,6 +540,16 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
     if (strcmp(name, "scan_path") == 0) {
         if (value < 0 || value > 2) return fail(DRESD_ERR_INVALID, "scan_path = %d outside 0..2", value);
         s->opt_path = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "wait_ms") == 0) {
+        if (value < 0 || value > 60000) return fail(DRESD_ERR_INVALID, "wait_ms = %d outside 0..60000", value);
+        s->opt_wait_ms = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "debug_lose_stage") == 0) {
+        if (value < 0) return fail(DRESD_ERR_INVALID, "debug_lose_stage = %d is negative", value);
+        s->opt_lose_stage = value;
         return DRESD_OK;
     }
     if (strcmp(name, "probe") == 0) {

@@ -54,6 +54,8 @@ struct ScanArgs {
     const int32_t *first_col;   // [N] first stored token of every key (compact copy)
     const int32_t *want_first;  // [B] of this launch
     int stages;             // pipeline depth
+    long long wait_cycles;  // bound of every device-side wait in cycles, 0 = default (~2 s)
+    int debug_lose_stage;   // test hook (streaming kernel): CTA 0 never receives stage (value-1); 0 = off
     int tile_stride;        // tcgen05 kernel: visit every tile_stride-th tile (probe pass), default 1
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.

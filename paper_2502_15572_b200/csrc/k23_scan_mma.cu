@@ -125,6 +125,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
     const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
     const int n_it = my_tiles * kch;
     bool dead = false;
+    const long long wait_limit = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;
 
     if (warp == kConsumerWarps) {
         // ------------------------------ producer ------------------------------
@@ -133,7 +134,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             int issued = 0;
             for (int it = 0; it < n_it; ++it) {
                 const int s = it % n_stages;
-                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
+                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1, wait_limit)) {
                     report_timeout(a.status);
                     break;
                 }
@@ -142,14 +143,17 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 const int nsl = KS > 0 ? KS : min(4, dslabs - kc * 4);
                 mbar_arrive_expect_tx(&full[s], (uint32_t)(nsl * S::kRows * kSlabBytes));
                 uint8_t *dst = stages + (size_t)s * kStageBytes;
-                for (int sl = 0; sl < nsl; ++sl)
+                // Test hook: one CTA "loses" the copies of one stage, so that the waits on it
+                // run out and the timeout path (status word, orderly exit) can be exercised.
+                const bool lose = a.debug_lose_stage > 0 && cta == 0 && it == a.debug_lose_stage - 1;
+                for (int sl = 0; sl < nsl && !lose; ++sl)
                     tma_load_2d(dst + (size_t)sl * S::kRows * kSlabBytes, &keys_map,
                                 (kc * 4 + sl) * kSlabElems, tile * S::kRows, &full[s]);
                 issued = it + 1;
             }
             // Do not leave while copies into this CTA's shared memory are in flight.
             for (int it = max(0, issued - n_stages); it < issued; ++it)
-                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1)) {
+                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1, wait_limit)) {
                     report_timeout(a.status);
                     break;
                 }
@@ -208,7 +212,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             for (int kc = 0; kc < kch; ++kc) {
                 const int it = tl * kch + kc;
                 const int s = it % n_stages;
-                if (!mbar_wait(&full[s], (it / n_stages) & 1)) {
+                if (!mbar_wait(&full[s], (it / n_stages) & 1, wait_limit)) {
                     report_timeout(a.status);
                     dead = true;
                     break;

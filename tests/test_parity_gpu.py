@@ -283,3 +283,29 @@ def test_argument_errors_on_device():
     with pytest.raises(binding.DresdError) as e:
         binding.Store(k, torch.zeros((8, 2), dtype=torch.int32, device="cuda"), "f16")
     assert e.value.status == -1
+
+
+def test_bounded_wait_reports_timeout_and_store_stays_usable():
+    """Failure detection without a GPU fault: one CTA never receives one pipeline stage
+    (a barrier that nothing completes); every wait on it runs out after 100 ms, the
+    kernel returns in an orderly way, the status word says TIMEOUT, and the next call
+    on the same store is correct again."""
+    N, d, dtype = 60013, 128, "f16"
+    keys, toks = synth.make_store(8401, N, d, 16, dtype, 4)
+    q, _ = synth.make_queries(8402, keys, dtype, 2, 0.1)
+    st = gpu_store(keys, toks, dtype)
+    st.set_option("scan_path", 1)
+    good = gpu_retrieve(st, q, 10, 4)
+    st.set_option("wait_ms", 100)
+    st.set_option("debug_lose_stage", 2)
+    import torch
+    st.retrieve(binding.to_device(q, dtype), 10, 4)
+    torch.cuda.synchronize()
+    with pytest.raises(binding.DresdError) as e:
+        st.status()
+    assert e.value.status == -5
+    st.set_option("debug_lose_stage", 0)
+    st.set_option("wait_ms", 0)
+    again = gpu_retrieve(st, q, 10, 4)               # status() inside: clean again
+    assert all(np.array_equal(a, b) for a, b in zip(good, again))
+    st.close()
