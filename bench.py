@@ -45,6 +45,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2_decode_b1_f16", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--rows", type=int, default=None, help="override N (debugging; not a bench value)")
+    ap.add_argument("--batch", type=int, default=None, help="override B (debugging; not a bench value)")
+    ap.add_argument("--top-n", type=int, default=None, help="override top_n (debugging; not a bench value)")
     ap.add_argument("--oracle-queries", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--first-token-filter", action="store_true",
@@ -85,6 +87,10 @@ def make_inputs(args):
     cfg = dict(synth.WORKLOADS[args.workload], name=args.workload)
     if args.rows:
         cfg["N"] = args.rows
+    if args.batch:
+        cfg["B"] = args.batch
+    if args.top_n:
+        cfg["top_n"] = args.top_n
     keys, toks = synth.make_store(cfg["seed"], cfg["N"], cfg["d"], cfg["C"], cfg["dtype"], cfg["stored_len"])
     nq = N_QUERIES if cfg["B"] == 1 else cfg["B"] * 16
     if "d_in" in cfg:       # queries arrive at the LLM's hidden width and are projected (Section 3.3)

@@ -159,7 +159,7 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "grid"       CTAs of the scoring kernel, 0 = one per SM.
  *   "probe"      large batches on large stores first run a probe pass over every
  *                value-th key tile to seed the selection filter; 0 = never,
- *                1 = default stride (256).
+ *                1 = default stride (128).
  *   "wait_ms"    bound of the device-side waits of the streaming kernels in
  *                milliseconds (0 = default, about 2 s).
  *   "debug_lose_stage"  test hook: in the next calls the streaming 16-bit kernel's

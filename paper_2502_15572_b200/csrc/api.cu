@@ -29,7 +29,7 @@ dresd_status fail_cuda(cudaError_t e, const char *what)
 }
 
 constexpr uint32_t kMagic = 0xD2E5D001u;
-constexpr int kProbeStride = 256;    // default: the probe pass visits every 256th tile
+constexpr int kProbeStride = 128;    // default: the probe pass visits every 128th tile
 constexpr float kEpsNorm = 1e-12f;   // epsilon of Eq. 2 (the paper leaves it open)
 
 bool is_device_ptr(const void *p)
@@ -255,6 +255,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
             ScanArgs pa = a;
             pa.tile_stride = pstride;
             pa.n_tiles = (n_tiles + pstride - 1) / pstride;
+            pa.probe_max = pa.n_tiles <= 32 * grid;      // tile bests fit a CTA's queue as they are
             int pgrid = grid < pa.n_tiles ? grid : pa.n_tiles;
             e = launch_scan_umma(s->map_umma, s->map_q[mi], pa, pgrid, stream);
             if (e == cudaSuccess) e = launch_merge_tau(s->cand, pgrid, B, top_n, s->gtau, stream);

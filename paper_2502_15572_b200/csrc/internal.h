@@ -57,6 +57,7 @@ struct ScanArgs {
     long long wait_cycles;  // bound of every device-side wait in cycles, 0 = default (~2 s)
     int debug_lose_stage;   // test hook (streaming kernel): CTA 0 never receives stage (value-1); 0 = off
     int tile_stride;        // tcgen05 kernel: visit every tile_stride-th tile (probe pass), default 1
+    int probe_max;          // tcgen05 kernel, probe pass: keep only each tile's best row per query
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.
 int scan_mma_tile_rows(int d);

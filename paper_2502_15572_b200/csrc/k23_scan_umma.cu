@@ -116,6 +116,30 @@ template <int CW> __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, u
         for (int c = 0; c < CW / 16; ++c) tmem_ld16p(taddr + 16 * c, r + 16 * c);
     }
 }
+// Column-wise maximum over the 32 lanes of a warp for C values per lane, with C-1
+// exchanges in total instead of 5 per value: at each step a lane keeps one half of its
+// values and hands the other half to its partner.  Afterwards v[0] of lane l holds the
+// maximum of column l >> (5 - log2 C) (the lanes of such a group all hold it).
+template <int C, int O> struct WarpColumnMax {
+    template <int N> static __device__ __forceinline__ void run(unsigned long long (&v)[N], int lane)
+    {
+        if constexpr (O >= 1) {
+            const bool upper = (lane & O) != 0;
+            if constexpr (C > 1) {
+#pragma unroll
+                for (int i = 0; i < C / 2; ++i) {
+                    const unsigned long long send = upper ? v[i] : v[i + C / 2];
+                    const unsigned long long keep = upper ? v[i + C / 2] : v[i];
+                    v[i] = umax64(keep, shfl_xor_u64(send, O));
+                }
+                WarpColumnMax<C / 2, O / 2>::run(v, lane);
+            } else {
+                v[0] = umax64(v[0], shfl_xor_u64(v[0], O));
+                WarpColumnMax<1, O / 2>::run(v, lane);
+            }
+        }
+    }
+};
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 struct EpiFlags {
@@ -146,7 +170,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     WarpTopN *sel = reinterpret_cast<WarpTopN *>(qres + (q_resident ? (size_t)dslabs * kQSlabBytes : 0));
     float *tau = reinterpret_cast<float *>(sel + NQ);
     int *want_s = reinterpret_cast<int *>(tau + NQ);        // first-token filter per query, -1 = off
-    uint64_t *full = reinterpret_cast<uint64_t *>(want_s + NQ);
+    unsigned long long *tilemax = reinterpret_cast<unsigned long long *>(want_s + NQ);   // probe pass: best of a tile
+    uint64_t *full = reinterpret_cast<uint64_t *>(tilemax + 4 * NQ);     // [lane group][query]
     uint64_t *empty = full + kMaxStages;
     uint64_t *tfull = empty + kMaxStages;                   // [2] accumulator ready
     uint64_t *tempty = tfull + 2;                           // [2] accumulator drained
@@ -182,6 +207,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             if (lane == 0) {
                 tau[q] = q < a.B ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
                 want_s[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
+                for (int g4 = 0; g4 < 4; ++g4) tilemax[g4 * NQ + q] = 0ull;
             }
         }
     }
@@ -310,6 +336,45 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             const long long row =
                 (long long)(cta + tl * G) * a.tile_stride * kTileRows + lane_grp * 32 + lane;
             const bool row_ok = !dead && row < a.N;
+            if (a.probe_max) {
+                // Probe pass: no filtering and no lists -- only the best row of this tile per
+                // query (at most 32 tiles per CTA, so the bests fit the queue as they are).
+                // The n-th largest of all CTAs' tile bests is a valid filter: at least n rows
+                // reach it.
+                if (!dead) {
+                    uint32_t r[CW];
+                    tmem_ld_cols<CW>(lane_addr + (uint32_t)(acc * NCOLS), r);
+                    tmem_ld_wait();
+                    unsigned long long v[QW];
+#pragma unroll
+                    for (int j = 0; j < QW; ++j) {
+                        const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
+                        const int w = want_s[qbase + j];
+                        const bool ok = row_ok && (w < 0 || tok == w) && s > -INFINITY;    // false for NaN too
+                        v[j] = ok ? pack_candidate(s, (uint32_t)row) : 0ull;
+                    }
+                    // per-query maximum over the warp's 32 rows: QW-1 exchanges for all queries
+                    WarpColumnMax<QW, 16>::run(v, lane);
+                    constexpr int kShift = QW == 32 ? 0 : QW == 16 ? 1 : QW == 8 ? 2 : 3;
+                    if ((lane & ((1 << kShift) - 1)) == 0)
+                        tilemax[lane_grp * NQ + qbase + (lane >> kShift)] = v[0];
+                } else if (lane < QW) {
+                    tilemax[lane_grp * NQ + qbase + lane] = 0ull;
+                }
+                epi_bar();                                   // all four lane groups have written
+                for (int q = ew; q < a.B; q += kEpiWarps) {
+                    if (lane == 0) {
+                        unsigned long long v = umax64(umax64(tilemax[q], tilemax[NQ + q]),
+                                                      umax64(tilemax[2 * NQ + q], tilemax[3 * NQ + q]));
+                        if (v && sel[q].count < kQueueCap) sel[q].queue[sel[q].count++] = v;
+                    }
+                }
+                epi_bar();                                   // slots may be rewritten for the next tile
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tempty[acc]);
+                continue;
+            }
             uint32_t pending = 0u;                          // queries whose candidate found the queue full
             bool first = true;
             while (true) {
@@ -426,7 +491,8 @@ Plan make_plan(int d, int B)
     const size_t qbytes = (size_t)dslabs * p.ncols * kSlabBytes;
     p.q_resident = qbytes <= (size_t)kResidentLimit;
     const size_t fixed = 1024 + (p.q_resident ? qbytes : 0) + sizeof(WarpTopN) * (p.ncols / 2) +
-                         (sizeof(float) + sizeof(int)) * (p.ncols / 2) + sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
+                         (sizeof(float) + sizeof(int) + 4 * sizeof(unsigned long long)) * (p.ncols / 2) +
+                         sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
     const size_t slab = kKeyStageBytes + (p.q_resident ? 0 : (size_t)p.ncols * kSlabBytes);
     // Largest slab group (fewest barrier round trips per tile) that still leaves
     // at least three groups in flight.

@@ -211,6 +211,12 @@ WORKLOADS = {
                          draft_len=10, stored_len=10, sigma=0.1, seed=1004),
     "c5a_hidden_bf16": dict(N=4_000_000, d=4096, dtype="bf16", C=1024, B=16, top_n=10,
                             draft_len=10, stored_len=10, sigma=0.1, seed=1005),
+    # shaped like the paper's own datastore (Table 1 / Section 5.2: 46.3M token embeddings reduced
+    # to 64 dimensions, about 20 stored continuation tokens), 10 drafts of 10 tokens (Section 5.4)
+    "paper_46m_d64_f16": dict(N=46_300_000, d=64, dtype="f16", C=4096, B=1, top_n=10,
+                              draft_len=10, stored_len=20, sigma=0.1, seed=1010),
+    "paper_46m_d64_f16_b16": dict(N=46_300_000, d=64, dtype="f16", C=4096, B=16, top_n=10,
+                                  draft_len=10, stored_len=20, sigma=0.1, seed=1010),
     "c5b_projected_bf16": dict(N=4_000_000, d=256, dtype="bf16", C=1024, B=16, top_n=10,
                                draft_len=10, stored_len=10, sigma=0.1, seed=1006,
                                d_in=4096, proj_seed=1007),
