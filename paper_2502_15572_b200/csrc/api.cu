@@ -122,7 +122,6 @@ struct dresd_store {
     // tensor-core kernel geometry (16-bit keys): 128-row key tiles, query operand maps
     CUtensorMap map_umma;
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
-    int n_tiles_umma;
     // options / bookkeeping
     int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage;
     double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
@@ -211,15 +210,16 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     s->last_key_passes = 0.0;
     const bool f32 = s->dtype == kF32;
     // 16-bit keys: the tcgen05 kernel serves any batch in one pass over the keys and is
-    // also the fastest for rows of at least four 64-element slabs (7.1 vs 6.8 TB/s at
-    // d = 256); for narrow rows and up to 8 queries the streaming mma.sync kernel wins
-    // (6.8 vs 6.0 TB/s at d = 128) because its per-tile cost is lower.
-    const bool umma = !f32 && (s->opt_path == 2 || (s->opt_path == 0 && (B > 8 || s->d > 192)));
+    // the fastest at every measured shape (7.1-7.2 TB/s at batch 1 for d = 64 and 256
+    // against 6.7-6.8 for the streaming mma.sync kernel), so it is the default; the
+    // streaming kernel stays available as "scan_path" 1 and serves the allocation-free call.
+    const bool umma = !f32 && s->opt_path != 1;
     const int op_rows = umma ? scan_umma_operand_rows(B) : 0;
     dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream);
     if (st != DRESD_OK) return st;
 
-    const int n_tiles = umma ? s->n_tiles_umma : s->n_tiles;
+    const int umma_rows = umma ? scan_umma_tile_rows(s->d, B) : 1;
+    const int n_tiles = umma ? (int)((s->N + umma_rows - 1) / umma_rows) : s->n_tiles;
     int grid = s->opt_grid > 0 ? s->opt_grid : s->num_sms;
     if (grid > s->max_grid) grid = s->max_grid;
     if (grid > n_tiles) grid = n_tiles;
@@ -255,7 +255,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
             ScanArgs pa = a;
             pa.tile_stride = pstride;
             pa.n_tiles = (n_tiles + pstride - 1) / pstride;
-            pa.probe_max = pa.n_tiles <= 32 * grid;      // tile bests fit a CTA's queue as they are
+            pa.probe_max = (long long)pa.n_tiles * (umma_rows / 128) <= 32LL * grid;   // the bests fit a queue
             int pgrid = grid < pa.n_tiles ? grid : pa.n_tiles;
             e = launch_scan_umma(s->map_umma, s->map_q[mi], pa, pgrid, stream);
             if (e == cudaSuccess) e = launch_merge_tau(s->cand, pgrid, B, top_n, s->gtau, stream);
@@ -373,8 +373,7 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
     s->tokens_dev_elems = (size_t)kMaxBatch * kMaxTopN * stored_len;
     ok = ok && cudaMalloc(&s->tokens_dev, sizeof(int32_t) * s->tokens_dev_elems) == cudaSuccess;
     if (ok && dtype != DRESD_F32) {
-        s->n_tiles_umma = (int)((N + scan_umma_tile_rows() - 1) / scan_umma_tile_rows());
-        bool mok = make_map(&s->map_umma, keys, s->dtype, N, d, scan_umma_tile_rows());
+        bool mok = make_map(&s->map_umma, keys, s->dtype, N, d, 128);
         for (int i = 0; i < 4; ++i)
             mok = mok && make_map(&s->map_q[i], s->qsplit, s->dtype, 2 * kMaxBatch, s->dpad, 16 << i);
         if (!mok) {

@@ -68,7 +68,7 @@ cudaError_t launch_scan_mma(const CUtensorMap &keys_map, const ScanArgs &a, int 
 
 // Batched tensor-core kernel (tcgen05/TMEM, 16-bit keys): 128-row tiles; the query
 // operand holds 2 rows per query, padded to 16/32/64/128 rows.
-int scan_umma_tile_rows();
+int scan_umma_tile_rows(int d, int B);      // 128 x sub-tiles per tile (narrow rows use several)
 int scan_umma_operand_rows(int B);
 cudaError_t launch_scan_umma(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
                              int grid, cudaStream_t stream);

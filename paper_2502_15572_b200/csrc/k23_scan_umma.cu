@@ -147,31 +147,35 @@ struct EpiFlags {
     int overflow;
 };
 
-template <typename T, int NCOLS>
+template <typename T, int NCOLS, int TSUB>
 __global__ void __launch_bounds__(kThreads, 1)
 scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_constant__ CUtensorMap q_map,
                  const ScanArgs a, const int q_resident, const int gs)
 {
     constexpr int NQ = NCOLS / 2;                           // queries (padded)
-    constexpr int kTmemCols = 2 * NCOLS < 32 ? 32 : 2 * NCOLS;
+    constexpr int kAccCols = TSUB * NCOLS;                  // one accumulator buffer
+    constexpr int kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;
+    static_assert(kTmemCols <= 512, "TMEM has 512 columns");
     constexpr int kQSlabBytes = NCOLS * kSlabBytes;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    // A pipeline stage holds a GROUP of `gs` consecutive 64-column slabs of one
-    // 128-row tile (one full/empty barrier pair, one wait and one commit per group).
+    // A tile is TSUB sub-tiles of 128 rows.  A pipeline stage (one full/empty barrier
+    // pair, one wait and one commit) holds a GROUP of slabs: for TSUB == 1, `gs`
+    // consecutive 64-column slabs of the tile; for TSUB > 1 (narrow rows) the whole
+    // tile, i.e. all slabs of all its sub-tiles.
     const int n_stages = a.stages;
     const int dslabs = (a.d + kSlabElems - 1) / kSlabElems;
-    const int gpt = (dslabs + gs - 1) / gs;                 // groups per tile
+    const int gpt = TSUB > 1 ? 1 : (dslabs + gs - 1) / gs;  // groups per tile
     const int slab_bytes = kKeyStageBytes + (q_resident ? 0 : kQSlabBytes);
-    const int stage_bytes = gs * slab_bytes;
+    const int stage_bytes = (TSUB > 1 ? TSUB * dslabs : gs) * slab_bytes;
     uint8_t *stages = base;
     uint8_t *qres = stages + (size_t)n_stages * stage_bytes;                 // resident query operand
     WarpTopN *sel = reinterpret_cast<WarpTopN *>(qres + (q_resident ? (size_t)dslabs * kQSlabBytes : 0));
     float *tau = reinterpret_cast<float *>(sel + NQ);
     int *want_s = reinterpret_cast<int *>(tau + NQ);        // first-token filter per query, -1 = off
-    unsigned long long *tilemax = reinterpret_cast<unsigned long long *>(want_s + NQ);   // probe pass: best of a tile
-    uint64_t *full = reinterpret_cast<uint64_t *>(tilemax + 4 * NQ);     // [lane group][query]
+    unsigned long long *tilemax = reinterpret_cast<unsigned long long *>(want_s + NQ);   // probe: [sub][lane group][query]
+    uint64_t *full = reinterpret_cast<uint64_t *>(tilemax + 4 * TSUB * NQ);
     uint64_t *empty = full + kMaxStages;
     uint64_t *tfull = empty + kMaxStages;                   // [2] accumulator ready
     uint64_t *tempty = tfull + 2;                           // [2] accumulator drained
@@ -183,6 +187,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     const int cta = blockIdx.x, G = gridDim.x;
     const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
     const int n_it = my_tiles * gpt;
+    constexpr int kRowsPerTile = kTileRows * TSUB;
 
     if (tid == 0) {
         for (int s = 0; s < n_stages; ++s) {
@@ -207,7 +212,6 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             if (lane == 0) {
                 tau[q] = q < a.B ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
                 want_s[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
-                for (int g4 = 0; g4 < 4; ++g4) tilemax[g4 * NQ + q] = 0ull;
             }
         }
     }
@@ -238,16 +242,25 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     break;
                 }
                 const int tile = (cta + (it / gpt) * G) * a.tile_stride;
-                const int sl0 = (it % gpt) * gs;
-                const int nsl = min(gs, dslabs - sl0);
                 uint8_t *dst = stages + (size_t)s * stage_bytes;
-                mbar_arrive_expect_tx(&full[s], (uint32_t)(nsl * slab_bytes));
-                for (int j = 0; j < nsl; ++j) {
-                    tma_load_2d(dst + (size_t)j * slab_bytes, &keys_map, (sl0 + j) * kSlabElems,
-                                tile * kTileRows, &full[s]);
-                    if (!q_resident)
-                        tma_load_2d(dst + (size_t)j * slab_bytes + kKeyStageBytes, &q_map,
-                                    (sl0 + j) * kSlabElems, 0, &full[s]);
+                if constexpr (TSUB > 1) {
+                    // narrow rows: every slab of every sub-tile (rows past N read as zeros)
+                    mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
+                    for (int sub = 0; sub < TSUB; ++sub)
+                        for (int j = 0; j < dslabs; ++j)
+                            tma_load_2d(dst + (size_t)(sub * dslabs + j) * slab_bytes, &keys_map, j * kSlabElems,
+                                        tile * kRowsPerTile + sub * kTileRows, &full[s]);
+                } else {
+                    const int sl0 = (it % gpt) * gs;
+                    const int nsl = min(gs, dslabs - sl0);
+                    mbar_arrive_expect_tx(&full[s], (uint32_t)(nsl * slab_bytes));
+                    for (int j = 0; j < nsl; ++j) {
+                        tma_load_2d(dst + (size_t)j * slab_bytes, &keys_map, (sl0 + j) * kSlabElems,
+                                    tile * kTileRows, &full[s]);
+                        if (!q_resident)
+                            tma_load_2d(dst + (size_t)j * slab_bytes + kKeyStageBytes, &q_map,
+                                        (sl0 + j) * kSlabElems, 0, &full[s]);
+                    }
                 }
                 issued = it + 1;
             }
@@ -271,23 +284,35 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 const int acc = tl & 1, use = tl >> 1;
                 if (use >= 1 && !mbar_wait(&tempty[acc], (use - 1) & 1)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * NCOLS);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
                 for (int g = 0; g < gpt; ++g) {
                     const int it = tl * gpt + g;
                     const int s = it % n_stages;
                     if (!mbar_wait(&full[s], (it / n_stages) & 1)) { ok = false; break; }
                     tc_fence_after();
-                    const int sl0 = g * gs;
-                    const int nsl = min(gs, dslabs - sl0);
                     const uint32_t st_addr = smem_u32(stages + (size_t)s * stage_bytes);
-                    for (int j = 0; j < nsl; ++j) {
-                        const uint32_t a_addr = st_addr + (uint32_t)(j * slab_bytes);
-                        const uint32_t b_addr = q_resident ? smem_u32(qres + (size_t)(sl0 + j) * kQSlabBytes)
-                                                           : a_addr + kKeyStageBytes;
-                        const uint64_t a_desc = make_desc(a_addr), b_desc = make_desc(b_addr);
+                    if constexpr (TSUB > 1) {
+                        for (int sub = 0; sub < TSUB; ++sub)
+                            for (int j = 0; j < dslabs; ++j) {
+                                const uint64_t a_desc = make_desc(st_addr + (uint32_t)((sub * dslabs + j) * slab_bytes));
+                                const uint64_t b_desc = make_desc(smem_u32(qres + (size_t)j * kQSlabBytes));
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
-                            umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
+                                for (int k = 0; k < 4; ++k)
+                                    umma_f16(d_tmem + (uint32_t)(sub * NCOLS), a_desc + 2 * k, b_desc + 2 * k, idesc,
+                                             (j + k) != 0);
+                            }
+                    } else {
+                        const int sl0 = g * gs;
+                        const int nsl = min(gs, dslabs - sl0);
+                        for (int j = 0; j < nsl; ++j) {
+                            const uint32_t a_addr = st_addr + (uint32_t)(j * slab_bytes);
+                            const uint32_t b_addr = q_resident ? smem_u32(qres + (size_t)(sl0 + j) * kQSlabBytes)
+                                                               : a_addr + kKeyStageBytes;
+                            const uint64_t a_desc = make_desc(a_addr), b_desc = make_desc(b_addr);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
+                                umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
+                        }
                     }
                     tc_commit(&empty[s]);             // group reusable once these MMAs have read it
                 }
@@ -298,8 +323,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         }
     } else {
         // ---------------------------------- epilogue ----------------------------------
-        // Eight warps: warp w may read TMEM lanes 32*(w&3)..+31 (one key row per thread);
-        // the two warps that share a lane group split the accumulator columns in halves.
+        // Eight warps: warp w may read TMEM lanes 32*(w&3)..+31 (one key row per thread and
+        // sub-tile); the two warps that share a lane group split the accumulator columns.
         constexpr int CW = NCOLS / 2;                       // columns per warp
         constexpr int QW = CW / 2;                          // queries per warp
         const int ew = warp - 2;                            // 0..7
@@ -321,10 +346,13 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         EpiFlags *fl = &flags[0];
         for (int tl = 0; tl < my_tiles; ++tl) {
             const int acc = tl & 1, use = tl >> 1;
-            // this row's first stored token (filtered calls), requested before the wait
-            const long long row_pre =
-                (long long)(cta + tl * G) * a.tile_stride * kTileRows + lane_grp * 32 + lane;
-            const int tok = (filtered && row_pre < a.N) ? a.first_col[row_pre] : 0;
+            const long long row0 =
+                (long long)(cta + tl * G) * a.tile_stride * kRowsPerTile + lane_grp * 32 + lane;
+            // first stored token of this thread's rows (filtered calls), requested before the wait
+            int tok[TSUB];
+#pragma unroll
+            for (int sub = 0; sub < TSUB; ++sub)
+                tok[sub] = (filtered && row0 + sub * kTileRows < a.N) ? a.first_col[row0 + sub * kTileRows] : 0;
             if (!dead && !mbar_wait(&tfull[acc], use & 1)) {
                 report_timeout(a.status);
                 dead = true;
@@ -333,40 +361,44 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             tc_fence_after();
             // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
             if ((tl & 3) == 0 && et < a.B) tau[et] = peek_tau(&a.gtau[et], tau[et]);
-            const long long row =
-                (long long)(cta + tl * G) * a.tile_stride * kTileRows + lane_grp * 32 + lane;
-            const bool row_ok = !dead && row < a.N;
+            const uint32_t acc_addr = lane_addr + (uint32_t)(acc * kAccCols);
             if (a.probe_max) {
-                // Probe pass: no filtering and no lists -- only the best row of this tile per
-                // query (at most 32 tiles per CTA, so the bests fit the queue as they are).
-                // The n-th largest of all CTAs' tile bests is a valid filter: at least n rows
-                // reach it.
-                if (!dead) {
-                    uint32_t r[CW];
-                    tmem_ld_cols<CW>(lane_addr + (uint32_t)(acc * NCOLS), r);
-                    tmem_ld_wait();
-                    unsigned long long v[QW];
+                // Probe pass: no filtering and no lists -- only the best row of each sub-tile
+                // per query (at most 32 per CTA, so they fit the queue as they are).  The n-th
+                // largest of all CTAs' bests is a valid filter: at least n rows reach it.
 #pragma unroll
-                    for (int j = 0; j < QW; ++j) {
-                        const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
-                        const int w = want_s[qbase + j];
-                        const bool ok = row_ok && (w < 0 || tok == w) && s > -INFINITY;    // false for NaN too
-                        v[j] = ok ? pack_candidate(s, (uint32_t)row) : 0ull;
+                for (int sub = 0; sub < TSUB; ++sub) {
+                    const long long row = row0 + sub * kTileRows;
+                    const bool row_ok = row < a.N;
+                    unsigned long long *slot = tilemax + (size_t)(sub * 4 + lane_grp) * NQ + qbase;
+                    if (!dead) {
+                        uint32_t r[CW];
+                        tmem_ld_cols<CW>(acc_addr + (uint32_t)(sub * NCOLS), r);
+                        tmem_ld_wait();
+                        unsigned long long v[QW];
+#pragma unroll
+                        for (int j = 0; j < QW; ++j) {
+                            const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
+                            const int w = want_s[qbase + j];
+                            const bool ok = row_ok && (w < 0 || tok[sub] == w) && s > -INFINITY;   // false for NaN
+                            v[j] = ok ? pack_candidate(s, (uint32_t)row) : 0ull;
+                        }
+                        // per-query maximum over the warp's 32 rows: QW-1 exchanges for all queries
+                        WarpColumnMax<QW, 16>::run(v, lane);
+                        constexpr int kShift = QW == 32 ? 0 : QW == 16 ? 1 : QW == 8 ? 2 : 3;
+                        if ((lane & ((1 << kShift) - 1)) == 0) slot[lane >> kShift] = v[0];
+                    } else if (lane < QW) {
+                        slot[lane] = 0ull;
                     }
-                    // per-query maximum over the warp's 32 rows: QW-1 exchanges for all queries
-                    WarpColumnMax<QW, 16>::run(v, lane);
-                    constexpr int kShift = QW == 32 ? 0 : QW == 16 ? 1 : QW == 8 ? 2 : 3;
-                    if ((lane & ((1 << kShift) - 1)) == 0)
-                        tilemax[lane_grp * NQ + qbase + (lane >> kShift)] = v[0];
-                } else if (lane < QW) {
-                    tilemax[lane_grp * NQ + qbase + lane] = 0ull;
                 }
-                epi_bar();                                   // all four lane groups have written
+                epi_bar();                                   // all lane groups have written
                 for (int q = ew; q < a.B; q += kEpiWarps) {
                     if (lane == 0) {
-                        unsigned long long v = umax64(umax64(tilemax[q], tilemax[NQ + q]),
-                                                      umax64(tilemax[2 * NQ + q], tilemax[3 * NQ + q]));
-                        if (v && sel[q].count < kQueueCap) sel[q].queue[sel[q].count++] = v;
+                        for (int sub = 0; sub < TSUB; ++sub) {
+                            const unsigned long long *m = tilemax + (size_t)(sub * 4) * NQ + q;
+                            const unsigned long long v = umax64(umax64(m[0], m[NQ]), umax64(m[2 * NQ], m[3 * NQ]));
+                            if (v && sel[q].count < kQueueCap) sel[q].queue[sel[q].count++] = v;
+                        }
                     }
                 }
                 epi_bar();                                   // slots may be rewritten for the next tile
@@ -375,13 +407,19 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 if (lane == 0) mbar_arrive(&tempty[acc]);
                 continue;
             }
-            uint32_t pending = 0u;                          // queries whose candidate found the queue full
+            uint32_t pending[TSUB];                         // queries whose candidate found the queue full
+#pragma unroll
+            for (int sub = 0; sub < TSUB; ++sub) pending[sub] = 0u;
             bool first = true;
             while (true) {
-                // warp-uniform decision: tcgen05.ld needs the whole warp
-                if (!dead && (first || __any_sync(0xFFFFFFFFu, pending != 0u))) {
+#pragma unroll
+                for (int sub = 0; sub < TSUB; ++sub) {
+                    const long long row = row0 + sub * kTileRows;
+                    const bool row_ok = !dead && row < a.N;
+                    // warp-uniform decision: tcgen05.ld needs the whole warp
+                    if (dead || !(first || __any_sync(0xFFFFFFFFu, pending[sub] != 0u))) continue;
                     uint32_t r[CW];
-                    tmem_ld_cols<CW>(lane_addr + (uint32_t)(acc * NCOLS), r);
+                    tmem_ld_cols<CW>(acc_addr + (uint32_t)(sub * NCOLS), r);
                     tmem_ld_wait();
                     // Hot part, branch-free and compact: one bit per query whose score
                     // reaches the filter.
@@ -399,16 +437,17 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     }
                     if (filtered) {                         // Section 3.5: drafts must start with x_{t+1}
                         uint32_t match = wild;
+                        const int tk = tok[sub];
 #pragma unroll
                         for (int j4 = 0; j4 < QW / 4; ++j4) {
                             const int4 w = want4[j4];
-                            match |= (tok == w.x ? 1u : 0u) << (4 * j4) | (tok == w.y ? 2u : 0u) << (4 * j4) |
-                                     (tok == w.z ? 4u : 0u) << (4 * j4) | (tok == w.w ? 8u : 0u) << (4 * j4);
+                            match |= ((tk == w.x ? 1u : 0u) | (tk == w.y ? 2u : 0u) | (tk == w.z ? 4u : 0u) |
+                                      (tk == w.w ? 8u : 0u)) << (4 * j4);
                         }
                         mask &= match;
                     }
-                    mask &= first ? (row_ok ? 0xFFFFFFFFu : 0u) : pending;
-                    pending = 0u;
+                    mask &= first ? (row_ok ? 0xFFFFFFFFu : 0u) : pending[sub];
+                    pending[sub] = 0u;
                     // Cold part (rare once the filter is warm), kept out of the hot code:
                     // a warp-uniform loop over the queries that have a survivor in some
                     // lane; the two accumulator columns are re-read from TMEM.
@@ -417,7 +456,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         const int j = __ffs(wm) - 1;
                         wm &= wm - 1;
                         uint32_t v0, v1;
-                        tmem_ld2(lane_addr + (uint32_t)(acc * NCOLS + 2 * j), v0, v1);
+                        tmem_ld2(acc_addr + (uint32_t)(sub * NCOLS + 2 * j), v0, v1);
                         tmem_ld_wait();
                         if ((mask >> j) & 1u) {
                             const float s = fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
@@ -427,7 +466,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                                 sel[q].queue[slot] = pack_candidate(s, (uint32_t)row);
                                 if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
                             } else {
-                                pending |= 1u << j;
+                                pending[sub] |= 1u << j;
                                 fl->overflow = 1;
                             }
                         }
@@ -479,50 +518,84 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
 }
 
 struct Plan {
-    int ncols, stages, q_resident, gs;
+    int ncols, tsub, stages, q_resident, gs;
     size_t smem;
 };
+
+int ncols_of(int B) { return B <= 8 ? 16 : B <= 16 ? 32 : B <= 32 ? 64 : 128; }
+// Narrow rows (one or two 64-element slabs): several 128-row sub-tiles per tile so that a
+// pipeline stage is 32-64 KB and the per-tile barrier round trips are amortised.
+int tsub_of(int d, int ncols)
+{
+    const int dslabs = (d + kSlabElems - 1) / kSlabElems;
+    if (dslabs > 2) return 1;
+    int t = 4 / dslabs;                              // 4 slabs per stage
+    while (2 * t * ncols > 512) t >>= 1;             // two accumulator buffers in 512 TMEM columns
+    return t;
+}
 
 Plan make_plan(int d, int B)
 {
     Plan p{};
-    p.ncols = B <= 8 ? 16 : B <= 16 ? 32 : B <= 32 ? 64 : 128;
+    p.ncols = ncols_of(B);
+    p.tsub = tsub_of(d, p.ncols);
     const int dslabs = (d + kSlabElems - 1) / kSlabElems;
     const size_t qbytes = (size_t)dslabs * p.ncols * kSlabBytes;
     p.q_resident = qbytes <= (size_t)kResidentLimit;
     const size_t fixed = 1024 + (p.q_resident ? qbytes : 0) + sizeof(WarpTopN) * (p.ncols / 2) +
-                         (sizeof(float) + sizeof(int) + 4 * sizeof(unsigned long long)) * (p.ncols / 2) +
+                         (sizeof(float) + sizeof(int) + 4 * p.tsub * sizeof(unsigned long long)) * (p.ncols / 2) +
                          sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
     const size_t slab = kKeyStageBytes + (p.q_resident ? 0 : (size_t)p.ncols * kSlabBytes);
-    // Largest slab group (fewest barrier round trips per tile) that still leaves
-    // at least three groups in flight.
-    for (int gs = 4; gs >= 1; gs >>= 1) {
-        if (gs > dslabs && gs > 1) continue;
-        long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)(gs * slab);
-        if (s > kMaxStages) s = kMaxStages;
-        p.gs = gs;
-        p.stages = (int)s;
-        if (s >= 3) break;
+    if (p.tsub > 1) {
+        p.gs = p.tsub * dslabs;
+        long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)(p.gs * slab);
+        p.stages = (int)(s > kMaxStages ? kMaxStages : s);
+    } else {
+        // Largest slab group (fewest barrier round trips per tile) that still leaves
+        // at least three groups in flight.
+        for (int gs = 4; gs >= 1; gs >>= 1) {
+            if (gs > dslabs && gs > 1) continue;
+            long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)(gs * slab);
+            if (s > kMaxStages) s = kMaxStages;
+            p.gs = gs;
+            p.stages = (int)s;
+            if (s >= 3) break;
+        }
     }
     p.smem = fixed + (size_t)(p.stages > 0 ? p.stages : 0) * p.gs * slab;
     return p;
 }
 
-template <typename T, int NCOLS>
+template <typename T, int NCOLS, int TSUB>
 cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a, const Plan &p,
                        int grid, cudaStream_t stream)
 {
-    auto kernel = scan_umma_kernel<T, NCOLS>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
-    if (e != cudaSuccess) return e;
-    kernel<<<grid, kThreads, p.smem, stream>>>(kmap, qmap, a, p.q_resident, p.gs);
-    return cudaGetLastError();
+    if constexpr (2 * TSUB * NCOLS > 512) {
+        return cudaErrorInvalidValue;
+    } else {
+        auto kernel = scan_umma_kernel<T, NCOLS, TSUB>;
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
+        if (e != cudaSuccess) return e;
+        kernel<<<grid, kThreads, p.smem, stream>>>(kmap, qmap, a, p.q_resident, p.gs);
+        return cudaGetLastError();
+    }
+}
+
+template <typename T, int NCOLS>
+cudaError_t launch_tsub(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a, const Plan &p,
+                        int grid, cudaStream_t stream)
+{
+    switch (p.tsub) {
+    case 4: return launch_one<T, NCOLS, 4>(kmap, qmap, a, p, grid, stream);
+    case 2: return launch_one<T, NCOLS, 2>(kmap, qmap, a, p, grid, stream);
+    default: return launch_one<T, NCOLS, 1>(kmap, qmap, a, p, grid, stream);
+    }
 }
 
 }  // namespace
 
-int scan_umma_tile_rows() { return kTileRows; }
-int scan_umma_operand_rows(int B) { return B <= 8 ? 16 : B <= 16 ? 32 : B <= 32 ? 64 : 128; }
+int scan_umma_tile_rows(int d, int B) { return kTileRows * tsub_of(d, ncols_of(B)); }
+int scan_umma_operand_rows(int B) { return ncols_of(B); }
 
 cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a_in, int grid,
                              cudaStream_t stream)
@@ -534,8 +607,8 @@ cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, c
     a.stages = p.stages;
     const bool h = a.dtype == kF16;
 #define DRESD_GO(N_)                                                                          \
-    return h ? launch_one<__half, N_>(kmap, qmap, a, p, grid, stream)                         \
-             : launch_one<__nv_bfloat16, N_>(kmap, qmap, a, p, grid, stream)
+    return h ? launch_tsub<__half, N_>(kmap, qmap, a, p, grid, stream)                        \
+             : launch_tsub<__nv_bfloat16, N_>(kmap, qmap, a, p, grid, stream)
     switch (p.ncols) {
     case 16: DRESD_GO(16);
     case 32: DRESD_GO(32);
