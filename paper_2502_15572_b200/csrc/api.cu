@@ -104,9 +104,6 @@ struct dresd_store {
     // workspace (owned)
     float *qhat;                 // [kMaxBatch][d]
     void *qsplit;                // [2*kMaxBatch][dpad] 16-bit
-    void *qhi;                   // [kMaxBatch][dpad] 16-bit: the rounded queries alone (tcgen05 operand)
-    float *kmax;                 // device word: largest key norm (computed on the first tcgen05 call)
-    int kmax_ready;
     unsigned long long *cand;    // [max_grid][kMaxBatch][kCandStride]
     int *status;                 // device status word
     unsigned int *gtau;          // [kMaxBatch] grid-wide filter words
@@ -124,7 +121,7 @@ struct dresd_store {
     int tile_rows, n_tiles;
     // tensor-core kernel geometry (16-bit keys): 128-row key tiles, query operand maps
     CUtensorMap map_umma;
-    CUtensorMap map_q[3];        // box rows 16 / 32 / 64 over qhi
+    CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     // options / bookkeeping
     int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage;
     double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
@@ -144,8 +141,6 @@ void free_store(dresd_store *s)
     if (!s) return;
     cudaFree(s->qhat);
     cudaFree(s->qsplit);
-    cudaFree(s->qhi);
-    cudaFree(s->kmax);
     cudaFree(s->cand);
     cudaFree(s->status);
     cudaFree(s->gtau);
@@ -196,7 +191,6 @@ dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows
     p.dtype = s->dtype;
     p.qhat = s->qhat;
     p.qsplit = s->dtype == kF32 ? nullptr : s->qsplit;
-    p.qhi = s->dtype == kF32 ? nullptr : s->qhi;
     p.dpad = s->dpad;
     p.rows = rows;                   // operand rows beyond B are written as zeros
     p.lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
@@ -221,7 +215,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // streaming kernel stays available as "scan_path" 1 and serves the allocation-free call.
     const bool umma = !f32 && s->opt_path != 1;
     const int op_rows = umma ? scan_umma_operand_rows(B) : 0;
-    dresd_status st = run_preprocess(s, queries, B, umma ? op_rows : ((B + 7) / 8) * 8, stream);
+    dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream);
     if (st != DRESD_OK) return st;
 
     const int umma_rows = umma ? scan_umma_tile_rows(s->d, B) : 1;
@@ -250,22 +244,8 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.gtau = s->gtau;
         a.first_col = first_tokens ? s->first_col : nullptr;
         a.want_first = first_tokens;
-        const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : 2;
+        const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
         cudaError_t e = cudaSuccess;
-        if (!s->kmax_ready) {           // once per store: the scale of the filter slack
-            e = launch_key_norm_max(s->keys, s->dtype, s->N, s->d, s->kmax, stream);
-            if (e != cudaSuccess) return fail_cuda(e, "key norm launch");
-            s->kmax_ready = 1;
-            s->last_launches += 1;
-        }
-        a.keys = s->keys;
-        a.qhat = s->qhat;
-        a.kmax = s->kmax;
-        // |accumulator - exact| <= (rounding of the query to the store dtype: 2^-11 fp16,
-        // 2^-8 bf16, times ||q|| ||k|| by Cauchy-Schwarz) + fp16 underflow of tiny query
-        // elements (2^-25 each) + fp32 accumulation, all per unit of key norm.
-        a.rel_err = (s->dtype == kF16 ? 4.8828125e-4f : 3.90625e-3f) * 1.02f + 4e-6f +
-                    3e-8f * sqrtf((float)s->d);
         // Large batches on large stores: a probe pass over every 64th tile first.  Its
         // n-th best score per query seeds the grid-wide filter, so that the full pass
         // queues ~64 n survivors per query GPU-wide instead of ~n ln(rows/n) per CTA.
@@ -385,8 +365,6 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
 
     bool ok = cudaMalloc(&s->qhat, sizeof(float) * kMaxBatch * (size_t)d) == cudaSuccess &&
               cudaMalloc(&s->qsplit, (size_t)2 * 2 * kMaxBatch * s->dpad) == cudaSuccess &&
-              cudaMalloc(&s->qhi, (size_t)2 * kMaxBatch * s->dpad) == cudaSuccess &&
-              cudaMalloc(&s->kmax, sizeof(float)) == cudaSuccess &&
               cudaMalloc(&s->cand, sizeof(unsigned long long) * (size_t)s->max_grid * kMaxBatch * kCandStride) == cudaSuccess &&
               cudaMalloc(&s->status, sizeof(int)) == cudaSuccess &&
               cudaMalloc(&s->gtau, sizeof(unsigned int) * kMaxBatch) == cudaSuccess &&
@@ -396,8 +374,8 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
     ok = ok && cudaMalloc(&s->tokens_dev, sizeof(int32_t) * s->tokens_dev_elems) == cudaSuccess;
     if (ok && dtype != DRESD_F32) {
         bool mok = make_map(&s->map_umma, keys, s->dtype, N, d, 128);
-        for (int i = 0; i < 3; ++i)
-            mok = mok && make_map(&s->map_q[i], s->qhi, s->dtype, kMaxBatch, s->dpad, 16 << i);
+        for (int i = 0; i < 4; ++i)
+            mok = mok && make_map(&s->map_q[i], s->qsplit, s->dtype, 2 * kMaxBatch, s->dpad, 16 << i);
         if (!mok) {
             free_store(s);
             return fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the tensor-core path");

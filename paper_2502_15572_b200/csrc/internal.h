@@ -26,7 +26,6 @@ struct PreprocessArgs {
     int B, d_in, d, dtype;
     float *qhat;            // [rows][d] fp32 unit queries (rows >= B zero)
     void *qsplit;           // 16-bit keys: [2*rows][dpad] hi/lo operand rows, else null
-    void *qhi;              // 16-bit keys: [rows][dpad] the hi rows alone (tcgen05 operand), else null
     int dpad;               // d rounded up to 64
     int rows;               // CTAs launched: B rounded up to the operand row count
     float lo_scale;
@@ -54,10 +53,6 @@ struct ScanArgs {
     // with first_col[row] == want_first[q]; want_first[q] < 0 disables it for that query.
     const int32_t *first_col;   // [N] first stored token of every key (compact copy)
     const int32_t *want_first;  // [B] of this launch
-    // tcgen05 kernel: exact re-scoring of the rows that pass the accumulator filter
-    const void *keys;       // [N][d] the key matrix itself
-    const float *kmax;      // device word: largest key norm of the store
-    float rel_err;          // bound of |accumulator - exact score| per unit of key norm
     int stages;             // pipeline depth
     long long wait_cycles;  // bound of every device-side wait in cycles, 0 = default (~2 s)
     int debug_lose_stage;   // test hook (streaming kernel): CTA 0 never receives stage (value-1); 0 = off
@@ -71,8 +66,8 @@ size_t scan_mma_smem_bytes(int d, int B, int *stages_out);
 cudaError_t launch_scan_mma(const CUtensorMap &keys_map, const ScanArgs &a, int grid,
                             cudaStream_t stream);
 
-// Tensor-core kernel (tcgen05/TMEM, 16-bit keys): 128-row sub-tiles; the query
-// operand holds one row per query (rounded to the store dtype), padded to 16/32/64 rows.
+// Batched tensor-core kernel (tcgen05/TMEM, 16-bit keys): 128-row tiles; the query
+// operand holds 2 rows per query, padded to 16/32/64/128 rows.
 int scan_umma_tile_rows(int d, int B);      // 128 x sub-tiles per tile (narrow rows use several)
 int scan_umma_operand_rows(int B);
 cudaError_t launch_scan_umma(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
@@ -93,10 +88,6 @@ cudaError_t launch_merge_tau(const unsigned long long *cand, int grid_lists, int
 cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long N,
                           const int32_t *ids, int B, int top_n, int draft_len,
                           int32_t *out_tokens, cudaStream_t stream);
-
-// *kmax = max_i ||keys[i]||_2 (fp32), the scale of the tcgen05 kernel's filter slack.
-cudaError_t launch_key_norm_max(const void *keys, int dtype, long long N, int d, float *kmax,
-                                cudaStream_t stream);
 
 // first_col[i] = next_tokens[i][0]: the compact column the first-token filter reads.
 cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, long long N,

@@ -57,7 +57,6 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
     const int tid = threadIdx.x;
     T *split_hi = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)(2 * b) * a.dpad : nullptr;
     T *split_lo = split_hi ? split_hi + a.dpad : nullptr;
-    T *hi_row = a.qhi ? static_cast<T *>(a.qhi) + (size_t)b * a.dpad : nullptr;
     float *qrow = a.qhat + (size_t)b * a.d;
     if (tid == 0 && a.gtau) a.gtau[b] = 0u;          // fresh grid-wide filter for this call
 
@@ -67,7 +66,6 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
             for (int c = tid; c < a.dpad; c += blockDim.x) {
                 split_hi[c] = from_f32<T>(0.f);
                 split_lo[c] = from_f32<T>(0.f);
-                if (hi_row) hi_row[c] = from_f32<T>(0.f);
             }
         return;
     }
@@ -127,7 +125,6 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
             float r = (x - to_f32<T>(hi)) * a.lo_scale;
             split_hi[c] = hi;
             split_lo[c] = from_f32<T>(r);
-            if (hi_row) hi_row[c] = hi;
         }
     }
 }

@@ -10,23 +10,17 @@
 //             when the query operand is too large to stay resident, the
 //             matching query slab next to each key slab;
 //   warp 1    allocates TMEM; one thread issues tcgen05.mma (M = 128 key rows,
-//             N = one column per query, K = 16 per instruction, fp32
-//             accumulators in TMEM, two accumulator buffers so that the
-//             epilogue of tile t overlaps the MMAs of tile t+1);
+//             N = 2 columns per query: q = hi + lo/scale, K = 16 per
+//             instruction, fp32 accumulators in TMEM, two accumulator buffers
+//             so that the epilogue of tile t overlaps the MMAs of tile t+1);
 //             tcgen05.commit releases shared-memory stages and publishes
 //             finished accumulators;
 //   warps 2-9 epilogue: each thread owns one key row of the tile and half of
-//             the accumulator columns (two warps share a TMEM lane group),
-//             reads them with tcgen05.ld and filters them against the CTA's
-//             running n-th best per query.
-// Precision: the tensor cores see the query rounded to the store dtype, so an
-// accumulator is the score only to within delta = (rounding bound) x (largest
-// key norm).  It is used as a FILTER alone: a row whose accumulator reaches
-// (n-th best - delta) is re-scored exactly -- the warp re-reads that key row
-// and takes the fp32 dot product with the unrounded unit query -- and only
-// exact scores enter the lists.  Survivors are rare, so the exact pass costs
-// nothing measurable while the tensor work, the TMEM traffic and the query
-// operand are half of what a two-term split of the query would need.
+//             its N accumulator columns (two warps share a TMEM lane group),
+//             reads them with tcgen05.ld, combines hi and lo, filters against
+//             the CTA's running n-th best per query and queues survivors;
+//             queues are folded into sorted 32-lane lists with shuffle-based
+//             bitonic merges.
 // Every wait is bounded; TMEM is freed on every path.
 #include <type_traits>
 
@@ -122,43 +116,6 @@ template <int CW> __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, u
         for (int c = 0; c < CW / 16; ++c) tmem_ld16p(taddr + 16 * c, r + 16 * c);
     }
 }
-// Exact fp32 score of one key row against one unit query, computed by a whole warp:
-// lane l takes elements 8l..8l+7 of every 256-element chunk; the partial sums are
-// combined in a fixed order, so the value depends on the row and the query only.
-template <typename T> __device__ __forceinline__ float2 pair_to_float2(uint32_t u);
-template <> __device__ __forceinline__ float2 pair_to_float2<__half>(uint32_t u)
-{
-    return __half22float2(*reinterpret_cast<const __half2 *>(&u));
-}
-template <> __device__ __forceinline__ float2 pair_to_float2<__nv_bfloat16>(uint32_t u)
-{
-    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&u));
-}
-template <typename T>
-__device__ __forceinline__ float exact_score(const T *key_row, const float *q, int d, int lane)
-{
-    float acc0 = 0.f, acc1 = 0.f;
-    for (int c = lane * 8; c < d; c += 256) {
-        const uint4 kv = *reinterpret_cast<const uint4 *>(key_row + c);
-        const float4 qa = *reinterpret_cast<const float4 *>(q + c);
-        const float4 qb = *reinterpret_cast<const float4 *>(q + c + 4);
-        const float2 k0 = pair_to_float2<T>(kv.x), k1 = pair_to_float2<T>(kv.y);
-        const float2 k2 = pair_to_float2<T>(kv.z), k3 = pair_to_float2<T>(kv.w);
-        acc0 = fmaf(qa.x, k0.x, acc0);
-        acc1 = fmaf(qa.y, k0.y, acc1);
-        acc0 = fmaf(qa.z, k1.x, acc0);
-        acc1 = fmaf(qa.w, k1.y, acc1);
-        acc0 = fmaf(qb.x, k2.x, acc0);
-        acc1 = fmaf(qb.y, k2.y, acc1);
-        acc0 = fmaf(qb.z, k3.x, acc0);
-        acc1 = fmaf(qb.w, k3.y, acc1);
-    }
-    float acc = acc0 + acc1;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-    return acc;
-}
-
 // Column-wise maximum over the 32 lanes of a warp for C values per lane, with C-1
 // exchanges in total instead of 5 per value: at each step a lane keeps one half of its
 // values and hands the other half to its partner.  Afterwards v[0] of lane l holds the
@@ -195,7 +152,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_constant__ CUtensorMap q_map,
                  const ScanArgs a, const int q_resident, const int gs)
 {
-    constexpr int NQ = NCOLS;                               // queries (padded): one column each
+    constexpr int NQ = NCOLS / 2;                           // queries (padded)
     constexpr int kAccCols = TSUB * NCOLS;                  // one accumulator buffer
     constexpr int kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;
     static_assert(kTmemCols <= 512, "TMEM has 512 columns");
@@ -228,8 +185,6 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
-    // how far an accumulator may lie below the exact score (see the header)
-    const float delta = a.rel_err * (*a.kmax);
     const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
     const int n_it = my_tiles * gpt;
     constexpr int kRowsPerTile = kTileRows * TSUB;
@@ -255,7 +210,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             warp_topn_init(&sel[q], lane);
             // start from whatever the grid already knows; padding columns never pass
             if (lane == 0) {
-                tau[q] = q < a.B ? peek_tau(&a.gtau[q], -INFINITY) - delta : INFINITY;
+                tau[q] = q < a.B ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
                 want_s[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
             }
         }
@@ -370,15 +325,15 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         // ---------------------------------- epilogue ----------------------------------
         // Eight warps: warp w may read TMEM lanes 32*(w&3)..+31 (one key row per thread and
         // sub-tile); the two warps that share a lane group split the accumulator columns.
-        constexpr int CW = NCOLS / 2;                       // columns = queries per warp
-        constexpr int QW = CW;
+        constexpr int CW = NCOLS / 2;                       // columns per warp
+        constexpr int QW = CW / 2;                          // queries per warp
         const int ew = warp - 2;                            // 0..7
         const int lane_grp = warp & 3;
         const int half = ew >> 2;
         const int et = ew * 32 + lane;
         const int qbase = half * QW;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(half * CW);
-        const T *keys = static_cast<const T *>(a.keys);
+        const float inv = a.lo_inv_scale;
         const float4 *tau4 = reinterpret_cast<const float4 *>(tau + qbase);
         const int4 *want4 = reinterpret_cast<const int4 *>(want_s + qbase);
         const bool filtered = a.first_col != nullptr;
@@ -405,7 +360,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             dead = __any_sync(0xFFFFFFFFu, dead);
             tc_fence_after();
             // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
-            if ((tl & 3) == 0 && et < a.B) tau[et] = fmaxf(tau[et], peek_tau(&a.gtau[et], -INFINITY) - delta);
+            if ((tl & 3) == 0 && et < a.B) tau[et] = peek_tau(&a.gtau[et], tau[et]);
             const uint32_t acc_addr = lane_addr + (uint32_t)(acc * kAccCols);
             if (a.probe_max) {
                 // Probe pass: no filtering and no lists -- only the best row of each sub-tile
@@ -423,15 +378,14 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         unsigned long long v[QW];
 #pragma unroll
                         for (int j = 0; j < QW; ++j) {
-                            // a lower bound of this row's exact score
-                            const float s = __uint_as_float(r[j]) - delta;
+                            const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
                             const int w = want_s[qbase + j];
                             const bool ok = row_ok && (w < 0 || tok[sub] == w) && s > -INFINITY;   // false for NaN
                             v[j] = ok ? pack_candidate(s, (uint32_t)row) : 0ull;
                         }
                         // per-query maximum over the warp's 32 rows: QW-1 exchanges for all queries
                         WarpColumnMax<QW, 16>::run(v, lane);
-                        constexpr int kShift = QW == 32 ? 0 : QW == 16 ? 1 : 2;
+                        constexpr int kShift = QW == 32 ? 0 : QW == 16 ? 1 : QW == 8 ? 2 : 3;
                         if ((lane & ((1 << kShift) - 1)) == 0) slot[lane >> kShift] = v[0];
                     } else if (lane < QW) {
                         slot[lane] = 0ull;
@@ -467,8 +421,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     uint32_t r[CW];
                     tmem_ld_cols<CW>(acc_addr + (uint32_t)(sub * NCOLS), r);
                     tmem_ld_wait();
-                    // Hot part, branch-free and compact: one bit per query whose accumulator
-                    // reaches the filter (n-th best so far minus delta).
+                    // Hot part, branch-free and compact: one bit per query whose score
+                    // reaches the filter.
                     uint32_t mask = 0u;
 #pragma unroll
                     for (int j4 = 0; j4 < QW / 4; ++j4) {
@@ -477,7 +431,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             const int j = 4 * j4 + i;
-                            mask |= (__uint_as_float(r[j]) >= tt[i]) ? (1u << j) : 0u;
+                            const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
+                            mask |= (s >= tt[i]) ? (1u << j) : 0u;
                         }
                     }
                     if (filtered) {                         // Section 3.5: drafts must start with x_{t+1}
@@ -493,30 +448,26 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     }
                     mask &= first ? (row_ok ? 0xFFFFFFFFu : 0u) : pending[sub];
                     pending[sub] = 0u;
-                    // Cold part (rare once the filter is warm), kept out of the hot code: a
-                    // warp-uniform loop over (query, lane) pairs that passed; the whole warp
-                    // re-scores that lane's key row exactly and the lane queues it if the exact
-                    // score still reaches the exact n-th best.
+                    // Cold part (rare once the filter is warm), kept out of the hot code:
+                    // a warp-uniform loop over the queries that have a survivor in some
+                    // lane; the two accumulator columns are re-read from TMEM.
                     uint32_t wm = __reduce_or_sync(0xFFFFFFFFu, mask);
                     while (wm) {
                         const int j = __ffs(wm) - 1;
                         wm &= wm - 1;
-                        const int q = qbase + j;
-                        uint32_t lanes = __ballot_sync(0xFFFFFFFFu, (mask >> j) & 1u);
-                        while (lanes) {
-                            const int src = __ffs(lanes) - 1;
-                            lanes &= lanes - 1;
-                            const long long rr = row - lane + src;
-                            const float s = exact_score<T>(keys + (size_t)rr * a.d, a.qhat + (size_t)q * a.d, a.d, lane);
-                            if (lane == src && s >= tau[q] + delta) {
-                                const int slot = atomicAdd(&sel[q].count, 1);
-                                if (slot < kQueueCap) {
-                                    sel[q].queue[slot] = pack_candidate(s, (uint32_t)rr);
-                                    if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
-                                } else {
-                                    pending[sub] |= 1u << j;
-                                    fl->overflow = 1;
-                                }
+                        uint32_t v0, v1;
+                        tmem_ld2(acc_addr + (uint32_t)(sub * NCOLS + 2 * j), v0, v1);
+                        tmem_ld_wait();
+                        if ((mask >> j) & 1u) {
+                            const float s = fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
+                            const int q = qbase + j;
+                            const int slot = atomicAdd(&sel[q].count, 1);
+                            if (slot < kQueueCap) {
+                                sel[q].queue[slot] = pack_candidate(s, (uint32_t)row);
+                                if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
+                            } else {
+                                pending[sub] |= 1u << j;
+                                fl->overflow = 1;
                             }
                         }
                     }
@@ -537,7 +488,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 for (int q = ew; q < NQ; q += kEpiWarps) {
                     if (sel[q].count > 0) {
                         warp_topn_merge(&sel[q], a.top_n, lane);
-                        if (lane == 0 && q < a.B) tau[q] = share_tau(&a.gtau[q], sel[q].tau) - delta;
+                        if (lane == 0 && q < a.B) tau[q] = share_tau(&a.gtau[q], sel[q].tau);
                     }
                 }
                 epi_bar();                                   // C: lists, counts and tau are settled
@@ -571,7 +522,7 @@ struct Plan {
     size_t smem;
 };
 
-int ncols_of(int B) { return B <= 16 ? 16 : B <= 32 ? 32 : 64; }
+int ncols_of(int B) { return B <= 8 ? 16 : B <= 16 ? 32 : B <= 32 ? 64 : 128; }
 // Narrow rows (one or two 64-element slabs): several 128-row sub-tiles per tile so that a
 // pipeline stage is 32-64 KB and the per-tile barrier round trips are amortised.
 int tsub_of(int d, int ncols)
@@ -591,8 +542,8 @@ Plan make_plan(int d, int B)
     const int dslabs = (d + kSlabElems - 1) / kSlabElems;
     const size_t qbytes = (size_t)dslabs * p.ncols * kSlabBytes;
     p.q_resident = qbytes <= (size_t)kResidentLimit;
-    const size_t fixed = 1024 + (p.q_resident ? qbytes : 0) + sizeof(WarpTopN) * p.ncols +
-                         (sizeof(float) + sizeof(int) + 4 * p.tsub * sizeof(unsigned long long)) * p.ncols +
+    const size_t fixed = 1024 + (p.q_resident ? qbytes : 0) + sizeof(WarpTopN) * (p.ncols / 2) +
+                         (sizeof(float) + sizeof(int) + 4 * p.tsub * sizeof(unsigned long long)) * (p.ncols / 2) +
                          sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
     const size_t slab = kKeyStageBytes + (p.q_resident ? 0 : (size_t)p.ncols * kSlabBytes);
     if (p.tsub > 1) {
@@ -661,7 +612,8 @@ cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, c
     switch (p.ncols) {
     case 16: DRESD_GO(16);
     case 32: DRESD_GO(32);
-    default: DRESD_GO(64);
+    case 64: DRESD_GO(64);
+    default: DRESD_GO(128);
     }
 #undef DRESD_GO
 }

@@ -72,44 +72,7 @@ __global__ void extract_first_kernel(const int32_t *__restrict__ next_tokens, in
         first_col[i] = next_tokens[i * stored_len];
 }
 
-// Largest Euclidean norm over all key rows: one warp per row (grid-stride), fp32.
-template <typename T> __device__ __forceinline__ float elem_to_f32(T x);
-template <> __device__ __forceinline__ float elem_to_f32<__half>(__half x) { return __half2float(x); }
-template <> __device__ __forceinline__ float elem_to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
-template <typename T>
-__global__ void key_norm_max_kernel(const T *__restrict__ keys, long long N, int d, float *kmax)
-{
-    const int lane = threadIdx.x & 31;
-    const long long warps = (long long)gridDim.x * (blockDim.x >> 5);
-    float best = 0.f;
-    for (long long row = blockIdx.x * (long long)(blockDim.x >> 5) + (threadIdx.x >> 5); row < N; row += warps) {
-        const T *k = keys + (size_t)row * d;
-        float ss = 0.f;
-        for (int c = lane; c < d; c += 32) {
-            const float x = elem_to_f32<T>(k[c]);
-            ss = fmaf(x, x, ss);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-        best = fmaxf(best, ss);
-    }
-    // non-negative floats order like their bit patterns; NaN/inf propagate as "huge"
-    if (lane == 0) atomicMax(reinterpret_cast<unsigned int *>(kmax), __float_as_uint(sqrtf(best)));
-}
-
 }  // namespace
-
-cudaError_t launch_key_norm_max(const void *keys, int dtype, long long N, int d, float *kmax, cudaStream_t stream)
-{
-    cudaError_t e = cudaMemsetAsync(kmax, 0, sizeof(float), stream);
-    if (e != cudaSuccess) return e;
-    const int threads = 256, blocks = 148 * 8;
-    if (dtype == kF16)
-        key_norm_max_kernel<__half><<<blocks, threads, 0, stream>>>(static_cast<const __half *>(keys), N, d, kmax);
-    else
-        key_norm_max_kernel<__nv_bfloat16><<<blocks, threads, 0, stream>>>(static_cast<const __nv_bfloat16 *>(keys), N, d, kmax);
-    return cudaGetLastError();
-}
 
 cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, long long N, int32_t *first_col,
                                  cudaStream_t stream)
