@@ -128,6 +128,36 @@ dresd_status dresd_retrieve_filtered(dresd_store *store, const void *queries, co
                                      int32_t *out_tokens, void *stream);
 
 /*
+ * Token-level half of batch verification, Section 3.6 and Fig. 3 (no LLM involved).
+ *
+ * dresd_drafts_prepare() turns the gathered continuations into the n x L draft
+ * matrix that is sent for verification:
+ *   tokens      device, int32 [B][n][L]  (out_tokens of dresd_retrieve, draft_len = L)
+ *   ids         device, int32 [B][n]     (out_ids; -1 = missing neighbour)
+ *   out_drafts  device, int32 [B][n][L]: every token after a draft's first eos_id is
+ *               eos_id (the EOS id is the padding); a missing neighbour is all eos_id
+ *   out_valid   device, int32 [B][n]: 0 for a missing neighbour and for a draft equal
+ *               (after padding) to a better-ranked draft of the same query, else 1.
+ *
+ * dresd_drafts_accept() accepts the longest draft that exactly matches the LLM:
+ *   llm_tokens  device, int32 [B][n][L+1]: llm_tokens[b][r][t] is the LLM's own token
+ *               at the position of drafts[b][r][t] given the context and the draft's
+ *               first t tokens (t = L: the token after the whole draft)
+ *   out_best    device, int32 [B]: the valid draft with the longest matching prefix
+ *               (ties to the better-ranked one), -1 when no draft is valid
+ *   out_len     device, int32 [B]: accepted tokens = matched prefix length + 1
+ *   out_tokens  device, int32 [B][L+1]: the matched prefix, then the LLM's token at
+ *               the first mismatch (so every step yields at least one token,
+ *               Section 3.1), then -1.
+ * n <= DRESD_MAX_TOP_N; n * L <= 12288.  Asynchronous on `stream`.
+ */
+dresd_status dresd_drafts_prepare(const int32_t *tokens, const int32_t *ids, int B, int n, int L,
+                                  int32_t eos_id, int32_t *out_drafts, int32_t *out_valid, void *stream);
+dresd_status dresd_drafts_accept(const int32_t *drafts, const int32_t *valid, const int32_t *llm_tokens,
+                                 int B, int n, int L, int32_t *out_best, int32_t *out_len,
+                                 int32_t *out_tokens, void *stream);
+
+/*
  * The same call for callers whose queries and results live in HOST memory
  * (ideally pinned): copies the queries to the device, runs dresd_retrieve(),
  * copies the three results back and waits for `stream`.  The datastore itself

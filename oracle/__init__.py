@@ -10,4 +10,6 @@ from .dresd_oracle import (  # noqa: F401
     scores,
     retrieve,
     OracleResult,
+    drafts_prepare,
+    drafts_accept,
 )

@@ -224,3 +224,63 @@ done:
     free(order);
     return rc;
 }
+
+/* ---- token-level half of batch verification (Section 3.6, Fig. 3) ----------
+ * prepare: tokens [B][n][L], ids [B][n] (-1 = missing neighbour).  drafts [B][n][L]:
+ * after a draft's first EOS every token is EOS (the EOS id is the padding); a missing
+ * neighbour is all EOS.  valid [B][n]: 0 for a missing neighbour and for a draft equal
+ * to a better-ranked (lower r) present draft, else 1.                               */
+int dresd_oracle_drafts_prepare(const int32_t *tokens, const int32_t *ids, int B, int n, int L,
+                                int32_t eos, int32_t *drafts, int32_t *valid)
+{
+    if (B < 0 || n < 1 || L < 1) return -1;
+    for (int b = 0; b < B; ++b)
+        for (int r = 0; r < n; ++r) {
+            const size_t row = ((size_t)b * n + r) * L;
+            int present = ids[(size_t)b * n + r] >= 0;
+            int ended = !present;
+            for (int t = 0; t < L; ++t) {
+                int32_t x = ended ? eos : tokens[row + t];
+                drafts[row + t] = x;
+                if (x == eos) ended = 1;
+            }
+            int ok = present;
+            for (int p = 0; p < r && ok; ++p) {
+                if (ids[(size_t)b * n + p] < 0) continue;
+                if (memcmp(drafts + ((size_t)b * n + p) * L, drafts + row, sizeof(int32_t) * (size_t)L) == 0) ok = 0;
+            }
+            valid[(size_t)b * n + r] = ok;
+        }
+    return 0;
+}
+
+/* accept: llm [B][n][L+1] = the LLM's own token at each draft position (and after the
+ * draft).  The valid draft with the longest exactly matching prefix wins (ties to the
+ * lower r); out_tokens [B][L+1] = that prefix, then the LLM's token at the first
+ * mismatch, then -1; out_len = prefix length + 1; out_best = -1 when no draft is valid
+ * (then the single token is the LLM's own next token, llm[b][0][0]).                 */
+int dresd_oracle_drafts_accept(const int32_t *drafts, const int32_t *valid, const int32_t *llm, int B, int n,
+                               int L, int32_t *out_best, int32_t *out_len, int32_t *out_tokens)
+{
+    if (B < 0 || n < 1 || L < 1) return -1;
+    for (int b = 0; b < B; ++b) {
+        int best = -1, best_len = -1;
+        for (int r = 0; r < n; ++r) {
+            if (!valid[(size_t)b * n + r]) continue;
+            int a = 0;
+            while (a < L && drafts[((size_t)b * n + r) * L + a] == llm[((size_t)b * n + r) * (L + 1) + a]) ++a;
+            if (a > best_len) { best_len = a; best = r; }
+        }
+        int len = best >= 0 ? best_len : 0;
+        int src = best >= 0 ? best : 0;
+        out_best[b] = best;
+        out_len[b] = len + 1;
+        for (int t = 0; t <= L; ++t) {
+            int32_t x = -1;
+            if (t < len) x = drafts[((size_t)b * n + src) * L + t];
+            else if (t == len) x = llm[((size_t)b * n + src) * (L + 1) + t];
+            out_tokens[(size_t)b * (L + 1) + t] = x;
+        }
+    }
+    return 0;
+}

@@ -171,3 +171,38 @@ def retrieve(keys, next_tokens, dtype: str, queries, top_n: int, draft_len: int,
     if rc != 0:
         raise ValueError("oracle retrieve: bad arguments")
     return OracleResult(ids, sc, tok, full)
+
+
+def drafts_prepare(tokens, ids, eos_id: int):
+    """Section 3.6 / Fig. 3: EOS-padded n x L draft matrices and their validity flags."""
+    tok = np.ascontiguousarray(tokens, dtype=np.int32)
+    idx = np.ascontiguousarray(ids, dtype=np.int32)
+    B, n, L = tok.shape
+    drafts = np.empty_like(tok)
+    valid = np.empty((B, n), dtype=np.int32)
+    lib = _load()
+    lib.dresd_oracle_drafts_prepare.restype = ctypes.c_int
+    lib.dresd_oracle_drafts_prepare.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                                ctypes.c_int, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+    if lib.dresd_oracle_drafts_prepare(_ptr(tok), _ptr(idx), B, n, L, eos_id, _ptr(drafts), _ptr(valid)) != 0:
+        raise ValueError("oracle drafts_prepare: bad arguments")
+    return drafts, valid
+
+
+def drafts_accept(drafts, valid, llm_tokens):
+    """Section 3.6: longest exactly matching draft prefix plus the LLM's own next token."""
+    d = np.ascontiguousarray(drafts, dtype=np.int32)
+    v = np.ascontiguousarray(valid, dtype=np.int32)
+    m = np.ascontiguousarray(llm_tokens, dtype=np.int32)
+    B, n, L = d.shape
+    if m.shape != (B, n, L + 1):
+        raise ValueError("llm_tokens must be [B][n][L+1]")
+    best = np.empty(B, dtype=np.int32)
+    length = np.empty(B, dtype=np.int32)
+    out = np.empty((B, L + 1), dtype=np.int32)
+    lib = _load()
+    lib.dresd_oracle_drafts_accept.restype = ctypes.c_int
+    lib.dresd_oracle_drafts_accept.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int] * 3 + [ctypes.c_void_p] * 3
+    if lib.dresd_oracle_drafts_accept(_ptr(d), _ptr(v), _ptr(m), B, n, L, _ptr(best), _ptr(length), _ptr(out)) != 0:
+        raise ValueError("oracle drafts_accept: bad arguments")
+    return best, length, out

@@ -28,7 +28,7 @@ EXPORTS = (
     "dresd_store_profile_read", "dresd_store_last_launches", "dresd_store_last_key_passes",
     "dresd_last_error",
     "dresd_store_destroy", "dresd_retrieve_noalloc", "dresd_store_enable_first_token_filter",
-    "dresd_retrieve_filtered",
+    "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
 )
 
 
@@ -82,6 +82,10 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_store_enable_first_token_filter.argtypes = [vp, vp]
     lib.dresd_retrieve_filtered.restype = i32
     lib.dresd_retrieve_filtered.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.dresd_drafts_prepare.restype = i32
+    lib.dresd_drafts_prepare.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp]
+    lib.dresd_drafts_accept.restype = i32
+    lib.dresd_drafts_accept.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_retrieve_noalloc.restype = i32
     lib.dresd_retrieve_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
     if path is None:
@@ -125,6 +129,17 @@ def dresd_retrieve_filtered(store: int, queries_ptr: int, first_tokens_ptr, B: i
                             out_ids_ptr: int, out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
     _check(load().dresd_retrieve_filtered(store, queries_ptr, first_tokens_ptr, B, top_n, draft_len,
                                           out_ids_ptr, out_scores_ptr, out_tokens_ptr, stream))
+
+
+def dresd_drafts_prepare(tokens_ptr: int, ids_ptr: int, B: int, n: int, L: int, eos_id: int,
+                         out_drafts_ptr: int, out_valid_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_drafts_prepare(tokens_ptr, ids_ptr, B, n, L, eos_id, out_drafts_ptr, out_valid_ptr, stream))
+
+
+def dresd_drafts_accept(drafts_ptr: int, valid_ptr: int, llm_ptr: int, B: int, n: int, L: int,
+                        out_best_ptr: int, out_len_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_drafts_accept(drafts_ptr, valid_ptr, llm_ptr, B, n, L, out_best_ptr, out_len_ptr,
+                                      out_tokens_ptr, stream))
 
 
 def dresd_retrieve_host(store: int, queries_ptr: int, B: int, top_n: int, draft_len: int,

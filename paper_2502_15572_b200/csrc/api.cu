@@ -603,6 +603,35 @@ dresd_status dresd_store_profile_read(dresd_store *s, double *scan_ms_total, int
     return DRESD_OK;
 }
 
+dresd_status dresd_drafts_prepare(const int32_t *tokens, const int32_t *ids, int B, int n, int L, int32_t eos_id,
+                                  int32_t *out_drafts, int32_t *out_valid, void *stream)
+{
+    if (B < 0 || n < 1 || L < 1) return fail(DRESD_ERR_INVALID, "bad B/n/L");
+    if (n > DRESD_MAX_TOP_N) return fail(DRESD_ERR_UNSUPPORTED, "n = %d exceeds DRESD_MAX_TOP_N", n);
+    if ((size_t)n * L * sizeof(int32_t) > 48 * 1024) return fail(DRESD_ERR_UNSUPPORTED, "n * L = %d exceeds 12288", n * L);
+    if (B == 0) return DRESD_OK;
+    if (!is_device_ptr(tokens) || !is_device_ptr(ids) || !is_device_ptr(out_drafts) || !is_device_ptr(out_valid))
+        return fail(DRESD_ERR_INVALID, "tokens/ids/out_* must be device pointers");
+    cudaError_t e = launch_drafts_prepare(tokens, ids, B, n, L, eos_id, out_drafts, out_valid,
+                                          static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "drafts_prepare launch");
+}
+
+dresd_status dresd_drafts_accept(const int32_t *drafts, const int32_t *valid, const int32_t *llm_tokens, int B,
+                                 int n, int L, int32_t *out_best, int32_t *out_len, int32_t *out_tokens,
+                                 void *stream)
+{
+    if (B < 0 || n < 1 || L < 1) return fail(DRESD_ERR_INVALID, "bad B/n/L");
+    if (n > DRESD_MAX_TOP_N) return fail(DRESD_ERR_UNSUPPORTED, "n = %d exceeds DRESD_MAX_TOP_N", n);
+    if (B == 0) return DRESD_OK;
+    if (!is_device_ptr(drafts) || !is_device_ptr(valid) || !is_device_ptr(llm_tokens) || !is_device_ptr(out_best) ||
+        !is_device_ptr(out_len) || !is_device_ptr(out_tokens))
+        return fail(DRESD_ERR_INVALID, "all buffers must be device pointers");
+    cudaError_t e = launch_drafts_accept(drafts, valid, llm_tokens, B, n, L, out_best, out_len, out_tokens,
+                                         static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "drafts_accept launch");
+}
+
 int dresd_store_last_launches(const dresd_store *s) { return valid(s) ? s->last_launches : 0; }
 
 double dresd_store_last_key_passes(const dresd_store *s) { return valid(s) ? s->last_key_passes : 0.0; }

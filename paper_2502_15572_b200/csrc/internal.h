@@ -93,6 +93,13 @@ cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long 
 cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, long long N,
                                  int32_t *first_col, cudaStream_t stream);
 
+// ---- K6: draft matrix preparation and longest-match acceptance (Section 3.6) ----
+cudaError_t launch_drafts_prepare(const int32_t *tokens, const int32_t *ids, int B, int n, int L, int eos,
+                                  int32_t *drafts, int32_t *valid, cudaStream_t stream);
+cudaError_t launch_drafts_accept(const int32_t *drafts, const int32_t *valid, const int32_t *llm, int B, int n,
+                                 int L, int32_t *out_best, int32_t *out_len, int32_t *out_tokens,
+                                 cudaStream_t stream);
+
 // Stores `msg` as the calling thread's dresd_last_error() text.
 void set_last_error(const char *msg);
 
