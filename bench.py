@@ -271,6 +271,30 @@ def run_ours(args):
     store.set_option("profile", 0)
     store.status()
 
+    # ---- latency per decode step (a synchronisation after every call) and the scan floor ----
+    lat = []
+    for i in range(min(args.steps, 200)):
+        t0 = time.perf_counter()
+        step(args.warmup + i)
+        torch.cuda.synchronize()
+        lat.append((time.perf_counter() - t0) * 1e3)
+    floor_ms = None
+    if dtype != "f32" and args.scan_path != 1:
+        store.set_option("debug_no_select", 1)
+        for i in range(3):
+            step(i)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        f0.record()
+        for i in range(min(args.steps, 200)):
+            step(args.warmup + i)
+        f1.record()
+        torch.cuda.synchronize()
+        floor_ms = f0.elapsed_time(f1) / min(args.steps, 200)
+        store.set_option("debug_no_select", 0)
+        step(0)
+        torch.cuda.synchronize()
+
     # ---- end to end: pinned host buffers in and out through dresd_retrieve_host ----
     hq = q.view(np.int16) if dtype == "bf16" else q
     hq = torch.from_numpy(np.ascontiguousarray(hq)).pin_memory()
@@ -323,6 +347,12 @@ def run_ours(args):
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "non_scan_share_of_step": 1.0 - scan_ms_avg / ms_step},
         "datastore_gbs_per_step": key_bytes / (ms_step * 1e-3) / 1e9,
+        "latency_ms": {"p50": float(np.percentile(lat, 50)), "p99": float(np.percentile(lat, 99)),
+                       "note": "wall clock per call with a device synchronisation after each"},
+        "selection_overhead": None if floor_ms is None else {
+            "floor_ms_per_step": floor_ms, "frac": ms_step / floor_ms - 1.0,
+            "note": "floor = the same call with a filter that nothing passes (keys streamed and scored, "
+                    "no candidate queued, merged or gathered beyond empty lists)"},
     }
     if world == 1 and not args.no_cpu_baseline:
         o_qps, threads, o_nq, o_dt, _ = time_oracle(cfg, keys, toks, q, args.oracle_queries)

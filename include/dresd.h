@@ -196,6 +196,10 @@ dresd_status dresd_store_status(dresd_store *store);
  *                first CTA never receives the copies of pipeline stage (value-1),
  *                so its waits run out: the kernel returns in an orderly way and
  *                dresd_store_status() reports DRESD_ERR_TIMEOUT.  0 = off.
+ *   "debug_no_select"  measurement hook: the tcgen05 scoring kernel streams and scores
+ *                every key but lets nothing pass its filter (results are empty); the
+ *                time of such a call is the floor against which the cost of
+ *                selection, merge and gather is measured.  0 = off.
  *   "profile"    > 0: record a CUDA-event pair around the scoring kernel(s) of
  *                each of the next `value` dresd_retrieve() calls (see
  *                dresd_store_profile_read); 0 = off (default).

@@ -123,7 +123,7 @@ struct dresd_store {
     CUtensorMap map_umma;
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     // options / bookkeeping
-    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage;
+    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select;
     double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
     cudaStream_t last_stream;
     int last_launches;
@@ -242,6 +242,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.cand_batch = B;
         a.status = s->status;
         a.gtau = s->gtau;
+        a.no_select = s->opt_no_select;
         a.first_col = first_tokens ? s->first_col : nullptr;
         a.want_first = first_tokens;
         const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
@@ -251,7 +252,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         // queues ~64 n survivors per query GPU-wide instead of ~n ln(rows/n) per CTA.
         // The filter only rejects rows that cannot be in the result.
         const int pstride = s->opt_probe;
-        if (pstride > 1 && B * top_n >= 256 && n_tiles >= pstride * grid) {
+        if (pstride > 1 && !s->opt_no_select && B * top_n >= 256 && n_tiles >= pstride * grid) {
             ScanArgs pa = a;
             pa.tile_stride = pstride;
             pa.n_tiles = (n_tiles + pstride - 1) / pstride;
@@ -540,6 +541,10 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
     if (strcmp(name, "scan_path") == 0) {
         if (value < 0 || value > 2) return fail(DRESD_ERR_INVALID, "scan_path = %d outside 0..2", value);
         s->opt_path = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "debug_no_select") == 0) {
+        s->opt_no_select = value != 0;
         return DRESD_OK;
     }
     if (strcmp(name, "wait_ms") == 0) {

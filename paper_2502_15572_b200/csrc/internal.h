@@ -58,6 +58,7 @@ struct ScanArgs {
     int debug_lose_stage;   // test hook (streaming kernel): CTA 0 never receives stage (value-1); 0 = off
     int tile_stride;        // tcgen05 kernel: visit every tile_stride-th tile (probe pass), default 1
     int probe_max;          // tcgen05 kernel, probe pass: keep only each tile's best row per query
+    int no_select;          // tcgen05 kernel, measurement only: nothing passes the filter (scan floor)
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.
 int scan_mma_tile_rows(int d);

@@ -210,7 +210,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             warp_topn_init(&sel[q], lane);
             // start from whatever the grid already knows; padding columns never pass
             if (lane == 0) {
-                tau[q] = q < a.B ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
+                tau[q] = (q < a.B && !a.no_select) ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
                 want_s[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
             }
         }
@@ -360,7 +360,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             dead = __any_sync(0xFFFFFFFFu, dead);
             tc_fence_after();
             // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
-            if ((tl & 3) == 0 && et < a.B) tau[et] = peek_tau(&a.gtau[et], tau[et]);
+            if ((tl & 3) == 0 && et < a.B && !a.no_select) tau[et] = peek_tau(&a.gtau[et], tau[et]);
             const uint32_t acc_addr = lane_addr + (uint32_t)(acc * kAccCols);
             if (a.probe_max) {
                 // Probe pass: no filtering and no lists -- only the best row of each sub-tile
