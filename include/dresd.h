@@ -158,6 +158,24 @@ dresd_status dresd_drafts_accept(const int32_t *drafts, const int32_t *valid, co
                                  int32_t *out_tokens, void *stream);
 
 /*
+ * Exchange step of a datastore whose rows are sharded over P GPUs.  Eq. 3 is an arg
+ * max over the whole datastore; with the rows split into disjoint shards, the top_n
+ * of the whole is the top_n of the union of the shards' top_n.  Each shard runs
+ * dresd_retrieve() on its own rows; the P results (B * top_n * (8 + 4 draft_len) bytes
+ * per shard) are gathered on one device -- NCCL all-gather, or peer copies -- and
+ * this call merges them.
+ *
+ *   ids, scores, tokens  device, [P][B][top_n] / [P][B][top_n] / [P][B][top_n][draft_len]:
+ *                        the shards' outputs, ids LOCAL to each shard (-1 = missing)
+ *   row_offsets          device, int64 [P]: global row index of each shard's row 0,
+ *                        ascending; global ids must stay below 2^31
+ *   out_*                as for dresd_retrieve(), ids global.
+ */
+dresd_status dresd_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens,
+                                const int64_t *row_offsets, int P, int B, int top_n, int draft_len,
+                                int32_t *out_ids, float *out_scores, int32_t *out_tokens, void *stream);
+
+/*
  * The same call for callers whose queries and results live in HOST memory
  * (ideally pinned): copies the queries to the device, runs dresd_retrieve(),
  * copies the three results back and waits for `stream`.  The datastore itself

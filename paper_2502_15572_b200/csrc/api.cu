@@ -637,6 +637,22 @@ dresd_status dresd_drafts_accept(const int32_t *drafts, const int32_t *valid, co
     return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "drafts_accept launch");
 }
 
+dresd_status dresd_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens,
+                                const int64_t *row_offsets, int P, int B, int top_n, int draft_len,
+                                int32_t *out_ids, float *out_scores, int32_t *out_tokens, void *stream)
+{
+    if (P < 1 || B < 0 || top_n < 1 || draft_len < 1) return fail(DRESD_ERR_INVALID, "bad P/B/top_n/draft_len");
+    if (top_n > DRESD_MAX_TOP_N) return fail(DRESD_ERR_UNSUPPORTED, "top_n = %d exceeds DRESD_MAX_TOP_N", top_n);
+    if (B == 0) return DRESD_OK;
+    if (!is_device_ptr(ids) || !is_device_ptr(scores) || !is_device_ptr(tokens) || !is_device_ptr(row_offsets) ||
+        !is_device_ptr(out_ids) || !is_device_ptr(out_scores) || !is_device_ptr(out_tokens))
+        return fail(DRESD_ERR_INVALID, "all buffers must be device pointers");
+    cudaError_t e = launch_merge_shards(ids, scores, tokens, reinterpret_cast<const long long *>(row_offsets), P, B,
+                                        top_n, draft_len, out_ids, out_scores, out_tokens,
+                                        static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "merge_shards launch");
+}
+
 int dresd_store_last_launches(const dresd_store *s) { return valid(s) ? s->last_launches : 0; }
 
 double dresd_store_last_key_passes(const dresd_store *s) { return valid(s) ? s->last_key_passes : 0.0; }

@@ -101,6 +101,11 @@ cudaError_t launch_drafts_accept(const int32_t *drafts, const int32_t *valid, co
                                  int L, int32_t *out_best, int32_t *out_len, int32_t *out_tokens,
                                  cudaStream_t stream);
 
+// Exchange step of a row-sharded datastore: P per-shard top-n lists -> the global top-n.
+cudaError_t launch_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens,
+                                const long long *offsets, int P, int B, int n, int L, int32_t *out_ids,
+                                float *out_scores, int32_t *out_tokens, cudaStream_t stream);
+
 // Stores `msg` as the calling thread's dresd_last_error() text.
 void set_last_error(const char *msg);
 

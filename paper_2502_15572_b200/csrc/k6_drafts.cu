@@ -90,3 +90,62 @@ cudaError_t launch_drafts_accept(const int32_t *drafts, const int32_t *valid, co
 }
 
 }  // namespace dresd
+
+// ---------------------------------------------------------------------------------
+// Row-sharded datastore: the exchange step.  Every shard (GPU) returns its own top-n
+// with LOCAL row ids; the top-n of the union is the top-n of the whole datastore
+// (Eq. 3 is an arg max over D, and D is the disjoint union of the shards).  One warp
+// per query folds the P sorted lists with the same bitonic merges as the grid merge,
+// on global ids (local id + the shard's row offset), then copies the winners' tokens.
+// ---------------------------------------------------------------------------------
+namespace dresd {
+namespace {
+
+__global__ void merge_shards_kernel(const int32_t *__restrict__ ids, const float *__restrict__ scores,
+                                    const int32_t *__restrict__ tokens, const long long *__restrict__ offsets,
+                                    int P, int B, int n, int L, int32_t *__restrict__ out_ids,
+                                    float *__restrict__ out_scores, int32_t *__restrict__ out_tokens)
+{
+    const int b = blockIdx.x, lane = threadIdx.x;
+    unsigned long long m = 0ull;
+    for (int p = 0; p < P; ++p) {
+        unsigned long long v = 0ull;
+        if (lane < n) {
+            const int32_t id = ids[((size_t)p * B + b) * n + lane];
+            if (id >= 0) v = pack_candidate(scores[((size_t)p * B + b) * n + lane], (uint32_t)(id + offsets[p]));
+        }
+        // a shard's list is sorted with its missing entries (id -1) last, so it is a valid input
+        m = warp_merge_top32(m, v, lane);
+    }
+    if (lane >= n) m = 0ull;
+    const long long gid = m ? (long long)candidate_id(m) : -1;
+    if (lane < n) {
+        out_ids[(size_t)b * n + lane] = (int32_t)gid;
+        out_scores[(size_t)b * n + lane] = m ? candidate_score(m) : -INFINITY;
+    }
+    // where did this winner come from?  shard = last offset <= gid; slot = its rank there
+    int p = -1, r = -1;
+    if (gid >= 0) {
+        p = 0;
+        while (p + 1 < P && offsets[p + 1] <= gid) ++p;
+        const int32_t local = (int32_t)(gid - offsets[p]);
+        for (int k = 0; k < n; ++k)
+            if (ids[((size_t)p * B + b) * n + k] == local) { r = k; break; }
+    }
+    if (lane < n)
+        for (int t = 0; t < L; ++t)
+            out_tokens[((size_t)b * n + lane) * L + t] =
+                r >= 0 ? tokens[(((size_t)p * B + b) * n + r) * L + t] : -1;
+}
+
+}  // namespace
+
+cudaError_t launch_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens,
+                                const long long *offsets, int P, int B, int n, int L, int32_t *out_ids,
+                                float *out_scores, int32_t *out_tokens, cudaStream_t stream)
+{
+    merge_shards_kernel<<<B, 32, 0, stream>>>(ids, scores, tokens, offsets, P, B, n, L, out_ids, out_scores, out_tokens);
+    return cudaGetLastError();
+}
+
+}  // namespace dresd

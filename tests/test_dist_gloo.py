@@ -61,3 +61,42 @@ def test_two_ranks_gloo_max_and_partition():
         assert p.exitcode == 0
     assert res[0][1] == res[1][1] == [11.0, 5.0, 501.0]          # element-wise max over both ranks
     assert res[0][2] == (0, 501) and res[1][2] == (501, 1001)    # disjoint, covering
+
+
+def _gather_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      LOCAL_RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        B, n, L = 3, 4, 2
+        rows = dist_util.shard_rows(1001, rank, world)
+        ids = torch.arange(B * n, dtype=torch.int32).reshape(B, n) + 100 * rank
+        scores = torch.full((B, n), float(rank), dtype=torch.float32)
+        tokens = torch.full((B, n, L), 7 + rank, dtype=torch.int32)
+        g = dist_util.gather_shard_results(ids, scores, tokens, rows.start)
+        out.put((rank, [t.tolist() for t in g]))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_gloo_gather_of_shard_results():
+    """The exchange step of the row-sharded mode: every rank ends up with all shards'
+    results stacked by rank, and with the shards' row offsets."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_gather_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res[0][1] == res[1][1]                                  # both ranks hold the same gathered view
+    ids, scores, tokens, offsets = res[0][1]
+    assert offsets == [0, 501]
+    assert ids[0][0] == [0, 1, 2, 3] and ids[1][0] == [100, 101, 102, 103]
+    assert scores[0][0][0] == 0.0 and scores[1][0][0] == 1.0
+    assert tokens[0][0][0] == [7, 7] and tokens[1][0][0] == [8, 8]

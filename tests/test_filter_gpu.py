@@ -73,3 +73,58 @@ def test_filtered_call_needs_the_column():
     st.retrieve_filtered(q, None, 2, 2)               # NULL = plain retrieve
     torch.cuda.synchronize()
     st.close()
+
+
+@pytest.mark.parametrize("filtered", [False, True])
+def test_row_sharded_merge_equals_whole_store(filtered):
+    """Exchange step of a row-sharded datastore on one GPU: three stores over row slices,
+    their results stacked as an all-gather would, merged by dresd_merge_shards."""
+    import torch
+    N, d, dtype, B, n, L = 50021, 128, "bf16", 9, 10, 4
+    vocab = 3000 if filtered else 32000
+    keys, toks = synth.make_store(9701, N, d, 16, dtype, L, vocab=vocab)
+    q, _ = synth.make_queries(9702, keys, dtype, B, 0.1)
+    ft = torch.from_numpy(np.random.default_rng(9703).integers(2000, 3000, size=B).astype(np.int32)).cuda()
+    dq = binding.to_device(q, dtype)
+
+    def run(k, t):
+        st = gpu_store(k, t, dtype)
+        if filtered:
+            st.enable_first_token_filter()
+            out = st.retrieve_filtered(dq, ft, n, L)
+        else:
+            out = st.retrieve(dq, n, L)
+        torch.cuda.synchronize()
+        st.close()
+        return out
+
+    whole = run(keys, toks)
+    cuts = [0, 12345, 30000, N]
+    parts = [run(keys[a:b], toks[a:b]) for a, b in zip(cuts[:-1], cuts[1:])]
+    g_ids = torch.stack([p[0] for p in parts]).contiguous()
+    g_sc = torch.stack([p[1] for p in parts]).contiguous()
+    g_tok = torch.stack([p[2] for p in parts]).contiguous()
+    offsets = torch.tensor(cuts[:-1], dtype=torch.int64, device="cuda")
+    out = (torch.empty_like(whole[0]), torch.empty_like(whole[1]), torch.empty_like(whole[2]))
+    binding.dresd_merge_shards(g_ids.data_ptr(), g_sc.data_ptr(), g_tok.data_ptr(), offsets.data_ptr(), 3, B, n, L,
+                               out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(),
+                               torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for a, b in zip(out, whole):
+        assert torch.equal(a, b)
+    if filtered:
+        assert (whole[0] == -1).any()          # scarce tokens: some queries have fewer than n matches
+
+
+def test_sharded_retrieve_single_process():
+    import torch
+    from paper_2502_15572_b200 import dist_util
+    keys, toks = synth.make_store(9801, 20011, 64, 8, "f16", 3)
+    q, _ = synth.make_queries(9802, keys, "f16", 2, 0.1)
+    st = gpu_store(keys, toks, "f16")
+    dq = binding.to_device(q, "f16")
+    ref = st.retrieve(dq, 5, 3)
+    got = dist_util.sharded_retrieve(st, 1000, dq, 5, 3)
+    torch.cuda.synchronize()
+    assert torch.equal(got[0], ref[0] + 1000) and torch.equal(got[1], ref[1]) and torch.equal(got[2], ref[2])
+    st.close()
