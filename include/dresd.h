@@ -158,6 +158,29 @@ dresd_status dresd_drafts_accept(const int32_t *drafts, const int32_t *valid, co
                                  int32_t *out_tokens, void *stream);
 
 /*
+ * Datastore-side preprocessing, Sections 3.2-3.5: the KEYS of the datastore are the
+ * token embeddings of the corpus after the same three steps the query takes -- Eq. 1
+ * (z-scoring), v_l <- v W_l, Eq. 2 (unit length).  This call applies them to N rows of
+ * LLM hidden states at once (a tensor-core GEMM [N x d_in] . [d_in x d] with the
+ * normalisations fused) and writes the key matrix that dresd_store_create() takes.
+ *
+ *   hidden     device, [N][d_in] row-major, fp16 or bf16 (`dtype`), 16-byte aligned;
+ *              d_in a multiple of 8, at most 16384
+ *   mean, var  device fp32 [d_in] (both or neither), eps_z: Eq. 1
+ *   W          device, [d_in][d] row-major in `dtype`; d = 32 .. 256 in steps of 32
+ *   pca_mean   device fp32 [d_in] or NULL, subtracted after Eq. 1
+ *   out_keys   device, [N][d] row-major in `dtype`: unit-length rows, rounded to
+ *              `dtype` from fp32 accumulation (hidden states enter exactly; W / sigma
+ *              is carried as a two-term 16-bit split)
+ *
+ * Offline operation: allocates a scratch copy of W (4 d d_in bytes), runs on `stream`
+ * and RETURNS AFTER THE STREAM HAS FINISHED (the scratch is freed on return).
+ */
+dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dtype dtype, const float *mean,
+                              const float *var, float eps_z, const void *W, int d, const float *pca_mean,
+                              void *out_keys, void *stream);
+
+/*
  * Exchange step of a datastore whose rows are sharded over P GPUs.  Eq. 3 is an arg
  * max over the whole datastore; with the rows split into disjoint shards, the top_n
  * of the whole is the top_n of the union of the shards' top_n.  Each shard runs

@@ -29,7 +29,7 @@ EXPORTS = (
     "dresd_last_error",
     "dresd_store_destroy", "dresd_retrieve_noalloc", "dresd_store_enable_first_token_filter",
     "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
-    "dresd_merge_shards",
+    "dresd_merge_shards", "dresd_build_keys",
 )
 
 
@@ -89,6 +89,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_drafts_accept.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_merge_shards.restype = i32
     lib.dresd_merge_shards.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.dresd_build_keys.restype = i32
+    lib.dresd_build_keys.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, i32, vp, vp, vp]
     lib.dresd_retrieve_noalloc.restype = i32
     lib.dresd_retrieve_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
     if path is None:
@@ -150,6 +152,13 @@ def dresd_merge_shards(ids_ptr: int, scores_ptr: int, tokens_ptr: int, offsets_p
                        stream: int = 0) -> None:
     _check(load().dresd_merge_shards(ids_ptr, scores_ptr, tokens_ptr, offsets_ptr, P, B, top_n, draft_len,
                                      out_ids_ptr, out_scores_ptr, out_tokens_ptr, stream))
+
+
+def dresd_build_keys(hidden_ptr: int, N: int, d_in: int, dtype: int, mean_ptr, var_ptr, eps_z: float, W_ptr: int,
+                     d: int, pca_mean_ptr, out_keys_ptr: int, stream: int = 0) -> None:
+    """Eq. 1 -> v W -> Eq. 2 over N rows of hidden states: builds the datastore's key matrix."""
+    _check(load().dresd_build_keys(hidden_ptr, N, d_in, dtype, mean_ptr, var_ptr, eps_z, W_ptr, d, pca_mean_ptr,
+                                   out_keys_ptr, stream))
 
 
 def dresd_retrieve_host(store: int, queries_ptr: int, B: int, top_n: int, draft_len: int,

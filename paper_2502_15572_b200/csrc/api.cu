@@ -653,6 +653,63 @@ dresd_status dresd_merge_shards(const int32_t *ids, const float *scores, const i
     return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "merge_shards launch");
 }
 
+dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dtype dtype, const float *mean,
+                              const float *var, float eps_z, const void *W, int d, const float *pca_mean,
+                              void *out_keys, void *stream_v)
+{
+    if (dtype != DRESD_F16 && dtype != DRESD_BF16)
+        return fail(DRESD_ERR_UNSUPPORTED, "dresd_build_keys builds 16-bit datastores (fp16 or bf16)");
+    if (N <= 0 || N > 2147483647LL) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1", (long long)N);
+    if (d_in < 8 || d_in % 8 != 0) return fail(DRESD_ERR_INVALID, "d_in = %d must be a positive multiple of 8", d_in);
+    if (d < 32 || d > 256 || d % 32 != 0) return fail(DRESD_ERR_UNSUPPORTED, "d = %d must be 32..256 in steps of 32", d);
+    if (d_in > 16384) return fail(DRESD_ERR_UNSUPPORTED, "d_in = %d exceeds 16384", d_in);
+    if ((mean == nullptr) != (var == nullptr)) return fail(DRESD_ERR_INVALID, "mean and var go together");
+    if (!(eps_z >= 0.f)) return fail(DRESD_ERR_INVALID, "eps_z must be >= 0");
+    if (!is_device_ptr(hidden) || !is_device_ptr(W) || !is_device_ptr(out_keys) || (mean && !is_device_ptr(mean)) ||
+        (var && !is_device_ptr(var)) || (pca_mean && !is_device_ptr(pca_mean)))
+        return fail(DRESD_ERR_INVALID, "hidden/W/out_keys/mean/var/pca_mean must be device pointers");
+    if (reinterpret_cast<uintptr_t>(hidden) % 16 != 0 || reinterpret_cast<uintptr_t>(out_keys) % 16 != 0)
+        return fail(DRESD_ERR_INVALID, "hidden / out_keys not 16-byte aligned");
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda(e, "cudaGetDevice");
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return fail_cuda(e, "SM count");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+
+    const size_t kpad = ((size_t)d_in + 63) / 64 * 64;
+    uint8_t *ws = nullptr;
+    if (cudaMalloc(&ws, build_keys_workspace_bytes(d_in, d)) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(DRESD_ERR_ALLOC, "workspace allocation failed");
+    }
+    void *wt_hi = ws, *wt_lo = ws + (size_t)d * kpad * 2;
+    float *bias = reinterpret_cast<float *>(ws + 2 * (size_t)d * kpad * 2);
+    int *status = reinterpret_cast<int *>(bias + 256);
+    dresd_status st = DRESD_OK;
+    CUtensorMap h_map, whi_map, wlo_map;
+    if (!make_map(&h_map, hidden, (int)dtype, N, d_in, 128) || !make_map(&whi_map, wt_hi, (int)dtype, d, (int)kpad, d) ||
+        !make_map(&wlo_map, wt_lo, (int)dtype, d, (int)kpad, d))
+        st = fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+    if (st == DRESD_OK && (e = cudaMemsetAsync(status, 0, sizeof(int), stream)) != cudaSuccess)
+        st = fail_cuda(e, "status reset");
+    if (st == DRESD_OK && (e = launch_build_prep(W, (int)dtype, mean, var, eps_z, pca_mean, d_in, d, wt_hi, wt_lo, bias,
+                                                 stream)) != cudaSuccess)
+        st = fail_cuda(e, "build prep launch");
+    if (st == DRESD_OK && (e = launch_build_keys(h_map, whi_map, wlo_map, (int)dtype, N, d_in, d, bias, out_keys,
+                                                 kEpsNorm, status, sms, stream)) != cudaSuccess)
+        st = fail_cuda(e, "build keys launch");
+    int word = 0;
+    if (st == DRESD_OK && (e = cudaMemcpyAsync(&word, status, sizeof(int), cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        st = fail_cuda(e, "status read");
+    e = cudaStreamSynchronize(stream);                 // the workspace is freed below: wait for the kernels
+    if (st == DRESD_OK && e != cudaSuccess) st = fail_cuda(e, "stream synchronize");
+    cudaFree(ws);
+    if (st == DRESD_OK && word != 0) st = fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
+    return st;
+}
+
 int dresd_store_last_launches(const dresd_store *s) { return valid(s) ? s->last_launches : 0; }
 
 double dresd_store_last_key_passes(const dresd_store *s) { return valid(s) ? s->last_key_passes : 0.0; }

@@ -1,0 +1,381 @@
+// K7 -- datastore-side preprocessing: the keys of the datastore are the token embeddings
+// of the corpus after the SAME three steps the query takes (Sections 3.2-3.4 of the paper:
+// Eq. 1 z-scoring, v_l <- v W_l, Eq. 2 unit length), applied to N rows of LLM hidden
+// states.  Unlike the per-step retrieval this is a real GEMM, [N x d_in] . [d_in x d], and
+// it is tensor-bound: tcgen05.mma with TMEM accumulators, TMA-fed.
+//
+// Algebra.  With sigma_j = sqrt(Var_j + eps):
+//     ((h - mu) / sigma - m) W  =  h W'  +  c,      W'[j][c] = W[j][c] / sigma_j,
+//                                                   c[c]     = -sum_j (mu_j / sigma_j + m_j) W[j][c].
+// The hidden states h enter the tensor cores exactly (they are stored in 16 bits); W' is
+// split into two 16-bit terms (W' = hi + lo) and both products accumulate into the same
+// fp32 accumulator, so the result carries fp32-level accuracy before the final rounding to
+// the store dtype.  c is computed in float64 by a small kernel.
+//
+// One persistent CTA per SM, ten warps: warp 0 = TMA producer (per 64-column k-slab: two
+// 128-row slabs of h, the hi and the lo slab of W'^T, all 128-byte swizzled); warp 1 =
+// TMEM allocation + MMA issue (a 256-row tile = two 128-row accumulators of d columns);
+// warps 2-9 = epilogue (a thread owns one row: adds c, takes the norm in a first pass over
+// its accumulator row, scales, rounds and stores in a second).  Every wait is bounded.
+#include <type_traits>
+
+#include "common.cuh"
+#include "internal.h"
+
+namespace dresd {
+namespace {
+
+constexpr int kThreads = 10 * 32;
+constexpr int kSubRows = 128;
+constexpr int kTileRows = 2 * kSubRows;
+constexpr int kSlabBytes = 128;
+constexpr int kSlabElems = 64;
+constexpr int kASlab = kSubRows * kSlabBytes;        // 16 KB
+constexpr int kMaxStages = 6;
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *smem_dst, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// K-major operand, 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr)
+{
+    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t *r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+template <typename T> __device__ __forceinline__ float w_to_f32(T x);
+template <> __device__ __forceinline__ float w_to_f32<__half>(__half x) { return __half2float(x); }
+template <> __device__ __forceinline__ float w_to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T w_from_f32(float x);
+template <> __device__ __forceinline__ __half w_from_f32<__half>(float x) { return __float2half_rn(x); }
+template <> __device__ __forceinline__ __nv_bfloat16 w_from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
+template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b)
+{
+    __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, float b)
+{
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+// W'^T = (W / sigma)^T split into hi + lo, [d][kpad] K-major, zero padded; bias in float64.
+template <typename T>
+__global__ void build_prep_kernel(const T *__restrict__ W, const float *__restrict__ mean,
+                                  const float *__restrict__ var, float eps_z, const float *__restrict__ pca_mean,
+                                  int d_in, int d, int kpad, T *__restrict__ wt_hi, T *__restrict__ wt_lo,
+                                  float *__restrict__ bias)
+{
+    const int c = blockIdx.x;                              // output column
+    __shared__ double red[32];
+    double acc = 0.0;
+    for (int j = threadIdx.x; j < kpad; j += blockDim.x) {
+        float hi = 0.f, lo = 0.f;
+        if (j < d_in) {
+            const float w = w_to_f32<T>(W[(size_t)j * d + c]);
+            const float sigma = mean ? sqrtf(var[j] + eps_z) : 1.f;
+            const float wp = w / sigma;
+            const T h = w_from_f32<T>(wp);
+            hi = w_to_f32<T>(h);
+            lo = w_to_f32<T>(w_from_f32<T>(wp - hi));
+            const double shift = (mean ? (double)mean[j] / (double)sigma : 0.0) + (pca_mean ? (double)pca_mean[j] : 0.0);
+            acc -= shift * (double)w;
+        }
+        wt_hi[(size_t)c * kpad + j] = w_from_f32<T>(hi);
+        wt_lo[(size_t)c * kpad + j] = w_from_f32<T>(lo);
+    }
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+        bias[c] = (float)t;
+    }
+}
+
+struct BuildArgs {
+    long long N;
+    int d_in, d, n_tiles, stages;
+    const float *bias;       // [d]
+    void *out;               // [N][d] store dtype
+    float eps_n;
+    int *status;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 1)
+build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_constant__ CUtensorMap whi_map,
+                  const __grid_constant__ CUtensorMap wlo_map, const BuildArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *base = reinterpret_cast<uint8_t *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int n_stages = a.stages;
+    const int kslabs = (a.d_in + kSlabElems - 1) / kSlabElems;
+    const int b_slab = a.d * kSlabBytes;                    // one 64-column slab of W'^T (hi or lo)
+    const int stage_bytes = 2 * kASlab + 2 * b_slab;
+    uint8_t *stages = base;
+    float *bias_s = reinterpret_cast<float *>(stages + (size_t)n_stages * stage_bytes);
+    uint64_t *full = reinterpret_cast<uint64_t *>(bias_s + 256);
+    uint64_t *empty = full + kMaxStages;
+    uint64_t *tfull = empty + kMaxStages;
+    uint64_t *tempty = tfull + 1;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(tempty + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x, G = gridDim.x;
+    const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
+    const int n_it = my_tiles * kslabs;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * a.d) tmem_cols <<= 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(tfull, 1);
+        mbar_init(tempty, 8);
+        mbar_fence_init();
+    }
+    for (int c = tid; c < a.d; c += kThreads) bias_s[c] = a.bias[c];
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&h_map);
+            tma_prefetch_desc(&whi_map);
+            tma_prefetch_desc(&wlo_map);
+            int issued = 0;
+            for (int it = 0; it < n_it; ++it) {
+                const int s = it % n_stages;
+                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
+                    report_timeout(a.status);
+                    break;
+                }
+                const int tile = cta + (it / kslabs) * G;
+                const int ks = it % kslabs;
+                uint8_t *dst = stages + (size_t)s * stage_bytes;
+                mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
+                tma_load_2d(dst, &h_map, ks * kSlabElems, tile * kTileRows, &full[s]);
+                tma_load_2d(dst + kASlab, &h_map, ks * kSlabElems, tile * kTileRows + kSubRows, &full[s]);
+                tma_load_2d(dst + 2 * kASlab, &whi_map, ks * kSlabElems, 0, &full[s]);
+                tma_load_2d(dst + 2 * kASlab + b_slab, &wlo_map, ks * kSlabElems, 0, &full[s]);
+                issued = it + 1;
+            }
+            for (int it = max(0, issued - n_stages); it < issued; ++it)
+                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1)) {
+                    report_timeout(a.status);
+                    break;
+                }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t kFmt = std::is_same<T, __nv_bfloat16>::value ? 1u : 0u;
+            const uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(a.d >> 3) << 17) |
+                                   ((uint32_t)(kSubRows >> 4) << 24);
+            bool ok = true;
+            for (int tl = 0; tl < my_tiles && ok; ++tl) {
+                // one accumulator set: wait until the epilogue has drained the previous tile
+                if (tl >= 1 && !mbar_wait(tempty, (tl - 1) & 1)) { ok = false; break; }
+                tc_fence_after();
+                for (int ks = 0; ks < kslabs; ++ks) {
+                    const int it = tl * kslabs + ks;
+                    const int s = it % n_stages;
+                    if (!mbar_wait(&full[s], (it / n_stages) & 1)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
+                    const uint64_t bhi = make_desc(st + 2 * kASlab), blo = make_desc(st + 2 * kASlab + b_slab);
+#pragma unroll
+                    for (int sub = 0; sub < 2; ++sub) {
+                        const uint64_t ad = make_desc(st + sub * kASlab);
+                        const uint32_t dt = tmem_base + (uint32_t)(sub * a.d);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            umma_f16(dt, ad + 2 * k, bhi + 2 * k, idesc, (ks | k) != 0);
+                            umma_f16(dt, ad + 2 * k, blo + 2 * k, idesc, 1);
+                        }
+                    }
+                    tc_commit(&empty[s]);
+                }
+                if (!ok) break;
+                tc_commit(tfull);
+            }
+            if (!ok) report_timeout(a.status);
+        }
+    } else {
+        // epilogue: warps 2-5 own sub-tile 0, warps 6-9 sub-tile 1; lane group = warp & 3
+        const int ew = warp - 2;
+        const int sub = ew >> 2;
+        const int lane_grp = warp & 3;
+        const uint32_t row_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(sub * a.d);
+        T *out = static_cast<T *>(a.out);
+        bool dead = false;
+        for (int tl = 0; tl < my_tiles; ++tl) {
+            if (!dead && !mbar_wait(tfull, tl & 1)) {
+                report_timeout(a.status);
+                dead = true;
+            }
+            dead = __any_sync(0xFFFFFFFFu, dead);
+            tc_fence_after();
+            const long long row = (long long)(cta + tl * G) * kTileRows + sub * kSubRows + lane_grp * 32 + lane;
+            if (!dead) {
+                float ss = 0.f;                                    // Eq. 2: squared length of v W' + c
+                for (int c0 = 0; c0 < a.d; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld32(row_addr + (uint32_t)c0, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float x = __uint_as_float(r[i]) + bias_s[c0 + i];
+                        ss = fmaf(x, x, ss);
+                    }
+                }
+                const float inv = 1.0f / fmaxf(sqrtf(ss), a.eps_n);
+                for (int c0 = 0; c0 < a.d; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld32(row_addr + (uint32_t)c0, r);
+                    tmem_ld_wait();
+                    if (row < a.N) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(out + (size_t)row * a.d + c0);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 o;
+                            const int i = 8 * v;
+                            o.x = pack2<T>((__uint_as_float(r[i + 0]) + bias_s[c0 + i + 0]) * inv,
+                                           (__uint_as_float(r[i + 1]) + bias_s[c0 + i + 1]) * inv);
+                            o.y = pack2<T>((__uint_as_float(r[i + 2]) + bias_s[c0 + i + 2]) * inv,
+                                           (__uint_as_float(r[i + 3]) + bias_s[c0 + i + 3]) * inv);
+                            o.z = pack2<T>((__uint_as_float(r[i + 4]) + bias_s[c0 + i + 4]) * inv,
+                                           (__uint_as_float(r[i + 5]) + bias_s[c0 + i + 5]) * inv);
+                            o.w = pack2<T>((__uint_as_float(r[i + 6]) + bias_s[c0 + i + 6]) * inv,
+                                           (__uint_as_float(r[i + 7]) + bias_s[c0 + i + 7]) * inv);
+                            dst[v] = o;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+}  // namespace
+
+size_t build_keys_workspace_bytes(int d_in, int d)
+{
+    const size_t kpad = ((size_t)d_in + 63) / 64 * 64;
+    return 2 * (size_t)d * kpad * 2 + 256 * sizeof(float) + 256;
+}
+
+cudaError_t launch_build_prep(const void *W, int dtype, const float *mean, const float *var, float eps_z,
+                              const float *pca_mean, int d_in, int d, void *wt_hi, void *wt_lo, float *bias,
+                              cudaStream_t stream)
+{
+    const int kpad = (d_in + 63) / 64 * 64;
+    if (dtype == kF16)
+        build_prep_kernel<__half><<<d, 256, 0, stream>>>(static_cast<const __half *>(W), mean, var, eps_z, pca_mean,
+                                                          d_in, d, kpad, static_cast<__half *>(wt_hi),
+                                                          static_cast<__half *>(wt_lo), bias);
+    else
+        build_prep_kernel<__nv_bfloat16><<<d, 256, 0, stream>>>(
+            static_cast<const __nv_bfloat16 *>(W), mean, var, eps_z, pca_mean, d_in, d, kpad,
+            static_cast<__nv_bfloat16 *>(wt_hi), static_cast<__nv_bfloat16 *>(wt_lo), bias);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_build_keys(const CUtensorMap &h_map, const CUtensorMap &whi_map, const CUtensorMap &wlo_map,
+                              int dtype, long long N, int d_in, int d, const float *bias, void *out, float eps_n,
+                              int *status, int grid, cudaStream_t stream)
+{
+    BuildArgs a{};
+    a.N = N;
+    a.d_in = d_in;
+    a.d = d;
+    a.n_tiles = (int)((N + kTileRows - 1) / kTileRows);
+    a.bias = bias;
+    a.out = out;
+    a.eps_n = eps_n;
+    a.status = status;
+    const size_t stage = 2 * (size_t)kASlab + 2 * (size_t)d * kSlabBytes;
+    const size_t fixed = 1024 + 256 * sizeof(float) + sizeof(uint64_t) * (2 * kMaxStages + 2) + 64;
+    long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)stage;
+    if (s > kMaxStages) s = kMaxStages;
+    if (s < 2) return cudaErrorInvalidValue;
+    a.stages = (int)s;
+    const size_t smem = fixed + (size_t)s * stage;
+    if (grid > a.n_tiles) grid = a.n_tiles;
+    cudaError_t e;
+    if (dtype == kF16) {
+        auto k = build_keys_kernel<__half>;
+        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k<<<grid, kThreads, smem, stream>>>(h_map, whi_map, wlo_map, a);
+    } else {
+        auto k = build_keys_kernel<__nv_bfloat16>;
+        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k<<<grid, kThreads, smem, stream>>>(h_map, whi_map, wlo_map, a);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace dresd

@@ -1,0 +1,87 @@
+"""Datastore-side preprocessing (dresd_build_keys: Eq. 1 -> v W -> Eq. 2 over N rows on the
+tensor cores) against the oracle's per-row float64 preprocessing, and end to end: keys built
+on the GPU, then searched, must give the oracle's neighbours."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2502_15572_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _ulp(x, dtype):
+    """Spacing of the store dtype at |x| (float64 array)."""
+    bits = 10 if dtype == "f16" else 7
+    e = np.floor(np.log2(np.maximum(np.abs(x), 2.0 ** -14)))
+    return 2.0 ** (e - bits)
+
+
+def _build(hidden, dtype, mean, var, W, pca_mean, eps_z=1e-5):
+    import torch
+    N, d_in = hidden.shape
+    d = W.shape[1]
+    dh = binding.to_device(hidden, dtype)
+    dW = binding.to_device(W, dtype)
+    t = lambda a: None if a is None else torch.from_numpy(np.asarray(a, dtype=np.float32)).cuda()
+    dm, dv, dp = t(mean), t(var), t(pca_mean)
+    out = torch.empty((N, d), dtype=dh.dtype, device="cuda")
+    ptr = lambda x: None if x is None else x.data_ptr()
+    binding.dresd_build_keys(dh.data_ptr(), N, d_in, binding.DTYPE_CODE[dtype], ptr(dm), ptr(dv), eps_z,
+                             dW.data_ptr(), d, ptr(dp), out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    return out
+
+
+@pytest.mark.parametrize("dtype,N,d_in,d,zscore,centre", [
+    ("bf16", 3000, 4096, 256, True, False),
+    ("f16", 1111, 512, 64, True, True),
+    ("bf16", 700, 200, 128, False, False),        # d_in not a multiple of 64, no z-scoring
+    ("f16", 257, 1024, 96, True, False),
+    ("bf16", 40000, 256, 32, True, True),         # many tiles per CTA
+])
+def test_build_keys_matches_oracle_preprocess(dtype, N, d_in, d, zscore, centre):
+    mean, var, W = synth.make_preprocess(6100 + d, d_in, d, dtype)
+    hidden = synth.make_hidden_queries(6200 + d, N, d_in, dtype)
+    pm = (0.02 * np.cos(np.arange(d_in))).astype(np.float32) if centre else None
+    if not zscore:
+        mean = var = None
+    got = _build(hidden, dtype, mean, var, W, pm)
+    got64 = synth.store_to_float32(got.cpu().view({"f16": __import__("torch").float16,
+                                                   "bf16": __import__("torch").int16}[dtype]).numpy()
+                                   if dtype == "f16" else got.cpu().view(__import__("torch").int16).numpy().view(np.uint16),
+                                   dtype).astype(np.float64)
+    want = oracle.preprocess(hidden, dtype, mean=mean, var=var, eps_z=1e-5, W=W, pca_mean=pm)
+    # Stored values: the float64 result rounded to the store dtype, up to the arithmetic
+    # error of the GEMM before that rounding.  That error is absolute (it scales with the
+    # row, not the element): W / sigma is carried as two 16-bit terms (2^-17 relative per
+    # product for bf16, 2^-22 for fp16) and 4096 products are summed in fp32.
+    ulp = _ulp(want, dtype)
+    err = np.abs(got64 - want)
+    abs_tol = 4e-5 if dtype == "bf16" else 6e-6
+    assert np.all(err <= 0.5 * ulp + abs_tol), f"max excess {np.max(err - 0.5 * ulp):.2e}"
+    assert np.mean(err <= 0.5 * ulp * 1.001) >= 0.9             # the great majority correctly rounded
+    np.testing.assert_allclose(np.linalg.norm(got64, axis=1), 1.0, atol=2.0 ** -7)
+
+
+def test_built_keys_are_searchable_end_to_end():
+    """Hidden states -> keys on the GPU -> store -> retrieval; the same hidden state as the
+    query (projected by K1) must find its own row first (Eq. 4: reciprocal rank 1)."""
+    import torch
+    dtype, N, d_in, d = "bf16", 20000, 1024, 128
+    mean, var, W = synth.make_preprocess(6301, d_in, d, dtype)
+    hidden = synth.make_hidden_queries(6302, N, d_in, dtype)
+    keys = _build(hidden, dtype, mean, var, W, None)
+    toks = torch.arange(N, dtype=torch.int32, device="cuda").reshape(N, 1).contiguous()
+    st = binding.Store(keys, toks, dtype)
+    dm, dv = torch.from_numpy(mean).cuda(), torch.from_numpy(var).cuda()
+    dW = binding.to_device(W, dtype)
+    st.set_preprocess(d_in, dm, dv, 1e-5, dW, None)
+    idx = np.random.default_rng(6303).integers(0, N, size=32)
+    ids, sc, tok = st.retrieve(binding.to_device(hidden[idx], dtype), 1, 1)
+    torch.cuda.synchronize()
+    st.status()
+    assert np.array_equal(ids.cpu().numpy()[:, 0], idx)
+    assert np.array_equal(tok.cpu().numpy()[:, 0, 0], idx)
+    np.testing.assert_allclose(sc.cpu().numpy()[:, 0], 1.0, atol=2.0 ** -7)
+    st.close()
