@@ -49,6 +49,10 @@ def parse_args():
     ap.add_argument("--top-n", type=int, default=None, help="override top_n (debugging; not a bench value)")
     ap.add_argument("--oracle-queries", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--build-keys", action="store_true",
+                    help="time dresd_build_keys (datastore-side Eq. 1 -> v W -> Eq. 2, a tensor-bound GEMM) instead")
+    ap.add_argument("--d-in", type=int, default=4096)
+    ap.add_argument("--d-out", type=int, default=256)
     ap.add_argument("--first-token-filter", action="store_true",
                     help="time dresd_retrieve_filtered: each query wants the first stored token of its source row")
     ap.add_argument("--probe", type=int, default=1, help="probe-pass tile stride (0 off, 1 default)")
@@ -364,9 +368,67 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_build_keys(args):
+    """Datastore-side preprocessing: rows/s and achieved tensor throughput of dresd_build_keys."""
+    import torch
+    from paper_2502_15572_b200 import binding, build as lib_build
+    lib_build.build()
+    torch.cuda.set_device(0)
+    torch.manual_seed(1234)
+    N, d_in, d = args.rows or 2_000_000, args.d_in, args.d_out
+    H = torch.randn((N, d_in), device="cuda", dtype=torch.bfloat16)
+    W = (torch.randn((d_in, d), device="cuda") / d_in ** 0.5).to(torch.bfloat16)
+    mean = 0.5 * torch.randn(d_in, device="cuda")
+    var = 0.5 + torch.rand(d_in, device="cuda")
+    out = torch.empty((N, d), device="cuda", dtype=torch.bfloat16)
+    s = torch.cuda.current_stream().cuda_stream
+
+    def step():
+        binding.dresd_build_keys(H.data_ptr(), N, d_in, binding.DRESD_BF16, mean.data_ptr(), var.data_ptr(), 1e-5,
+                                 W.data_ptr(), d, None, out.data_ptr(), s)
+
+    steps, warm = min(args.steps, 20), max(3, min(args.warmup, 5))
+    for _ in range(warm):
+        step()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1) / steps            # includes the per-call scratch set-up of W
+    flops = 2.0 * N * d_in * d * 2                # the two 16-bit terms of W / sigma are both multiplied
+    peak = 1404.5
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        peak = float(json.load(open(pk))["bf16_tflops_sustained"])
+    tf = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "datastore rows preprocessed/s (Eq. 1 -> v W -> Eq. 2), bf16 hidden states",
+        "value": N / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1, "steps": steps, "warmup": warm,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 accumulate over bf16 operands", "data": "synthetic",
+        "config": {"workload": "build_keys", "N": N, "d_in": d_in, "d": d,
+                   "l2": "hidden states are %.1f GB per step: no flush needed" % (N * d_in * 2 / 1e9)},
+        "gpu_launches": 2 * steps,
+        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
+        "roofline": {"bound": "tensor", "kernel": "build_keys (tcgen05 GEMM + fused normalisation)",
+                     "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                     "peak_source": "measured (MEASURED_PEAKS.json bf16_tflops_sustained)", "traffic": None,
+                     "hbm_read_gbs": N * d_in * 2 / (ms * 1e-3) / 1e9},
+    }))
+
+
 if __name__ == "__main__":
     a = parse_args()
-    if a.impl == "reference":
+    if a.build_keys:
+        run_build_keys(a)
+    elif a.impl == "reference":
         run_reference(a)
     else:
         run_ours(a)

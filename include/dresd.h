@@ -173,8 +173,9 @@ dresd_status dresd_drafts_accept(const int32_t *drafts, const int32_t *valid, co
  *              `dtype` from fp32 accumulation (hidden states enter exactly; W / sigma
  *              is carried as a two-term 16-bit split)
  *
- * Offline operation: allocates a scratch copy of W (4 d d_in bytes), runs on `stream`
- * and RETURNS AFTER THE STREAM HAS FINISHED (the scratch is freed on return).
+ * Offline operation: keeps a scratch copy of W per device (4 d d_in bytes, allocated on
+ * the first call and reused), runs on `stream` and RETURNS AFTER THE STREAM HAS
+ * FINISHED; one build per device at a time.
  */
 dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dtype dtype, const float *mean,
                               const float *var, float eps_z, const void *W, int d, const float *pca_mean,

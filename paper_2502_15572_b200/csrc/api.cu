@@ -4,6 +4,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "../../include/dresd.h"
@@ -679,11 +680,25 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
 
     const size_t kpad = ((size_t)d_in + 63) / 64 * 64;
-    uint8_t *ws = nullptr;
-    if (cudaMalloc(&ws, build_keys_workspace_bytes(d_in, d)) != cudaSuccess) {
-        cudaGetLastError();
-        return fail(DRESD_ERR_ALLOC, "workspace allocation failed");
+    // Scratch for the split copy of W: kept per device between calls (grow-only), so that
+    // building a datastore chunk by chunk does not allocate and free on every call.
+    static std::mutex ws_mutex;
+    static uint8_t *ws_ptr[64] = {};
+    static size_t ws_size[64] = {};
+    if (dev < 0 || dev >= 64) return fail(DRESD_ERR_UNSUPPORTED, "device ordinal beyond 63");
+    std::lock_guard<std::mutex> ws_lock(ws_mutex);      // one build per device at a time
+    const size_t need = build_keys_workspace_bytes(d_in, d);
+    if (ws_size[dev] < need) {
+        cudaFree(ws_ptr[dev]);
+        ws_ptr[dev] = nullptr;
+        ws_size[dev] = 0;
+        if (cudaMalloc(&ws_ptr[dev], need) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(DRESD_ERR_ALLOC, "workspace allocation failed");
+        }
+        ws_size[dev] = need;
     }
+    uint8_t *ws = ws_ptr[dev];
     void *wt_hi = ws, *wt_lo = ws + (size_t)d * kpad * 2;
     float *bias = reinterpret_cast<float *>(ws + 2 * (size_t)d * kpad * 2);
     int *status = reinterpret_cast<int *>(bias + 256);
@@ -703,9 +718,8 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
     int word = 0;
     if (st == DRESD_OK && (e = cudaMemcpyAsync(&word, status, sizeof(int), cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
         st = fail_cuda(e, "status read");
-    e = cudaStreamSynchronize(stream);                 // the workspace is freed below: wait for the kernels
+    e = cudaStreamSynchronize(stream);                 // the scratch is reused by the next call
     if (st == DRESD_OK && e != cudaSuccess) st = fail_cuda(e, "stream synchronize");
-    cudaFree(ws);
     if (st == DRESD_OK && word != 0) st = fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
     return st;
 }
