@@ -7,6 +7,7 @@ from .dresd_oracle import (  # noqa: F401
     build,
     decode,
     preprocess,
+    fit_zscore,
     scores,
     retrieve,
     OracleResult,

@@ -27,7 +27,8 @@
  *     x_{t+1} rules out drafts that do not start with it) is applied BEFORE
  *     the selection: only keys whose first stored token equals first_token[b]
  *     are candidates; when fewer than n exist the tail is id -1, score
- *     -infinity, tokens -1.  first_token NULL or -1 = no filter.
+ *     -infinity, tokens -1.  first_token NULL or -1 = no filter;
+ *   - Var[V] of Eq. 1 is the population variance of the sample (divide by N).
  *
  * Pins (tests/test_oracle_*.py): hand-computed cases, closed forms
  * (unit norm, scale invariance, identity keys), brute-force cross-check
@@ -135,6 +136,30 @@ int dresd_oracle_preprocess(const void *queries, int B, int d_in, int dtype,
         for (int c = 0; c < d; ++c) vl[c] /= den;
     }
     free(v);
+    return 0;
+}
+
+/* ---- statistics of Eq. 1 (Section 3.2): E[V] and Var[V] per dimension -----
+ * V [N][d_in] in `dtype` is the sample of full-size embeddings the statistics
+ * are estimated from.  Two plain passes in float64: the mean, then the mean of
+ * the squared deviations from it.  Reading: Var[V] is the population variance
+ * (divide by N), as in the batch-normalisation form the equation is written in.
+ * mean, var: float64 [d_in] out.  Returns 0, or -1 on bad arguments.          */
+int dresd_oracle_fit_zscore(const void *V, int64_t N, int d_in, int dtype, double *mean, double *var)
+{
+    if (N <= 0 || d_in <= 0) return -1;
+    for (int j = 0; j < d_in; ++j) {
+        double s = 0.0;
+        for (int64_t i = 0; i < N; ++i) s += load_elem(V, i * d_in + j, dtype);
+        const double m = s / (double)N;
+        double q = 0.0;
+        for (int64_t i = 0; i < N; ++i) {
+            const double t = load_elem(V, i * d_in + j, dtype) - m;
+            q += t * t;
+        }
+        mean[j] = m;
+        var[j] = q / (double)N;
+    }
     return 0;
 }
 

@@ -42,6 +42,8 @@ def _load():
         lib.dresd_oracle_preprocess.argtypes = [
             c.c_void_p, c.c_int, c.c_int, c.c_int, c.c_void_p, c.c_void_p, c.c_double,
             c.c_void_p, c.c_int, c.c_void_p, c.c_double, c.c_void_p]
+        lib.dresd_oracle_fit_zscore.restype = c.c_int
+        lib.dresd_oracle_fit_zscore.argtypes = [c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_void_p, c.c_void_p]
         lib.dresd_oracle_scores.restype = c.c_int
         lib.dresd_oracle_scores.argtypes = [c.c_void_p, c.c_int64, c.c_int, c.c_int,
                                             c.c_void_p, c.c_void_p, c.c_int]
@@ -107,6 +109,19 @@ def preprocess(queries, dtype: str, mean=None, var=None, eps_z: float = 1e-5,
     if rc != 0:
         raise ValueError("oracle preprocess: bad arguments")
     return out
+
+
+def fit_zscore(sample, dtype: str):
+    """Statistics of Eq. 1 (Section 3.2) from a sample ``[N][d_in]`` of stored embeddings:
+    ``(mean, var)`` float64 ``[d_in]``, var = population variance."""
+    v = _store_array(sample, dtype)
+    N, d_in = v.shape
+    mean = np.empty(d_in, dtype=np.float64)
+    var = np.empty(d_in, dtype=np.float64)
+    rc = _load().dresd_oracle_fit_zscore(_ptr(v), N, d_in, _DTYPE_CODE[dtype], _ptr(mean), _ptr(var))
+    if rc != 0:
+        raise ValueError("oracle fit_zscore: bad arguments")
+    return mean, var
 
 
 def scores(keys, dtype: str, qhat, threads: int = 1) -> np.ndarray:

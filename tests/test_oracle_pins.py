@@ -315,3 +315,55 @@ def test_first_token_filter_equals_search_of_the_matching_subset():
         assert np.all(got.ids[b, k:] == -1) and np.all(np.isneginf(got.scores[b, k:]))
         if ft[b] >= 0:
             assert np.all(got.tokens[b, :k, 0] == ft[b])
+
+
+# --------------------------------------------------------------------------
+# statistics of Eq. 1 (Section 3.2): E[V], Var[V] from a sample
+# --------------------------------------------------------------------------
+def _as_store(a, dtype):
+    return synth.cast_to_store(np.asarray(a, dtype=np.float32), dtype)
+
+
+@pytest.mark.parametrize("case", GOLDEN["fit_zscore"], ids=lambda c: c["cite"])
+def test_fit_zscore_hand_cases(case):
+    for dtype in case.get("dtypes", ["f32", "f16", "bf16"]):
+        mean, var = oracle.fit_zscore(_as_store(case["V"], dtype), dtype)
+        np.testing.assert_allclose(mean, case["mean"], rtol=0, atol=1e-12)
+        np.testing.assert_allclose(var, case["var"], rtol=1e-12, atol=1e-12)
+
+
+def test_fit_zscore_closed_forms():
+    # 0..N-1 in one column: mean (N-1)/2, population variance (N^2-1)/12
+    N = 1000
+    V = np.stack([np.arange(N), 3.0 - 2.0 * np.arange(N)], axis=1).astype(np.float32)
+    mean, var = oracle.fit_zscore(V, "f32")
+    np.testing.assert_allclose(mean, [(N - 1) / 2, 3.0 - (N - 1)], rtol=1e-14)
+    np.testing.assert_allclose(var, [(N * N - 1) / 12, 4 * (N * N - 1) / 12], rtol=1e-13)
+    # +-1 alternating: mean 0, variance 1; a constant shift moves the mean only
+    pm = np.where(np.arange(64) % 2 == 0, 1.0, -1.0).astype(np.float32)[:, None]
+    for shift in (0.0, 512.0):
+        mean, var = oracle.fit_zscore(_as_store(pm + shift, "f16"), "f16")
+        assert mean[0] == shift and var[0] == 1.0
+
+
+def test_fit_zscore_then_eq1_standardises_the_sample():
+    """Feeding the fitted statistics to Eq. 1 gives the sample mean 0 and variance
+    Var/(Var + eps) per dimension: the definition the statistics exist for."""
+    rng = np.random.default_rng(77)
+    V = (rng.normal(size=(500, 6)) * np.array([0.1, 1, 5, 20, 1, 1]) + np.array([0, 3, -7, 40, 0, 0])).astype(np.float32)
+    Vs = _as_store(V, "bf16")
+    mean, var = oracle.fit_zscore(Vs, "bf16")
+    x = synth.store_to_float32(Vs, "bf16").astype(np.float64)
+    eps = 1e-5
+    z = (x - mean) / np.sqrt(var + eps)
+    np.testing.assert_allclose(z.mean(axis=0), 0.0, atol=1e-12)
+    np.testing.assert_allclose((z * z).mean(axis=0), var / (var + eps), rtol=1e-12)
+    # row order and duplication of the whole sample change nothing
+    m2, v2 = oracle.fit_zscore(np.concatenate([Vs[::-1], Vs]), "bf16")
+    np.testing.assert_allclose(m2, mean, rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(v2, var, rtol=1e-12)
+
+
+def test_fit_zscore_bad_arguments():
+    with pytest.raises(ValueError):
+        oracle.fit_zscore(np.zeros((0, 4), dtype=np.float32), "f32")
