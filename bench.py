@@ -51,6 +51,10 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--build-keys", action="store_true",
                     help="time dresd_build_keys (datastore-side Eq. 1 -> v W -> Eq. 2, a tensor-bound GEMM) instead")
+    ap.add_argument("--fit-zscore", action="store_true",
+                    help="time dresd_fit_zscore (Eq. 1 statistics over --rows x --d-in bf16 embeddings) instead")
+    ap.add_argument("--no-zscore", action="store_true",
+                    help="--build-keys: projection and Eq. 2 only (W is exact in 16 bits: one tensor-core term)")
     ap.add_argument("--d-in", type=int, default=4096)
     ap.add_argument("--d-out", type=int, default=256)
     ap.add_argument("--first-token-filter", action="store_true",
@@ -382,9 +386,11 @@ def run_build_keys(args):
     var = 0.5 + torch.rand(d_in, device="cuda")
     out = torch.empty((N, d), device="cuda", dtype=torch.bfloat16)
     s = torch.cuda.current_stream().cuda_stream
+    terms = 1 if args.no_zscore else 2
+    m_ptr, v_ptr = (None, None) if args.no_zscore else (mean.data_ptr(), var.data_ptr())
 
     def step():
-        binding.dresd_build_keys(H.data_ptr(), N, d_in, binding.DRESD_BF16, mean.data_ptr(), var.data_ptr(), 1e-5,
+        binding.dresd_build_keys(H.data_ptr(), N, d_in, binding.DRESD_BF16, m_ptr, v_ptr, 1e-5,
                                  W.data_ptr(), d, None, out.data_ptr(), s)
 
     steps, warm = min(args.steps, 20), max(3, min(args.warmup, 5))
@@ -402,7 +408,7 @@ def run_build_keys(args):
     torch.cuda.synchronize()
     clocks = sampler.stop()
     ms = ev0.elapsed_time(ev1) / steps            # includes the per-call scratch set-up of W
-    flops = 2.0 * N * d_in * d * 2                # the two 16-bit terms of W / sigma are both multiplied
+    flops = 2.0 * N * d_in * d * terms            # with Eq. 1, both 16-bit terms of W / sigma are multiplied
     peak = 1404.5
     pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(pk):
@@ -413,7 +419,8 @@ def run_build_keys(args):
         "value": N / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1, "steps": steps, "warmup": warm,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 accumulate over bf16 operands", "data": "synthetic",
-        "config": {"workload": "build_keys", "N": N, "d_in": d_in, "d": d,
+        "config": {"workload": "build_keys", "N": N, "d_in": d_in, "d": d, "zscore": not args.no_zscore,
+                   "tensor_terms": terms,
                    "l2": "hidden states are %.1f GB per step: no flush needed" % (N * d_in * 2 / 1e9)},
         "gpu_launches": 2 * steps,
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
@@ -424,9 +431,61 @@ def run_build_keys(args):
     }))
 
 
+def run_fit_zscore(args):
+    """Statistics of Eq. 1 over a sample of embeddings: rows/s and achieved HBM bandwidth of dresd_fit_zscore."""
+    import torch
+    from paper_2502_15572_b200 import binding, build as lib_build
+    lib_build.build()
+    torch.cuda.set_device(0)
+    torch.manual_seed(4321)
+    N, d_in = args.rows or 1_000_000, args.d_in
+    V = (torch.randn((N, d_in), device="cuda") * 2.0 + 0.5).to(torch.bfloat16)
+    mean = torch.empty(d_in, device="cuda")
+    var = torch.empty(d_in, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+
+    def step():
+        binding.dresd_fit_zscore(V.data_ptr(), N, d_in, binding.DRESD_BF16, mean.data_ptr(), var.data_ptr(), s)
+
+    steps, warm = min(args.steps, 50), max(3, min(args.warmup, 5))
+    for _ in range(warm):
+        step()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1) / steps            # three launches and the call's stream synchronisation
+    peak, src = 6650.0, "fallback"
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        peak, src = float(json.load(open(pk))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    gbs = N * d_in * 2 / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "sample rows reduced/s (Eq. 1 statistics E[V], Var[V]), bf16 embeddings",
+        "value": N / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1, "steps": steps, "warmup": warm,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32 chunk sums folded into f64", "data": "synthetic",
+        "config": {"workload": "fit_zscore", "N": N, "d_in": d_in,
+                   "l2": "the sample is %.1f GB per step: no flush needed" % (N * d_in * 2 / 1e9)},
+        "gpu_launches": 3 * steps,
+        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
+        "roofline": {"bound": "hbm", "kernel": "fit_sums_kernel (whole call timed)", "achieved": gbs, "peak": peak,
+                     "unit": "GB/s", "frac": gbs / peak, "peak_source": src, "traffic": None},
+    }))
+
+
 if __name__ == "__main__":
     a = parse_args()
-    if a.build_keys:
+    if a.fit_zscore:
+        run_fit_zscore(a)
+    elif a.build_keys:
         run_build_keys(a)
     elif a.impl == "reference":
         run_reference(a)

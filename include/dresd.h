@@ -171,7 +171,8 @@ dresd_status dresd_drafts_accept(const int32_t *drafts, const int32_t *valid, co
  *   pca_mean   device fp32 [d_in] or NULL, subtracted after Eq. 1
  *   out_keys   device, [N][d] row-major in `dtype`: unit-length rows, rounded to
  *              `dtype` from fp32 accumulation (hidden states enter exactly; W / sigma
- *              is carried as a two-term 16-bit split)
+ *              is carried as a two-term 16-bit split; without mean/var W itself is
+ *              exact and a single term is multiplied, at half the tensor work)
  *
  * Offline operation: keeps a scratch copy of W per device (4 d d_in bytes, allocated on
  * the first call and reused), runs on `stream` and RETURNS AFTER THE STREAM HAS
@@ -180,6 +181,27 @@ dresd_status dresd_drafts_accept(const int32_t *drafts, const int32_t *valid, co
 dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dtype dtype, const float *mean,
                               const float *var, float eps_z, const void *W, int d, const float *pca_mean,
                               void *out_keys, void *stream);
+
+/*
+ * The statistics of Eq. 1, Section 3.2: E[V] and Var[V] per embedding dimension,
+ * estimated from a sample V of full-size token embeddings (the paper samples about
+ * a million rows of the datastore's hidden states).  Var is the population variance
+ * (divide by N; the equation has the batch-normalisation form).  One streaming pass.
+ *
+ *   sample     device, [N][d_in] row-major, fp16 or bf16 (`dtype`), 16-byte aligned;
+ *              N >= 1, d_in a multiple of 8, at most 16384
+ *   out_mean   device fp32 [d_in]
+ *   out_var    device fp32 [d_in]; exactly 0 for a constant column
+ *
+ * The outputs are what dresd_store_set_preprocess() and dresd_build_keys() take as
+ * mean / var.  Sums are shifted per column and carried in float64, so the result is
+ * accurate to fp32 rounding also when |E| >> sqrt(Var); it does not depend on the
+ * launch (fixed summation order).  Offline operation like dresd_build_keys(): uses the
+ * same per-device scratch, runs on `stream` and RETURNS AFTER THE STREAM HAS FINISHED.
+ * Fitting W (the PCA of Section 3.3, an eigen-decomposition) is not part of this library.
+ */
+dresd_status dresd_fit_zscore(const void *sample, int64_t N, int d_in, dresd_dtype dtype, float *out_mean,
+                              float *out_var, void *stream);
 
 /*
  * Exchange step of a datastore whose rows are sharded over P GPUs.  Eq. 3 is an arg

@@ -29,7 +29,7 @@ EXPORTS = (
     "dresd_last_error",
     "dresd_store_destroy", "dresd_retrieve_noalloc", "dresd_store_enable_first_token_filter",
     "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
-    "dresd_merge_shards", "dresd_build_keys",
+    "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore",
 )
 
 
@@ -91,6 +91,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_merge_shards.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_build_keys.restype = i32
     lib.dresd_build_keys.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, i32, vp, vp, vp]
+    lib.dresd_fit_zscore.restype = i32
+    lib.dresd_fit_zscore.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     lib.dresd_retrieve_noalloc.restype = i32
     lib.dresd_retrieve_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
     if path is None:
@@ -159,6 +161,12 @@ def dresd_build_keys(hidden_ptr: int, N: int, d_in: int, dtype: int, mean_ptr, v
     """Eq. 1 -> v W -> Eq. 2 over N rows of hidden states: builds the datastore's key matrix."""
     _check(load().dresd_build_keys(hidden_ptr, N, d_in, dtype, mean_ptr, var_ptr, eps_z, W_ptr, d, pca_mean_ptr,
                                    out_keys_ptr, stream))
+
+
+def dresd_fit_zscore(sample_ptr: int, N: int, d_in: int, dtype: int, out_mean_ptr: int, out_var_ptr: int,
+                     stream: int = 0) -> None:
+    """E[V] and population Var[V] of Eq. 1 from a sample of N stored embeddings."""
+    _check(load().dresd_fit_zscore(sample_ptr, N, d_in, dtype, out_mean_ptr, out_var_ptr, stream))
 
 
 def dresd_retrieve_host(store: int, queries_ptr: int, B: int, top_n: int, draft_len: int,

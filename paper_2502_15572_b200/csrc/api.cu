@@ -311,6 +311,32 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
 
 }  // namespace
 
+namespace {
+// Scratch of the datastore-building calls (the split copy of W, partial sums): kept per device
+// between calls and only ever grown, so that building a datastore chunk by chunk does not
+// allocate and free on every call.  Callers hold g_scratch_mutex until their work has finished.
+constexpr int kScratchDevices = 64;
+std::mutex g_scratch_mutex;
+uint8_t *g_scratch_ptr[kScratchDevices] = {};
+size_t g_scratch_size[kScratchDevices] = {};
+
+uint8_t *device_scratch(int dev, size_t need)
+{
+    if (g_scratch_size[dev] < need) {
+        cudaFree(g_scratch_ptr[dev]);
+        g_scratch_ptr[dev] = nullptr;
+        g_scratch_size[dev] = 0;
+        if (cudaMalloc(&g_scratch_ptr[dev], need) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        g_scratch_size[dev] = need;
+    }
+    return g_scratch_ptr[dev];
+}
+
+}  // namespace
+
 extern "C" {
 
 dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, int64_t N, int d,
@@ -680,25 +706,10 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
 
     const size_t kpad = ((size_t)d_in + 63) / 64 * 64;
-    // Scratch for the split copy of W: kept per device between calls (grow-only), so that
-    // building a datastore chunk by chunk does not allocate and free on every call.
-    static std::mutex ws_mutex;
-    static uint8_t *ws_ptr[64] = {};
-    static size_t ws_size[64] = {};
-    if (dev < 0 || dev >= 64) return fail(DRESD_ERR_UNSUPPORTED, "device ordinal beyond 63");
-    std::lock_guard<std::mutex> ws_lock(ws_mutex);      // one build per device at a time
-    const size_t need = build_keys_workspace_bytes(d_in, d);
-    if (ws_size[dev] < need) {
-        cudaFree(ws_ptr[dev]);
-        ws_ptr[dev] = nullptr;
-        ws_size[dev] = 0;
-        if (cudaMalloc(&ws_ptr[dev], need) != cudaSuccess) {
-            cudaGetLastError();
-            return fail(DRESD_ERR_ALLOC, "workspace allocation failed");
-        }
-        ws_size[dev] = need;
-    }
-    uint8_t *ws = ws_ptr[dev];
+    if (dev < 0 || dev >= kScratchDevices) return fail(DRESD_ERR_UNSUPPORTED, "device ordinal beyond 63");
+    std::lock_guard<std::mutex> ws_lock(g_scratch_mutex);      // one build per device at a time
+    uint8_t *ws = device_scratch(dev, build_keys_workspace_bytes(d_in, d));
+    if (!ws) return fail(DRESD_ERR_ALLOC, "workspace allocation failed");
     void *wt_hi = ws, *wt_lo = ws + (size_t)d * kpad * 2;
     float *bias = reinterpret_cast<float *>(ws + 2 * (size_t)d * kpad * 2);
     int *status = reinterpret_cast<int *>(bias + 256);
@@ -712,7 +723,7 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
     if (st == DRESD_OK && (e = launch_build_prep(W, (int)dtype, mean, var, eps_z, pca_mean, d_in, d, wt_hi, wt_lo, bias,
                                                  stream)) != cudaSuccess)
         st = fail_cuda(e, "build prep launch");
-    if (st == DRESD_OK && (e = launch_build_keys(h_map, whi_map, wlo_map, (int)dtype, N, d_in, d, bias, out_keys,
+    if (st == DRESD_OK && (e = launch_build_keys(h_map, whi_map, wlo_map, (int)dtype, N, d_in, d, mean ? 2 : 1, bias, out_keys,
                                                  kEpsNorm, status, sms, stream)) != cudaSuccess)
         st = fail_cuda(e, "build keys launch");
     int word = 0;
@@ -721,6 +732,36 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
     e = cudaStreamSynchronize(stream);                 // the scratch is reused by the next call
     if (st == DRESD_OK && e != cudaSuccess) st = fail_cuda(e, "stream synchronize");
     if (st == DRESD_OK && word != 0) st = fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
+    return st;
+}
+
+dresd_status dresd_fit_zscore(const void *sample, int64_t N, int d_in, dresd_dtype dtype, float *out_mean,
+                              float *out_var, void *stream_v)
+{
+    if (dtype != DRESD_F16 && dtype != DRESD_BF16)
+        return fail(DRESD_ERR_UNSUPPORTED, "dresd_fit_zscore reads 16-bit embeddings (fp16 or bf16)");
+    if (N <= 0) return fail(DRESD_ERR_INVALID, "N = %lld must be positive", (long long)N);
+    if (d_in < 8 || d_in % 8 != 0) return fail(DRESD_ERR_INVALID, "d_in = %d must be a positive multiple of 8", d_in);
+    if (d_in > 16384) return fail(DRESD_ERR_UNSUPPORTED, "d_in = %d exceeds 16384", d_in);
+    if (!is_device_ptr(sample) || !is_device_ptr(out_mean) || !is_device_ptr(out_var))
+        return fail(DRESD_ERR_INVALID, "sample/out_mean/out_var must be device pointers");
+    if (reinterpret_cast<uintptr_t>(sample) % 16 != 0) return fail(DRESD_ERR_INVALID, "sample not 16-byte aligned");
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail_cuda(e, "cudaGetDevice");
+    if (dev < 0 || dev >= kScratchDevices) return fail(DRESD_ERR_UNSUPPORTED, "device ordinal beyond 63");
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return fail_cuda(e, "SM count");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    std::lock_guard<std::mutex> ws_lock(g_scratch_mutex);
+    uint8_t *ws = device_scratch(dev, fit_zscore_workspace_bytes(N, d_in, sms));
+    if (!ws) return fail(DRESD_ERR_ALLOC, "workspace allocation failed");
+    dresd_status st = DRESD_OK;
+    if ((e = launch_fit_zscore(sample, (int)dtype, N, d_in, sms, ws, out_mean, out_var, stream)) != cudaSuccess)
+        st = fail_cuda(e, "fit_zscore launch");
+    e = cudaStreamSynchronize(stream);                 // the scratch is reused by the next call
+    if (st == DRESD_OK && e != cudaSuccess) st = fail_cuda(e, "stream synchronize");
     return st;
 }
 

@@ -139,6 +139,7 @@ __global__ void build_prep_kernel(const T *__restrict__ W, const float *__restri
 struct BuildArgs {
     long long N;
     int d_in, d, n_tiles, stages;
+    int terms;               // 2: W' = hi + lo; 1: W' is exact in 16 bits (no z-score), lo is not read
     const float *bias;       // [d]
     void *out;               // [N][d] store dtype
     float eps_n;
@@ -156,7 +157,7 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
     const int n_stages = a.stages;
     const int kslabs = (a.d_in + kSlabElems - 1) / kSlabElems;
     const int b_slab = a.d * kSlabBytes;                    // one 64-column slab of W'^T (hi or lo)
-    const int stage_bytes = 2 * kASlab + 2 * b_slab;
+    const int stage_bytes = 2 * kASlab + a.terms * b_slab;
     uint8_t *stages = base;
     float *bias_s = reinterpret_cast<float *>(stages + (size_t)n_stages * stage_bytes);
     uint64_t *full = reinterpret_cast<uint64_t *>(bias_s + 256);
@@ -210,7 +211,7 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
                 tma_load_2d(dst, &h_map, ks * kSlabElems, tile * kTileRows, &full[s]);
                 tma_load_2d(dst + kASlab, &h_map, ks * kSlabElems, tile * kTileRows + kSubRows, &full[s]);
                 tma_load_2d(dst + 2 * kASlab, &whi_map, ks * kSlabElems, 0, &full[s]);
-                tma_load_2d(dst + 2 * kASlab + b_slab, &wlo_map, ks * kSlabElems, 0, &full[s]);
+                if (a.terms == 2) tma_load_2d(dst + 2 * kASlab + b_slab, &wlo_map, ks * kSlabElems, 0, &full[s]);
                 issued = it + 1;
             }
             for (int it = max(0, issued - n_stages); it < issued; ++it)
@@ -225,6 +226,7 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
             const uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(a.d >> 3) << 17) |
                                    ((uint32_t)(kSubRows >> 4) << 24);
             bool ok = true;
+            const bool two = a.terms == 2;
             for (int tl = 0; tl < my_tiles && ok; ++tl) {
                 // one accumulator set: wait until the epilogue has drained the previous tile
                 if (tl >= 1 && !mbar_wait(tempty, (tl - 1) & 1)) { ok = false; break; }
@@ -243,7 +245,7 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
                             umma_f16(dt, ad + 2 * k, bhi + 2 * k, idesc, (ks | k) != 0);
-                            umma_f16(dt, ad + 2 * k, blo + 2 * k, idesc, 1);
+                            if (two) umma_f16(dt, ad + 2 * k, blo + 2 * k, idesc, 1);
                         }
                     }
                     tc_commit(&empty[s]);
@@ -343,10 +345,11 @@ cudaError_t launch_build_prep(const void *W, int dtype, const float *mean, const
 }
 
 cudaError_t launch_build_keys(const CUtensorMap &h_map, const CUtensorMap &whi_map, const CUtensorMap &wlo_map,
-                              int dtype, long long N, int d_in, int d, const float *bias, void *out, float eps_n,
-                              int *status, int grid, cudaStream_t stream)
+                              int dtype, long long N, int d_in, int d, int terms, const float *bias, void *out,
+                              float eps_n, int *status, int grid, cudaStream_t stream)
 {
     BuildArgs a{};
+    a.terms = terms == 1 ? 1 : 2;
     a.N = N;
     a.d_in = d_in;
     a.d = d;
@@ -355,7 +358,7 @@ cudaError_t launch_build_keys(const CUtensorMap &h_map, const CUtensorMap &whi_m
     a.out = out;
     a.eps_n = eps_n;
     a.status = status;
-    const size_t stage = 2 * (size_t)kASlab + 2 * (size_t)d * kSlabBytes;
+    const size_t stage = 2 * (size_t)kASlab + (size_t)a.terms * d * kSlabBytes;
     const size_t fixed = 1024 + 256 * sizeof(float) + sizeof(uint64_t) * (2 * kMaxStages + 2) + 64;
     long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)stage;
     if (s > kMaxStages) s = kMaxStages;

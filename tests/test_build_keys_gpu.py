@@ -39,6 +39,10 @@ def _build(hidden, dtype, mean, var, W, pca_mean, eps_z=1e-5):
     ("bf16", 700, 200, 128, False, False),        # d_in not a multiple of 64, no z-scoring
     ("f16", 257, 1024, 96, True, False),
     ("bf16", 40000, 256, 32, True, True),         # many tiles per CTA
+    # projection only: W is exact in 16 bits, the kernel multiplies by one term
+    ("bf16", 2500, 4096, 256, False, True),
+    ("f16", 900, 1024, 64, False, False),
+    ("f16", 38000, 320, 160, False, True),
 ])
 def test_build_keys_matches_oracle_preprocess(dtype, N, d_in, d, zscore, centre):
     mean, var, W = synth.make_preprocess(6100 + d, d_in, d, dtype)
