@@ -53,6 +53,8 @@ def parse_args():
                     help="time dresd_build_keys (datastore-side Eq. 1 -> v W -> Eq. 2, a tensor-bound GEMM) instead")
     ap.add_argument("--fit-zscore", action="store_true",
                     help="time dresd_fit_zscore (Eq. 1 statistics over --rows x --d-in bf16 embeddings) instead")
+    ap.add_argument("--single-cta", action="store_true",
+                    help="--build-keys: one CTA per tile instead of CTA pairs (cta_group::2)")
     ap.add_argument("--no-zscore", action="store_true",
                     help="--build-keys: projection and Eq. 2 only (W is exact in 16 bits: one tensor-core term)")
     ap.add_argument("--d-in", type=int, default=4096)
@@ -387,6 +389,7 @@ def run_build_keys(args):
     out = torch.empty((N, d), device="cuda", dtype=torch.bfloat16)
     s = torch.cuda.current_stream().cuda_stream
     terms = 1 if args.no_zscore else 2
+    binding.dresd_set_global_option("build_keys_pairs", 0 if args.single_cta else 1)
     m_ptr, v_ptr = (None, None) if args.no_zscore else (mean.data_ptr(), var.data_ptr())
 
     def step():
@@ -420,7 +423,7 @@ def run_build_keys(args):
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32 accumulate over bf16 operands", "data": "synthetic",
         "config": {"workload": "build_keys", "N": N, "d_in": d_in, "d": d, "zscore": not args.no_zscore,
-                   "tensor_terms": terms,
+                   "tensor_terms": terms, "cta_pairs": not args.single_cta,
                    "l2": "hidden states are %.1f GB per step: no flush needed" % (N * d_in * 2 / 1e9)},
         "gpu_launches": 2 * steps,
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},

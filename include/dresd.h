@@ -204,6 +204,15 @@ dresd_status dresd_fit_zscore(const void *sample, int64_t N, int d_in, dresd_dty
                               float *out_var, void *stream);
 
 /*
+ * Process-wide switches (not part of the paper; for measurement and tests).
+ *   "build_keys_pairs"  1 (default): dresd_build_keys runs on CTA pairs -- clusters of two
+ *                       CTAs, one tensor-core instruction spanning both SMs, each CTA staging
+ *                       half of the weight slab; 0: one CTA per tile.  Results are identical.
+ * Unknown names and values outside the stated set return DRESD_ERR_INVALID.
+ */
+dresd_status dresd_set_global_option(const char *name, int value);
+
+/*
  * Exchange step of a datastore whose rows are sharded over P GPUs.  Eq. 3 is an arg
  * max over the whole datastore; with the rows split into disjoint shards, the top_n
  * of the whole is the top_n of the union of the shards' top_n.  Each shard runs

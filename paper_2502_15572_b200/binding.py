@@ -29,7 +29,7 @@ EXPORTS = (
     "dresd_last_error",
     "dresd_store_destroy", "dresd_retrieve_noalloc", "dresd_store_enable_first_token_filter",
     "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
-    "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore",
+    "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore", "dresd_set_global_option",
 )
 
 
@@ -91,6 +91,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_merge_shards.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_build_keys.restype = i32
     lib.dresd_build_keys.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, i32, vp, vp, vp]
+    lib.dresd_set_global_option.restype = i32
+    lib.dresd_set_global_option.argtypes = [ctypes.c_char_p, i32]
     lib.dresd_fit_zscore.restype = i32
     lib.dresd_fit_zscore.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     lib.dresd_retrieve_noalloc.restype = i32
@@ -161,6 +163,10 @@ def dresd_build_keys(hidden_ptr: int, N: int, d_in: int, dtype: int, mean_ptr, v
     """Eq. 1 -> v W -> Eq. 2 over N rows of hidden states: builds the datastore's key matrix."""
     _check(load().dresd_build_keys(hidden_ptr, N, d_in, dtype, mean_ptr, var_ptr, eps_z, W_ptr, d, pca_mean_ptr,
                                    out_keys_ptr, stream))
+
+
+def dresd_set_global_option(name: str, value: int) -> None:
+    _check(load().dresd_set_global_option(name.encode(), int(value)))
 
 
 def dresd_fit_zscore(sample_ptr: int, N: int, d_in: int, dtype: int, out_mean_ptr: int, out_var_ptr: int,

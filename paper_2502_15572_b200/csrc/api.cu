@@ -4,6 +4,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 #include <new>
 
@@ -319,6 +320,8 @@ constexpr int kScratchDevices = 64;
 std::mutex g_scratch_mutex;
 uint8_t *g_scratch_ptr[kScratchDevices] = {};
 size_t g_scratch_size[kScratchDevices] = {};
+
+std::atomic<int> g_build_pairs{1};      // dresd_build_keys on CTA pairs (cta_group::2); 0 = one CTA per tile
 
 uint8_t *device_scratch(int dev, size_t need)
 {
@@ -715,15 +718,18 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
     int *status = reinterpret_cast<int *>(bias + 256);
     dresd_status st = DRESD_OK;
     CUtensorMap h_map, whi_map, wlo_map;
-    if (!make_map(&h_map, hidden, (int)dtype, N, d_in, 128) || !make_map(&whi_map, wt_hi, (int)dtype, d, (int)kpad, d) ||
-        !make_map(&wlo_map, wt_lo, (int)dtype, d, (int)kpad, d))
+    const int pair = g_build_pairs.load() != 0 ? 1 : 0;            // CTA pairs stage half of W' each
+    const int w_box = pair ? d / 2 : d;
+    if (!make_map(&h_map, hidden, (int)dtype, N, d_in, 128) ||
+        !make_map(&whi_map, wt_hi, (int)dtype, d, (int)kpad, w_box) ||
+        !make_map(&wlo_map, wt_lo, (int)dtype, d, (int)kpad, w_box))
         st = fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed");
     if (st == DRESD_OK && (e = cudaMemsetAsync(status, 0, sizeof(int), stream)) != cudaSuccess)
         st = fail_cuda(e, "status reset");
     if (st == DRESD_OK && (e = launch_build_prep(W, (int)dtype, mean, var, eps_z, pca_mean, d_in, d, wt_hi, wt_lo, bias,
                                                  stream)) != cudaSuccess)
         st = fail_cuda(e, "build prep launch");
-    if (st == DRESD_OK && (e = launch_build_keys(h_map, whi_map, wlo_map, (int)dtype, N, d_in, d, mean ? 2 : 1, bias, out_keys,
+    if (st == DRESD_OK && (e = launch_build_keys(h_map, whi_map, wlo_map, (int)dtype, N, d_in, d, mean ? 2 : 1, pair, bias, out_keys,
                                                  kEpsNorm, status, sms, stream)) != cudaSuccess)
         st = fail_cuda(e, "build keys launch");
     int word = 0;
@@ -733,6 +739,17 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
     if (st == DRESD_OK && e != cudaSuccess) st = fail_cuda(e, "stream synchronize");
     if (st == DRESD_OK && word != 0) st = fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
     return st;
+}
+
+dresd_status dresd_set_global_option(const char *name, int value)
+{
+    if (!name) return fail(DRESD_ERR_INVALID, "option name is NULL");
+    if (std::strcmp(name, "build_keys_pairs") == 0) {
+        if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "build_keys_pairs takes 0 or 1");
+        g_build_pairs.store(value);
+        return DRESD_OK;
+    }
+    return fail(DRESD_ERR_INVALID, "unknown global option '%s'", name);
 }
 
 dresd_status dresd_fit_zscore(const void *sample, int64_t N, int d_in, dresd_dtype dtype, float *out_mean,

@@ -108,14 +108,15 @@ cudaError_t launch_merge_shards(const int32_t *ids, const float *scores, const i
 
 // ---- K7: datastore-side preprocessing (Eq. 1 -> v W -> Eq. 2 over N rows), a tcgen05 GEMM ----
 // `terms` = 2 multiplies by W' = hi + lo (needed when Eq. 1 scales the weights), 1 by hi alone
-// (exact when there is no z-score: W' is W).
+// (exact when there is no z-score: W' is W).  `pair` != 0 runs the kernel on CTA pairs
+// (cta_group::2, clusters of two); the W' tensor maps must then have boxes of d/2 rows.
 size_t build_keys_workspace_bytes(int d_in, int d);
 cudaError_t launch_build_prep(const void *W, int dtype, const float *mean, const float *var, float eps_z,
                               const float *pca_mean, int d_in, int d, void *wt_hi, void *wt_lo, float *bias,
                               cudaStream_t stream);
 cudaError_t launch_build_keys(const CUtensorMap &h_map, const CUtensorMap &whi_map, const CUtensorMap &wlo_map,
-                              int dtype, long long N, int d_in, int d, int terms, const float *bias, void *out,
-                              float eps_n, int *status, int grid, cudaStream_t stream);
+                              int dtype, long long N, int d_in, int d, int terms, int pair, const float *bias,
+                              void *out, float eps_n, int *status, int grid, cudaStream_t stream);
 
 // ---- K8: statistics of Eq. 1 (Section 3.2) from a sample of embeddings, one streaming pass ----
 size_t fit_zscore_workspace_bytes(long long N, int d_in, int sms);

@@ -44,7 +44,16 @@ def _build(hidden, dtype, mean, var, W, pca_mean, eps_z=1e-5):
     ("f16", 900, 1024, 64, False, False),
     ("f16", 38000, 320, 160, False, True),
 ])
-def test_build_keys_matches_oracle_preprocess(dtype, N, d_in, d, zscore, centre):
+@pytest.mark.parametrize("pairs", [1, 0], ids=["cta_pairs", "single_cta"])
+def test_build_keys_matches_oracle_preprocess(dtype, N, d_in, d, zscore, centre, pairs):
+    binding.dresd_set_global_option("build_keys_pairs", pairs)
+    try:
+        _check_build(dtype, N, d_in, d, zscore, centre)
+    finally:
+        binding.dresd_set_global_option("build_keys_pairs", 1)
+
+
+def _check_build(dtype, N, d_in, d, zscore, centre):
     mean, var, W = synth.make_preprocess(6100 + d, d_in, d, dtype)
     hidden = synth.make_hidden_queries(6200 + d, N, d_in, dtype)
     pm = (0.02 * np.cos(np.arange(d_in))).astype(np.float32) if centre else None
@@ -66,6 +75,29 @@ def test_build_keys_matches_oracle_preprocess(dtype, N, d_in, d, zscore, centre)
     assert np.all(err <= 0.5 * ulp + abs_tol), f"max excess {np.max(err - 0.5 * ulp):.2e}"
     assert np.mean(err <= 0.5 * ulp * 1.001) >= 0.9             # the great majority correctly rounded
     np.testing.assert_allclose(np.linalg.norm(got64, axis=1), 1.0, atol=2.0 ** -7)
+
+
+def test_pairs_and_single_cta_give_identical_keys():
+    """The two launch forms run the same products in the same order per row: bit-identical output."""
+    import torch
+    dtype, N, d_in, d = "bf16", 70001, 768, 192
+    mean, var, W = synth.make_preprocess(6401, d_in, d, dtype)
+    hidden = synth.make_hidden_queries(6402, N, d_in, dtype)
+    outs = []
+    for pairs in (1, 0):
+        binding.dresd_set_global_option("build_keys_pairs", pairs)
+        try:
+            outs.append(_build(hidden, dtype, mean, var, W, None).view(torch.int16).cpu())
+        finally:
+            binding.dresd_set_global_option("build_keys_pairs", 1)
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_global_option_rejects_unknown_names():
+    with pytest.raises(binding.DresdError):
+        binding.dresd_set_global_option("no_such_option", 1)
+    with pytest.raises(binding.DresdError):
+        binding.dresd_set_global_option("build_keys_pairs", 7)
 
 
 def test_built_keys_are_searchable_end_to_end():
