@@ -62,6 +62,8 @@ def parse_args():
     ap.add_argument("--first-token-filter", action="store_true",
                     help="time dresd_retrieve_filtered: each query wants the first stored token of its source row")
     ap.add_argument("--probe", type=int, default=1, help="probe-pass tile stride (0 off, 1 default)")
+    ap.add_argument("--keys-as-m", type=int, default=0, choices=[0, 1],
+                    help="1: keep the keys as the M operand of the tcgen05 kernel also for 33-64 queries")
     ap.add_argument("--scan-path", type=int, default=0, choices=[0, 1, 2],
                     help="0 auto, 1 streaming mma.sync kernel, 2 tcgen05 kernel (16-bit keys)")
     return ap.parse_args()
@@ -233,6 +235,7 @@ def run_ours(args):
         store.set_preprocess(cfg["d_in"], W=dW)
     store.set_option("scan_path", args.scan_path)
     store.set_option("probe", args.probe)
+    store.set_option("keys_as_m", args.keys_as_m)
     dft = None
     if args.first_token_filter:
         if "first_tokens" not in cfg:

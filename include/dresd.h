@@ -263,6 +263,10 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "probe"      large batches on large stores first run a probe pass over every
  *                value-th key tile to seed the selection filter; 0 = never,
  *                1 = default stride (128).
+ *   "keys_as_m"  0 (default): batches of 33-64 queries on rows of 129-256 elements run the
+ *                tcgen05 kernel with the queries as the M = 128 and the keys as the
+ *                N = 256 operand of the instruction; 1 = keys as the M operand at every
+ *                batch size (the form all other shapes use).  Results do not change.
  *   "wait_ms"    bound of the device-side waits of the streaming kernels in
  *                milliseconds (0 = default, about 2 s).
  *   "debug_lose_stage"  test hook: in the next calls the streaming 16-bit kernel's

@@ -125,7 +125,7 @@ struct dresd_store {
     CUtensorMap map_umma;
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     // options / bookkeeping
-    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select;
+    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m;
     double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
     cudaStream_t last_stream;
     int last_launches;
@@ -177,7 +177,8 @@ dresd_status check_retrieve_args(const dresd_store *s, const void *queries, int 
 }
 
 // K1 for B queries into the store's workspace.
-dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows, cudaStream_t stream)
+dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows, cudaStream_t stream,
+                            int split_blocked = 0)
 {
     PreprocessArgs p{};
     p.queries = queries;
@@ -197,6 +198,7 @@ dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows
     p.rows = rows;                   // operand rows beyond B are written as zeros
     p.lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
     p.gtau = s->gtau;
+    p.split_blocked = split_blocked;
     cudaError_t e = launch_preprocess(p, stream);
     if (e != cudaSuccess) return fail_cuda(e, "preprocess launch");
     s->last_launches += 1;
@@ -217,10 +219,12 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // streaming kernel stays available as "scan_path" 1 and serves the allocation-free call.
     const bool umma = !f32 && s->opt_path != 1;
     const int op_rows = umma ? scan_umma_operand_rows(B) : 0;
-    dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream);
+    // the kernel with the keys as the N operand reads hi and lo of a query from one TMEM fragment
+    const int blocked = umma && !s->opt_keys_as_m && scan_ummat_eligible(s->d, B);
+    dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream, blocked);
     if (st != DRESD_OK) return st;
 
-    const int umma_rows = umma ? scan_umma_tile_rows(s->d, B) : 1;
+    const int umma_rows = umma ? scan_umma_tile_rows(s->d, B, s->opt_keys_as_m) : 1;
     const int n_tiles = umma ? (int)((s->N + umma_rows - 1) / umma_rows) : s->n_tiles;
     int grid = s->opt_grid > 0 ? s->opt_grid : s->num_sms;
     if (grid > s->max_grid) grid = s->max_grid;
@@ -245,6 +249,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.status = s->status;
         a.gtau = s->gtau;
         a.no_select = s->opt_no_select;
+        a.keys_as_m = s->opt_keys_as_m;
         a.first_col = first_tokens ? s->first_col : nullptr;
         a.want_first = first_tokens;
         const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
@@ -585,6 +590,11 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
     if (strcmp(name, "debug_lose_stage") == 0) {
         if (value < 0) return fail(DRESD_ERR_INVALID, "debug_lose_stage = %d is negative", value);
         s->opt_lose_stage = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "keys_as_m") == 0) {
+        if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "keys_as_m takes 0 or 1");
+        s->opt_keys_as_m = value;
         return DRESD_OK;
     }
     if (strcmp(name, "probe") == 0) {

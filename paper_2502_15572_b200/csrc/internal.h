@@ -30,6 +30,7 @@ struct PreprocessArgs {
     int rows;               // CTAs launched: B rounded up to the operand row count
     float lo_scale;
     unsigned int *gtau;     // [rows] grid-wide filter words, reset to 0 ("nothing known") here
+    int split_blocked;      // qsplit rows: 0 = (2b, 2b+1); 1 = 16-row blocks, hi rows 0-7, lo rows 8-15
 };
 cudaError_t launch_preprocess(const PreprocessArgs &a, cudaStream_t stream);
 
@@ -59,6 +60,7 @@ struct ScanArgs {
     int tile_stride;        // tcgen05 kernel: visit every tile_stride-th tile (probe pass), default 1
     int probe_max;          // tcgen05 kernel, probe pass: keep only each tile's best row per query
     int no_select;          // tcgen05 kernel, measurement only: nothing passes the filter (scan floor)
+    int keys_as_m;          // tcgen05 kernels: never use the form with the keys as the N = 256 operand
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.
 int scan_mma_tile_rows(int d);
@@ -69,10 +71,16 @@ cudaError_t launch_scan_mma(const CUtensorMap &keys_map, const ScanArgs &a, int 
 
 // Batched tensor-core kernel (tcgen05/TMEM, 16-bit keys): 128-row tiles; the query
 // operand holds 2 rows per query, padded to 16/32/64/128 rows.
-int scan_umma_tile_rows(int d, int B);      // 128 x sub-tiles per tile (narrow rows use several)
+int scan_umma_tile_rows(int d, int B, int keys_as_m);   // rows per tile of the kernel that will run
 int scan_umma_operand_rows(int B);
 cudaError_t launch_scan_umma(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
                              int grid, cudaStream_t stream);
+
+// Same path for 33-64 queries on rows of 129-256 elements: queries as the M = 128 operand,
+// keys as the N = 256 operand (256-key tiles).  launch_scan_umma() dispatches to it.
+bool scan_ummat_eligible(int d, int B);
+cudaError_t launch_scan_ummat(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
+                              int grid, cudaStream_t stream);
 
 int scan_f32_tile_rows(int d);
 int scan_f32_queries_per_launch(int d, int B);

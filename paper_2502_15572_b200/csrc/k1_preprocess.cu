@@ -55,8 +55,12 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
-    T *split_hi = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)(2 * b) * a.dpad : nullptr;
-    T *split_lo = split_hi ? split_hi + a.dpad : nullptr;
+    // operand rows of query b: (2b, 2b+1), or -- blocked layout -- rows (b % 8) and 8 + (b % 8)
+    // of the 16-row block b / 8, so that a 16-lane TMEM fragment holds hi and lo of 8 queries
+    const int row_hi = a.split_blocked ? 16 * (b >> 3) + (b & 7) : 2 * b;
+    const int row_lo = a.split_blocked ? row_hi + 8 : row_hi + 1;
+    T *split_hi = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)row_hi * a.dpad : nullptr;
+    T *split_lo = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)row_lo * a.dpad : nullptr;
     float *qrow = a.qhat + (size_t)b * a.d;
     if (tid == 0 && a.gtau) a.gtau[b] = 0u;          // fresh grid-wide filter for this call
 

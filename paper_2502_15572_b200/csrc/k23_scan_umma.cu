@@ -39,46 +39,6 @@ constexpr int kKeyStageBytes = kTileRows * kSlabBytes;     // 16 KB
 constexpr int kMaxStages = 12;
 constexpr int kResidentLimit = 64 * 1024;                  // query operand kept in smem up to this size
 
-// ------------------------------- tcgen05 wrappers -------------------------------
-__device__ __forceinline__ void tmem_alloc(uint32_t *smem_dst, uint32_t ncols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
-                 "r"(ncols)
-                 : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish()
-{
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t *bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
-}
-// D[tmem] (+)= A[smem desc] * B[smem desc]; fp16/bf16 inputs, fp32 accumulate.
-__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                         uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// K-major operand, 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr)
-{
-    return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           (1ull << 46) | (2ull << 61);
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t *r)
 {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
@@ -92,10 +52,6 @@ __device__ __forceinline__ void tmem_ld16p(uint32_t taddr, uint32_t *r)
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld2(uint32_t taddr, uint32_t &v0, uint32_t &v1)
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0,%1}, [%2];" : "=r"(v0), "=r"(v1) : "r"(taddr));
 }
 // CW consecutive accumulator columns of this thread's TMEM lane -> registers.
 template <int CW> __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[CW])
@@ -585,12 +541,18 @@ cudaError_t launch_tsub(const CUtensorMap &kmap, const CUtensorMap &qmap, const 
 
 }  // namespace
 
-int scan_umma_tile_rows(int d, int B) { return kTileRows * tsub_of(d, ncols_of(B)); }
+int scan_umma_tile_rows(int d, int B, int keys_as_m)
+{
+    if (!keys_as_m && scan_ummat_eligible(d, B)) return 256;        // keys are the N = 256 operand there
+    return kTileRows * tsub_of(d, ncols_of(B));
+}
 int scan_umma_operand_rows(int B) { return ncols_of(B); }
 
 cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a_in, int grid,
                              cudaStream_t stream)
 {
+    if (!a_in.keys_as_m && scan_ummat_eligible(a_in.d, a_in.B))
+        return launch_scan_ummat(kmap, qmap, a_in, grid, stream);
     ScanArgs a = a_in;
     if (a.tile_stride < 1) a.tile_stride = 1;
     const Plan p = make_plan(a.d, a.B);
