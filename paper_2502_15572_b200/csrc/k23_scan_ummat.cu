@@ -334,62 +334,83 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
             int next_unit = 0;
             uint32_t pend = 0u;
             bool resume = false;
-            while (true) {
-                const float tau0 = tau[qq0], tau1 = tau[qq0 + 8];
-                if (!dead) {
-                    int u = next_unit;
-                    for (; u < 4; ++u) {                    // warp-uniform
-                        const float tau_r = (u >> 1) ? tau1 : tau0;
-                        const int q = qq0 + 8 * (u >> 1);
-                        uint32_t r[32];
-                        tmem_ld_frag8(unit_addr(u), r);
-                        tmem_ld_wait();
-                        uint32_t m = 0u;
+            // scores of one unit against the filter, survivors queued; true = stop here (queue full)
+            auto process = [&](int u, const uint32_t (&r)[32], float tau_r) -> bool {
+                const int q = qq0 + 8 * (u >> 1);
+                uint32_t m = 0u;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int g = i >> 1, e = i & 1;
-                            const float s = fmaf(__uint_as_float(r[4 * g + 2 + e]), inv, __uint_as_float(r[4 * g + e]));
-                            m |= (s >= tau_r) ? (1u << i) : 0u;
-                        }
-                        if (resume) {
-                            m &= pend;                      // only what was left over in this unit
-                            pend = 0u;
-                            resume = false;
-                        } else if (m) {
-                            m &= slot_mask(u);
-                        }
-                        // Cold part (rare once the filter is warm): a warp-uniform loop over the
-                        // 8-column groups with a survivor in some lane; the group is re-read.
-                        uint32_t wm = __reduce_or_sync(0xFFFFFFFFu, m);
-                        while (wm) {
-                            const int g = (__ffs(wm) - 1) >> 1;
-                            wm &= ~(3u << (2 * g));
-                            uint32_t v[4];                  // hi, hi, lo, lo of my two columns of the group
-                            tmem_ld_frag1(unit_addr(u) + (uint32_t)(8 * g), v);
-                            tmem_ld_wait();
+                for (int i = 0; i < 16; ++i) {
+                    const int g = i >> 1, e = i & 1;
+                    const float s = fmaf(__uint_as_float(r[4 * g + 2 + e]), inv, __uint_as_float(r[4 * g + e]));
+                    m |= (s >= tau_r) ? (1u << i) : 0u;
+                }
+                if (resume) {
+                    m &= pend;                              // only what was left over in this unit
+                    pend = 0u;
+                    resume = false;
+                } else if (m) {
+                    m &= slot_mask(u);
+                }
+                // Cold part (rare once the filter is warm): a warp-uniform loop over the
+                // 8-column groups with a survivor in some lane; the group is re-read.
+                uint32_t wm = __reduce_or_sync(0xFFFFFFFFu, m);
+                if (wm == 0u) return false;
+                while (wm) {
+                    const int g = (__ffs(wm) - 1) >> 1;
+                    wm &= ~(3u << (2 * g));
+                    uint32_t v[4];                          // hi, hi, lo, lo of my two columns of the group
+                    tmem_ld_frag1(unit_addr(u) + (uint32_t)(8 * g), v);
+                    tmem_ld_wait();
 #pragma unroll
-                            for (int e = 0; e < 2; ++e) {
-                                if ((m >> (2 * g + e)) & 1u) {
-                                    const float s = fmaf(__uint_as_float(v[2 + e]), inv, __uint_as_float(v[e]));
-                                    const int slot = atomicAdd(&sel[q].count, 1);
-                                    if (slot < kQueueCap) {
-                                        sel[q].queue[slot] =
-                                            pack_candidate(s, (uint32_t)(key0 + 64 * (u & 1) + 8 * g + e));
-                                        if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
-                                    } else {
-                                        pend |= 1u << (2 * g + e);
-                                        fl->overflow = 1;
-                                    }
-                                }
+                    for (int e = 0; e < 2; ++e) {
+                        if ((m >> (2 * g + e)) & 1u) {
+                            const float s = fmaf(__uint_as_float(v[2 + e]), inv, __uint_as_float(v[e]));
+                            const int slot = atomicAdd(&sel[q].count, 1);
+                            if (slot < kQueueCap) {
+                                sel[q].queue[slot] = pack_candidate(s, (uint32_t)(key0 + 64 * (u & 1) + 8 * g + e));
+                                if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
+                            } else {
+                                pend |= 1u << (2 * g + e);
+                                fl->overflow = 1;
                             }
                         }
-                        if (__any_sync(0xFFFFFFFFu, pend != 0u)) {
-                            resume = true;
+                    }
+                }
+                if (__any_sync(0xFFFFFFFFu, pend != 0u)) {
+                    resume = true;
+                    return true;
+                }
+                return false;
+            };
+            bool first_round = true;
+            while (true) {
+                const float tau0 = tau[qq0], tau1 = tau[qq0 + 8];
+                if (!dead && first_round) {
+                    // all four units, the fragment of the next one in flight while this one is scored
+                    uint32_t ra[32], rb[32];
+                    tmem_ld_frag8(unit_addr(0), ra);
+                    next_unit = 4;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        tmem_ld_wait();
+                        if (u + 1 < 4) tmem_ld_frag8(unit_addr(u + 1), (u & 1) ? ra : rb);
+                        if (process(u, (u & 1) ? rb : ra, (u >> 1) ? tau1 : tau0)) {
+                            next_unit = u;
                             break;
                         }
                     }
+                    tmem_ld_wait();                         // nothing in flight towards registers past this point
+                } else if (!dead) {
+                    int u = next_unit;
+                    for (; u < 4; ++u) {                    // warp-uniform
+                        uint32_t r[32];
+                        tmem_ld_frag8(unit_addr(u), r);
+                        tmem_ld_wait();
+                        if (process(u, r, (u >> 1) ? tau1 : tau0)) break;
+                    }
                     next_unit = u;
                 }
+                first_round = false;
                 epi_bar();                                   // A: every push of this round is visible
                 const int need = fl->need_merge, over = fl->overflow;
                 // Flags rotate over three slots: the slot of the previous round was read by
@@ -436,7 +457,9 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
 
 }  // namespace
 
-// The transposed kernel serves 33-64 queries on rows of three or four 64-element slabs.
+// This kernel serves 33-64 queries on rows of three or four 64-element slabs (129-256 elements).
+// On narrower rows it works too but measured no better than the other tcgen05 kernel (the
+// epilogue, ~2.7 k cycles per 256 keys, is then slower than the memory stream in both).
 bool scan_ummat_eligible(int d, int B)
 {
     const int dslabs = (d + kSlabElems - 1) / kSlabElems;
