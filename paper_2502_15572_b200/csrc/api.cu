@@ -307,11 +307,10 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         cudaEventRecord(s->prof_events[2 * s->prof_count + 1], stream);
         s->prof_count += 1;
     }
-    cudaError_t e = launch_merge(s->cand, grid, B, top_n, out_ids, out_scores, stream);
-    if (e != cudaSuccess) return fail_cuda(e, "merge launch");
-    e = launch_gather(s->next_tokens, s->stored_len, s->N, out_ids, B, top_n, draft_len, out_tokens, stream);
-    if (e != cudaSuccess) return fail_cuda(e, "gather launch");
-    s->last_launches += 2;
+    cudaError_t e = launch_merge_gather(s->cand, grid, B, top_n, out_ids, out_scores, s->next_tokens, s->stored_len,
+                                        s->N, draft_len, out_tokens, stream);
+    if (e != cudaSuccess) return fail_cuda(e, "merge/gather launch");
+    s->last_launches += 1;
     return DRESD_OK;
 }
 

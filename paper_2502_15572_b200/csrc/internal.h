@@ -88,15 +88,14 @@ cudaError_t launch_scan_f32(const CUtensorMap &keys_map, const ScanArgs &a, int 
                             cudaStream_t stream);
 
 // ---- K4: merge the per-CTA lists;  K5: gather continuations ----------------
-cudaError_t launch_merge(const unsigned long long *cand, int grid_lists, int B, int top_n,
-                         int32_t *out_ids, float *out_scores, cudaStream_t stream);
+// Merge of the per-CTA lists and gather of the winners' stored tokens, one kernel.
+cudaError_t launch_merge_gather(const unsigned long long *cand, int grid_lists, int B, int top_n, int32_t *out_ids,
+                                float *out_scores, const int32_t *next_tokens, int stored_len, long long N,
+                                int draft_len, int32_t *out_tokens, cudaStream_t stream);
 // Same merge, but only the n-th best score of each query is kept, as a grid-wide
 // filter word (see share_tau); 0 when fewer than top_n candidates exist.
 cudaError_t launch_merge_tau(const unsigned long long *cand, int grid_lists, int B, int top_n,
                              unsigned int *gtau, cudaStream_t stream);
-cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long N,
-                          const int32_t *ids, int B, int top_n, int draft_len,
-                          int32_t *out_tokens, cudaStream_t stream);
 
 // first_col[i] = next_tokens[i][0]: the compact column the first-token filter reads.
 cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, long long N,

@@ -3,25 +3,32 @@
 // extended to the n best; ties to the lower row index).
 // K5 -- value lookup f_D of Section 3.5: copy the first draft_len stored
 // continuation tokens of every selected key into the n x L draft matrix.
+// Both run in one kernel: the CTA that merged a query's lists gathers its tokens.
 #include "common.cuh"
 #include "internal.h"
 
 namespace dresd {
 namespace {
 
-constexpr int kMergeWarps = 8;
+constexpr int kMergeWarps = 16;
 
+// One CTA per query.  Each warp folds every 16th per-CTA list (four loads in flight before
+// the dependent merge chain), the 16 partial lists are folded pairwise in four rounds, and --
+// fused K5 -- the whole CTA then copies the winners' stored tokens.  Probe pass (gtau set):
+// only the n-th best score is kept, as the grid-wide filter word.
 __global__ void __launch_bounds__(kMergeWarps * 32)
-merge_kernel(const unsigned long long *__restrict__ cand, int lists, int B, int top_n,
-             int32_t *__restrict__ out_ids, float *__restrict__ out_scores, unsigned int *__restrict__ gtau)
+merge_gather_kernel(const unsigned long long *__restrict__ cand, int lists, int B, int top_n,
+                    int32_t *__restrict__ out_ids, float *__restrict__ out_scores, unsigned int *__restrict__ gtau,
+                    const int32_t *__restrict__ next_tokens, int stored_len, long long N, int draft_len,
+                    int32_t *__restrict__ out_tokens)
 {
     __shared__ unsigned long long part[kMergeWarps][kListLen];
+    __shared__ int win[kListLen];
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     unsigned long long m = 0ull;
     int g = warp;
-    // Four loads in flight per lane before the dependent merge chain starts.
     for (; g + 3 * kMergeWarps < lists; g += 4 * kMergeWarps) {
         unsigned long long l0 = cand[((size_t)(g + 0 * kMergeWarps) * B + b) * kCandStride + lane];
         unsigned long long l1 = cand[((size_t)(g + 1 * kMergeWarps) * B + b) * kCandStride + lane];
@@ -36,29 +43,31 @@ merge_kernel(const unsigned long long *__restrict__ cand, int lists, int B, int 
         m = warp_merge_top32(m, cand[((size_t)g * B + b) * kCandStride + lane], lane);
     part[warp][lane] = m;
     __syncthreads();
-    if (warp == 0) {
-        m = part[0][lane];
-        for (int w = 1; w < kMergeWarps; ++w) m = warp_merge_top32(m, part[w][lane], lane);
-        if (gtau) {                       // probe pass: publish the n-th best as the filter
-            if (lane == top_n - 1) gtau[b] = m ? float_to_ordered(candidate_score(m)) : 0u;
-        } else if (lane < top_n) {
-            out_ids[(size_t)b * top_n + lane] = m ? (int32_t)candidate_id(m) : -1;
-            out_scores[(size_t)b * top_n + lane] = m ? candidate_score(m) : -INFINITY;
+    for (int span = kMergeWarps / 2; span >= 1; span >>= 1) {
+        if (warp < span) {
+            m = warp_merge_top32(part[warp][lane], part[warp + span][lane], lane);
+            part[warp][lane] = m;
         }
+        __syncthreads();
     }
-}
-
-__global__ void gather_kernel(const int32_t *__restrict__ next_tokens, int stored_len, long long N,
-                              const int32_t *__restrict__ ids, int top_n, int draft_len,
-                              int32_t *__restrict__ out_tokens)
-{
-    const int b = blockIdx.x;
+    m = part[0][lane];
+    if (gtau) {                           // probe pass: publish the n-th best as the filter
+        if (warp == 0 && lane == top_n - 1) gtau[b] = m ? float_to_ordered(candidate_score(m)) : 0u;
+        return;
+    }
+    if (warp == 0 && lane < top_n) {
+        const int id = m ? (int32_t)candidate_id(m) : -1;
+        out_ids[(size_t)b * top_n + lane] = id;
+        out_scores[(size_t)b * top_n + lane] = m ? candidate_score(m) : -INFINITY;
+        win[lane] = id;
+    }
+    __syncthreads();
+    // K5: the first draft_len stored tokens of every winner (Section 3.5, f_D: k -> v)
     const int total = top_n * draft_len;
     for (int i = threadIdx.x; i < total; i += blockDim.x) {
         const int r = i / draft_len, t = i - r * draft_len;
-        const long long id = ids[(size_t)b * top_n + r];
-        out_tokens[(size_t)b * total + i] =
-            (id >= 0 && id < N) ? next_tokens[(size_t)id * stored_len + t] : -1;
+        const long long id = win[r];
+        out_tokens[(size_t)b * total + i] = (id >= 0 && id < N) ? next_tokens[(size_t)id * stored_len + t] : -1;
     }
 }
 
@@ -84,26 +93,20 @@ cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, lon
     return cudaGetLastError();
 }
 
-cudaError_t launch_merge(const unsigned long long *cand, int lists, int B, int top_n,
-                         int32_t *out_ids, float *out_scores, cudaStream_t stream)
+cudaError_t launch_merge_gather(const unsigned long long *cand, int lists, int B, int top_n, int32_t *out_ids,
+                                float *out_scores, const int32_t *next_tokens, int stored_len, long long N,
+                                int draft_len, int32_t *out_tokens, cudaStream_t stream)
 {
-    merge_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, out_ids, out_scores, nullptr);
+    merge_gather_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, out_ids, out_scores, nullptr,
+                                                           next_tokens, stored_len, N, draft_len, out_tokens);
     return cudaGetLastError();
 }
 
 cudaError_t launch_merge_tau(const unsigned long long *cand, int lists, int B, int top_n, unsigned int *gtau,
                              cudaStream_t stream)
 {
-    merge_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, nullptr, nullptr, gtau);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_gather(const int32_t *next_tokens, int stored_len, long long N, const int32_t *ids,
-                          int B, int top_n, int draft_len, int32_t *out_tokens, cudaStream_t stream)
-{
-    int threads = top_n * draft_len;
-    threads = threads < 32 ? 32 : threads > 512 ? 512 : ((threads + 31) / 32) * 32;
-    gather_kernel<<<B, threads, 0, stream>>>(next_tokens, stored_len, N, ids, top_n, draft_len, out_tokens);
+    merge_gather_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, nullptr, nullptr, gtau, nullptr, 0,
+                                                           0, 0, nullptr);
     return cudaGetLastError();
 }
 

@@ -196,9 +196,8 @@ extern "C" dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *
         cudaError_t e = f32 ? launch_scan_f32(map, a, grid, stream) : launch_scan_mma(map, a, grid, stream);
         if (e != cudaSuccess) return na_fail(DRESD_ERR_CUDA, "scan launch failed");
     }
-    if (launch_merge(cand, grid, B, top_n, out_ids, out_scores, stream) != cudaSuccess)
-        return na_fail(DRESD_ERR_CUDA, "merge launch failed");
-    if (launch_gather(next_tokens, stored_len, N, out_ids, B, top_n, draft_len, out_tokens, stream) != cudaSuccess)
-        return na_fail(DRESD_ERR_CUDA, "gather launch failed");
+    if (launch_merge_gather(cand, grid, B, top_n, out_ids, out_scores, next_tokens, stored_len, N, draft_len,
+                            out_tokens, stream) != cudaSuccess)
+        return na_fail(DRESD_ERR_CUDA, "merge/gather launch failed");
     return DRESD_OK;
 }
