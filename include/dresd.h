@@ -78,7 +78,10 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
  *   pca_mean   fp32 [d_in] subtracted before the projection, or NULL (the
  *              paper's formula has no centring).
  *
- * Without this call queries are [B][d] and only Eq. 2 is applied.
+ * Without this call queries are [B][d] and only Eq. 2 is applied.  A set-up call:
+ * it may allocate (a staging buffer for the host-buffer call and, with W, 8 MB for
+ * the partial products of the projection, which is split over d_in so that W is
+ * read once per call for all queries); the retrieval calls allocate nothing.
  */
 dresd_status dresd_store_set_preprocess(dresd_store *store, int d_in, const float *mean,
                                         const float *var, float eps_z, const void *W,

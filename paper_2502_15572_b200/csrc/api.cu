@@ -127,6 +127,8 @@ struct dresd_store {
     // options / bookkeeping
     int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m;
     double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
+    float *proj_ws;              // partial products of the split projection (allocated with W)
+    size_t proj_ws_bytes;
     cudaStream_t last_stream;
     int last_launches;
     // optional timing of the scoring kernel (option "profile")
@@ -148,6 +150,7 @@ void free_store(dresd_store *s)
     cudaFree(s->gtau);
     cudaFree(s->first_col);
     cudaFree(s->q_stage);
+    cudaFree(s->proj_ws);
     cudaFree(s->ids_dev);
     cudaFree(s->scores_dev);
     cudaFree(s->tokens_dev);
@@ -199,9 +202,13 @@ dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows
     p.lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
     p.gtau = s->gtau;
     p.split_blocked = split_blocked;
+    if (s->W && s->proj_ws && reinterpret_cast<uintptr_t>(s->W) % 16 == 0) {     // 16-byte loads of W rows
+        preprocess_split_plan(s->d_in, s->d, B, (int)elem_bytes(s->dtype), s->proj_ws_bytes, &p.slices, &p.rows_per_slice);
+        if (p.slices > 0) p.partial = s->proj_ws;
+    }
     cudaError_t e = launch_preprocess(p, stream);
     if (e != cudaSuccess) return fail_cuda(e, "preprocess launch");
-    s->last_launches += 1;
+    s->last_launches += p.partial ? 2 : 1;
     return DRESD_OK;
 }
 
@@ -451,6 +458,17 @@ dresd_status dresd_store_set_preprocess(dresd_store *s, int d_in, const float *m
         cudaFree(s->q_stage);
         s->q_stage = p;
         s->q_stage_bytes = need;
+    }
+    if (W && !s->proj_ws) {
+        // workspace of the split projection; without it every query's CTA walks all of W (slow, not wrong)
+        const size_t bytes = (size_t)8 << 20;
+        void *p = nullptr;
+        if (cudaMalloc(&p, bytes) == cudaSuccess) {
+            s->proj_ws = static_cast<float *>(p);
+            s->proj_ws_bytes = bytes;
+        } else {
+            cudaGetLastError();
+        }
     }
     s->d_in = d_in;
     s->mean = mean;

@@ -31,7 +31,13 @@ struct PreprocessArgs {
     float lo_scale;
     unsigned int *gtau;     // [rows] grid-wide filter words, reset to 0 ("nothing known") here
     int split_blocked;      // qsplit rows: 0 = (2b, 2b+1); 1 = 16-row blocks, hi rows 0-7, lo rows 8-15
+    // Split projection (W given): `slices` CTAs of `rows_per_slice` rows of W each write
+    // partial[slice][B][d]; null = every query's CTA walks all of W itself.
+    float *partial;
+    int slices, rows_per_slice;
 };
+// Slices and rows per slice of the split projection for a workspace of `bytes` (0 slices = do not split).
+void preprocess_split_plan(int d_in, int d, int B, int elem_bytes, size_t bytes, int *slices, int *rows_per_slice);
 cudaError_t launch_preprocess(const PreprocessArgs &a, cudaStream_t stream);
 
 // ---- K2+K3: score every key, keep a per-CTA top-n per query ----------------

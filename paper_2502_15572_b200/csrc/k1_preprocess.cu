@@ -44,6 +44,126 @@ __device__ __forceinline__ float block_sum(float x, float *scratch /*[32]*/)
     return t;                             // every thread holds the total
 }
 
+// K1a -- the projection v W of ALL queries of the call, split over d_in: CTA s takes the
+// rows [s * rps, (s+1) * rps) of W (read once, coalesced, for every query), applies Eq. 1 and
+// the centring to the matching slice of each query, and writes the partial products
+// partial[s][b][c].  K1b adds the slices in a fixed order, so the result does not depend on
+// the launch.  (One CTA per query reading all of W, as K1b does without a workspace, is
+// latency-bound: 130 us for 16 queries x 4096 x 256; this form takes a few microseconds.)
+constexpr int kProjThreads = 256;
+constexpr int kProjWarps = kProjThreads / 32;
+constexpr int kProjChunk = 8;            // queries per register block
+
+template <typename T> struct ProjVec;    // 16 bytes of a W row
+template <> struct ProjVec<float> { static constexpr int N = 4; };
+template <> struct ProjVec<__half> { static constexpr int N = 8; };
+template <> struct ProjVec<__nv_bfloat16> { static constexpr int N = 8; };
+template <typename T> __device__ __forceinline__ void unpack_w(const uint4 &v, float *w);
+template <> __device__ __forceinline__ void unpack_w<float>(const uint4 &v, float *w)
+{
+    w[0] = __uint_as_float(v.x); w[1] = __uint_as_float(v.y); w[2] = __uint_as_float(v.z); w[3] = __uint_as_float(v.w);
+}
+template <> __device__ __forceinline__ void unpack_w<__half>(const uint4 &v, float *w)
+{
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&u[i]));
+        w[2 * i] = f.x;
+        w[2 * i + 1] = f.y;
+    }
+}
+template <> __device__ __forceinline__ void unpack_w<__nv_bfloat16>(const uint4 &v, float *w)
+{
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        w[2 * i] = __uint_as_float(u[i] << 16);
+        w[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
+    }
+}
+
+// The CTA first copies its slice of W to shared memory with every 16-byte load in flight at
+// once (W does not survive in L2 between calls -- the scan streams gigabytes through it -- so
+// these are DRAM reads, and a loop that waits for each row costs ~1.2 k cycles per row).  Then
+// warp w takes the queries w, w + 8, ... (at most 8 of the 64) and a lane 16 bytes (4 or 8
+// columns) of every row; no sum crosses a warp.
+// QW = queries per warp (1, 2, 4 or 8, chosen from B): the inner loops are branch-free.
+template <typename T, int QW>
+__global__ void __launch_bounds__(kProjThreads) project_partial_kernel(PreprocessArgs a)
+{
+    constexpr int VEC = ProjVec<T>::N;
+    extern __shared__ __align__(16) uint8_t proj_smem[];
+    const int rps = a.rows_per_slice;
+    const int s = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int j0 = s * rps, nr = min(a.d_in, j0 + rps) - j0;
+    uint4 *ws = reinterpret_cast<uint4 *>(proj_smem);                        // [nr][d / VEC]: the slice of W
+    float *vs = reinterpret_cast<float *>(proj_smem + (size_t)rps * a.d * sizeof(T));   // [B][rps]: the queries' slices
+    const int cblocks = a.d / VEC;        // 16-byte column blocks per row (d is a multiple of VEC)
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(static_cast<const T *>(a.W) + (size_t)j0 * a.d);
+        const int total = nr * cblocks;
+        for (int i0 = tid; i0 < total; i0 += 8 * kProjThreads) {
+            uint4 v[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                const int i = i0 + r * kProjThreads;
+                v[r] = i < total ? __ldg(src + i) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                const int i = i0 + r * kProjThreads;
+                if (i < total) ws[i] = v[r];
+            }
+        }
+    }
+    const T *Q = static_cast<const T *>(a.queries);
+    for (int i = tid; i < a.B * rps; i += kProjThreads) {
+        const int b = i / rps, jj = i - b * rps;
+        float x = 0.f;
+        if (jj < nr) {
+            const int j = j0 + jj;
+            x = to_f32<T>(Q[(size_t)b * a.d_in + j]);
+            if (a.mean) x = (x - a.mean[j]) / sqrtf(a.var[j] + a.eps_z);      // Eq. 1
+            if (a.pca_mean) x -= a.pca_mean[j];
+        }
+        vs[i] = x;
+    }
+    __syncthreads();
+    if (warp >= a.B) return;
+    int qrow[QW];                         // my queries w, w + 8, ...; past B: the last one again (not stored)
+#pragma unroll
+    for (int u = 0; u < QW; ++u) qrow[u] = min(warp + kProjWarps * u, a.B - 1) * rps;
+    for (int cb = lane; cb < cblocks; cb += 32) {
+        float acc[QW][VEC];
+#pragma unroll
+        for (int u = 0; u < QW; ++u)
+#pragma unroll
+            for (int k = 0; k < VEC; ++k) acc[u][k] = 0.f;
+#pragma unroll 4
+        for (int jj = 0; jj < nr; ++jj) {
+            float w[VEC];
+            unpack_w<T>(ws[jj * cblocks + cb], w);
+#pragma unroll
+            for (int u = 0; u < QW; ++u) {
+                const float x = vs[qrow[u] + jj];
+#pragma unroll
+                for (int k = 0; k < VEC; ++k) acc[u][k] = fmaf(x, w[k], acc[u][k]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < QW; ++u) {
+            const int b = warp + kProjWarps * u;
+            if (b < a.B) {
+                float *o = a.partial + ((size_t)s * a.B + b) * a.d + (size_t)cb * VEC;
+#pragma unroll
+                for (int k = 0; k < VEC; k += 4)
+                    *reinterpret_cast<float4 *>(o + k) = make_float4(acc[u][k], acc[u][k + 1], acc[u][k + 2], acc[u][k + 3]);
+            }
+        }
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
 {
@@ -75,7 +195,8 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
     }
 
     const T *q = static_cast<const T *>(a.queries) + (size_t)b * a.d_in;
-    for (int j = tid; j < a.d_in; j += blockDim.x) {
+    const bool presummed = a.W && a.partial;             // K1a has done Eq. 1 and the products
+    for (int j = tid; j < a.d_in && !presummed; j += blockDim.x) {
         float x = to_f32<T>(q[j]);
         if (a.mean) x = (x - a.mean[j]) / sqrtf(a.var[j] + a.eps_z);      // Eq. 1
         if (a.W && a.pca_mean) x -= a.pca_mean[j];
@@ -83,7 +204,32 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
     }
     __syncthreads();
 
-    if (a.W) {                                                             // v_l = v W
+    if (presummed) {                                                       // v_l = sum of K1a's slices
+        // threads arranged [group][column]: group g adds slices g, g + groups, ... (loads of
+        // different slices in flight together), then the groups' sums are added in order
+        int ct = 1;
+        while (ct * 2 <= a.d && ct * 2 <= (int)blockDim.x) ct *= 2;
+        const int groups = blockDim.x / ct;
+        const int grp = tid / ct, cl = tid % ct;
+        for (int c = cl; c < a.d; c += ct) {
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            int sl = grp;
+            for (; sl + 3 * groups < a.slices; sl += 4 * groups) {
+                s0 += a.partial[((size_t)(sl + 0 * groups) * a.B + b) * a.d + c];
+                s1 += a.partial[((size_t)(sl + 1 * groups) * a.B + b) * a.d + c];
+                s2 += a.partial[((size_t)(sl + 2 * groups) * a.B + b) * a.d + c];
+                s3 += a.partial[((size_t)(sl + 3 * groups) * a.B + b) * a.d + c];
+            }
+            for (; sl < a.slices; sl += groups) s0 += a.partial[((size_t)sl * a.B + b) * a.d + c];
+            part[(size_t)grp * a.d + c] = (s0 + s1) + (s2 + s3);
+        }
+        __syncthreads();
+        for (int c = tid; c < a.d; c += blockDim.x) {
+            float t = 0.f;
+            for (int g = 0; g < groups; ++g) t += part[(size_t)g * a.d + c];
+            vl[c] = t;
+        }
+    } else if (a.W) {                                                      // v_l = v W
         // Threads are arranged [slice][column]: consecutive threads read
         // consecutive columns of one W row (coalesced); slices split d_in.
         int ct = 1;
@@ -135,9 +281,56 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
 
 }  // namespace
 
+void preprocess_split_plan(int d_in, int d, int B, int elem_bytes, size_t bytes, int *slices, int *rows_per_slice)
+{
+    *slices = 0;
+    *rows_per_slice = 0;
+    if (B <= 0 || bytes == 0) return;
+    const size_t per_slice = sizeof(float) * (size_t)B * d;
+    const long long cap = (long long)(bytes / per_slice);
+    if (cap < 2) return;                                  // no room: the unsplit form runs
+    // a CTA holds its slice of W (rows x d) and of the queries (B x rows) in 48 KB of shared memory
+    auto fits = [&](int rps) { return (size_t)rps * d * elem_bytes + sizeof(float) * (size_t)B * rps <= 48 * 1024; };
+    int rps = 64;
+    while (rps > 1 && !fits(rps)) rps /= 2;
+    if (!fits(rps)) return;
+    const long long n = (d_in + rps - 1) / rps;
+    if (n > cap || n > 1024) return;                      // too many slices for the workspace: unsplit form
+    *slices = (int)n;
+    *rows_per_slice = rps;
+}
+
 cudaError_t launch_preprocess(const PreprocessArgs &a, cudaStream_t stream)
 {
     if (a.rows <= 0) return cudaSuccess;
+    if (a.W && a.partial && a.B > 0) {
+        const size_t eb = a.dtype == kF32 ? 4 : 2;
+        const size_t psm = (size_t)a.rows_per_slice * a.d * eb + sizeof(float) * (size_t)a.B * a.rows_per_slice;
+        const int per_warp = (a.B + kProjWarps - 1) / kProjWarps;
+        const int qw = per_warp <= 1 ? 1 : per_warp <= 2 ? 2 : per_warp <= 4 ? 4 : 8;
+        auto launch = [&](auto k1, auto k2, auto k4, auto k8) {
+            if (qw == 1) k1<<<a.slices, kProjThreads, psm, stream>>>(a);
+            else if (qw == 2) k2<<<a.slices, kProjThreads, psm, stream>>>(a);
+            else if (qw == 4) k4<<<a.slices, kProjThreads, psm, stream>>>(a);
+            else k8<<<a.slices, kProjThreads, psm, stream>>>(a);
+        };
+        switch (a.dtype) {
+        case kF32:
+            launch(project_partial_kernel<float, 1>, project_partial_kernel<float, 2>,
+                   project_partial_kernel<float, 4>, project_partial_kernel<float, 8>);
+            break;
+        case kF16:
+            launch(project_partial_kernel<__half, 1>, project_partial_kernel<__half, 2>,
+                   project_partial_kernel<__half, 4>, project_partial_kernel<__half, 8>);
+            break;
+        default:
+            launch(project_partial_kernel<__nv_bfloat16, 1>, project_partial_kernel<__nv_bfloat16, 2>,
+                   project_partial_kernel<__nv_bfloat16, 4>, project_partial_kernel<__nv_bfloat16, 8>);
+            break;
+        }
+        cudaError_t pe = cudaGetLastError();
+        if (pe != cudaSuccess) return pe;
+    }
     int ct = 1;
     while (ct * 2 <= a.d && ct * 2 <= kThreads) ct *= 2;
     const int slices = a.W ? kThreads / ct : 0;
