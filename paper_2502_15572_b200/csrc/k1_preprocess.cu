@@ -52,7 +52,6 @@ __device__ __forceinline__ float block_sum(float x, float *scratch /*[32]*/)
 // latency-bound: 130 us for 16 queries x 4096 x 256; this form takes a few microseconds.)
 constexpr int kProjThreads = 256;
 constexpr int kProjWarps = kProjThreads / 32;
-constexpr int kProjChunk = 8;            // queries per register block
 
 template <typename T> struct ProjVec;    // 16 bytes of a W row
 template <> struct ProjVec<float> { static constexpr int N = 4; };
