@@ -350,3 +350,44 @@ def test_wide_batch_adversarial_order_and_agreement_of_both_forms():
         assert same >= 0.99                               # near-ties may swap within fp32 rounding
     finally:
         st.close()
+
+
+def test_retrieve_can_be_captured_in_a_cuda_graph_and_replayed():
+    """dresd_retrieve enqueues kernels only (no allocation, no host synchronisation), so a
+    serving loop can capture it once and replay it: the replay must use the CURRENT contents
+    of the query buffer and give the same result as a direct call."""
+    import torch
+    dtype, N, d, B, n, L = "f16", 60011, 256, 4, 10, 5
+    keys, toks = synth.make_store(7600, N, d, 16, dtype, L)
+    q1, _ = synth.make_queries(7601, keys, dtype, B, 0.1)
+    q2, _ = synth.make_queries(7602, keys, dtype, B, 0.1)
+    st = gpu_store(keys, toks, dtype)
+    try:
+        want1 = gpu_retrieve(st, q1, n, L)
+        want2 = gpu_retrieve(st, q2, n, L)
+        qbuf = binding.to_device(q1, dtype)
+        ids = torch.empty((B, n), dtype=torch.int32, device="cuda")
+        sc = torch.empty((B, n), dtype=torch.float32, device="cuda")
+        tok = torch.empty((B, n, L), dtype=torch.int32, device="cuda")
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(2):          # warm-up outside the capture (function attributes, lazy loading)
+                binding.dresd_retrieve(st.handle, qbuf.data_ptr(), B, n, L, ids.data_ptr(), sc.data_ptr(),
+                                       tok.data_ptr(), side.cuda_stream)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            binding.dresd_retrieve(st.handle, qbuf.data_ptr(), B, n, L, ids.data_ptr(), sc.data_ptr(),
+                                   tok.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        for q, want in ((q1, want1), (q2, want2), (q1, want1)):
+            qbuf.copy_(binding.to_device(q, dtype))
+            g.replay()
+            torch.cuda.synchronize()
+            st.status()
+            assert np.array_equal(ids.cpu().numpy(), want[0])
+            assert np.array_equal(sc.cpu().numpy(), want[1])
+            assert np.array_equal(tok.cpu().numpy(), want[2])
+    finally:
+        st.close()
