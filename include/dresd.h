@@ -104,7 +104,7 @@ dresd_status dresd_store_set_preprocess(dresd_store *store, int d_in, const floa
  *               stored tokens of each neighbour, verbatim.
  *
  * Non-finite inputs give unspecified results but neither hang nor fault.
-  * The call only enqueues kernels: it can be captured into a CUDA graph and replayed
+ * The call only enqueues kernels: it can be captured into a CUDA graph and replayed
  * (the replay reads the query buffer as it is then; tested).
  */
 dresd_status dresd_retrieve(dresd_store *store, const void *queries, int B, int top_n,
