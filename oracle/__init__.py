@@ -13,4 +13,8 @@ from .dresd_oracle import (  # noqa: F401
     OracleResult,
     drafts_prepare,
     drafts_accept,
+    e4m3_decode,
+    e4m3_encode,
+    quantised_scores,
+    retrieve_quantised,
 )

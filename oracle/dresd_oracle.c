@@ -250,6 +250,85 @@ done:
     return rc;
 }
 
+/* ---- quantised candidate search (the approximation the paper's search library makes) ----
+ * The paper does not search exactly: it uses an approximate nearest-neighbour library
+ * (Section 3.5), whose core device is scoring against a quantised copy of the keys.  The
+ * CUDA library offers that as: 8-bit keys (E4M3: 1 sign, 4 exponent bits with bias 7, 3
+ * mantissa bits, largest finite value 448, no infinities), candidates by approximate score,
+ * exact re-ranking of the candidates.  Stated here step by step, exact arithmetic throughout:
+ *   k8_ij = e4m3(256 k_ij)            round to nearest, ties to even, saturating at +-448
+ *   h1_j  = e4m3(256 q_j),   h2_j = e4m3(16 (256 q_j - h1_j))        (two-term query)
+ *   a_i   = sum_j (h1_j + h2_j / 16) k8_ij / 65536                    (approximate score)
+ * The caller takes the m best a_i (ties to the lower row), scores those exactly and keeps
+ * the n best.  Nothing here is printed in the paper; it is this library's definition.   */
+double dresd_oracle_e4m3_decode(uint32_t code)
+{
+    const int sign = (code >> 7) & 1, e = (code >> 3) & 15, m = code & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;                       /* the only NaN pattern (and its negative) */
+    if (e == 0) v = ldexp((double)m / 8.0, -6);              /* subnormal */
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+uint32_t dresd_oracle_e4m3_encode(double x)
+{
+    if (x != x) return 0x7F;
+    const uint32_t sign = (x < 0.0 || (x == 0.0 && 1.0 / x < 0.0)) ? 0x80u : 0u;
+    const double ax = fabs(x);
+    /* nearest of the 127 finite non-negative values 0x00..0x7E (increasing with the code);
+       a tie goes to the even code, which is the even mantissa */
+    uint32_t best = 0;
+    double best_err = ax;                                    /* code 0 = 0.0 */
+    for (uint32_t c = 1; c <= 0x7E; ++c) {
+        const double err = fabs(ax - dresd_oracle_e4m3_decode(c));
+        if (err < best_err || (err == best_err && (c & 1u) == 0u)) {
+            best_err = err;
+            best = c;
+        }
+    }
+    return sign | best;                                      /* values beyond 448 end at 0x7E */
+}
+
+/* approx[i] for one unit query qhat (float64 [d]) over all keys.  Returns 0 or -1.   */
+int dresd_oracle_quantised_scores(const void *keys, int64_t N, int d, int dtype, const double *qhat,
+                                  double *approx, int threads)
+{
+    if (N < 0 || d <= 0) return -1;
+    double *qq = (double *)malloc(sizeof(double) * (size_t)d);
+    if (!qq) return -1;
+    for (int j = 0; j < d; ++j) {
+        const double q256 = 256.0 * qhat[j];
+        const double h1 = dresd_oracle_e4m3_decode(dresd_oracle_e4m3_encode(q256));
+        const double h2 = dresd_oracle_e4m3_decode(dresd_oracle_e4m3_encode(16.0 * (q256 - h1)));
+        qq[j] = h1 + h2 / 16.0;
+    }
+    if (threads < 1) threads = 1;
+    /* 16-bit stores: the quantised value of every possible stored bit pattern, once */
+    double *k8_of = NULL;
+    if (dtype == ORACLE_F16 || dtype == ORACLE_BF16) {
+        k8_of = (double *)malloc(sizeof(double) * 65536);
+        if (!k8_of) { free(qq); return -1; }
+        for (uint32_t b = 0; b < 65536; ++b) {
+            const uint16_t h = (uint16_t)b;
+            k8_of[b] = dresd_oracle_e4m3_decode(dresd_oracle_e4m3_encode(256.0 * load_elem(&h, 0, dtype)));
+        }
+    }
+#pragma omp parallel for num_threads(threads) schedule(static)
+    for (int64_t i = 0; i < N; ++i) {
+        double acc = 0.0;
+        for (int j = 0; j < d; ++j) {
+            const double k8 = k8_of ? k8_of[((const uint16_t *)keys)[i * d + j]]
+                                    : dresd_oracle_e4m3_decode(dresd_oracle_e4m3_encode(256.0 * load_elem(keys, i * d + j, dtype)));
+            acc += qq[j] * k8;
+        }
+        approx[i] = acc / 65536.0;
+    }
+    free(k8_of);
+    free(qq);
+    return 0;
+}
+
 /* ---- token-level half of batch verification (Section 3.6, Fig. 3) ----------
  * prepare: tokens [B][n][L], ids [B][n] (-1 = missing neighbour).  drafts [B][n][L]:
  * after a draft's first EOS every token is EOS (the EOS id is the padding); a missing

@@ -44,6 +44,13 @@ def _load():
             c.c_void_p, c.c_int, c.c_void_p, c.c_double, c.c_void_p]
         lib.dresd_oracle_fit_zscore.restype = c.c_int
         lib.dresd_oracle_fit_zscore.argtypes = [c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_void_p, c.c_void_p]
+        lib.dresd_oracle_e4m3_decode.restype = c.c_double
+        lib.dresd_oracle_e4m3_decode.argtypes = [c.c_uint32]
+        lib.dresd_oracle_e4m3_encode.restype = c.c_uint32
+        lib.dresd_oracle_e4m3_encode.argtypes = [c.c_double]
+        lib.dresd_oracle_quantised_scores.restype = c.c_int
+        lib.dresd_oracle_quantised_scores.argtypes = [c.c_void_p, c.c_int64, c.c_int, c.c_int, c.c_void_p,
+                                                     c.c_void_p, c.c_int]
         lib.dresd_oracle_scores.restype = c.c_int
         lib.dresd_oracle_scores.argtypes = [c.c_void_p, c.c_int64, c.c_int, c.c_int,
                                             c.c_void_p, c.c_void_p, c.c_int]
@@ -221,3 +228,58 @@ def drafts_accept(drafts, valid, llm_tokens):
     if lib.dresd_oracle_drafts_accept(_ptr(d), _ptr(v), _ptr(m), B, n, L, _ptr(best), _ptr(length), _ptr(out)) != 0:
         raise ValueError("oracle drafts_accept: bad arguments")
     return best, length, out
+
+
+def e4m3_decode(code: int) -> float:
+    """Value of one E4M3 code (0..255); the two NaN codes give nan."""
+    return float(_load().dresd_oracle_e4m3_decode(int(code) & 0xFF))
+
+
+def e4m3_encode(x: float) -> int:
+    """E4M3 code of x: round to nearest, ties to even, saturating at +-448."""
+    return int(_load().dresd_oracle_e4m3_encode(float(x)))
+
+
+def quantised_scores(keys, dtype: str, qhat, threads: int = 1) -> np.ndarray:
+    """Approximate scores of one float64 unit query against the 8-bit copy of every key."""
+    k = _store_array(keys, dtype)
+    N, d = k.shape
+    qh = np.ascontiguousarray(qhat, dtype=np.float64)
+    if qh.shape != (d,):
+        raise ValueError("qhat must be [d]")
+    out = np.empty(N, dtype=np.float64)
+    rc = _load().dresd_oracle_quantised_scores(_ptr(k), N, d, _DTYPE_CODE[dtype], _ptr(qh), _ptr(out), threads)
+    if rc != 0:
+        raise ValueError("oracle quantised_scores: bad arguments")
+    return out
+
+
+def retrieve_quantised(keys, next_tokens, dtype: str, queries, top_n: int, draft_len: int, candidates: int,
+                       mean=None, var=None, eps_z: float = 1e-5, W=None, pca_mean=None, threads: int = 1):
+    """Candidates by approximate (8-bit) score, exact re-ranking, value lookup.
+
+    For each query: the `candidates` rows with the largest approximate score (ties to the
+    lower row) are scored exactly; the `top_n` best of them (score descending, row
+    ascending) are returned with their stored tokens.  Returns ``(ids, scores, tokens,
+    approx, exact)`` with approx / exact the full float64 score vectors ``[B][N]``."""
+    toks = np.ascontiguousarray(next_tokens, dtype=np.int32)
+    N = toks.shape[0]
+    if not (1 <= top_n <= candidates <= N) or not (1 <= draft_len <= toks.shape[1]):
+        raise ValueError("need 1 <= top_n <= candidates <= N and 1 <= draft_len <= stored_len")
+    qhat = preprocess(queries, dtype, mean=mean, var=var, eps_z=eps_z, W=W, pca_mean=pca_mean)
+    B = qhat.shape[0]
+    ids = np.empty((B, top_n), dtype=np.int32)
+    sc = np.empty((B, top_n), dtype=np.float64)
+    tok = np.empty((B, top_n, draft_len), dtype=np.int32)
+    approx = np.empty((B, N), dtype=np.float64)
+    exact = np.empty((B, N), dtype=np.float64)
+    rows = np.arange(N)
+    for b in range(B):
+        approx[b] = quantised_scores(keys, dtype, qhat[b], threads)
+        exact[b] = scores(keys, dtype, qhat[b], threads)
+        cand = np.lexsort((rows, -approx[b]))[:candidates]          # approx descending, row ascending
+        order = cand[np.lexsort((cand, -exact[b][cand]))][:top_n]    # exact descending, row ascending
+        ids[b] = order
+        sc[b] = exact[b][order]
+        tok[b] = toks[order, :draft_len]
+    return ids, sc, tok, approx, exact

@@ -367,3 +367,85 @@ def test_fit_zscore_then_eq1_standardises_the_sample():
 def test_fit_zscore_bad_arguments():
     with pytest.raises(ValueError):
         oracle.fit_zscore(np.zeros((0, 4), dtype=np.float32), "f32")
+
+
+# --------------------------------------------------------------------------
+# quantised candidate search: E4M3 codes, approximate scores, re-ranking
+# --------------------------------------------------------------------------
+def test_e4m3_decode_all_codes_match_the_format_definition():
+    """1 sign, 4 exponent bits (bias 7), 3 mantissa bits; exponent 0 is subnormal; only
+    S.1111.111 is NaN (the format has no infinities), so the largest finite value is 448."""
+    for code in range(256):
+        s, e, m = code >> 7, (code >> 3) & 15, code & 7
+        got = oracle.e4m3_decode(code)
+        if e == 15 and m == 7:
+            assert np.isnan(got)
+            continue
+        want = (m / 8.0) * 2.0 ** -6 if e == 0 else (1 + m / 8.0) * 2.0 ** (e - 7)
+        assert got == (-want if s else want)
+    assert oracle.e4m3_decode(0x7E) == 448.0 and oracle.e4m3_decode(0x01) == 2.0 ** -9
+    assert oracle.e4m3_decode(0x38) == 1.0 and oracle.e4m3_decode(0xB8) == -1.0
+
+
+def test_e4m3_encode_known_values_ties_and_saturation():
+    enc, dec = oracle.e4m3_encode, oracle.e4m3_decode
+    for code in range(256):                              # every finite code encodes back to itself
+        if (code & 0x7F) != 0x7F:
+            assert enc(dec(code)) == code
+    assert enc(1.0) == 0x38 and enc(-2.0) == 0xC0 and enc(448.0) == 0x7E
+    assert enc(1e6) == 0x7E and enc(-1e6) == 0xFE and enc(449.0) == 0x7E      # saturating, never NaN
+    assert enc(float("nan")) & 0x7F == 0x7F
+    # ties go to the even mantissa: 1.0625 is halfway between 1.0 (m=0) and 1.125 (m=1)
+    assert enc(1.0625) == 0x38 and enc(1.1875) == 0x3A        # 1.1875: between 1.125 (m=1) and 1.25 (m=2)
+    assert enc(1.0626) == 0x39 and enc(1.0624) == 0x38
+    # below half of the smallest subnormal (2^-10) -> 0; exactly half -> 0 (even); just above -> 2^-9
+    assert enc(2.0 ** -10) == 0x00 and enc(2.0 ** -10 * 1.001) == 0x01 and enc(2.0 ** -11) == 0x00
+    # monotone
+    xs = np.linspace(-500, 500, 20001)
+    codes = np.array([dec(enc(x)) for x in xs])
+    assert np.all(np.diff(codes) >= 0)
+
+
+def test_e4m3_encode_matches_an_independent_library_conversion():
+    torch = pytest.importorskip("torch")
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("this torch has no float8_e4m3fn")
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.normal(size=4000) * 20, rng.normal(size=2000) * 0.01, rng.uniform(-448, 448, 2000),
+                        np.array([0.0, 448.0, -448.0, 2.0 ** -9, 2.0 ** -10 * 3])]).astype(np.float32)
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).to(torch.float32).numpy()
+    got = np.array([oracle.e4m3_decode(oracle.e4m3_encode(float(v))) for v in x], dtype=np.float32)
+    assert np.array_equal(got, want)
+
+
+def test_quantised_scores_hand_case_and_exactly_representable_inputs():
+    # keys and query whose 256-fold multiples are E4M3 values: the approximate score is the exact one
+    keys = np.array([[0.5, 0.25, 0.0, -0.125], [1.0, 0.0, 0.0, 0.0], [0.0, -0.75, 0.5, 0.5]], dtype=np.float32)
+    q = np.array([0.5, -0.5, 0.25, 0.0])
+    a = oracle.quantised_scores(keys, "f32", q)
+    np.testing.assert_allclose(a, keys.astype(np.float64) @ q, rtol=0, atol=1e-15)
+    # hand case with rounding: k = 0.3 -> 76.8 -> e4m3 80 (grid step 8 above 64); q = 0.3:
+    # h1 = 80, residual -3.2 -> 16 * -3.2 = -51.2 -> e4m3 -52 (step 4 above 32) -> q ~ 80 - 52/16 = 76.75
+    a = oracle.quantised_scores(np.array([[0.3]], dtype=np.float32), "f32", np.array([0.3]))
+    np.testing.assert_allclose(a, [76.75 * 80 / 65536], rtol=1e-12)
+
+
+def test_quantised_scores_are_close_to_exact_and_reranking_recovers_the_neighbours():
+    dtype, N, d = "bf16", 6000, 64
+    keys, toks = synth.make_store(910, N, d, 8, dtype, 3)
+    q, _ = synth.make_queries(911, keys, dtype, 4, 0.1)
+    ids, sc, tok, approx, exact = oracle.retrieve_quantised(keys, toks, dtype, q, 5, 3, 40)
+    # error model: keys carry 3 mantissa bits (relative error <= 2^-4 per element), the query two terms
+    assert np.max(np.abs(approx - exact)) < 0.02
+    ref = oracle.retrieve(keys, toks, dtype, q, 5, 3)
+    assert np.mean(ids == ref.ids) >= 0.9                   # recall of the exact neighbours on this easy store
+    # with every row a candidate the result IS the exact one
+    ids_all, sc_all, tok_all, _, _ = oracle.retrieve_quantised(keys, toks, dtype, q, 5, 3, N)
+    assert np.array_equal(ids_all, ref.ids) and np.array_equal(tok_all, ref.tokens)
+    np.testing.assert_allclose(sc_all, ref.scores, rtol=0, atol=1e-12)
+    # the returned rows are candidates, sorted by exact score, tokens copied verbatim
+    for b in range(4):
+        cut = np.sort(approx[b])[-40]
+        assert np.all(approx[b][ids[b]] >= cut)
+        assert np.all(np.diff(sc[b]) <= 0)
+        assert np.array_equal(tok[b], toks[ids[b], :3])
