@@ -209,6 +209,36 @@ dresd_status dresd_fit_zscore(const void *sample, int64_t N, int d_in, dresd_dty
                               float *out_var, void *stream);
 
 /*
+ * Quantised candidate search.  The paper searches its datastore with an approximate
+ * nearest-neighbour library (Section 3.5); the counterpart here scores an 8-bit copy of
+ * the keys -- half the bytes of a 16-bit store, so about twice the queries per second of
+ * the memory-bound exact scan -- and re-ranks the best candidates exactly.  Every step is
+ * defined exactly (E4M3: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, largest
+ * finite value 448; conversions round to nearest even and saturate):
+ *
+ *     k8[i][j] = e4m3(256 k[i][j])
+ *     h1[j] = e4m3(256 q[j]),   h2[j] = e4m3(16 (256 q[j] - h1[j]))      q = unit query
+ *     a[i]  = sum_j (h1[j] + h2[j] / 16) k8[i][j] / 65536                 approximate score
+ *
+ * The `candidates` rows with the largest a[i] (ties to the lower row) are scored exactly
+ * against the 16-bit keys (fp32) and the top_n best of them returned like dresd_retrieve().
+ * The result is NOT always the exact top_n: a true neighbour whose approximate score falls
+ * below the candidate cut is missed (recall is measured by bench.py --quantised).
+ *
+ * dresd_quantise_keys       keys: device [N][d] fp16/bf16, d a multiple of 16; out_q8: device
+ *                           [N][d] bytes; both 16-byte aligned.  Asynchronous on `stream`.
+ * dresd_store_attach_quantised   the 8-bit copy of the store's keys (borrowed until destroy);
+ *                           a set-up call, may allocate.  16-bit stores with d <= 2048.
+ * dresd_retrieve_quantised  as dresd_retrieve() plus `candidates` in top_n .. DRESD_MAX_TOP_N.
+ *                           Asynchronous on `stream`; no allocation.
+ */
+dresd_status dresd_quantise_keys(const void *keys, int64_t N, int d, dresd_dtype dtype, void *out_q8, void *stream);
+dresd_status dresd_store_attach_quantised(dresd_store *store, const void *keys_q8);
+dresd_status dresd_retrieve_quantised(dresd_store *store, const void *queries, int B, int top_n, int draft_len,
+                                      int candidates, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
+                                      void *stream);
+
+/*
  * Process-wide switches (not part of the paper; for measurement and tests).
  *   "build_keys_pairs"  1 (default): dresd_build_keys runs on CTA pairs -- clusters of two
  *                       CTAs, one tensor-core instruction spanning both SMs, each CTA staging

@@ -29,7 +29,8 @@ EXPORTS = (
     "dresd_last_error",
     "dresd_store_destroy", "dresd_retrieve_noalloc", "dresd_store_enable_first_token_filter",
     "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
-    "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore", "dresd_set_global_option",
+    "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore", "dresd_set_global_option", "dresd_quantise_keys", "dresd_store_attach_quantised",
+    "dresd_retrieve_quantised",
 )
 
 
@@ -91,6 +92,12 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_merge_shards.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_build_keys.restype = i32
     lib.dresd_build_keys.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, i32, vp, vp, vp]
+    lib.dresd_quantise_keys.restype = i32
+    lib.dresd_quantise_keys.argtypes = [vp, i64, i32, i32, vp, vp]
+    lib.dresd_store_attach_quantised.restype = i32
+    lib.dresd_store_attach_quantised.argtypes = [vp, vp]
+    lib.dresd_retrieve_quantised.restype = i32
+    lib.dresd_retrieve_quantised.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_set_global_option.restype = i32
     lib.dresd_set_global_option.argtypes = [ctypes.c_char_p, i32]
     lib.dresd_fit_zscore.restype = i32
@@ -163,6 +170,20 @@ def dresd_build_keys(hidden_ptr: int, N: int, d_in: int, dtype: int, mean_ptr, v
     """Eq. 1 -> v W -> Eq. 2 over N rows of hidden states: builds the datastore's key matrix."""
     _check(load().dresd_build_keys(hidden_ptr, N, d_in, dtype, mean_ptr, var_ptr, eps_z, W_ptr, d, pca_mean_ptr,
                                    out_keys_ptr, stream))
+
+
+def dresd_quantise_keys(keys_ptr: int, N: int, d: int, dtype: int, out_q8_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_quantise_keys(keys_ptr, N, d, dtype, out_q8_ptr, stream))
+
+
+def dresd_store_attach_quantised(store: int, keys_q8_ptr: int) -> None:
+    _check(load().dresd_store_attach_quantised(store, keys_q8_ptr))
+
+
+def dresd_retrieve_quantised(store: int, queries_ptr: int, B: int, top_n: int, draft_len: int, candidates: int,
+                             out_ids_ptr: int, out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_retrieve_quantised(store, queries_ptr, B, top_n, draft_len, candidates, out_ids_ptr,
+                                           out_scores_ptr, out_tokens_ptr, stream))
 
 
 def dresd_set_global_option(name: str, value: int) -> None:
@@ -307,6 +328,31 @@ class Store:
         dresd_retrieve_filtered(self.handle, queries.data_ptr(),
                                 None if first_tokens is None else first_tokens.data_ptr(), B, top_n, draft_len,
                                 ids.data_ptr(), scores.data_ptr(), tokens.data_ptr(), s)
+        return ids, scores, tokens
+
+    def attach_quantised(self, stream=None):
+        """Build the 8-bit (E4M3) copy of the keys on the device and attach it; returns the copy."""
+        torch = _torch()
+        s = (stream or torch.cuda.current_stream()).cuda_stream
+        q8 = torch.empty((self.N, self.d), dtype=torch.uint8, device=self.keys.device)
+        dresd_quantise_keys(self.keys.data_ptr(), self.N, self.d, DTYPE_CODE[self.dtype], q8.data_ptr(), s)
+        dresd_store_attach_quantised(self.handle, q8.data_ptr())
+        self.keys_q8 = q8                                # keep the borrowed buffer alive
+        return q8
+
+    def retrieve_quantised(self, queries, top_n: int, draft_len: int, candidates: int, out=None, stream=None):
+        """Candidates by 8-bit approximate score, exact re-ranking of `candidates` rows per query."""
+        torch = _torch()
+        B = queries.shape[0]
+        if out is None:
+            dev = queries.device
+            out = (torch.empty((B, top_n), dtype=torch.int32, device=dev),
+                   torch.empty((B, top_n), dtype=torch.float32, device=dev),
+                   torch.empty((B, top_n, draft_len), dtype=torch.int32, device=dev))
+        ids, scores, tokens = out
+        s = (stream or torch.cuda.current_stream()).cuda_stream
+        dresd_retrieve_quantised(self.handle, queries.data_ptr(), B, top_n, draft_len, candidates,
+                                 ids.data_ptr(), scores.data_ptr(), tokens.data_ptr(), s)
         return ids, scores, tokens
 
     def retrieve_host(self, queries, top_n: int, draft_len: int, out, stream=None):

@@ -127,6 +127,10 @@ struct dresd_store {
     // options / bookkeeping
     int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m;
     double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
+    const void *k8;              // 8-bit (E4M3) copy of the keys, borrowed; null = none attached
+    void *qsplit8;               // [2 * kMaxBatch][dpad8] 8-bit query operand
+    int dpad8;                   // d rounded up to 128 bytes
+    CUtensorMap map_k8, map_q8[4];
     float *proj_ws;              // partial products of the split projection (allocated with W)
     size_t proj_ws_bytes;
     cudaStream_t last_stream;
@@ -151,6 +155,7 @@ void free_store(dresd_store *s)
     cudaFree(s->first_col);
     cudaFree(s->q_stage);
     cudaFree(s->proj_ws);
+    cudaFree(s->qsplit8);
     cudaFree(s->ids_dev);
     cudaFree(s->scores_dev);
     cudaFree(s->tokens_dev);
@@ -214,8 +219,11 @@ dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows
 
 dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n, int draft_len,
                           int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream,
-                          const int32_t *first_tokens = nullptr)
+                          const int32_t *first_tokens = nullptr, int quantised_m = 0)
 {
+    // quantised_m > 0: candidates by approximate score over the 8-bit copy of the keys (the same
+    // tcgen05 kernel, other instruction kind), then exact re-ranking of the quantised_m best
+    const bool q8 = quantised_m > 0;
     s->last_stream = stream;
     s->last_launches = 0;
     s->last_key_passes = 0.0;
@@ -224,14 +232,20 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // the fastest at every measured shape (7.1-7.2 TB/s at batch 1 for d = 64 and 256
     // against 6.7-6.8 for the streaming mma.sync kernel), so it is the default; the
     // streaming kernel stays available as "scan_path" 1 and serves the allocation-free call.
-    const bool umma = !f32 && s->opt_path != 1;
+    const bool umma = q8 || (!f32 && s->opt_path != 1);
     const int op_rows = umma ? scan_umma_operand_rows(B) : 0;
     // the kernel with the keys as the N operand reads hi and lo of a query from one TMEM fragment
-    const int blocked = umma && !s->opt_keys_as_m && scan_ummat_eligible(s->d, B);
+    const int blocked = umma && !q8 && !s->opt_keys_as_m && scan_ummat_eligible(s->d, B);
     dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream, blocked);
     if (st != DRESD_OK) return st;
 
-    const int umma_rows = umma ? scan_umma_tile_rows(s->d, B, s->opt_keys_as_m) : 1;
+    if (q8) {
+        cudaError_t e8 = launch_split_queries_e4m3(s->qhat, B, op_rows / 2, s->d, s->qsplit8, s->dpad8, stream);
+        if (e8 != cudaSuccess) return fail_cuda(e8, "query split launch");
+        s->last_launches += 1;
+    }
+    const int scan_d = q8 ? s->d / 2 : s->d;          // the 8-bit store is scanned as rows of d/2 two-byte units
+    const int umma_rows = umma ? scan_umma_tile_rows(scan_d, B, q8 ? 1 : s->opt_keys_as_m) : 1;
     const int n_tiles = umma ? (int)((s->N + umma_rows - 1) / umma_rows) : s->n_tiles;
     int grid = s->opt_grid > 0 ? s->opt_grid : s->num_sms;
     if (grid > s->max_grid) grid = s->max_grid;
@@ -244,19 +258,22 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     if (umma) {
         ScanArgs a{};
         a.N = s->N;
-        a.d = s->d;
-        a.dpad = s->dpad;
-        a.dtype = s->dtype;
+        a.d = scan_d;
+        a.dpad = q8 ? s->dpad8 / 2 : s->dpad;
+        a.dtype = q8 ? kE4M3 : s->dtype;
         a.n_tiles = n_tiles;
         a.B = B;
-        a.top_n = top_n;
-        a.lo_inv_scale = 1.0f / lo_scale;
+        a.top_n = q8 ? quantised_m : top_n;
+        a.lo_inv_scale = q8 ? 1.0f / 16.0f : 1.0f / lo_scale;
         a.cand = s->cand;
         a.cand_batch = B;
         a.status = s->status;
         a.gtau = s->gtau;
         a.no_select = s->opt_no_select;
-        a.keys_as_m = s->opt_keys_as_m;
+        a.keys_as_m = q8 ? 1 : s->opt_keys_as_m;
+        const CUtensorMap &kmap = q8 ? s->map_k8 : s->map_umma;
+        const CUtensorMap *qmaps = q8 ? s->map_q8 : s->map_q;
+        const int sel_n = a.top_n;
         a.first_col = first_tokens ? s->first_col : nullptr;
         a.want_first = first_tokens;
         const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
@@ -266,19 +283,19 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         // queues ~64 n survivors per query GPU-wide instead of ~n ln(rows/n) per CTA.
         // The filter only rejects rows that cannot be in the result.
         const int pstride = s->opt_probe;
-        if (pstride > 1 && !s->opt_no_select && B * top_n >= 256 && n_tiles >= pstride * grid) {
+        if (pstride > 1 && !s->opt_no_select && B * sel_n >= 256 && n_tiles >= pstride * grid) {
             ScanArgs pa = a;
             pa.tile_stride = pstride;
             pa.n_tiles = (n_tiles + pstride - 1) / pstride;
             pa.probe_max = (long long)pa.n_tiles * (umma_rows / 128) <= 32LL * grid;   // the bests fit a queue
             int pgrid = grid < pa.n_tiles ? grid : pa.n_tiles;
-            e = launch_scan_umma(s->map_umma, s->map_q[mi], pa, pgrid, stream);
-            if (e == cudaSuccess) e = launch_merge_tau(s->cand, pgrid, B, top_n, s->gtau, stream);
+            e = launch_scan_umma(kmap, qmaps[mi], pa, pgrid, stream);
+            if (e == cudaSuccess) e = launch_merge_tau(s->cand, pgrid, B, sel_n, s->gtau, stream);
             if (e != cudaSuccess) return fail_cuda(e, "probe launch");
             s->last_launches += 2;
             s->last_key_passes += 1.0 / pstride;
         }
-        e = launch_scan_umma(s->map_umma, s->map_q[mi], a, grid, stream);
+        e = launch_scan_umma(kmap, qmaps[mi], a, grid, stream);
         if (e != cudaSuccess) return fail_cuda(e, "scan launch");
         s->last_launches += 1;
         s->last_key_passes += 1.0;
@@ -313,6 +330,17 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     if (prof) {
         cudaEventRecord(s->prof_events[2 * s->prof_count + 1], stream);
         s->prof_count += 1;
+    }
+    if (q8) {
+        // the m candidates of every query (approximate scores are not returned), then the exact pass
+        cudaError_t e = launch_merge_gather(s->cand, grid, B, quantised_m, s->ids_dev, s->scores_dev, nullptr, 0, s->N, 0,
+                                            nullptr, stream);
+        if (e == cudaSuccess)
+            e = launch_rerank(s->keys, s->dtype, s->d, s->N, s->qhat, s->ids_dev, B, quantised_m, top_n, s->next_tokens,
+                              s->stored_len, draft_len, out_ids, out_scores, out_tokens, stream);
+        if (e != cudaSuccess) return fail_cuda(e, "merge / re-rank launch");
+        s->last_launches += 2;
+        return DRESD_OK;
     }
     cudaError_t e = launch_merge_gather(s->cand, grid, B, top_n, out_ids, out_scores, s->next_tokens, s->stored_len,
                                         s->N, draft_len, out_tokens, stream);
@@ -766,6 +794,61 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
     if (st == DRESD_OK && e != cudaSuccess) st = fail_cuda(e, "stream synchronize");
     if (st == DRESD_OK && word != 0) st = fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
     return st;
+}
+
+dresd_status dresd_quantise_keys(const void *keys, int64_t N, int d, dresd_dtype dtype, void *out_q8, void *stream)
+{
+    if (dtype != DRESD_F16 && dtype != DRESD_BF16)
+        return fail(DRESD_ERR_UNSUPPORTED, "dresd_quantise_keys reads 16-bit datastores (fp16 or bf16)");
+    if (N <= 0 || N > 2147483647LL) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1", (long long)N);
+    if (d < 16 || d % 16 != 0) return fail(DRESD_ERR_INVALID, "d = %d must be a positive multiple of 16", d);
+    if (!is_device_ptr(keys) || !is_device_ptr(out_q8)) return fail(DRESD_ERR_INVALID, "keys / out_q8 must be device pointers");
+    if (reinterpret_cast<uintptr_t>(keys) % 16 != 0 || reinterpret_cast<uintptr_t>(out_q8) % 16 != 0)
+        return fail(DRESD_ERR_INVALID, "keys / out_q8 not 16-byte aligned");
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return fail_cuda(e, "device query");
+    e = launch_quantise_keys(keys, (int)dtype, N, d, out_q8, sms, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "quantise launch");
+}
+
+dresd_status dresd_store_attach_quantised(dresd_store *s, const void *keys_q8)
+{
+    if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+    if (s->dtype == kF32) return fail(DRESD_ERR_UNSUPPORTED, "the quantised search needs a 16-bit store");
+    if (s->d % 16 != 0) return fail(DRESD_ERR_UNSUPPORTED, "d = %d must be a multiple of 16 for the 8-bit copy", s->d);
+    if (s->d > 2048) return fail(DRESD_ERR_UNSUPPORTED, "d = %d exceeds 2048 for the 8-bit copy", s->d);
+    if (!is_device_ptr(keys_q8) || reinterpret_cast<uintptr_t>(keys_q8) % 16 != 0)
+        return fail(DRESD_ERR_INVALID, "keys_q8 must be a 16-byte aligned device pointer");
+    if (!s->qsplit8) {
+        s->dpad8 = (s->d + 127) / 128 * 128;
+        if (cudaMalloc(&s->qsplit8, (size_t)2 * kMaxBatch * s->dpad8) != cudaSuccess) {
+            cudaGetLastError();
+            s->qsplit8 = nullptr;
+            return fail(DRESD_ERR_ALLOC, "workspace allocation failed");
+        }
+    }
+    // The scan kernels see the 8-bit store as rows of d/2 two-byte units (TMA moves bytes).
+    bool ok = make_map(&s->map_k8, keys_q8, kF16, s->N, s->d / 2, 128);
+    for (int i = 0; i < 4; ++i) ok = ok && make_map(&s->map_q8[i], s->qsplit8, kF16, 2 * kMaxBatch, s->dpad8 / 2, 16 << i);
+    if (!ok) return fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the 8-bit copy");
+    s->k8 = keys_q8;
+    return DRESD_OK;
+}
+
+dresd_status dresd_retrieve_quantised(dresd_store *s, const void *queries, int B, int top_n, int draft_len,
+                                      int candidates, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
+                                      void *stream)
+{
+    dresd_status st = check_retrieve_args(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens, true);
+    if (st != DRESD_OK) return st;
+    if (!s->k8) return fail(DRESD_ERR_INVALID, "no 8-bit copy attached (dresd_store_attach_quantised)");
+    if (candidates < top_n || candidates > DRESD_MAX_TOP_N || candidates > s->N)
+        return fail(DRESD_ERR_INVALID, "candidates = %d outside top_n..min(%d, N)", candidates, DRESD_MAX_TOP_N);
+    if (B == 0) return DRESD_OK;
+    return run_retrieve(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens,
+                        static_cast<cudaStream_t>(stream), nullptr, candidates);
 }
 
 dresd_status dresd_set_global_option(const char *name, int value)

@@ -7,7 +7,7 @@
 
 namespace dresd {
 
-enum { kF32 = 0, kF16 = 1, kBF16 = 2 };
+enum { kF32 = 0, kF16 = 1, kBF16 = 2, kE4M3 = 3 };   // kE4M3: the 8-bit copy of a 16-bit store (internal)
 
 constexpr int kMaxBatch = 64;
 constexpr int kMaxTopN = 32;
@@ -135,6 +135,16 @@ cudaError_t launch_build_keys(const CUtensorMap &h_map, const CUtensorMap &whi_m
 size_t fit_zscore_workspace_bytes(long long N, int d_in, int sms);
 cudaError_t launch_fit_zscore(const void *V, int dtype, long long N, int d_in, int sms, void *workspace,
                               float *mean, float *var, cudaStream_t stream);
+
+// ---- K9: quantised candidate search (8-bit E4M3 keys, exact re-ranking) ----
+cudaError_t launch_quantise_keys(const void *keys, int dtype, long long N, int d, void *out_q8, int sms,
+                                 cudaStream_t stream);
+// qsplit8: [2 * rows][dpad8] bytes, rows 2b / 2b+1 = the two 8-bit terms of query b
+cudaError_t launch_split_queries_e4m3(const float *qhat, int B, int rows, int d, void *qsplit8, int dpad8,
+                                      cudaStream_t stream);
+cudaError_t launch_rerank(const void *keys, int dtype, int d, long long N, const float *qhat, const int32_t *cand,
+                          int B, int m, int top_n, const int32_t *next_tokens, int stored_len, int draft_len,
+                          int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream);
 
 // Stores `msg` as the calling thread's dresd_last_error() text.
 void set_last_error(const char *msg);

@@ -222,6 +222,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     } else if (warp == 1) {
         // ---------------------------------- MMA issuer ----------------------------------
         if (lane == 0) {
+            // operand formats: kind::f16 -- 0 = fp16, 1 = bf16; kind::f8f6f4 -- 0 = E4M3
+            constexpr bool kIs8 = std::is_same<T, E4M3Keys>::value;
             constexpr uint32_t kFmt = std::is_same<T, __nv_bfloat16>::value ? 1u : 0u;
             constexpr uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(NCOLS >> 3) << 17) |
                                        ((uint32_t)(kTileRows >> 4) << 24);
@@ -245,8 +247,12 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                                 const uint64_t b_desc = make_desc(smem_u32(qres + (size_t)j * kQSlabBytes));
 #pragma unroll
                                 for (int k = 0; k < 4; ++k)
-                                    umma_f16(d_tmem + (uint32_t)(sub * NCOLS), a_desc + 2 * k, b_desc + 2 * k, idesc,
-                                             (j + k) != 0);
+                                    if constexpr (kIs8)
+                                        umma_f8(d_tmem + (uint32_t)(sub * NCOLS), a_desc + 2 * k, b_desc + 2 * k, idesc,
+                                                (j + k) != 0);
+                                    else
+                                        umma_f16(d_tmem + (uint32_t)(sub * NCOLS), a_desc + 2 * k, b_desc + 2 * k, idesc,
+                                                 (j + k) != 0);
                             }
                     } else {
                         const int sl0 = g * gs;
@@ -258,7 +264,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                             const uint64_t a_desc = make_desc(a_addr), b_desc = make_desc(b_addr);
 #pragma unroll
                             for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
-                                umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
+                                if constexpr (kIs8) umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
+                                else umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
                         }
                     }
                     tc_commit(&empty[s]);             // group reusable once these MMAs have read it
@@ -551,17 +558,18 @@ int scan_umma_operand_rows(int B) { return ncols_of(B); }
 cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a_in, int grid,
                              cudaStream_t stream)
 {
-    if (!a_in.keys_as_m && scan_ummat_eligible(a_in.d, a_in.B))
+    if (!a_in.keys_as_m && a_in.dtype != kE4M3 && scan_ummat_eligible(a_in.d, a_in.B))
         return launch_scan_ummat(kmap, qmap, a_in, grid, stream);
     ScanArgs a = a_in;
     if (a.tile_stride < 1) a.tile_stride = 1;
     const Plan p = make_plan(a.d, a.B);
     if (p.stages < 2) return cudaErrorInvalidValue;
     a.stages = p.stages;
-    const bool h = a.dtype == kF16;
+    const bool h = a.dtype == kF16, q8 = a.dtype == kE4M3;
 #define DRESD_GO(N_)                                                                          \
-    return h ? launch_tsub<__half, N_>(kmap, qmap, a, p, grid, stream)                        \
-             : launch_tsub<__nv_bfloat16, N_>(kmap, qmap, a, p, grid, stream)
+    return q8 ? launch_tsub<E4M3Keys, N_>(kmap, qmap, a, p, grid, stream)                     \
+           : h ? launch_tsub<__half, N_>(kmap, qmap, a, p, grid, stream)                      \
+               : launch_tsub<__nv_bfloat16, N_>(kmap, qmap, a, p, grid, stream)
     switch (p.ncols) {
     case 16: DRESD_GO(16);
     case 32: DRESD_GO(32);
