@@ -62,6 +62,9 @@ def parse_args():
     ap.add_argument("--first-token-filter", action="store_true",
                     help="time dresd_retrieve_filtered: each query wants the first stored token of its source row")
     ap.add_argument("--probe", type=int, default=1, help="probe-pass tile stride (0 off, 1 default)")
+    ap.add_argument("--quantised", type=int, default=0, metavar="M",
+                    help="candidates by approximate score over an 8-bit (E4M3) copy of the keys, exact re-ranking "
+                         "of the M best (top_n <= M <= 32); reports recall against the exact path")
     ap.add_argument("--keys-as-m", type=int, default=0, choices=[0, 1],
                     help="1: keep the keys as the M operand of the tcgen05 kernel also for 33-64 queries")
     ap.add_argument("--scan-path", type=int, default=0, choices=[0, 1, 2],
@@ -246,9 +249,27 @@ def run_ours(args):
            torch.empty((B, n), dtype=torch.float32, device="cuda"),
            torch.empty((B, n, L), dtype=torch.int32, device="cuda"))
 
+    recall = None
+    if args.quantised:
+        if dft is not None:
+            raise SystemExit("--quantised and --first-token-filter are separate paths")
+        store.attach_quantised()
+        # recall of the exact neighbours (the exact path is the parity-checked one)
+        hit = tot = 0
+        for i in range(min(nq, 64)):
+            j = (q_first + i) * B
+            ex = store.retrieve(dq[j:j + B], n, L)[0].cpu().numpy()
+            ap_ = store.retrieve_quantised(dq[j:j + B], n, L, args.quantised)[0].cpu().numpy()
+            for b in range(B):
+                hit += len(set(ex[b].tolist()) & set(ap_[b].tolist()))
+                tot += n
+        recall = hit / tot
+
     def step(i):
         j = (q_first + i % nq) * B
-        if dft is None:
+        if args.quantised:
+            store.retrieve_quantised(dq[j:j + B], n, L, args.quantised, out=out)
+        elif dft is None:
             store.retrieve(dq[j:j + B], n, L, out=out)
         else:
             store.retrieve_filtered(dq[j:j + B], dft[j:j + B], n, L, out=out)
@@ -314,13 +335,26 @@ def run_ours(args):
     hout = (torch.empty((B, n), dtype=torch.int32).pin_memory(),
             torch.empty((B, n), dtype=torch.float32).pin_memory(),
             torch.empty((B, n, L), dtype=torch.int32).pin_memory())
+    dq_stage = dq[:B].clone()
+
+    def host_call(j):
+        if not args.quantised:
+            store.retrieve_host(hq[j:j + B], n, L, hout)
+            return
+        # the quantised call takes device buffers: the same copies, issued here
+        dq_stage.view(torch.int16 if dtype != "f32" else torch.float32).copy_(
+            hq[j:j + B].view(torch.int16 if dtype != "f32" else torch.float32), non_blocking=True)
+        store.retrieve_quantised(dq_stage, n, L, args.quantised, out=out)
+        for h, o_ in zip(hout, out):
+            h.copy_(o_, non_blocking=True)
+        torch.cuda.synchronize()
+
     for i in range(min(args.warmup, 3)):
-        store.retrieve_host(hq[(q_first + i % nq) * B:(q_first + i % nq) * B + B], n, L, hout)
+        host_call((q_first + i % nq) * B)
     barrier()
     t0 = time.perf_counter()
     for i in range(args.steps):
-        j = (q_first + (args.warmup + i) % nq) * B
-        store.retrieve_host(hq[j:j + B], n, L, hout)
+        host_call((q_first + (args.warmup + i) % nq) * B)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     barrier()
@@ -337,11 +371,12 @@ def run_ours(args):
     qps = dist_util.aggregate_throughput(B, args.steps, world, ms_total)
     e2e_qps = dist_util.aggregate_throughput(B, args.steps, world, e2e_ms_total)
     eb = synth.DTYPE_BYTES[dtype]
-    key_bytes = cfg["N"] * cfg["d"] * eb                    # algorithmic bytes of one scoring launch
+    key_bytes = cfg["N"] * cfg["d"] * (1 if args.quantised else eb)   # algorithmic bytes of one scoring launch
     peak, peak_src = peaks()
     achieved = passes * key_bytes / (scan_ms_avg * 1e-3) / 1e9
     line = {
-        "metric": metric_name(cfg), "value": qps, "unit": "queries/s", "n_gpus": world,
+        "metric": metric_name(cfg) + (" -- 8-bit candidates, exact re-rank of %d" % args.quantised
+                                      if args.quantised else ""), "value": qps, "unit": "queries/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate over %s keys" % dtype,
         "data": "synthetic", "config": workload_config(cfg),
@@ -367,6 +402,10 @@ def run_ours(args):
             "note": "floor = the same call with a filter that nothing passes (keys streamed and scored, "
                     "no candidate queued, merged or gathered beyond empty lists)"},
     }
+    if args.quantised:
+        line["quantised"] = {"candidates": args.quantised, "recall_at_n_vs_exact_path": recall,
+                             "queries_compared": min(nq, 64) * B, "key_format": "E4M3 (k8 = e4m3(256 k))"}
+        line["dtype"] = "f32 accumulate over E4M3 keys, exact re-rank over %s keys" % dtype
     if world == 1 and not args.no_cpu_baseline:
         o_qps, threads, o_nq, o_dt, _ = time_oracle(cfg, keys, toks, q, args.oracle_queries)
         line["cpu_baseline"] = {"value": o_qps, "unit": "queries/s", "cores": threads, "kind": "oracle",
