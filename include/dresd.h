@@ -298,6 +298,9 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "probe"      large batches on large stores first run a probe pass over every
  *                value-th key tile to seed the selection filter; 0 = never,
  *                1 = default stride (128).
+ *   "pack2"      1 (default): the quantised search of a store with d = 64 scans the 8-bit copy
+ *                as rows of two keys (one 128-byte line), up to 32 queries per call; 0 = one
+ *                key per row.  Results do not change.
  *   "keys_as_m"  0 (default): batches of 33-64 queries on rows of 129-256 elements run the
  *                tcgen05 kernel with the queries as the M = 128 and the keys as the
  *                N = 256 operand of the instruction; 1 = keys as the M operand at every

@@ -125,12 +125,14 @@ struct dresd_store {
     CUtensorMap map_umma;
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     // options / bookkeeping
-    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m;
+    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m, opt_pack2;
     double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
     const void *k8;              // 8-bit (E4M3) copy of the keys, borrowed; null = none attached
     void *qsplit8;               // [2 * kMaxBatch][dpad8] 8-bit query operand
     int dpad8;                   // d rounded up to 128 bytes
     CUtensorMap map_k8, map_q8[4];
+    CUtensorMap map_k8p;         // d = 64: the 8-bit copy as N/2 rows of two keys (128 bytes)
+    int k8_packable;
     float *proj_ws;              // partial products of the split projection (allocated with W)
     size_t proj_ws_bytes;
     cudaStream_t last_stream;
@@ -224,6 +226,8 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // quantised_m > 0: candidates by approximate score over the 8-bit copy of the keys (the same
     // tcgen05 kernel, other instruction kind), then exact re-ranking of the quantised_m best
     const bool q8 = quantised_m > 0;
+    // 64-element keys are 64 bytes in the 8-bit copy: two per 128-byte row, two column pairs per query
+    const bool pack2 = q8 && s->k8_packable && B <= kMaxBatch / 2 && s->opt_pack2;
     s->last_stream = stream;
     s->last_launches = 0;
     s->last_key_passes = 0.0;
@@ -233,20 +237,23 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // against 6.7-6.8 for the streaming mma.sync kernel), so it is the default; the
     // streaming kernel stays available as "scan_path" 1 and serves the allocation-free call.
     const bool umma = q8 || (!f32 && s->opt_path != 1);
-    const int op_rows = umma ? scan_umma_operand_rows(B) : 0;
+    const int op_rows = umma ? scan_umma_operand_rows(pack2 ? 2 * B : B) : 0;
     // the kernel with the keys as the N operand reads hi and lo of a query from one TMEM fragment
     const int blocked = umma && !q8 && !s->opt_keys_as_m && scan_ummat_eligible(s->d, B);
     dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream, blocked);
     if (st != DRESD_OK) return st;
 
     if (q8) {
-        cudaError_t e8 = launch_split_queries_e4m3(s->qhat, B, op_rows / 2, s->d, s->qsplit8, s->dpad8, stream);
+        cudaError_t e8 = launch_split_queries_e4m3(s->qhat, B, pack2 ? op_rows / 4 : op_rows / 2, s->d, s->qsplit8,
+                                                   s->dpad8, pack2 ? 1 : 0, stream);
         if (e8 != cudaSuccess) return fail_cuda(e8, "query split launch");
         s->last_launches += 1;
     }
-    const int scan_d = q8 ? s->d / 2 : s->d;          // the 8-bit store is scanned as rows of d/2 two-byte units
-    const int umma_rows = umma ? scan_umma_tile_rows(scan_d, B, q8 ? 1 : s->opt_keys_as_m) : 1;
-    const int n_tiles = umma ? (int)((s->N + umma_rows - 1) / umma_rows) : s->n_tiles;
+    // the 8-bit store is scanned as rows of d/2 two-byte units (packed: N/2 rows of 64 units)
+    const int scan_d = pack2 ? 64 : q8 ? s->d / 2 : s->d;
+    const long long scan_rows = pack2 ? s->N / 2 : s->N;
+    const int umma_rows = umma ? scan_umma_tile_rows(scan_d, pack2 ? 2 * B : B, q8 ? 1 : s->opt_keys_as_m) : 1;
+    const int n_tiles = umma ? (int)((scan_rows + umma_rows - 1) / umma_rows) : s->n_tiles;
     int grid = s->opt_grid > 0 ? s->opt_grid : s->num_sms;
     if (grid > s->max_grid) grid = s->max_grid;
     if (grid > n_tiles) grid = n_tiles;
@@ -257,7 +264,8 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     if (prof) cudaEventRecord(s->prof_events[2 * s->prof_count], stream);
     if (umma) {
         ScanArgs a{};
-        a.N = s->N;
+        a.N = scan_rows;
+        a.pack2 = pack2 ? 1 : 0;
         a.d = scan_d;
         a.dpad = q8 ? s->dpad8 / 2 : s->dpad;
         a.dtype = q8 ? kE4M3 : s->dtype;
@@ -271,7 +279,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.gtau = s->gtau;
         a.no_select = s->opt_no_select;
         a.keys_as_m = q8 ? 1 : s->opt_keys_as_m;
-        const CUtensorMap &kmap = q8 ? s->map_k8 : s->map_umma;
+        const CUtensorMap &kmap = pack2 ? s->map_k8p : q8 ? s->map_k8 : s->map_umma;
         const CUtensorMap *qmaps = q8 ? s->map_q8 : s->map_q;
         const int sel_n = a.top_n;
         a.first_col = first_tokens ? s->first_col : nullptr;
@@ -336,8 +344,9 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         cudaError_t e = launch_merge_gather(s->cand, grid, B, quantised_m, s->ids_dev, s->scores_dev, nullptr, 0, s->N, 0,
                                             nullptr, stream);
         if (e == cudaSuccess)
-            e = launch_rerank(s->keys, s->dtype, s->d, s->N, s->qhat, s->ids_dev, B, quantised_m, top_n, s->next_tokens,
-                              s->stored_len, draft_len, out_ids, out_scores, out_tokens, stream);
+            e = launch_rerank(s->keys, s->dtype, s->d, s->N, s->qhat, s->ids_dev, B, quantised_m, top_n,
+                              pack2 && (s->N & 1) ? s->N - 1 : -1, s->next_tokens, s->stored_len, draft_len, out_ids,
+                              out_scores, out_tokens, stream);
         if (e != cudaSuccess) return fail_cuda(e, "merge / re-rank launch");
         s->last_launches += 2;
         return DRESD_OK;
@@ -425,6 +434,7 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
     s->eps_z = 1e-5f;
     s->max_grid = 2 * s->num_sms;
     s->opt_probe = kProbeStride;
+    s->opt_pack2 = 1;
 
     s->tile_rows = dtype == DRESD_F32 ? scan_f32_tile_rows(d) : scan_mma_tile_rows(d);
     s->n_tiles = (int)((N + s->tile_rows - 1) / s->tile_rows);
@@ -637,6 +647,11 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
         s->opt_lose_stage = value;
         return DRESD_OK;
     }
+    if (strcmp(name, "pack2") == 0) {
+        if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "pack2 takes 0 or 1");
+        s->opt_pack2 = value;
+        return DRESD_OK;
+    }
     if (strcmp(name, "keys_as_m") == 0) {
         if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "keys_as_m takes 0 or 1");
         s->opt_keys_as_m = value;
@@ -833,6 +848,12 @@ dresd_status dresd_store_attach_quantised(dresd_store *s, const void *keys_q8)
     bool ok = make_map(&s->map_k8, keys_q8, kF16, s->N, s->d / 2, 128);
     for (int i = 0; i < 4; ++i) ok = ok && make_map(&s->map_q8[i], s->qsplit8, kF16, 2 * kMaxBatch, s->dpad8 / 2, 16 << i);
     if (!ok) return fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the 8-bit copy");
+    s->k8_packable = 0;
+    if (s->d == 64 && s->N >= 2) {
+        if (!make_map(&s->map_k8p, keys_q8, kF16, s->N / 2, 64, 128))
+            return fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the packed 8-bit copy");
+        s->k8_packable = 1;
+    }
     s->k8 = keys_q8;
     return DRESD_OK;
 }

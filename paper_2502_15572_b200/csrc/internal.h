@@ -67,6 +67,7 @@ struct ScanArgs {
     int probe_max;          // tcgen05 kernel, probe pass: keep only each tile's best row per query
     int no_select;          // tcgen05 kernel, measurement only: nothing passes the filter (scan floor)
     int keys_as_m;          // tcgen05 kernels: never use the form with the keys as the N = 256 operand
+    int pack2;              // 8-bit keys of 64 elements: a 128-byte row holds two keys (N = rows, ids = 2 row + parity)
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.
 int scan_mma_tile_rows(int d);
@@ -140,11 +141,14 @@ cudaError_t launch_fit_zscore(const void *V, int dtype, long long N, int d_in, i
 cudaError_t launch_quantise_keys(const void *keys, int dtype, long long N, int d, void *out_q8, int sms,
                                  cudaStream_t stream);
 // qsplit8: [2 * rows][dpad8] bytes, rows 2b / 2b+1 = the two 8-bit terms of query b
+// pack2: four rows per query, (h1|0), (h2|0), (0|h1), (0|h2), for two 64-byte keys per 128-byte row
 cudaError_t launch_split_queries_e4m3(const float *qhat, int B, int rows, int d, void *qsplit8, int dpad8,
-                                      cudaStream_t stream);
+                                      int pack2, cudaStream_t stream);
+// extra_id >= 0: one more candidate for every query (the last key of an odd-sized packed store)
 cudaError_t launch_rerank(const void *keys, int dtype, int d, long long N, const float *qhat, const int32_t *cand,
-                          int B, int m, int top_n, const int32_t *next_tokens, int stored_len, int draft_len,
-                          int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream);
+                          int B, int m, int top_n, long long extra_id, const int32_t *next_tokens, int stored_len,
+                          int draft_len, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
+                          cudaStream_t stream);
 
 // Stores `msg` as the calling thread's dresd_last_error() text.
 void set_last_error(const char *msg);

@@ -94,7 +94,12 @@ struct EpiFlags {
     int overflow;
 };
 
-template <typename T, int NCOLS, int TSUB>
+// PACK2 (8-bit keys of 64 elements): a 128-byte row of the store holds TWO keys.  Query j then
+// owns four operand rows -- (h1|0), (h2|0), (0|h1), (0|h2) -- i.e. two "virtual" queries 2j, 2j+1
+// that score the even and the odd key of a row; both feed the lists and the filter of query j,
+// and a candidate's id is 2 * row + parity.  tau[] is kept per virtual query (two equal
+// entries per query) so that the hot loop is the same code.
+template <typename T, int NCOLS, int TSUB, bool PACK2 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_constant__ CUtensorMap q_map,
                  const ScanArgs a, const int q_resident, const int gs)
@@ -157,8 +162,9 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             warp_topn_init(&sel[q], lane);
             // start from whatever the grid already knows; padding columns never pass
             if (lane == 0) {
-                tau[q] = (q < a.B && !a.no_select) ? peek_tau(&a.gtau[q], -INFINITY) : INFINITY;
-                want_s[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
+                const int rq = PACK2 ? q >> 1 : q;          // the query this column pair belongs to
+                tau[q] = (rq < a.B && !a.no_select) ? peek_tau(&a.gtau[rq], -INFINITY) : INFINITY;
+                want_s[q] = (!PACK2 && a.first_col && q < a.B) ? a.want_first[q] : -1;
             }
         }
     }
@@ -314,7 +320,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             dead = __any_sync(0xFFFFFFFFu, dead);
             tc_fence_after();
             // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
-            if ((tl & 3) == 0 && et < a.B && !a.no_select) tau[et] = peek_tau(&a.gtau[et], tau[et]);
+            if ((tl & 3) == 0 && et < a.B && !a.no_select) {
+                if constexpr (PACK2) tau[2 * et] = tau[2 * et + 1] = peek_tau(&a.gtau[et], tau[2 * et]);
+                else tau[et] = peek_tau(&a.gtau[et], tau[et]);
+            }
             const uint32_t acc_addr = lane_addr + (uint32_t)(acc * kAccCols);
             if (a.probe_max) {
                 // Probe pass: no filtering and no lists -- only the best row of each sub-tile
@@ -335,7 +344,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                             const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
                             const int w = want_s[qbase + j];
                             const bool ok = row_ok && (w < 0 || tok[sub] == w) && s > -INFINITY;   // false for NaN
-                            v[j] = ok ? pack_candidate(s, (uint32_t)row) : 0ull;
+                            const uint32_t id = PACK2 ? (uint32_t)(2 * row + ((qbase + j) & 1)) : (uint32_t)row;
+                            v[j] = ok ? pack_candidate(s, id) : 0ull;
                         }
                         // per-query maximum over the warp's 32 rows: QW-1 exchanges for all queries
                         WarpColumnMax<QW, 16>::run(v, lane);
@@ -349,8 +359,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 for (int q = ew; q < a.B; q += kEpiWarps) {
                     if (lane == 0) {
                         for (int sub = 0; sub < TSUB; ++sub) {
-                            const unsigned long long *m = tilemax + (size_t)(sub * 4) * NQ + q;
-                            const unsigned long long v = umax64(umax64(m[0], m[NQ]), umax64(m[2 * NQ], m[3 * NQ]));
+                            const unsigned long long *m = tilemax + (size_t)(sub * 4) * NQ + (PACK2 ? 2 * q : q);
+                            unsigned long long v = umax64(umax64(m[0], m[NQ]), umax64(m[2 * NQ], m[3 * NQ]));
+                            if constexpr (PACK2)               // the odd keys of the same rows
+                                v = umax64(v, umax64(umax64(m[1], m[NQ + 1]), umax64(m[2 * NQ + 1], m[3 * NQ + 1])));
                             if (v && sel[q].count < kQueueCap) sel[q].queue[sel[q].count++] = v;
                         }
                     }
@@ -414,10 +426,11 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         tmem_ld_wait();
                         if ((mask >> j) & 1u) {
                             const float s = fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
-                            const int q = qbase + j;
+                            const int q = PACK2 ? (qbase + j) >> 1 : qbase + j;
+                            const uint32_t id = PACK2 ? (uint32_t)(2 * row + ((qbase + j) & 1)) : (uint32_t)row;
                             const int slot = atomicAdd(&sel[q].count, 1);
                             if (slot < kQueueCap) {
-                                sel[q].queue[slot] = pack_candidate(s, (uint32_t)row);
+                                sel[q].queue[slot] = pack_candidate(s, id);
                                 if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
                             } else {
                                 pending[sub] |= 1u << j;
@@ -442,7 +455,11 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 for (int q = ew; q < NQ; q += kEpiWarps) {
                     if (sel[q].count > 0) {
                         warp_topn_merge(&sel[q], a.top_n, lane);
-                        if (lane == 0 && q < a.B) tau[q] = share_tau(&a.gtau[q], sel[q].tau);
+                        if (lane == 0 && q < a.B) {
+                            const float t = share_tau(&a.gtau[q], sel[q].tau);
+                            if constexpr (PACK2) tau[2 * q] = tau[2 * q + 1] = t;
+                            else tau[q] = t;
+                        }
                     }
                 }
                 epi_bar();                                   // C: lists, counts and tau are settled
@@ -520,14 +537,14 @@ Plan make_plan(int d, int B)
     return p;
 }
 
-template <typename T, int NCOLS, int TSUB>
+template <typename T, int NCOLS, int TSUB, bool PACK2 = false>
 cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a, const Plan &p,
                        int grid, cudaStream_t stream)
 {
     if constexpr (2 * TSUB * NCOLS > 512) {
         return cudaErrorInvalidValue;
     } else {
-        auto kernel = scan_umma_kernel<T, NCOLS, TSUB>;
+        auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2>;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
         if (e != cudaSuccess) return e;
         kernel<<<grid, kThreads, p.smem, stream>>>(kmap, qmap, a, p.q_resident, p.gs);
@@ -535,14 +552,14 @@ cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const S
     }
 }
 
-template <typename T, int NCOLS>
+template <typename T, int NCOLS, bool PACK2 = false>
 cudaError_t launch_tsub(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a, const Plan &p,
                         int grid, cudaStream_t stream)
 {
     switch (p.tsub) {
-    case 4: return launch_one<T, NCOLS, 4>(kmap, qmap, a, p, grid, stream);
-    case 2: return launch_one<T, NCOLS, 2>(kmap, qmap, a, p, grid, stream);
-    default: return launch_one<T, NCOLS, 1>(kmap, qmap, a, p, grid, stream);
+    case 4: return launch_one<T, NCOLS, 4, PACK2>(kmap, qmap, a, p, grid, stream);
+    case 2: return launch_one<T, NCOLS, 2, PACK2>(kmap, qmap, a, p, grid, stream);
+    default: return launch_one<T, NCOLS, 1, PACK2>(kmap, qmap, a, p, grid, stream);
     }
 }
 
@@ -562,11 +579,13 @@ cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, c
         return launch_scan_ummat(kmap, qmap, a_in, grid, stream);
     ScanArgs a = a_in;
     if (a.tile_stride < 1) a.tile_stride = 1;
-    const Plan p = make_plan(a.d, a.B);
+    const bool h = a.dtype == kF16, q8 = a.dtype == kE4M3;
+    const bool pack2 = q8 && a.pack2;
+    const Plan p = make_plan(a.d, pack2 ? 2 * a.B : a.B);        // two operand-row pairs per query when packed
     if (p.stages < 2) return cudaErrorInvalidValue;
     a.stages = p.stages;
-    const bool h = a.dtype == kF16, q8 = a.dtype == kE4M3;
 #define DRESD_GO(N_)                                                                          \
+    if (pack2) return launch_tsub<E4M3Keys, N_, true>(kmap, qmap, a, p, grid, stream);        \
     return q8 ? launch_tsub<E4M3Keys, N_>(kmap, qmap, a, p, grid, stream)                     \
            : h ? launch_tsub<__half, N_>(kmap, qmap, a, p, grid, stream)                      \
                : launch_tsub<__nv_bfloat16, N_>(kmap, qmap, a, p, grid, stream)

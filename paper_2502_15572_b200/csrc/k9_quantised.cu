@@ -77,11 +77,32 @@ __global__ void __launch_bounds__(256) quantise_keys_kernel(const T *__restrict_
 }
 
 // One CTA per operand query: rows 2b (h1) and 2b+1 (h2) of the 8-bit operand, zero-padded to
-// dpad8 bytes; queries past B are zero rows.
+// dpad8 bytes; queries past B are zero rows.  pack2 (d = 64, dpad8 = 128: two keys per store
+// row): rows 4b .. 4b+3 = (h1|0), (h2|0), (0|h1), (0|h2).
 __global__ void split_queries_e4m3_kernel(const float *__restrict__ qhat, int B, int d, uint8_t *__restrict__ qsplit8,
-                                          int dpad8)
+                                          int dpad8, int pack2)
 {
     const int b = blockIdx.x;
+    if (pack2) {
+        uint8_t *r0 = qsplit8 + (size_t)(4 * b) * dpad8;
+        for (int j = threadIdx.x; j < 64; j += blockDim.x) {
+            uint32_t c1 = 0u, c2 = 0u;
+            if (b < B) {
+                const float q256 = 256.f * qhat[(size_t)b * d + j];
+                c1 = to_e4m3(q256);
+                c2 = to_e4m3(16.f * (q256 - from_e4m3(c1)));
+            }
+            r0[j] = (uint8_t)c1;
+            r0[64 + j] = 0;
+            r0[dpad8 + j] = (uint8_t)c2;
+            r0[dpad8 + 64 + j] = 0;
+            r0[2 * dpad8 + j] = 0;
+            r0[2 * dpad8 + 64 + j] = (uint8_t)c1;
+            r0[3 * dpad8 + j] = 0;
+            r0[3 * dpad8 + 64 + j] = (uint8_t)c2;
+        }
+        return;
+    }
     uint8_t *h1 = qsplit8 + (size_t)(2 * b) * dpad8, *h2 = h1 + dpad8;
     for (int j = threadIdx.x; j < dpad8; j += blockDim.x) {
         uint32_t c1 = 0u, c2 = 0u;
@@ -102,16 +123,18 @@ __global__ void split_queries_e4m3_kernel(const float *__restrict__ qhat, int B,
 template <typename T>
 __global__ void __launch_bounds__(256) rerank_kernel(const T *__restrict__ keys, int d, long long N,
                                                      const float *__restrict__ qhat, const int32_t *__restrict__ cand,
-                                                     int m, int top_n, const int32_t *__restrict__ next_tokens,
+                                                     int m, int top_n, long long extra_id,
+                                                     const int32_t *__restrict__ next_tokens,
                                                      int stored_len, int draft_len, int32_t *__restrict__ out_ids,
                                                      float *__restrict__ out_scores, int32_t *__restrict__ out_tokens)
 {
-    __shared__ unsigned long long packed[kListLen];
+    __shared__ unsigned long long packed[kListLen + 1];
     __shared__ int win[kListLen];
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const float *q = qhat + (size_t)b * d;
-    for (int r = warp; r < kListLen; r += 8) {
-        const long long id = r < m ? cand[(size_t)b * m + r] : -1;
+    // slot kListLen: one extra candidate (the last key of an odd-sized packed store), never a duplicate
+    for (int r = warp; r <= kListLen; r += 8) {
+        const long long id = r < m ? cand[(size_t)b * m + r] : r == kListLen ? extra_id : -1;
         unsigned long long p = 0ull;
         if (id >= 0 && id < N) {                             // warp-uniform
             const uint4 *row = reinterpret_cast<const uint4 *>(keys + (size_t)id * d);
@@ -133,7 +156,8 @@ __global__ void __launch_bounds__(256) rerank_kernel(const T *__restrict__ keys,
     }
     __syncthreads();
     if (warp == 0) {
-        const unsigned long long x = warp_sort_desc(packed[lane], lane);
+        unsigned long long x = warp_sort_desc(packed[lane], lane);
+        x = warp_merge_top32(x, lane == 0 ? packed[kListLen] : 0ull, lane);      // a sorted list of one
         if (lane < top_n) {
             const int id = x ? (int32_t)candidate_id(x) : -1;
             out_ids[(size_t)b * top_n + lane] = id;
@@ -169,23 +193,24 @@ cudaError_t launch_quantise_keys(const void *keys, int dtype, long long N, int d
 }
 
 cudaError_t launch_split_queries_e4m3(const float *qhat, int B, int rows, int d, void *qsplit8, int dpad8,
-                                      cudaStream_t stream)
+                                      int pack2, cudaStream_t stream)
 {
-    split_queries_e4m3_kernel<<<rows, 256, 0, stream>>>(qhat, B, d, static_cast<uint8_t *>(qsplit8), dpad8);
+    split_queries_e4m3_kernel<<<rows, 256, 0, stream>>>(qhat, B, d, static_cast<uint8_t *>(qsplit8), dpad8, pack2);
     return cudaGetLastError();
 }
 
 cudaError_t launch_rerank(const void *keys, int dtype, int d, long long N, const float *qhat, const int32_t *cand,
-                          int B, int m, int top_n, const int32_t *next_tokens, int stored_len, int draft_len,
-                          int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream)
+                          int B, int m, int top_n, long long extra_id, const int32_t *next_tokens, int stored_len,
+                          int draft_len, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
+                          cudaStream_t stream)
 {
     if (dtype == kF16)
         rerank_kernel<__half><<<B, 256, 0, stream>>>(static_cast<const __half *>(keys), d, N, qhat, cand, m, top_n,
-                                                      next_tokens, stored_len, draft_len, out_ids, out_scores,
+                                                      extra_id, next_tokens, stored_len, draft_len, out_ids, out_scores,
                                                       out_tokens);
     else
         rerank_kernel<__nv_bfloat16><<<B, 256, 0, stream>>>(static_cast<const __nv_bfloat16 *>(keys), d, N, qhat,
-                                                            cand, m, top_n, next_tokens, stored_len, draft_len,
+                                                            cand, m, top_n, extra_id, next_tokens, stored_len, draft_len,
                                                             out_ids, out_scores, out_tokens);
     return cudaGetLastError();
 }

@@ -162,3 +162,55 @@ def test_quantised_argument_errors():
             binding.dresd_store_attach_quantised(s32.handle, torch.zeros(300 * 64, dtype=torch.uint8, device="cuda").data_ptr())
     finally:
         s32.close()
+
+
+# d = 64: the 8-bit copy is scanned as rows of two keys (one 128-byte line).  Odd and even N
+# (the last key of an odd store is handed to the re-ranking as an extra candidate), batch
+# sizes on both sides of the 32-query limit of the packed form, and the unpacked form.
+@pytest.mark.parametrize("pack2", [1, 0], ids=["two_keys_per_row", "one_key_per_row"])
+@pytest.mark.parametrize("dtype,B,n,L,m,N", [
+    ("f16", 1, 10, 4, 32, 148 * 512 * 2 + 37),
+    ("bf16", 16, 5, 3, 20, 50022),
+    ("f16", 32, 4, 2, 16, 40009),
+    ("bf16", 33, 4, 2, 16, 30011),             # more than 32 queries: one key per row in both runs
+    ("f16", 3, 3, 2, 3, 7),                    # three packed rows and an odd key
+    ("bf16", 2, 1, 1, 1, 2),                   # a single packed row
+])
+def test_quantised_retrieval_d64_packed_rows(pack2, dtype, B, n, L, m, N):
+    import torch
+    d = 64
+    keys, toks = synth.make_store(8500 + B, N, d, 8, dtype, L + 1)
+    q, _ = synth.make_queries(8550 + B, keys, dtype, B, 0.1)
+    n, m = min(n, N), min(m, N)
+    st = gpu_store(keys, toks, dtype)
+    try:
+        st.attach_quantised()
+        outs = []
+        for p in (pack2, 1 - pack2):
+            st.set_option("pack2", p)
+            o = st.retrieve_quantised(binding.to_device(q, dtype), n, L, m)
+            torch.cuda.synchronize()
+            st.status()
+            outs.append([t.cpu().numpy() for t in o])
+    finally:
+        st.close()
+    # the two forms visit the same keys with the same arithmetic: identical results
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(a, b)
+    # and against the oracle (the first form)
+    ids, sc, tok = outs[0]
+    _, _, _, approx, exact = oracle.retrieve_quantised(keys, toks, dtype, q, n, L, m,
+                                                       threads=oracle.dresd_oracle.default_threads())
+    for b in range(B):
+        cut = np.sort(approx[b])[-m]
+        got = ids[b]
+        assert len(set(got.tolist())) == n and np.all(got >= 0) and np.all(got < N)
+        # the last key of an odd packed store is always re-ranked, whatever its approximate score
+        extra = N - 1 if (N % 2 == 1 and B <= 32) else -1
+        assert np.all((approx[b][got] >= cut - DELTA) | (got == extra))
+        np.testing.assert_allclose(sc[b], exact[b][got], rtol=0, atol=SCORE_TOL)
+        assert np.all(np.diff(exact[b][got]) <= 2 * EPS_ACC)
+        safe = np.flatnonzero(approx[b] >= cut + DELTA)
+        nth = exact[b][got[-1]]
+        assert not [i for i in safe if exact[b][i] > nth + 2 * EPS_ACC and i not in set(got.tolist())]
+        assert np.array_equal(tok[b], toks[got, :L])
