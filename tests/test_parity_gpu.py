@@ -391,3 +391,40 @@ def test_retrieve_can_be_captured_in_a_cuda_graph_and_replayed():
             assert np.array_equal(tok.cpu().numpy(), want[2])
     finally:
         st.close()
+
+
+@pytest.mark.parametrize("dtype,d,B", [("f16", 256, 2), ("bf16", 256, 40), ("f32", 128, 3), ("f16", 64, 1)])
+def test_non_finite_inputs_neither_hang_nor_fault(dtype, d, B):
+    """NaN keys never enter a result (a comparison with NaN is false); the other rows are ranked
+    as if the NaN rows scored nothing; a NaN query selects nothing at all.  The calls return, the
+    health word stays clean and the store remains usable."""
+    import torch
+    N, n, L = 30011, 10, 3
+    keys, toks = synth.make_store(7700 + d, N, d, 16, dtype, L)
+    q, _ = synth.make_queries(7701 + d, keys, dtype, B, 0.1)
+    bad = np.array([0, 5, 777, 12345, N - 1])
+    poisoned = keys.copy()
+    nan_bits = {"f16": np.float16(np.nan), "f32": np.float32(np.nan)}.get(dtype)
+    if dtype == "bf16":
+        poisoned[bad, 3] = np.uint16(0x7FC0)
+    else:
+        poisoned[bad, 3] = nan_bits
+    zeroed = keys.copy()
+    zeroed[bad] = 0                                     # a zero row scores 0, far below the neighbours
+    st = gpu_store(poisoned, toks, dtype)
+    try:
+        ids, sc, tok = gpu_retrieve(st, q, n, L)
+        assert not np.isin(ids, bad).any() and np.all(ids >= 0) and np.all(np.isfinite(sc))
+        o = oracle.retrieve(zeroed, toks, dtype, q, n, L, want_full_scores=True)
+        checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids)
+        qn = q.copy()
+        if dtype == "bf16":
+            qn[:, 0] = np.uint16(0x7FC0)
+        else:
+            qn[:, 0] = nan_bits
+        ids2, sc2, tok2 = gpu_retrieve(st, qn, n, L)    # gpu_retrieve checks the health word
+        assert np.all(ids2 == -1) and np.all(sc2 == -np.inf) and np.all(tok2 == -1)
+        ids3, _, _ = gpu_retrieve(st, q, n, L)          # and the store still answers
+        assert np.array_equal(ids3, ids)
+    finally:
+        st.close()
