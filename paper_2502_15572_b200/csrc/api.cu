@@ -187,8 +187,9 @@ dresd_status check_retrieve_args(const dresd_store *s, const void *queries, int 
 }
 
 // K1 for B queries into the store's workspace.
+// quantised: 0 = no, 1 = also write the 8-bit query terms, 2 = in the packed (two keys per row) layout
 dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows, cudaStream_t stream,
-                            int split_blocked = 0)
+                            int split_blocked = 0, int quantised = 0)
 {
     PreprocessArgs p{};
     p.queries = queries;
@@ -209,6 +210,11 @@ dresd_status run_preprocess(dresd_store *s, const void *queries, int B, int rows
     p.lo_scale = s->dtype == kF16 ? kHiLoScaleF16 : kHiLoScaleBF16;
     p.gtau = s->gtau;
     p.split_blocked = split_blocked;
+    if (quantised) {
+        p.qsplit8 = static_cast<uint8_t *>(s->qsplit8);
+        p.dpad8 = s->dpad8;
+        p.pack2 = quantised == 2;
+    }
     if (s->W && s->proj_ws && reinterpret_cast<uintptr_t>(s->W) % 16 == 0) {     // 16-byte loads of W rows
         preprocess_split_plan(s->d_in, s->d, B, (int)elem_bytes(s->dtype), s->proj_ws_bytes, &p.slices, &p.rows_per_slice);
         if (p.slices > 0) p.partial = s->proj_ws;
@@ -240,15 +246,11 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     const int op_rows = umma ? scan_umma_operand_rows(pack2 ? 2 * B : B) : 0;
     // the kernel with the keys as the N operand reads hi and lo of a query from one TMEM fragment
     const int blocked = umma && !q8 && !s->opt_keys_as_m && scan_ummat_eligible(s->d, B);
-    dresd_status st = run_preprocess(s, queries, B, umma ? op_rows / 2 : ((B + 7) / 8) * 8, stream, blocked);
+    // one CTA per operand query: two operand rows each, four in the packed 8-bit layout
+    const int pre_rows = pack2 ? op_rows / 4 : umma ? op_rows / 2 : ((B + 7) / 8) * 8;
+    dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, blocked, pack2 ? 2 : q8 ? 1 : 0);
     if (st != DRESD_OK) return st;
 
-    if (q8) {
-        cudaError_t e8 = launch_split_queries_e4m3(s->qhat, B, pack2 ? op_rows / 4 : op_rows / 2, s->d, s->qsplit8,
-                                                   s->dpad8, pack2 ? 1 : 0, stream);
-        if (e8 != cudaSuccess) return fail_cuda(e8, "query split launch");
-        s->last_launches += 1;
-    }
     // the 8-bit store is scanned as rows of d/2 two-byte units (packed: N/2 rows of 64 units)
     const int scan_d = pack2 ? 64 : q8 ? s->d / 2 : s->d;
     const long long scan_rows = pack2 ? s->N / 2 : s->N;
@@ -340,15 +342,12 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         s->prof_count += 1;
     }
     if (q8) {
-        // the m candidates of every query (approximate scores are not returned), then the exact pass
-        cudaError_t e = launch_merge_gather(s->cand, grid, B, quantised_m, s->ids_dev, s->scores_dev, nullptr, 0, s->N, 0,
-                                            nullptr, stream);
-        if (e == cudaSuccess)
-            e = launch_rerank(s->keys, s->dtype, s->d, s->N, s->qhat, s->ids_dev, B, quantised_m, top_n,
-                              pack2 && (s->N & 1) ? s->N - 1 : -1, s->next_tokens, s->stored_len, draft_len, out_ids,
-                              out_scores, out_tokens, stream);
+        // fold the approximate lists, score the m survivors exactly, sort, gather: one launch
+        cudaError_t e = launch_merge_rerank(s->cand, grid, B, s->keys, s->dtype, s->d, s->N, s->qhat, quantised_m, top_n,
+                                            pack2 && (s->N & 1) ? s->N - 1 : -1, s->next_tokens, s->stored_len,
+                                            draft_len, out_ids, out_scores, out_tokens, stream);
         if (e != cudaSuccess) return fail_cuda(e, "merge / re-rank launch");
-        s->last_launches += 2;
+        s->last_launches += 1;
         return DRESD_OK;
     }
     cudaError_t e = launch_merge_gather(s->cand, grid, B, top_n, out_ids, out_scores, s->next_tokens, s->stored_len,

@@ -11,6 +11,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -289,6 +290,42 @@ __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// E4M3 conversions (round to nearest even, saturating at +-448) and the two-term 8-bit query:
+// h1 = e4m3(256 q), h2 = e4m3(16 (256 q - h1)).  Rows 2b / 2b+1 of the operand hold h1 / h2 of
+// query b; in the packed form (two 64-byte keys per 128-byte store row) rows 4b .. 4b+3 hold
+// (h1|0), (h2|0), (0|h1), (0|h2).
+__device__ __forceinline__ uint32_t to_e4m3(float x)
+{
+    return (uint32_t)__nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3);
+}
+__device__ __forceinline__ float from_e4m3(uint32_t c)
+{
+    const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)c, __NV_E4M3);
+    return __half2float(*reinterpret_cast<const __half *>(&h));
+}
+__device__ __forceinline__ void store_query_e4m3(uint8_t *qsplit8, int dpad8, int pack2, int b, int c, float q)
+{
+    const float q256 = 256.f * q;
+    const uint32_t c1 = to_e4m3(q256);
+    const uint32_t c2 = to_e4m3(16.f * (q256 - from_e4m3(c1)));
+    if (pack2) {
+        if (c >= 64) return;
+        uint8_t *r0 = qsplit8 + (size_t)(4 * b) * dpad8;
+        r0[c] = (uint8_t)c1;
+        r0[64 + c] = 0;
+        r0[dpad8 + c] = (uint8_t)c2;
+        r0[dpad8 + 64 + c] = 0;
+        r0[2 * dpad8 + c] = 0;
+        r0[2 * dpad8 + 64 + c] = (uint8_t)c1;
+        r0[3 * dpad8 + c] = 0;
+        r0[3 * dpad8 + 64 + c] = (uint8_t)c2;
+    } else {
+        uint8_t *h1 = qsplit8 + (size_t)(2 * b) * dpad8;
+        h1[c] = (uint8_t)c1;
+        h1[dpad8 + c] = (uint8_t)c2;
+    }
+}
+
 // Element-type tag of the 8-bit copy of a datastore: the scan kernels see such a store as rows
 // of d/2 two-byte units (TMA moves bytes) and only switch the instruction kind.
 struct E4M3Keys {};

@@ -35,6 +35,9 @@ struct PreprocessArgs {
     // partial[slice][B][d]; null = every query's CTA walks all of W itself.
     float *partial;
     int slices, rows_per_slice;
+    // Quantised search: also write the two E4M3 terms of every query (see store_query_e4m3); null = not needed.
+    uint8_t *qsplit8;
+    int dpad8, pack2;
 };
 // Slices and rows per slice of the split projection for a workspace of `bytes` (0 slices = do not split).
 void preprocess_split_plan(int d_in, int d, int B, int elem_bytes, size_t bytes, int *slices, int *rows_per_slice);
@@ -140,15 +143,12 @@ cudaError_t launch_fit_zscore(const void *V, int dtype, long long N, int d_in, i
 // ---- K9: quantised candidate search (8-bit E4M3 keys, exact re-ranking) ----
 cudaError_t launch_quantise_keys(const void *keys, int dtype, long long N, int d, void *out_q8, int sms,
                                  cudaStream_t stream);
-// qsplit8: [2 * rows][dpad8] bytes, rows 2b / 2b+1 = the two 8-bit terms of query b
-// pack2: four rows per query, (h1|0), (h2|0), (0|h1), (0|h2), for two 64-byte keys per 128-byte row
-cudaError_t launch_split_queries_e4m3(const float *qhat, int B, int rows, int d, void *qsplit8, int dpad8,
-                                      int pack2, cudaStream_t stream);
-// extra_id >= 0: one more candidate for every query (the last key of an odd-sized packed store)
-cudaError_t launch_rerank(const void *keys, int dtype, int d, long long N, const float *qhat, const int32_t *cand,
-                          int B, int m, int top_n, long long extra_id, const int32_t *next_tokens, int stored_len,
-                          int draft_len, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
-                          cudaStream_t stream);
+// Fold of the per-CTA approximate lists, exact re-ranking of the survivors, value lookup: one kernel.
+// extra_id >= 0: one more candidate for every query (the last key of an odd-sized packed store).
+cudaError_t launch_merge_rerank(const unsigned long long *cand, int lists, int B, const void *keys, int dtype, int d,
+                                long long N, const float *qhat, int mcand, int top_n, long long extra_id,
+                                const int32_t *next_tokens, int stored_len, int draft_len, int32_t *out_ids,
+                                float *out_scores, int32_t *out_tokens, cudaStream_t stream);
 
 // Stores `msg` as the calling thread's dresd_last_error() text.
 void set_last_error(const char *msg);

@@ -190,6 +190,8 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
                 split_hi[c] = from_f32<T>(0.f);
                 split_lo[c] = from_f32<T>(0.f);
             }
+        if (a.qsplit8)
+            for (int c = tid; c < a.dpad8; c += blockDim.x) store_query_e4m3(a.qsplit8, a.dpad8, a.pack2, b, c, 0.f);
         return;
     }
 
@@ -276,6 +278,9 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
             split_lo[c] = from_f32<T>(r);
         }
     }
+    if (a.qsplit8)                                       // the two 8-bit terms of the quantised search
+        for (int c = tid; c < a.dpad8; c += blockDim.x)
+            store_query_e4m3(a.qsplit8, a.dpad8, a.pack2, b, c, c < a.d ? vl[c] / den : 0.f);
 }
 
 }  // namespace

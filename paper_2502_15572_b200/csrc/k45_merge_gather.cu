@@ -61,7 +61,6 @@ merge_gather_kernel(const unsigned long long *__restrict__ cand, int lists, int 
         out_scores[(size_t)b * top_n + lane] = m ? candidate_score(m) : -INFINITY;
         win[lane] = id;
     }
-    if (!next_tokens) return;             // candidates only (the quantised search re-ranks them itself)
     __syncthreads();
     // K5: the first draft_len stored tokens of every winner (Section 3.5, f_D: k -> v)
     const int total = top_n * draft_len;

@@ -12,8 +12,9 @@
 // E4M3: 1 sign, 4 exponent bits (bias 7), 3 mantissa bits, largest finite value 448, no
 // infinities; conversions round to nearest even and saturate.
 //
-// This file holds the three small kernels around the scan: the key quantiser (HBM-bound, run
-// once per datastore), the query splitter, and the exact re-ranking with the value lookup.
+// This file holds the kernels around the scan: the key quantiser (HBM-bound, run once per
+// datastore) and the exact re-ranking with the value lookup; the query terms are written by
+// the preprocessing kernel.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
@@ -23,16 +24,6 @@
 
 namespace dresd {
 namespace {
-
-__device__ __forceinline__ uint32_t to_e4m3(float x)
-{
-    return (uint32_t)__nv_cvt_float_to_fp8(x, __NV_SATFINITE, __NV_E4M3);
-}
-__device__ __forceinline__ float from_e4m3(uint32_t c)
-{
-    const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)c, __NV_E4M3);
-    return __half2float(*reinterpret_cast<const __half *>(&h));
-}
 
 template <typename T> __device__ __forceinline__ void unpack16(const uint4 &v, float *x);
 template <> __device__ __forceinline__ void unpack16<__half>(const uint4 &v, float *x)
@@ -76,74 +67,64 @@ __global__ void __launch_bounds__(256) quantise_keys_kernel(const T *__restrict_
     }
 }
 
-// One CTA per operand query: rows 2b (h1) and 2b+1 (h2) of the 8-bit operand, zero-padded to
-// dpad8 bytes; queries past B are zero rows.  pack2 (d = 64, dpad8 = 128: two keys per store
-// row): rows 4b .. 4b+3 = (h1|0), (h2|0), (0|h1), (0|h2).
-__global__ void split_queries_e4m3_kernel(const float *__restrict__ qhat, int B, int d, uint8_t *__restrict__ qsplit8,
-                                          int dpad8, int pack2)
-{
-    const int b = blockIdx.x;
-    if (pack2) {
-        uint8_t *r0 = qsplit8 + (size_t)(4 * b) * dpad8;
-        for (int j = threadIdx.x; j < 64; j += blockDim.x) {
-            uint32_t c1 = 0u, c2 = 0u;
-            if (b < B) {
-                const float q256 = 256.f * qhat[(size_t)b * d + j];
-                c1 = to_e4m3(q256);
-                c2 = to_e4m3(16.f * (q256 - from_e4m3(c1)));
-            }
-            r0[j] = (uint8_t)c1;
-            r0[64 + j] = 0;
-            r0[dpad8 + j] = (uint8_t)c2;
-            r0[dpad8 + 64 + j] = 0;
-            r0[2 * dpad8 + j] = 0;
-            r0[2 * dpad8 + 64 + j] = (uint8_t)c1;
-            r0[3 * dpad8 + j] = 0;
-            r0[3 * dpad8 + 64 + j] = (uint8_t)c2;
-        }
-        return;
-    }
-    uint8_t *h1 = qsplit8 + (size_t)(2 * b) * dpad8, *h2 = h1 + dpad8;
-    for (int j = threadIdx.x; j < dpad8; j += blockDim.x) {
-        uint32_t c1 = 0u, c2 = 0u;
-        if (b < B && j < d) {
-            const float q256 = 256.f * qhat[(size_t)b * d + j];
-            c1 = to_e4m3(q256);
-            c2 = to_e4m3(16.f * (q256 - from_e4m3(c1)));
-        }
-        h1[j] = (uint8_t)c1;
-        h2[j] = (uint8_t)c2;
-    }
-}
+// Grid merge of the approximate lists + exact re-ranking + value lookup, one CTA (16 warps) per
+// query.  The per-CTA lists (sorted by approximate score, m entries each) are folded as in the
+// exact path; the m survivors are then scored exactly, a warp per candidate: s = sum_j q_j k_ij
+// in fp32 (the 16-bit key element converts exactly; four partial sums per lane, fixed reduction
+// order); the candidates are sorted by (score descending, row ascending), the n best written
+// out and their stored tokens copied (Section 3.5, f_D: k -> v).  extra_id >= 0 is one more
+// candidate for every query (the last key of an odd-sized packed store).
+constexpr int kRerankWarps = 16;
 
-// Exact re-ranking: one CTA per query, a warp per candidate.  s = sum_j q_j k_ij in fp32 (the
-// 16-bit key element converts exactly; four partial sums per lane, fixed reduction order),
-// then the m candidates are sorted by (score descending, row ascending), the n best written
-// out and their stored tokens copied (Section 3.5, f_D: k -> v).
 template <typename T>
-__global__ void __launch_bounds__(256) rerank_kernel(const T *__restrict__ keys, int d, long long N,
-                                                     const float *__restrict__ qhat, const int32_t *__restrict__ cand,
-                                                     int m, int top_n, long long extra_id,
-                                                     const int32_t *__restrict__ next_tokens,
-                                                     int stored_len, int draft_len, int32_t *__restrict__ out_ids,
-                                                     float *__restrict__ out_scores, int32_t *__restrict__ out_tokens)
+__global__ void __launch_bounds__(kRerankWarps * 32)
+merge_rerank_kernel(const unsigned long long *__restrict__ cand, int lists, int B, const T *__restrict__ keys, int d,
+                    long long N, const float *__restrict__ qhat, int mcand, int top_n, long long extra_id,
+                    const int32_t *__restrict__ next_tokens, int stored_len, int draft_len,
+                    int32_t *__restrict__ out_ids, float *__restrict__ out_scores, int32_t *__restrict__ out_tokens)
 {
+    __shared__ unsigned long long part[kRerankWarps][kListLen];
     __shared__ unsigned long long packed[kListLen + 1];
     __shared__ int win[kListLen];
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    unsigned long long m = 0ull;
+    int g = warp;
+    for (; g + 3 * kRerankWarps < lists; g += 4 * kRerankWarps) {
+        unsigned long long l0 = cand[((size_t)(g + 0 * kRerankWarps) * B + b) * kCandStride + lane];
+        unsigned long long l1 = cand[((size_t)(g + 1 * kRerankWarps) * B + b) * kCandStride + lane];
+        unsigned long long l2 = cand[((size_t)(g + 2 * kRerankWarps) * B + b) * kCandStride + lane];
+        unsigned long long l3 = cand[((size_t)(g + 3 * kRerankWarps) * B + b) * kCandStride + lane];
+        m = warp_merge_top32(m, l0, lane);
+        m = warp_merge_top32(m, l1, lane);
+        m = warp_merge_top32(m, l2, lane);
+        m = warp_merge_top32(m, l3, lane);
+    }
+    for (; g < lists; g += kRerankWarps)
+        m = warp_merge_top32(m, cand[((size_t)g * B + b) * kCandStride + lane], lane);
+    part[warp][lane] = m;
+    __syncthreads();
+    for (int span = kRerankWarps / 2; span >= 1; span >>= 1) {
+        if (warp < span) {
+            m = warp_merge_top32(part[warp][lane], part[warp + span][lane], lane);
+            part[warp][lane] = m;
+        }
+        __syncthreads();
+    }
+    // part[0]: the best approximate scores with their rows; the first mcand of them are the candidates
     const float *q = qhat + (size_t)b * d;
-    // slot kListLen: one extra candidate (the last key of an odd-sized packed store), never a duplicate
-    for (int r = warp; r <= kListLen; r += 8) {
-        const long long id = r < m ? cand[(size_t)b * m + r] : r == kListLen ? extra_id : -1;
+    for (int r = warp; r <= kListLen; r += kRerankWarps) {
+        const unsigned long long c = r < mcand ? part[0][r] : 0ull;       // exactly the m best, as defined
+        const long long id = r < kListLen ? (c ? (long long)candidate_id(c) : -1) : extra_id;
         unsigned long long p = 0ull;
         if (id >= 0 && id < N) {                             // warp-uniform
             const uint4 *row = reinterpret_cast<const uint4 *>(keys + (size_t)id * d);
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-            for (int c = lane; c < d / 8; c += 32) {          // d is a multiple of 16
+            for (int cc = lane; cc < d / 8; cc += 32) {       // d is a multiple of 16
                 float x[8];
-                unpack16<T>(__ldg(row + c), x);
-                const float4 q0 = *reinterpret_cast<const float4 *>(q + 8 * c);
-                const float4 q1 = *reinterpret_cast<const float4 *>(q + 8 * c + 4);
+                unpack16<T>(__ldg(row + cc), x);
+                const float4 q0 = *reinterpret_cast<const float4 *>(q + 8 * cc);
+                const float4 q1 = *reinterpret_cast<const float4 *>(q + 8 * cc + 4);
                 a0 = fmaf(q0.x, x[0], a0); a1 = fmaf(q0.y, x[1], a1); a2 = fmaf(q0.z, x[2], a2); a3 = fmaf(q0.w, x[3], a3);
                 a0 = fmaf(q1.x, x[4], a0); a1 = fmaf(q1.y, x[5], a1); a2 = fmaf(q1.z, x[6], a2); a3 = fmaf(q1.w, x[7], a3);
             }
@@ -192,26 +173,19 @@ cudaError_t launch_quantise_keys(const void *keys, int dtype, long long N, int d
     return cudaGetLastError();
 }
 
-cudaError_t launch_split_queries_e4m3(const float *qhat, int B, int rows, int d, void *qsplit8, int dpad8,
-                                      int pack2, cudaStream_t stream)
-{
-    split_queries_e4m3_kernel<<<rows, 256, 0, stream>>>(qhat, B, d, static_cast<uint8_t *>(qsplit8), dpad8, pack2);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_rerank(const void *keys, int dtype, int d, long long N, const float *qhat, const int32_t *cand,
-                          int B, int m, int top_n, long long extra_id, const int32_t *next_tokens, int stored_len,
-                          int draft_len, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
-                          cudaStream_t stream)
+cudaError_t launch_merge_rerank(const unsigned long long *cand, int lists, int B, const void *keys, int dtype, int d,
+                                long long N, const float *qhat, int mcand, int top_n, long long extra_id,
+                                const int32_t *next_tokens, int stored_len, int draft_len, int32_t *out_ids,
+                                float *out_scores, int32_t *out_tokens, cudaStream_t stream)
 {
     if (dtype == kF16)
-        rerank_kernel<__half><<<B, 256, 0, stream>>>(static_cast<const __half *>(keys), d, N, qhat, cand, m, top_n,
-                                                      extra_id, next_tokens, stored_len, draft_len, out_ids, out_scores,
-                                                      out_tokens);
+        merge_rerank_kernel<__half><<<B, kRerankWarps * 32, 0, stream>>>(
+            cand, lists, B, static_cast<const __half *>(keys), d, N, qhat, mcand, top_n, extra_id, next_tokens, stored_len,
+            draft_len, out_ids, out_scores, out_tokens);
     else
-        rerank_kernel<__nv_bfloat16><<<B, 256, 0, stream>>>(static_cast<const __nv_bfloat16 *>(keys), d, N, qhat,
-                                                            cand, m, top_n, extra_id, next_tokens, stored_len, draft_len,
-                                                            out_ids, out_scores, out_tokens);
+        merge_rerank_kernel<__nv_bfloat16><<<B, kRerankWarps * 32, 0, stream>>>(
+            cand, lists, B, static_cast<const __nv_bfloat16 *>(keys), d, N, qhat, mcand, top_n, extra_id, next_tokens,
+            stored_len, draft_len, out_ids, out_scores, out_tokens);
     return cudaGetLastError();
 }
 
