@@ -229,14 +229,17 @@ dresd_status dresd_fit_zscore(const void *sample, int64_t N, int d_in, dresd_dty
  *                           [N][d] bytes; both 16-byte aligned.  Asynchronous on `stream`.
  * dresd_store_attach_quantised   the 8-bit copy of the store's keys (borrowed until destroy);
  *                           a set-up call, may allocate.  16-bit stores with d <= 2048.
- * dresd_retrieve_quantised  as dresd_retrieve() plus `candidates` in top_n .. DRESD_MAX_TOP_N.
+ * dresd_retrieve_quantised  as dresd_retrieve_filtered() plus `candidates` in top_n .. DRESD_MAX_TOP_N:
+ *                           first_tokens NULL (or -1 per query) = no first-token filter; with it only
+ *                           keys whose first stored token matches are candidates (Section 3.5), and
+ *                           missing neighbours are id -1, score -inf, tokens -1.
  *                           Asynchronous on `stream`; no allocation.
  */
 dresd_status dresd_quantise_keys(const void *keys, int64_t N, int d, dresd_dtype dtype, void *out_q8, void *stream);
 dresd_status dresd_store_attach_quantised(dresd_store *store, const void *keys_q8);
-dresd_status dresd_retrieve_quantised(dresd_store *store, const void *queries, int B, int top_n, int draft_len,
-                                      int candidates, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
-                                      void *stream);
+dresd_status dresd_retrieve_quantised(dresd_store *store, const void *queries, const int32_t *first_tokens, int B,
+                                      int top_n, int draft_len, int candidates, int32_t *out_ids, float *out_scores,
+                                      int32_t *out_tokens, void *stream);
 
 /*
  * Process-wide switches (not part of the paper; for measurement and tests).

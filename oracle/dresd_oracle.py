@@ -255,7 +255,8 @@ def quantised_scores(keys, dtype: str, qhat, threads: int = 1) -> np.ndarray:
 
 
 def retrieve_quantised(keys, next_tokens, dtype: str, queries, top_n: int, draft_len: int, candidates: int,
-                       mean=None, var=None, eps_z: float = 1e-5, W=None, pca_mean=None, threads: int = 1):
+                       mean=None, var=None, eps_z: float = 1e-5, W=None, pca_mean=None, threads: int = 1,
+                       first_token=None):
     """Candidates by approximate (8-bit) score, exact re-ranking, value lookup.
 
     For each query: the `candidates` rows with the largest approximate score (ties to the
@@ -277,9 +278,14 @@ def retrieve_quantised(keys, next_tokens, dtype: str, queries, top_n: int, draft
     for b in range(B):
         approx[b] = quantised_scores(keys, dtype, qhat[b], threads)
         exact[b] = scores(keys, dtype, qhat[b], threads)
-        cand = np.lexsort((rows, -approx[b]))[:candidates]          # approx descending, row ascending
+        pool = rows
+        if first_token is not None and int(first_token[b]) >= 0:
+            pool = rows[toks[:, 0] == int(first_token[b])]
+        cand = pool[np.lexsort((pool, -approx[b][pool]))][:candidates]   # approx descending, row ascending
         order = cand[np.lexsort((cand, -exact[b][cand]))][:top_n]    # exact descending, row ascending
-        ids[b] = order
-        sc[b] = exact[b][order]
-        tok[b] = toks[order, :draft_len]
+        k = len(order)
+        ids[b], sc[b], tok[b] = -1, -np.inf, -1
+        ids[b, :k] = order
+        sc[b, :k] = exact[b][order]
+        tok[b, :k] = toks[order, :draft_len]
     return ids, sc, tok, approx, exact

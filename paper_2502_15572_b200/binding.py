@@ -97,7 +97,7 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_store_attach_quantised.restype = i32
     lib.dresd_store_attach_quantised.argtypes = [vp, vp]
     lib.dresd_retrieve_quantised.restype = i32
-    lib.dresd_retrieve_quantised.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.dresd_retrieve_quantised.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_set_global_option.restype = i32
     lib.dresd_set_global_option.argtypes = [ctypes.c_char_p, i32]
     lib.dresd_fit_zscore.restype = i32
@@ -180,10 +180,11 @@ def dresd_store_attach_quantised(store: int, keys_q8_ptr: int) -> None:
     _check(load().dresd_store_attach_quantised(store, keys_q8_ptr))
 
 
-def dresd_retrieve_quantised(store: int, queries_ptr: int, B: int, top_n: int, draft_len: int, candidates: int,
-                             out_ids_ptr: int, out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
-    _check(load().dresd_retrieve_quantised(store, queries_ptr, B, top_n, draft_len, candidates, out_ids_ptr,
-                                           out_scores_ptr, out_tokens_ptr, stream))
+def dresd_retrieve_quantised(store: int, queries_ptr: int, first_tokens_ptr, B: int, top_n: int, draft_len: int,
+                             candidates: int, out_ids_ptr: int, out_scores_ptr: int, out_tokens_ptr: int,
+                             stream: int = 0) -> None:
+    _check(load().dresd_retrieve_quantised(store, queries_ptr, first_tokens_ptr, B, top_n, draft_len, candidates,
+                                           out_ids_ptr, out_scores_ptr, out_tokens_ptr, stream))
 
 
 def dresd_set_global_option(name: str, value: int) -> None:
@@ -340,8 +341,10 @@ class Store:
         self.keys_q8 = q8                                # keep the borrowed buffer alive
         return q8
 
-    def retrieve_quantised(self, queries, top_n: int, draft_len: int, candidates: int, out=None, stream=None):
-        """Candidates by 8-bit approximate score, exact re-ranking of `candidates` rows per query."""
+    def retrieve_quantised(self, queries, top_n: int, draft_len: int, candidates: int, out=None, stream=None,
+                           first_tokens=None):
+        """Candidates by 8-bit approximate score, exact re-ranking of `candidates` rows per query;
+        first_tokens (int32 device tensor [B], -1 = any) restricts the candidates per query."""
         torch = _torch()
         B = queries.shape[0]
         if out is None:
@@ -351,8 +354,9 @@ class Store:
                    torch.empty((B, top_n, draft_len), dtype=torch.int32, device=dev))
         ids, scores, tokens = out
         s = (stream or torch.cuda.current_stream()).cuda_stream
-        dresd_retrieve_quantised(self.handle, queries.data_ptr(), B, top_n, draft_len, candidates,
-                                 ids.data_ptr(), scores.data_ptr(), tokens.data_ptr(), s)
+        dresd_retrieve_quantised(self.handle, queries.data_ptr(),
+                                 None if first_tokens is None else first_tokens.data_ptr(), B, top_n, draft_len,
+                                 candidates, ids.data_ptr(), scores.data_ptr(), tokens.data_ptr(), s)
         return ids, scores, tokens
 
     def retrieve_host(self, queries, top_n: int, draft_len: int, out, stream=None):

@@ -233,7 +233,8 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // tcgen05 kernel, other instruction kind), then exact re-ranking of the quantised_m best
     const bool q8 = quantised_m > 0;
     // 64-element keys are 64 bytes in the 8-bit copy: two per 128-byte row, two column pairs per query
-    const bool pack2 = q8 && s->k8_packable && B <= kMaxBatch / 2 && s->opt_pack2;
+    // (the packed form has no first-token test: filtered calls scan one key per row)
+    const bool pack2 = q8 && s->k8_packable && B <= kMaxBatch / 2 && s->opt_pack2 && !first_tokens;
     s->last_stream = stream;
     s->last_launches = 0;
     s->last_key_passes = 0.0;
@@ -857,18 +858,22 @@ dresd_status dresd_store_attach_quantised(dresd_store *s, const void *keys_q8)
     return DRESD_OK;
 }
 
-dresd_status dresd_retrieve_quantised(dresd_store *s, const void *queries, int B, int top_n, int draft_len,
-                                      int candidates, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
-                                      void *stream)
+dresd_status dresd_retrieve_quantised(dresd_store *s, const void *queries, const int32_t *first_tokens, int B,
+                                      int top_n, int draft_len, int candidates, int32_t *out_ids, float *out_scores,
+                                      int32_t *out_tokens, void *stream)
 {
     dresd_status st = check_retrieve_args(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens, true);
     if (st != DRESD_OK) return st;
+    if (first_tokens) {
+        if (!s->first_col) return fail(DRESD_ERR_INVALID, "call dresd_store_enable_first_token_filter() first");
+        if (B > 0 && !is_device_ptr(first_tokens)) return fail(DRESD_ERR_INVALID, "first_tokens must be a device pointer");
+    }
     if (!s->k8) return fail(DRESD_ERR_INVALID, "no 8-bit copy attached (dresd_store_attach_quantised)");
     if (candidates < top_n || candidates > DRESD_MAX_TOP_N || candidates > s->N)
         return fail(DRESD_ERR_INVALID, "candidates = %d outside top_n..min(%d, N)", candidates, DRESD_MAX_TOP_N);
     if (B == 0) return DRESD_OK;
     return run_retrieve(s, queries, B, top_n, draft_len, out_ids, out_scores, out_tokens,
-                        static_cast<cudaStream_t>(stream), nullptr, candidates);
+                        static_cast<cudaStream_t>(stream), first_tokens, candidates);
 }
 
 dresd_status dresd_set_global_option(const char *name, int value)

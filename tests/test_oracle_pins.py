@@ -449,3 +449,24 @@ def test_quantised_scores_are_close_to_exact_and_reranking_recovers_the_neighbou
         assert np.all(approx[b][ids[b]] >= cut)
         assert np.all(np.diff(sc[b]) <= 0)
         assert np.array_equal(tok[b], toks[ids[b], :3])
+
+
+def test_quantised_first_token_filter_equals_search_of_the_matching_subset():
+    dtype, N, d = "f16", 3000, 64
+    keys, toks = synth.make_store(920, N, d, 8, dtype, 3)
+    q, _ = synth.make_queries(921, keys, dtype, 3, 0.1)
+    vals, counts = np.unique(toks[:, 0], return_counts=True)
+    common = int(vals[np.argmax(counts)])
+    rare = int(vals[np.argmin(counts)])                       # fewer matches than top_n: padding
+    ft = np.array([common, -1, rare], dtype=np.int32)
+    ids, sc, tok, approx, exact = oracle.retrieve_quantised(keys, toks, dtype, q, 4, 3, 8, first_token=ft)
+    for b, want in enumerate(ft):
+        sub = np.arange(N) if want < 0 else np.flatnonzero(toks[:, 0] == want)
+        m = min(8, len(sub))
+        r = oracle.retrieve_quantised(keys[sub], toks[sub], dtype, q[b:b + 1], min(4, len(sub)), 3, m)
+        k = min(4, len(sub))
+        assert np.array_equal(ids[b, :k], sub[r[0][0]])
+        np.testing.assert_allclose(sc[b, :k], r[1][0], rtol=0, atol=1e-12)
+        assert np.array_equal(tok[b, :k], r[2][0])
+        assert np.all(ids[b, k:] == -1) and np.all(sc[b, k:] == -np.inf) and np.all(tok[b, k:] == -1)
+    assert np.sum(toks[:, 0] == rare) < 4                      # the padding case really occurred

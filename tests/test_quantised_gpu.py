@@ -214,3 +214,47 @@ def test_quantised_retrieval_d64_packed_rows(pack2, dtype, B, n, L, m, N):
         nth = exact[b][got[-1]]
         assert not [i for i in safe if exact[b][i] > nth + 2 * EPS_ACC and i not in set(got.tolist())]
         assert np.array_equal(tok[b], toks[got, :L])
+
+
+@pytest.mark.parametrize("dtype,d,B,N", [("bf16", 256, 6, 40009), ("f16", 64, 5, 30011)])
+def test_quantised_retrieval_with_first_token_filter(dtype, d, B, N):
+    """Only keys whose first stored token matches are candidates (Section 3.5); -1 switches the
+    filter off for a query; a rare token leaves slots empty (id -1, score -inf, tokens -1).
+    d = 64 checks that a filtered call leaves the packed form."""
+    import torch
+    n, L, m = 6, 3, 24
+    keys, toks = synth.make_store(8600 + d, N, d, 16, dtype, L)
+    q, src = synth.make_queries(8601 + d, keys, dtype, B, 0.1)
+    vals, counts = np.unique(toks[:, 0], return_counts=True)
+    ft = toks[src, 0].astype(np.int32)                         # the token of the query's source row
+    ft[1] = -1
+    ft[2] = int(vals[np.argmin(counts)])                       # rare: fewer than n matches
+    st = gpu_store(keys, toks, dtype)
+    try:
+        st.attach_quantised()
+        st.enable_first_token_filter()
+        ids, sc, tok = st.retrieve_quantised(binding.to_device(q, dtype), n, L, m,
+                                             first_tokens=torch.from_numpy(ft).cuda())
+        torch.cuda.synchronize()
+        st.status()
+        ids, sc, tok = ids.cpu().numpy(), sc.cpu().numpy(), tok.cpu().numpy()
+    finally:
+        st.close()
+    o_ids, o_sc, o_tok, approx, exact = oracle.retrieve_quantised(keys, toks, dtype, q, n, L, m, first_token=ft,
+                                                                  threads=oracle.dresd_oracle.default_threads())
+    for b in range(B):
+        ok_rows = np.arange(N) if ft[b] < 0 else np.flatnonzero(toks[:, 0] == ft[b])
+        k = min(n, len(ok_rows))
+        got = ids[b, :k]
+        assert np.all(ids[b, k:] == -1) and np.all(sc[b, k:] == -np.inf) and np.all(tok[b, k:] == -1)
+        assert np.all(np.isin(got, ok_rows)) and len(set(got.tolist())) == k
+        cut = np.sort(approx[b][ok_rows])[-min(m, len(ok_rows))]
+        assert np.all(approx[b][got] >= cut - DELTA)
+        np.testing.assert_allclose(sc[b, :k], exact[b][got], rtol=0, atol=SCORE_TOL)
+        assert np.all(np.diff(exact[b][got]) <= 2 * EPS_ACC)
+        safe = ok_rows[approx[b][ok_rows] >= cut + DELTA]
+        if k:
+            nth = exact[b][got[-1]]
+            assert not [i for i in safe if exact[b][i] > nth + 2 * EPS_ACC and i not in set(got.tolist())]
+        assert np.array_equal(tok[b, :k], toks[got, :L])
+    assert np.sum(toks[:, 0] == ft[2]) < n
