@@ -251,24 +251,26 @@ def run_ours(args):
 
     recall = None
     if args.quantised:
-        if dft is not None:
-            raise SystemExit("--quantised and --first-token-filter are separate paths")
         store.attach_quantised()
         # recall of the exact neighbours (the exact path is the parity-checked one)
         hit = tot = 0
         for i in range(min(nq, 64)):
             j = (q_first + i) * B
-            ex = store.retrieve(dq[j:j + B], n, L)[0].cpu().numpy()
-            ap_ = store.retrieve_quantised(dq[j:j + B], n, L, args.quantised)[0].cpu().numpy()
+            ftk = None if dft is None else dft[j:j + B]
+            ex = (store.retrieve(dq[j:j + B], n, L) if dft is None
+                  else store.retrieve_filtered(dq[j:j + B], ftk, n, L))[0].cpu().numpy()
+            ap_ = store.retrieve_quantised(dq[j:j + B], n, L, args.quantised, first_tokens=ftk)[0].cpu().numpy()
             for b in range(B):
-                hit += len(set(ex[b].tolist()) & set(ap_[b].tolist()))
-                tot += n
+                want = set(ex[b].tolist()) - {-1}
+                hit += len(want & set(ap_[b].tolist()))
+                tot += len(want)
         recall = hit / tot
 
     def step(i):
         j = (q_first + i % nq) * B
         if args.quantised:
-            store.retrieve_quantised(dq[j:j + B], n, L, args.quantised, out=out)
+            store.retrieve_quantised(dq[j:j + B], n, L, args.quantised, out=out,
+                                     first_tokens=None if dft is None else dft[j:j + B])
         elif dft is None:
             store.retrieve(dq[j:j + B], n, L, out=out)
         else:
@@ -344,7 +346,8 @@ def run_ours(args):
         # the quantised call takes device buffers: the same copies, issued here
         dq_stage.view(torch.int16 if dtype != "f32" else torch.float32).copy_(
             hq[j:j + B].view(torch.int16 if dtype != "f32" else torch.float32), non_blocking=True)
-        store.retrieve_quantised(dq_stage, n, L, args.quantised, out=out)
+        store.retrieve_quantised(dq_stage, n, L, args.quantised, out=out,
+                                 first_tokens=None if dft is None else dft[j:j + B])
         for h, o_ in zip(hout, out):
             h.copy_(o_, non_blocking=True)
         torch.cuda.synchronize()
