@@ -233,8 +233,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // tcgen05 kernel, other instruction kind), then exact re-ranking of the quantised_m best
     const bool q8 = quantised_m > 0;
     // 64-element keys are 64 bytes in the 8-bit copy: two per 128-byte row, two column pairs per query
-    // (the packed form has no first-token test: filtered calls scan one key per row)
-    const bool pack2 = q8 && s->k8_packable && B <= kMaxBatch / 2 && s->opt_pack2 && !first_tokens;
+    const bool pack2 = q8 && s->k8_packable && B <= kMaxBatch / 2 && s->opt_pack2;
     s->last_stream = stream;
     s->last_launches = 0;
     s->last_key_passes = 0.0;
@@ -345,7 +344,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     if (q8) {
         // fold the approximate lists, score the m survivors exactly, sort, gather: one launch
         cudaError_t e = launch_merge_rerank(s->cand, grid, B, s->keys, s->dtype, s->d, s->N, s->qhat, quantised_m, top_n,
-                                            pack2 && (s->N & 1) ? s->N - 1 : -1, s->next_tokens, s->stored_len,
+                                            pack2 && (s->N & 1) ? s->N - 1 : -1, first_tokens, s->next_tokens, s->stored_len,
                                             draft_len, out_ids, out_scores, out_tokens, stream);
         if (e != cudaSuccess) return fail_cuda(e, "merge / re-rank launch");
         s->last_launches += 1;

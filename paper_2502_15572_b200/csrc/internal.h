@@ -147,8 +147,8 @@ cudaError_t launch_quantise_keys(const void *keys, int dtype, long long N, int d
 // extra_id >= 0: one more candidate for every query (the last key of an odd-sized packed store).
 cudaError_t launch_merge_rerank(const unsigned long long *cand, int lists, int B, const void *keys, int dtype, int d,
                                 long long N, const float *qhat, int mcand, int top_n, long long extra_id,
-                                const int32_t *next_tokens, int stored_len, int draft_len, int32_t *out_ids,
-                                float *out_scores, int32_t *out_tokens, cudaStream_t stream);
+                                const int32_t *want_first, const int32_t *next_tokens, int stored_len, int draft_len,
+                                int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream);
 
 // Stores `msg` as the calling thread's dresd_last_error() text.
 void set_last_error(const char *msg);

@@ -164,7 +164,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             if (lane == 0) {
                 const int rq = PACK2 ? q >> 1 : q;          // the query this column pair belongs to
                 tau[q] = (rq < a.B && !a.no_select) ? peek_tau(&a.gtau[rq], -INFINITY) : INFINITY;
-                want_s[q] = (!PACK2 && a.first_col && q < a.B) ? a.want_first[q] : -1;
+                want_s[q] = (a.first_col && rq < a.B) ? a.want_first[rq] : -1;
             }
         }
     }
@@ -309,10 +309,22 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             const long long row0 =
                 (long long)(cta + tl * G) * a.tile_stride * kRowsPerTile + lane_grp * 32 + lane;
             // first stored token of this thread's rows (filtered calls), requested before the wait
-            int tok[TSUB];
+            // (PACK2: of the row's two keys -- first_col is indexed by key, two per row)
+            int tok[TSUB], tok1[TSUB];
 #pragma unroll
-            for (int sub = 0; sub < TSUB; ++sub)
-                tok[sub] = (filtered && row0 + sub * kTileRows < a.N) ? a.first_col[row0 + sub * kTileRows] : 0;
+            for (int sub = 0; sub < TSUB; ++sub) {
+                const long long r = row0 + sub * kTileRows;
+                tok[sub] = tok1[sub] = 0;
+                if (filtered && r < a.N) {
+                    if constexpr (PACK2) {
+                        const int2 t = *reinterpret_cast<const int2 *>(a.first_col + 2 * r);
+                        tok[sub] = t.x;
+                        tok1[sub] = t.y;
+                    } else {
+                        tok[sub] = a.first_col[r];
+                    }
+                }
+            }
             if (!dead && !mbar_wait(&tfull[acc], use & 1)) {
                 report_timeout(a.status);
                 dead = true;
@@ -343,7 +355,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         for (int j = 0; j < QW; ++j) {
                             const float s = fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
                             const int w = want_s[qbase + j];
-                            const bool ok = row_ok && (w < 0 || tok[sub] == w) && s > -INFINITY;   // false for NaN
+                            const int tkj = (PACK2 && ((qbase + j) & 1)) ? tok1[sub] : tok[sub];
+                            const bool ok = row_ok && (w < 0 || tkj == w) && s > -INFINITY;        // false for NaN
                             const uint32_t id = PACK2 ? (uint32_t)(2 * row + ((qbase + j) & 1)) : (uint32_t)row;
                             v[j] = ok ? pack_candidate(s, id) : 0ull;
                         }
@@ -403,12 +416,13 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     }
                     if (filtered) {                         // Section 3.5: drafts must start with x_{t+1}
                         uint32_t match = wild;
-                        const int tk = tok[sub];
+                        // column pairs alternate between the row's even and odd key when packed (qbase is even)
+                        const int tk = tok[sub], tko = PACK2 ? tok1[sub] : tok[sub];
 #pragma unroll
                         for (int j4 = 0; j4 < QW / 4; ++j4) {
                             const int4 w = want4[j4];
-                            match |= ((tk == w.x ? 1u : 0u) | (tk == w.y ? 2u : 0u) | (tk == w.z ? 4u : 0u) |
-                                      (tk == w.w ? 8u : 0u)) << (4 * j4);
+                            match |= ((tk == w.x ? 1u : 0u) | (tko == w.y ? 2u : 0u) | (tk == w.z ? 4u : 0u) |
+                                      (tko == w.w ? 8u : 0u)) << (4 * j4);
                         }
                         mask &= match;
                     }

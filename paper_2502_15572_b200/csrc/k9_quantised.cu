@@ -80,7 +80,7 @@ template <typename T>
 __global__ void __launch_bounds__(kRerankWarps * 32)
 merge_rerank_kernel(const unsigned long long *__restrict__ cand, int lists, int B, const T *__restrict__ keys, int d,
                     long long N, const float *__restrict__ qhat, int mcand, int top_n, long long extra_id,
-                    const int32_t *__restrict__ next_tokens, int stored_len, int draft_len,
+                    const int32_t *__restrict__ want_first, const int32_t *__restrict__ next_tokens, int stored_len, int draft_len,
                     int32_t *__restrict__ out_ids, float *__restrict__ out_scores, int32_t *__restrict__ out_tokens)
 {
     __shared__ unsigned long long part[kRerankWarps][kListLen];
@@ -115,7 +115,11 @@ merge_rerank_kernel(const unsigned long long *__restrict__ cand, int lists, int 
     const float *q = qhat + (size_t)b * d;
     for (int r = warp; r <= kListLen; r += kRerankWarps) {
         const unsigned long long c = r < mcand ? part[0][r] : 0ull;       // exactly the m best, as defined
-        const long long id = r < kListLen ? (c ? (long long)candidate_id(c) : -1) : extra_id;
+        long long id = r < kListLen ? (c ? (long long)candidate_id(c) : -1) : extra_id;
+        // the extra candidate did not pass the scan's first-token test: apply it here
+        if (r == kListLen && id >= 0 && want_first && want_first[b] >= 0 &&
+            next_tokens[(size_t)id * stored_len] != want_first[b])
+            id = -1;
         unsigned long long p = 0ull;
         if (id >= 0 && id < N) {                             // warp-uniform
             const uint4 *row = reinterpret_cast<const uint4 *>(keys + (size_t)id * d);
@@ -175,16 +179,18 @@ cudaError_t launch_quantise_keys(const void *keys, int dtype, long long N, int d
 
 cudaError_t launch_merge_rerank(const unsigned long long *cand, int lists, int B, const void *keys, int dtype, int d,
                                 long long N, const float *qhat, int mcand, int top_n, long long extra_id,
-                                const int32_t *next_tokens, int stored_len, int draft_len, int32_t *out_ids,
-                                float *out_scores, int32_t *out_tokens, cudaStream_t stream)
+                                const int32_t *want_first, const int32_t *next_tokens, int stored_len, int draft_len,
+                                int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream)
 {
     if (dtype == kF16)
         merge_rerank_kernel<__half><<<B, kRerankWarps * 32, 0, stream>>>(
-            cand, lists, B, static_cast<const __half *>(keys), d, N, qhat, mcand, top_n, extra_id, next_tokens, stored_len,
+            cand, lists, B, static_cast<const __half *>(keys), d, N, qhat, mcand, top_n, extra_id, want_first, next_tokens,
+            stored_len,
             draft_len, out_ids, out_scores, out_tokens);
     else
         merge_rerank_kernel<__nv_bfloat16><<<B, kRerankWarps * 32, 0, stream>>>(
-            cand, lists, B, static_cast<const __nv_bfloat16 *>(keys), d, N, qhat, mcand, top_n, extra_id, next_tokens,
+            cand, lists, B, static_cast<const __nv_bfloat16 *>(keys), d, N, qhat, mcand, top_n, extra_id, want_first,
+            next_tokens,
             stored_len, draft_len, out_ids, out_scores, out_tokens);
     return cudaGetLastError();
 }

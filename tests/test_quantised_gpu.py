@@ -220,7 +220,9 @@ def test_quantised_retrieval_d64_packed_rows(pack2, dtype, B, n, L, m, N):
 def test_quantised_retrieval_with_first_token_filter(dtype, d, B, N):
     """Only keys whose first stored token matches are candidates (Section 3.5); -1 switches the
     filter off for a query; a rare token leaves slots empty (id -1, score -inf, tokens -1).
-    d = 64 checks that a filtered call leaves the packed form."""
+    At d = 64 the packed form (two keys, two first tokens per row; N is odd, so the last key
+    reaches the re-ranking as an extra candidate and is filtered there) must agree with the
+    unpacked one."""
     import torch
     n, L, m = 6, 3, 24
     keys, toks = synth.make_store(8600 + d, N, d, 16, dtype, L)
@@ -233,11 +235,28 @@ def test_quantised_retrieval_with_first_token_filter(dtype, d, B, N):
     try:
         st.attach_quantised()
         st.enable_first_token_filter()
-        ids, sc, tok = st.retrieve_quantised(binding.to_device(q, dtype), n, L, m,
-                                             first_tokens=torch.from_numpy(ft).cuda())
+        dft = torch.from_numpy(ft).cuda()
+        ids, sc, tok = st.retrieve_quantised(binding.to_device(q, dtype), n, L, m, first_tokens=dft)
         torch.cuda.synchronize()
         st.status()
         ids, sc, tok = ids.cpu().numpy(), sc.cpu().numpy(), tok.cpu().numpy()
+        if d == 64:
+            st.set_option("pack2", 0)
+            other = st.retrieve_quantised(binding.to_device(q, dtype), n, L, m, first_tokens=dft)
+            torch.cuda.synchronize()
+            assert np.array_equal(other[0].cpu().numpy(), ids) and np.array_equal(other[1].cpu().numpy(), sc)
+            # the last key as a query: it must be found through the extra-candidate route, and only
+            # when its first token is the wanted one
+            st.set_option("pack2", 1)
+            last = binding.to_device(keys[N - 1:N], dtype)
+            for want, expect in ((int(toks[N - 1, 0]), N - 1), (int(toks[N - 1, 0]) + 1, None)):
+                o = st.retrieve_quantised(last, 1, L, 4, first_tokens=torch.tensor([want], dtype=torch.int32, device="cuda"))
+                torch.cuda.synchronize()
+                got0 = int(o[0].cpu().numpy()[0, 0])
+                if expect is None:
+                    assert got0 != N - 1
+                else:
+                    assert np.array_equal(keys[got0], keys[N - 1])     # the key itself (or an earlier duplicate)
     finally:
         st.close()
     o_ids, o_sc, o_tok, approx, exact = oracle.retrieve_quantised(keys, toks, dtype, q, n, L, m, first_token=ft,
