@@ -428,3 +428,19 @@ def test_non_finite_inputs_neither_hang_nor_fault(dtype, d, B):
         assert np.array_equal(ids3, ids)
     finally:
         st.close()
+
+
+# The corners of the supported envelope: the widest rows with the widest batch (query operand
+# streamed with the keys), the narrowest rows the loader accepts (16 bytes), the longest lists.
+@pytest.mark.parametrize("dtype,d,B,n,L,N", [
+    ("bf16", 4096, 64, 32, 2, 1501),
+    ("f16", 8, 1, 1, 1, 100),
+    ("f16", 8, 64, 32, 1, 5000),
+    ("f32", 4096, 8, 32, 2, 1201),
+    ("f32", 4, 9, 3, 1, 777),
+    ("bf16", 264, 64, 32, 1, 30011),           # five slabs: the 33-64 query kernel hands over to the other form
+])
+def test_parity_envelope_corners(dtype, d, B, n, L, N):
+    keys, toks = synth.make_store(7800 + d + B, N, d, 8, dtype, L)
+    q, _ = synth.make_queries(7850 + d + B, keys, dtype, B, 0.1)
+    _check(keys, toks, dtype, q, n, L)
