@@ -8,6 +8,11 @@
 // one row per thread, read it with conflict-free LDS.128 against queries
 // broadcast from shared memory, and keep four partial sums per query so that
 // the accumulation error stays near d/4 ulps.  Up to QB queries per launch.
+// The running top-n lists are shared by the CTA (one per query): survivors of
+// the filter are queued with a shared-memory atomic, a named barrier per tile
+// publishes them, and a queue that reaches 16 entries is folded by one warp
+// (the four warps fold different queries at once).  Per-warp lists would cost
+// a small store four cold starts per query instead of one.
 #include "common.cuh"
 #include "internal.h"
 
@@ -23,6 +28,15 @@ constexpr int kSlabsPerStage = 2;
 constexpr int kStageBytes = kRows * kSlabsPerStage * kSlabBytes;   // 32 KB
 constexpr int kMaxStages = 6;
 
+struct SelFlags {
+    int need_merge;
+    int overflow;
+};
+__device__ __forceinline__ void consumer_bar()
+{
+    asm volatile("bar.sync 2, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+}
+
 template <int QB>
 __global__ void __launch_bounds__(kThreads, 1)
 scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
@@ -32,10 +46,11 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     const int n_stages = a.stages;
     uint8_t *stages = base;
-    WarpTopN *sel = reinterpret_cast<WarpTopN *>(stages + (size_t)n_stages * kStageBytes);
-    uint64_t *full = reinterpret_cast<uint64_t *>(sel + kConsumerWarps * QB);
+    WarpTopN *sel = reinterpret_cast<WarpTopN *>(stages + (size_t)n_stages * kStageBytes);   // [QB], CTA-wide
+    uint64_t *full = reinterpret_cast<uint64_t *>(sel + QB);
     uint64_t *empty = full + kMaxStages;
-    float *qs = reinterpret_cast<float *>(empty + kMaxStages);     // [QB][dpad]
+    SelFlags *flags = reinterpret_cast<SelFlags *>(empty + kMaxStages);   // [3], rotating
+    float *qs = reinterpret_cast<float *>(flags + 4);              // [QB][dpad]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
@@ -47,10 +62,17 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], kConsumerWarps);
         }
+        for (int i = 0; i < 3; ++i) {
+            flags[i].need_merge = 0;
+            flags[i].overflow = 0;
+        }
         mbar_fence_init();
     }
     if (warp < kConsumerWarps)
-        for (int q = 0; q < QB; ++q) warp_topn_init(&sel[warp * QB + q], lane);
+        for (int q = warp; q < QB; q += kConsumerWarps) {
+            warp_topn_init(&sel[q], lane);
+            if (lane == 0 && q < a.B) sel[q].tau = peek_tau(&a.gtau[q], -INFINITY);
+        }
     for (int i = tid; i < QB * dpad; i += kThreads) {
         int q = i / dpad, c = i % dpad;
         qs[i] = (q < a.B && c < a.d) ? a.qhat[(size_t)q * a.d + c] : 0.f;
@@ -88,17 +110,20 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 }
         }
     } else {
-        WarpTopN *my_sel = &sel[warp * QB];
         const int row_in_tile = tid;                  // 0..127
         const uint32_t swz = (uint32_t)(row_in_tile & 7);
+        // A warp whose wait expired goes "dead": it does no more work and no more waits,
+        // but keeps taking part in every barrier so that nobody is left behind.
         bool dead = false;
+        int round = 0;                                 // barrier-A count: selects the flag slot
+        SelFlags *fl = &flags[0];
         int want[QB];                                  // first-token filter, -1 = off
 #pragma unroll
         for (int q = 0; q < QB; ++q) want[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
-        for (int tl = 0; tl < my_tiles && !dead; ++tl) {
+        for (int tl = 0; tl < my_tiles; ++tl) {
             // this row's first stored token, requested before the tile is waited for
-            const long long row_pre = (long long)(cta + tl * G) * kRows + row_in_tile;
-            const int tok = (a.first_col && row_pre < a.N) ? a.first_col[row_pre] : 0;
+            const long long row = (long long)(cta + tl * G) * kRows + row_in_tile;
+            const int tok = (a.first_col && row < a.N) ? a.first_col[row] : 0;
             float acc[QB][4];
 #pragma unroll
             for (int q = 0; q < QB; ++q)
@@ -107,11 +132,12 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             for (int kc = 0; kc < kch; ++kc) {
                 const int it = tl * kch + kc;
                 const int s = it % n_stages;
-                if (!mbar_wait(&full[s], (it / n_stages) & 1)) {
+                if (!dead && !mbar_wait(&full[s], (it / n_stages) & 1)) {
                     report_timeout(a.status);
                     dead = true;
-                    break;
                 }
+                dead = __any_sync(0xFFFFFFFFu, dead);
+                if (dead) continue;
                 const uint8_t *rowp = stages + (size_t)s * kStageBytes + (size_t)row_in_tile * kSlabBytes;
                 const int nsl = min(kSlabsPerStage, dslabs - kc * kSlabsPerStage);
                 for (int sl = 0; sl < nsl; ++sl) {
@@ -133,39 +159,66 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[s]);
             }
-            if (dead) break;
+            // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
+            if ((tl & 3) == 0 && tid < a.B && tid < QB) sel[tid].tau = peek_tau(&a.gtau[tid], sel[tid].tau);
 
-            const long long row = (long long)(cta + tl * G) * kRows + row_in_tile;
             float sc[QB];
-            bool take[QB];
-            bool any = false;
+            uint32_t pend = 0u;                        // queries for which this row is (still) a candidate
 #pragma unroll
             for (int q = 0; q < QB; ++q) {
                 sc[q] = (acc[q][0] + acc[q][1]) + (acc[q][2] + acc[q][3]);
-                take[q] = q < a.B && row < a.N && sc[q] >= my_sel[q].tau && (want[q] < 0 || tok == want[q]);
-                any |= take[q];
+                const bool take = !dead && q < a.B && row < a.N && sc[q] >= sel[q].tau && (want[q] < 0 || tok == want[q]);
+                pend |= take ? (1u << q) : 0u;
             }
-            if (__any_sync(0xFFFFFFFFu, any)) {
-                // Rare path: pull the grid-wide filter, re-test, queue, publish ours.
-                if (lane < QB && lane < a.B) my_sel[lane].tau = peek_tau(&a.gtau[lane], my_sel[lane].tau);
-                __syncwarp();
+            // Queue the survivors; when a queue is full the candidate waits (`pend`) until the CTA
+            // has folded the queues, so that adversarial row orders stay exact.
+            while (true) {
+                // claim the slots first (independent shared-memory atomics in flight together), then fill them
+                int slot[QB];
 #pragma unroll
-                for (int q = 0; q < QB; ++q)
-                    warp_topn_push(&my_sel[q], a.top_n, lane, take[q] && sc[q] >= my_sel[q].tau, sc[q], (uint32_t)row);
-                if (lane < QB && lane < a.B) my_sel[lane].tau = share_tau(&a.gtau[lane], my_sel[lane].tau);
-                __syncwarp();
+                for (int q = 0; q < QB; ++q) {
+                    if (((pend >> q) & 1u) && !(sc[q] >= sel[q].tau)) pend &= ~(1u << q);   // the filter has tightened
+                    slot[q] = ((pend >> q) & 1u) ? atomicAdd(&sel[q].count, 1) : 0;
+                }
+#pragma unroll
+                for (int q = 0; q < QB; ++q) {
+                    if ((pend >> q) & 1u) {
+                        if (slot[q] < kQueueCap) {
+                            sel[q].queue[slot[q]] = pack_candidate(sc[q], (uint32_t)row);
+                            if (slot[q] + 1 >= kMergeLevel) fl->need_merge = 1;
+                            pend &= ~(1u << q);
+                        } else {
+                            fl->overflow = 1;
+                        }
+                    }
+                }
+                consumer_bar();                         // A: every push of this pass is visible
+                const int need = fl->need_merge, over = fl->overflow;
+                // Flags rotate over three slots: the slot of the previous pass was read by everyone
+                // before arriving at A and is not written again before the next A.
+                if (tid == 0) {
+                    SelFlags *prev = &flags[(round + 2) % 3];
+                    prev->need_merge = 0;
+                    prev->overflow = 0;
+                }
+                round += 1;
+                fl = &flags[round % 3];
+                if (!(need | over)) break;
+                for (int q = warp; q < QB; q += kConsumerWarps) {
+                    if (sel[q].count > 0) {
+                        warp_topn_merge(&sel[q], a.top_n, lane);
+                        if (lane == 0 && q < a.B) sel[q].tau = share_tau(&a.gtau[q], sel[q].tau);
+                    }
+                }
+                consumer_bar();                         // C: lists, counts and tau are settled
+                if (!over) break;
             }
         }
-        for (int q = 0; q < QB; ++q)
-            if (my_sel[q].count > 0) warp_topn_merge(&my_sel[q], a.top_n, lane);
-    }
-    __syncthreads();
-
-    if (warp < kConsumerWarps) {
+        // flush and publish this CTA's lists
+        consumer_bar();
         for (int q = warp; q < min(QB, a.B); q += kConsumerWarps) {
+            if (sel[q].count > 0) warp_topn_merge(&sel[q], a.top_n, lane);
             unsigned long long m = sel[q].list[lane];
-            for (int w = 1; w < kConsumerWarps; ++w)
-                m = warp_merge_top32(m, sel[w * QB + q].list[lane], lane);
             if (lane >= a.top_n) m = 0ull;
             a.cand[((size_t)cta * a.cand_batch + q) * kCandStride + lane] = m;
         }
@@ -176,7 +229,7 @@ template <int QB>
 size_t smem_bytes(int d, int *stages_out)
 {
     const int dpad = ((d + kSlabElems - 1) / kSlabElems) * kSlabElems;
-    size_t fixed = 1024 + sizeof(WarpTopN) * kConsumerWarps * QB + 2 * kMaxStages * sizeof(uint64_t) +
+    size_t fixed = 1024 + sizeof(WarpTopN) * QB + 2 * kMaxStages * sizeof(uint64_t) + 4 * sizeof(SelFlags) +
                    sizeof(float) * (size_t)QB * dpad;
     int stages = (int)((227 * 1024 - (long long)fixed) / kStageBytes);
     if (stages > kMaxStages) stages = kMaxStages;
