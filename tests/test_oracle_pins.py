@@ -470,3 +470,25 @@ def test_quantised_first_token_filter_equals_search_of_the_matching_subset():
         assert np.array_equal(tok[b, :k], r[2][0])
         assert np.all(ids[b, k:] == -1) and np.all(sc[b, k:] == -np.inf) and np.all(tok[b, k:] == -1)
     assert np.sum(toks[:, 0] == rare) < 4                      # the padding case really occurred
+
+
+def test_quantised_scores_match_an_independent_formulation():
+    """The same three rules written with a library's E4M3 conversion and a float64 matmul."""
+    torch = pytest.importorskip("torch")
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("this torch has no float8_e4m3fn")
+    rng = np.random.default_rng(31)
+    N, d = 500, 48
+    keys = rng.normal(size=(N, d)).astype(np.float32)
+    keys /= np.linalg.norm(keys, axis=1, keepdims=True)
+    k16 = keys.astype(np.float16)                               # the store: fp16 bit patterns
+    q = rng.normal(size=d).astype(np.float32)
+    q /= np.linalg.norm(q)                                      # float32 values, handed over exactly
+    f8 = lambda x: torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.float8_e4m3fn).to(torch.float32).numpy().astype(np.float64)
+    k8 = f8(k16.astype(np.float32) * 256.0)
+    q256 = q.astype(np.float64) * 256.0
+    h1 = f8(q256)
+    h2 = f8((q256 - h1) * 16.0)
+    want = k8 @ (h1 + h2 / 16.0) / 65536.0
+    got = oracle.quantised_scores(k16, "f16", q.astype(np.float64))
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-13)
