@@ -269,10 +269,13 @@ dresd_status dresd_merge_shards(const int32_t *ids, const float *scores, const i
                                 int32_t *out_ids, float *out_scores, int32_t *out_tokens, void *stream);
 
 /*
- * The same call for callers whose queries and results live in HOST memory
- * (ideally pinned): copies the queries to the device, runs dresd_retrieve(),
- * copies the three results back and waits for `stream`.  The datastore itself
- * stays on the device.  Returns the device status word as well (see below).
+ * The same call for callers whose queries and results live in HOST memory, and
+ * waits for `stream`.  When all four buffers are page-locked and mapped (e.g.
+ * cudaHostAlloc, cudaHostRegister, a pinned framework tensor), the kernels read the
+ * queries and write the results across the bus themselves (B * d_in elements in,
+ * B * top_n * (8 + 4 draft_len) bytes out) and no copy is enqueued; otherwise the
+ * queries are copied to a staging buffer and the three results copied back.  The
+ * datastore itself stays on the device.  Returns the device status word as well.
  */
 dresd_status dresd_retrieve_host(dresd_store *store, const void *queries_host, int B, int top_n,
                                  int draft_len, int32_t *out_ids_host, float *out_scores_host,

@@ -67,6 +67,17 @@ size_t elem_bytes(int dtype) { return dtype == kF32 ? 4 : 2; }
 
 // 2-D map over a row-major [rows][cols] matrix; box = one 128-byte swizzle row
 // wide, box_rows tall; out-of-range elements read as zero.
+// Device-side address of a page-locked host buffer that the device can reach, else null.
+void *mapped_device_ptr(const void *host)
+{
+    cudaPointerAttributes at{};
+    if (!host || cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 bool make_map(CUtensorMap *map, const void *base, int dtype, long long rows, int cols, int box_rows)
 {
     EncodeTiledFn fn = encode_tiled_fn();
@@ -534,19 +545,33 @@ dresd_status dresd_retrieve_host(dresd_store *s, const void *queries_host, int B
     if (st != DRESD_OK || B == 0) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const size_t qbytes = (size_t)B * s->d_in * elem_bytes(s->dtype);
-    cudaError_t e = cudaMemcpyAsync(s->q_stage, queries_host, qbytes, cudaMemcpyHostToDevice, stream);
-    if (e != cudaSuccess) return fail_cuda(e, "query upload");
-    st = run_retrieve(s, s->q_stage, B, top_n, draft_len, s->ids_dev, s->scores_dev, s->tokens_dev, stream);
-    if (st != DRESD_OK) return st;
-    int dev_status = 0;
     const size_t n = (size_t)B * top_n;
-    e = cudaMemcpyAsync(out_ids_host, s->ids_dev, n * sizeof(int32_t), cudaMemcpyDeviceToHost, stream);
-    if (e == cudaSuccess)
-        e = cudaMemcpyAsync(out_scores_host, s->scores_dev, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
-    if (e == cudaSuccess)
-        e = cudaMemcpyAsync(out_tokens_host, s->tokens_dev, n * draft_len * sizeof(int32_t),
-                            cudaMemcpyDeviceToHost, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(&dev_status, s->status, sizeof(int), cudaMemcpyDeviceToHost, stream);
+    int dev_status = 0;
+    cudaError_t e;
+    // Pinned (page-locked, mapped) host buffers are reachable from the device: the kernels then
+    // read the queries and write the results across the bus themselves, and no copy is enqueued
+    // around them.  Any pageable buffer sends the call through staging copies instead.
+    const void *dq = mapped_device_ptr(queries_host);
+    int32_t *dids = static_cast<int32_t *>(mapped_device_ptr(out_ids_host));
+    float *dsc = static_cast<float *>(mapped_device_ptr(out_scores_host));
+    int32_t *dtok = static_cast<int32_t *>(mapped_device_ptr(out_tokens_host));
+    if (dq && dids && dsc && dtok) {
+        st = run_retrieve(s, dq, B, top_n, draft_len, dids, dsc, dtok, stream);
+        if (st != DRESD_OK) return st;
+        e = cudaMemcpyAsync(&dev_status, s->status, sizeof(int), cudaMemcpyDeviceToHost, stream);
+    } else {
+        e = cudaMemcpyAsync(s->q_stage, queries_host, qbytes, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return fail_cuda(e, "query upload");
+        st = run_retrieve(s, s->q_stage, B, top_n, draft_len, s->ids_dev, s->scores_dev, s->tokens_dev, stream);
+        if (st != DRESD_OK) return st;
+        e = cudaMemcpyAsync(out_ids_host, s->ids_dev, n * sizeof(int32_t), cudaMemcpyDeviceToHost, stream);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(out_scores_host, s->scores_dev, n * sizeof(float), cudaMemcpyDeviceToHost, stream);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(out_tokens_host, s->tokens_dev, n * draft_len * sizeof(int32_t),
+                                cudaMemcpyDeviceToHost, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(&dev_status, s->status, sizeof(int), cudaMemcpyDeviceToHost, stream);
+    }
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return fail_cuda(e, "result download");
     if (dev_status != 0) {

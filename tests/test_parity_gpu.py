@@ -444,3 +444,28 @@ def test_parity_envelope_corners(dtype, d, B, n, L, N):
     keys, toks = synth.make_store(7800 + d + B, N, d, 8, dtype, L)
     q, _ = synth.make_queries(7850 + d + B, keys, dtype, B, 0.1)
     _check(keys, toks, dtype, q, n, L)
+
+
+def test_host_call_with_pinned_and_with_pageable_buffers():
+    """Pinned buffers are read and written by the kernels directly; pageable ones go through
+    staging copies.  Same results either way, equal to the device-buffer call."""
+    import torch
+    dtype, N, d, B, n, L = "f16", 40009, 128, 5, 10, 4
+    keys, toks = synth.make_store(7900, N, d, 16, dtype, L)
+    q, _ = synth.make_queries(7901, keys, dtype, B, 0.1)
+    st = gpu_store(keys, toks, dtype)
+    try:
+        ref = gpu_retrieve(st, q, n, L)
+        for pinned in (True, False):
+            qh = torch.from_numpy(q.copy())
+            outs = [torch.full((B, n), -7, dtype=torch.int32), torch.full((B, n), -7.0, dtype=torch.float32),
+                    torch.full((B, n, L), -7, dtype=torch.int32)]
+            if pinned:
+                qh = qh.pin_memory()
+                outs = [o.pin_memory() for o in outs]
+            assert qh.is_pinned() == pinned
+            st.retrieve_host(qh, n, L, tuple(outs))
+            for a, b in zip(ref, outs):
+                assert np.array_equal(a, b.numpy())
+    finally:
+        st.close()
