@@ -277,3 +277,39 @@ def test_quantised_retrieval_with_first_token_filter(dtype, d, B, N):
             assert not [i for i in safe if exact[b][i] > nth + 2 * EPS_ACC and i not in set(got.tolist())]
         assert np.array_equal(tok[b, :k], toks[got, :L])
     assert np.sum(toks[:, 0] == ft[2]) < n
+
+
+def test_quantised_packed_rows_with_probe_pass_against_oracle():
+    """d = 64, 16 queries x 32 candidates on a store large enough for the probe pass of the packed
+    form (tile-best rows of even and odd keys seed the filter): full check against the oracle."""
+    dtype, d, B, n, L, m = "f16", 64, 16, 10, 2, 32
+    N = 148 * 512 * 130 + 1                                     # odd: the last key is the extra candidate
+    keys, toks = synth.make_store(8700, N, d, 256, dtype, L)
+    q, _ = synth.make_queries(8701, keys, dtype, B, 0.1)
+    q[3] = keys[N - 1]                                          # one query IS the last key
+    import torch
+    st = gpu_store(keys, toks, dtype)
+    try:
+        st.attach_quantised()
+        st.set_option("probe", 32)                              # every 32nd tile: this store has 9,620 tiles
+        ids, sc, tok = st.retrieve_quantised(binding.to_device(q, dtype), n, L, m)
+        torch.cuda.synchronize()
+        st.status()
+        assert st.last_launches() == 5                          # K1, probe scan + its merge, scan, merge/re-rank
+        ids, sc, tok = ids.cpu().numpy(), sc.cpu().numpy(), tok.cpu().numpy()
+    finally:
+        st.close()
+    _, _, _, approx, exact = oracle.retrieve_quantised(keys, toks, dtype, q, n, L, m,
+                                                       threads=oracle.dresd_oracle.default_threads())
+    assert np.array_equal(keys[ids[3, 0]], keys[N - 1])
+    for b in range(B):
+        cut = np.sort(approx[b])[-m]
+        got = ids[b]
+        assert len(set(got.tolist())) == n and np.all(got >= 0) and np.all(got < N)
+        assert np.all((approx[b][got] >= cut - DELTA) | (got == N - 1))
+        np.testing.assert_allclose(sc[b], exact[b][got], rtol=0, atol=SCORE_TOL)
+        assert np.all(np.diff(exact[b][got]) <= 2 * EPS_ACC)
+        safe = np.flatnonzero(approx[b] >= cut + DELTA)
+        nth = exact[b][got[-1]]
+        assert not [i for i in safe if exact[b][i] > nth + 2 * EPS_ACC and i not in set(got.tolist())]
+        assert np.array_equal(tok[b], toks[got, :L])
