@@ -92,3 +92,43 @@ def test_config5b_projected_full_size():
                         threads=oracle.dresd_oracle.default_threads())
     rate = checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids)
     assert rate >= 0.9
+
+
+def test_config2_quantised_full_size():
+    """10M x 256 fp16, single queries through the quantised search (8-bit candidates, exact
+    re-ranking of 32), as `bench.py --quantised 32` issues them: 32 calls checked by
+    properties (rows distinct and in range, exact scores in order, stored tokens), 3 against
+    the oracle's statement of the same rules, and the recall of the exact path's rows."""
+    import torch
+    w = synth.make_workload("c2_decode_b1_f16")
+    keys, toks, dtype, n, L, m = w["keys"], w["next_tokens"], "f16", w["top_n"], w["draft_len"], 32
+    q, _ = synth.make_queries(w["seed"] + 200, keys, dtype, 32, w["sigma"])
+    st = gpu_store(keys, toks, dtype)
+    try:
+        st.attach_quantised()
+        dq = binding.to_device(q, dtype)
+        outs, exact_ids = [], []
+        for j in range(q.shape[0]):
+            o = st.retrieve_quantised(dq[j:j + 1], n, L, m)
+            outs.append([t.cpu().numpy() for t in o])
+            exact_ids.append(st.retrieve(dq[j:j + 1], n, L)[0].cpu().numpy())
+        torch.cuda.synchronize()
+        st.status()
+    finally:
+        st.close()
+    ids = np.concatenate([o[0] for o in outs])
+    sc = np.concatenate([o[1] for o in outs])
+    tok = np.concatenate([o[2] for o in outs])
+    _properties(keys, toks, dtype, q, ids, sc, tok, n, L)
+    recall = np.mean([len(set(a.tolist()) & set(b[0].tolist())) / n for a, b in zip(ids, exact_ids)])
+    assert recall >= 0.95
+    sample = [0, 13, 31]
+    _, _, _, approx, exact = oracle.retrieve_quantised(keys, toks, dtype, q[sample], n, L, m,
+                                                       threads=oracle.dresd_oracle.default_threads())
+    for k, b in enumerate(sample):
+        cut = np.sort(approx[k])[-m]
+        got = ids[b]
+        assert np.all(approx[k][got] >= cut - 5e-4)
+        safe = np.flatnonzero(approx[k] >= cut + 5e-4)
+        nth = exact[k][got[-1]]
+        assert not [i for i in safe if exact[k][i] > nth + 2e-5 and i not in set(got.tolist())]
