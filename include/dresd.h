@@ -324,6 +324,10 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "profile"    > 0: record a CUDA-event pair around the scoring kernel(s) of
  *                each of the next `value` dresd_retrieve() calls (see
  *                dresd_store_profile_read); 0 = off (default).
+ *   "profile_stride"  k >= 1 (default 1): while "profile" is armed, only every k-th call is
+ *                timed.  The events sit between the kernels of a call and hold up the overlap
+ *                of one kernel's set-up with its predecessor's tail, so a sparse sample
+ *                disturbs a throughput measurement less.
  * Unknown names return DRESD_ERR_INVALID.
  */
 dresd_status dresd_store_set_option(dresd_store *store, const char *name, int value);

@@ -246,6 +246,33 @@ __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map)
 }
 
 // ---------------------------------------------------------------------------
+// Programmatic dependent launch: the kernels of one retrieve call form a chain (K1 -> scan ->
+// merge).  A kernel launched with launch_dependent() may start while its predecessor still
+// runs: it sets up (barriers, TMEM) and then blocks in pdl_wait() until the predecessor has
+// completed and its writes are visible; a kernel calls pdl_launch_dependents() as early as it
+// likes to let its successor be scheduled.  Both are no-ops in a kernel launched the plain way.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args &&...args)
+{
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// ---------------------------------------------------------------------------
 // tcgen05 / TMEM wrappers (5th-generation tensor cores)
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t *smem_dst, uint32_t ncols)

@@ -174,6 +174,7 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
 
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
+    pdl_launch_dependents();              // the scan may set itself up while this kernel runs
     // operand rows of query b: (2b, 2b+1), or -- blocked layout -- rows (b % 8) and 8 + (b % 8)
     // of the 16-row block b / 8, so that a 16-lane TMEM fragment holds hi and lo of 8 queries
     const int row_hi = a.split_blocked ? 16 * (b >> 3) + (b & 7) : 2 * b;

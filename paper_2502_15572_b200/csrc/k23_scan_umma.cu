@@ -157,6 +157,14 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         }
         mbar_fence_init();
     }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    // Everything above is independent of the preceding kernel; what follows reads its output
+    // (the query operand, the reset filter words).
+    pdl_wait();
+    pdl_launch_dependents();
     if (warp >= 2) {
         for (int q = warp - 2; q < NQ; q += kEpiWarps) {
             warp_topn_init(&sel[q], lane);
@@ -167,10 +175,6 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 want_s[q] = (a.first_col && rq < a.B) ? a.want_first[rq] : -1;
             }
         }
-    }
-    if (warp == 1) {
-        tmem_alloc(tmem_slot, kTmemCols);
-        tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
@@ -561,8 +565,7 @@ cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const S
         auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2>;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
         if (e != cudaSuccess) return e;
-        kernel<<<grid, kThreads, p.smem, stream>>>(kmap, qmap, a, p.q_resident, p.gs);
-        return cudaGetLastError();
+        return launch_dependent(kernel, dim3(grid), dim3(kThreads), p.smem, stream, kmap, qmap, a, p.q_resident, p.gs);
     }
 }
 

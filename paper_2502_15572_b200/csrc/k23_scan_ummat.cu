@@ -138,6 +138,13 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
         }
         mbar_fence_init();
     }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    // Everything above is independent of the preceding kernel; what follows reads its output.
+    pdl_wait();
+    pdl_launch_dependents();
     if (warp >= 2) {
         for (int q = warp - 2; q < kNQ; q += kEpiWarps) {
             warp_topn_init(&sel[q], lane);
@@ -148,10 +155,6 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
                 best[q] = 0ull;
             }
         }
-    }
-    if (warp == 1) {
-        tmem_alloc(tmem_slot, kTmemCols);
-        tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
@@ -482,14 +485,13 @@ cudaError_t launch_scan_ummat(const CUtensorMap &kmap, const CUtensorMap &qmap, 
         auto k = scan_ummat_kernel<__half>;
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k<<<grid, kThreads, smem, stream>>>(kmap, qmap, a);
+        return launch_dependent(k, dim3(grid), dim3(kThreads), smem, stream, kmap, qmap, a);
     } else {
         auto k = scan_ummat_kernel<__nv_bfloat16>;
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        k<<<grid, kThreads, smem, stream>>>(kmap, qmap, a);
+        return launch_dependent(k, dim3(grid), dim3(kThreads), smem, stream, kmap, qmap, a);
     }
-    return cudaGetLastError();
 }
 
 }  // namespace dresd

@@ -26,6 +26,8 @@ merge_gather_kernel(const unsigned long long *__restrict__ cand, int lists, int 
     __shared__ int win[kListLen];
     const int b = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_wait();                           // the scan's lists are complete and visible
+    pdl_launch_dependents();
 
     unsigned long long m = 0ull;
     int g = warp;
@@ -97,17 +99,16 @@ cudaError_t launch_merge_gather(const unsigned long long *cand, int lists, int B
                                 float *out_scores, const int32_t *next_tokens, int stored_len, long long N,
                                 int draft_len, int32_t *out_tokens, cudaStream_t stream)
 {
-    merge_gather_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, out_ids, out_scores, nullptr,
-                                                           next_tokens, stored_len, N, draft_len, out_tokens);
-    return cudaGetLastError();
+    return launch_dependent(merge_gather_kernel, dim3(B), dim3(kMergeWarps * 32), 0, stream, cand, lists, B, top_n, out_ids,
+                            out_scores, (unsigned int *)nullptr, next_tokens, stored_len, N, draft_len, out_tokens);
 }
 
 cudaError_t launch_merge_tau(const unsigned long long *cand, int lists, int B, int top_n, unsigned int *gtau,
                              cudaStream_t stream)
 {
-    merge_gather_kernel<<<B, kMergeWarps * 32, 0, stream>>>(cand, lists, B, top_n, nullptr, nullptr, gtau, nullptr, 0,
-                                                           0, 0, nullptr);
-    return cudaGetLastError();
+    return launch_dependent(merge_gather_kernel, dim3(B), dim3(kMergeWarps * 32), 0, stream, cand, lists, B, top_n,
+                            (int32_t *)nullptr, (float *)nullptr, gtau, (const int32_t *)nullptr, 0, 0LL, 0,
+                            (int32_t *)nullptr);
 }
 
 }  // namespace dresd

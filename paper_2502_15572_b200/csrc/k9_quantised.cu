@@ -87,6 +87,8 @@ merge_rerank_kernel(const unsigned long long *__restrict__ cand, int lists, int 
     __shared__ unsigned long long packed[kListLen + 1];
     __shared__ int win[kListLen];
     const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_wait();                           // the scan's lists are complete and visible
+    pdl_launch_dependents();
 
     unsigned long long m = 0ull;
     int g = warp;
@@ -183,16 +185,12 @@ cudaError_t launch_merge_rerank(const unsigned long long *cand, int lists, int B
                                 int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream)
 {
     if (dtype == kF16)
-        merge_rerank_kernel<__half><<<B, kRerankWarps * 32, 0, stream>>>(
-            cand, lists, B, static_cast<const __half *>(keys), d, N, qhat, mcand, top_n, extra_id, want_first, next_tokens,
-            stored_len,
-            draft_len, out_ids, out_scores, out_tokens);
-    else
-        merge_rerank_kernel<__nv_bfloat16><<<B, kRerankWarps * 32, 0, stream>>>(
-            cand, lists, B, static_cast<const __nv_bfloat16 *>(keys), d, N, qhat, mcand, top_n, extra_id, want_first,
-            next_tokens,
-            stored_len, draft_len, out_ids, out_scores, out_tokens);
-    return cudaGetLastError();
+        return launch_dependent(merge_rerank_kernel<__half>, dim3(B), dim3(kRerankWarps * 32), 0, stream, cand, lists, B,
+                                static_cast<const __half *>(keys), d, N, qhat, mcand, top_n, extra_id, want_first,
+                                next_tokens, stored_len, draft_len, out_ids, out_scores, out_tokens);
+    return launch_dependent(merge_rerank_kernel<__nv_bfloat16>, dim3(B), dim3(kRerankWarps * 32), 0, stream, cand, lists,
+                            B, static_cast<const __nv_bfloat16 *>(keys), d, N, qhat, mcand, top_n, extra_id, want_first,
+                            next_tokens, stored_len, draft_len, out_ids, out_scores, out_tokens);
 }
 
 }  // namespace dresd
