@@ -52,7 +52,7 @@ enum {
  *   keys         device, [N][d] row-major in `dtype`; base 16-byte aligned and
  *                d * sizeof(dtype) a multiple of 16 (rows are fetched by TMA).
  *   next_tokens  device, int32 [N][stored_len] row-major.
- *   N            1 .. 2^31-1 rows;  d: 8 .. DRESD_MAX_DIM.
+ *   N            1 .. 2^31-1024 rows (tile coordinates are 32-bit);  d: 8 .. DRESD_MAX_DIM.
  *   stored_len   tokens stored per key (the paper's "next N tokens"), >= 1.
  *   out_store    host pointer receiving the handle.
  *

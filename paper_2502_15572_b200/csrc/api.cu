@@ -410,7 +410,7 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
     *out_store = nullptr;
     if (dtype != DRESD_F32 && dtype != DRESD_F16 && dtype != DRESD_BF16)
         return fail(DRESD_ERR_INVALID, "unknown dtype %d", (int)dtype);
-    if (N <= 0 || N > 2147483647LL) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1", (long long)N);
+    if (N <= 0 || N > kMaxRows) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1024", (long long)N);
     if (d <= 0) return fail(DRESD_ERR_INVALID, "d = %d", d);
     if (stored_len < 1) return fail(DRESD_ERR_INVALID, "stored_len = %d", stored_len);
     const size_t eb = elem_bytes((int)dtype);
@@ -792,7 +792,7 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
 {
     if (dtype != DRESD_F16 && dtype != DRESD_BF16)
         return fail(DRESD_ERR_UNSUPPORTED, "dresd_build_keys builds 16-bit datastores (fp16 or bf16)");
-    if (N <= 0 || N > 2147483647LL) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1", (long long)N);
+    if (N <= 0 || N > kMaxRows) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1024", (long long)N);
     if (d_in < 8 || d_in % 8 != 0) return fail(DRESD_ERR_INVALID, "d_in = %d must be a positive multiple of 8", d_in);
     if (d < 32 || d > 256 || d % 32 != 0) return fail(DRESD_ERR_UNSUPPORTED, "d = %d must be 32..256 in steps of 32", d);
     if (d_in > 16384) return fail(DRESD_ERR_UNSUPPORTED, "d_in = %d exceeds 16384", d_in);
@@ -848,7 +848,7 @@ dresd_status dresd_quantise_keys(const void *keys, int64_t N, int d, dresd_dtype
 {
     if (dtype != DRESD_F16 && dtype != DRESD_BF16)
         return fail(DRESD_ERR_UNSUPPORTED, "dresd_quantise_keys reads 16-bit datastores (fp16 or bf16)");
-    if (N <= 0 || N > 2147483647LL) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1", (long long)N);
+    if (N <= 0 || N > kMaxRows) return fail(DRESD_ERR_INVALID, "N = %lld outside 1..2^31-1024", (long long)N);
     if (d < 16 || d % 16 != 0) return fail(DRESD_ERR_INVALID, "d = %d must be a positive multiple of 16", d);
     if (!is_device_ptr(keys) || !is_device_ptr(out_q8)) return fail(DRESD_ERR_INVALID, "keys / out_q8 must be device pointers");
     if (reinterpret_cast<uintptr_t>(keys) % 16 != 0 || reinterpret_cast<uintptr_t>(out_q8) % 16 != 0)

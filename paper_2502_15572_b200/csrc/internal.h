@@ -12,6 +12,7 @@ enum { kF32 = 0, kF16 = 1, kBF16 = 2, kE4M3 = 3 };   // kE4M3: the 8-bit copy of
 constexpr int kMaxBatch = 64;
 constexpr int kMaxTopN = 32;
 constexpr int kCandStride = 32;          // u64 slots per (CTA, query) in the workspace
+constexpr long long kMaxRows = 2147483647LL - 1023;   // row coordinates of the last (partly filled) tile stay within int32
 constexpr float kHiLoScaleF16 = 2048.f;  // low half of an fp16-split query is stored x 2^11
 constexpr float kHiLoScaleBF16 = 256.f;  // low half of a bf16-split query is stored x 2^8
 

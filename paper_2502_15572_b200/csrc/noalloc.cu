@@ -113,7 +113,7 @@ extern "C" dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *
 {
     if (dtype != DRESD_F32 && dtype != DRESD_F16 && dtype != DRESD_BF16)
         return na_fail(DRESD_ERR_INVALID, "unknown dtype");
-    if (N <= 0 || N > 2147483647LL) return na_fail(DRESD_ERR_INVALID, "N outside 1..2^31-1");
+    if (N <= 0 || N > kMaxRows) return na_fail(DRESD_ERR_INVALID, "N outside 1..2^31-1024");
     if (d <= 0 || stored_len < 1) return na_fail(DRESD_ERR_INVALID, "bad d or stored_len");
     const size_t eb = dtype == DRESD_F32 ? 4 : 2;
     if (((size_t)d * eb) % 16 != 0) return na_fail(DRESD_ERR_INVALID, "row size is not a multiple of 16 bytes");

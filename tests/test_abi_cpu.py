@@ -40,6 +40,7 @@ def test_validation_needs_no_device(lib):
         binding.dresd_store_create(0, 0, 10, 64, binding.DRESD_F16, 4)
     assert e.value.status == -1 and "NULL" in e.value.message
     for kwargs, status in [
+        (dict(N=2 ** 31 - 1023, d=64, dtype=1, stored_len=4), -1),   # last tile's row coordinate would pass 2^31
         (dict(N=0, d=64, dtype=1, stored_len=4), -1),
         (dict(N=2 ** 31, d=64, dtype=1, stored_len=4), -1),
         (dict(N=10, d=12, dtype=1, stored_len=4), -1),        # 24-byte rows
