@@ -61,6 +61,9 @@ def parse_args():
     ap.add_argument("--d-out", type=int, default=256)
     ap.add_argument("--first-token-filter", action="store_true",
                     help="time dresd_retrieve_filtered: each query wants the first stored token of its source row")
+    ap.add_argument("--sorted-store", action="store_true",
+                    help="with --first-token-filter: rows sorted by first stored token and indexed, so that a call "
+                         "scans only the rows of its queries' tokens (same result as the filtered full scan)")
     ap.add_argument("--probe", type=int, default=1, help="probe-pass tile stride (0 off, 1 default)")
     ap.add_argument("--quantised", type=int, default=0, metavar="M",
                     help="candidates by approximate score over an 8-bit (E4M3) copy of the keys, exact re-ranking "
@@ -93,6 +96,8 @@ def workload_config(cfg):
             "key_dtype": cfg["dtype"],
             "batch": cfg["B"], "top_n": cfg["top_n"], "draft_len": cfg["draft_len"],
             "first_token_filter": bool(cfg.get("filter_on", False)),
+            "sorted_by_first_token": "rows_scanned_per_step_mean" in cfg,
+            "rows_scanned_per_step_mean": cfg.get("rows_scanned_per_step_mean"),
             "mixture_components": cfg["C"], "query_noise_sigma": cfg["sigma"], "seed": cfg["seed"],
             "l2": "keys are %.2f GB per step, far larger than the 126 MB L2: no flush needed"
                   % (cfg["N"] * cfg["d"] * synth.DTYPE_BYTES[cfg["dtype"]] / 1e9)}
@@ -115,6 +120,8 @@ def make_inputs(args):
     else:
         q, src = synth.make_queries(cfg["seed"] + 100, keys, cfg["dtype"], nq, cfg["sigma"])
         cfg["first_tokens"] = np.ascontiguousarray(toks[src, 0])      # the token the LLM would have produced
+        if args.sorted_store:
+            keys, toks = synth.sort_by_first_token(keys, toks)
     return cfg, keys, toks, q
 
 
@@ -245,6 +252,8 @@ def run_ours(args):
             raise SystemExit("--first-token-filter needs a workload whose queries have source rows")
         store.enable_first_token_filter()
         dft = torch.from_numpy(cfg["first_tokens"]).cuda()
+        if args.sorted_store:
+            store.index_first_tokens()
     out = (torch.empty((B, n), dtype=torch.int32, device="cuda"),
            torch.empty((B, n), dtype=torch.float32, device="cuda"),
            torch.empty((B, n, L), dtype=torch.int32, device="cuda"))
@@ -342,16 +351,22 @@ def run_ours(args):
             torch.empty((B, n), dtype=torch.float32).pin_memory(),
             torch.empty((B, n, L), dtype=torch.int32).pin_memory())
     dq_stage = dq[:B].clone()
+    hft = None if dft is None else torch.from_numpy(cfg["first_tokens"]).pin_memory()
+    ft_stage = None if dft is None else dft[:B].clone()
 
     def host_call(j):
-        if not args.quantised:
+        if not args.quantised and dft is None:
             store.retrieve_host(hq[j:j + B], n, L, hout)
             return
-        # the quantised call takes device buffers: the same copies, issued here
+        # the quantised and the filtered calls take device buffers: the same copies, issued here
         dq_stage.view(torch.int16 if dtype != "f32" else torch.float32).copy_(
             hq[j:j + B].view(torch.int16 if dtype != "f32" else torch.float32), non_blocking=True)
-        store.retrieve_quantised(dq_stage, n, L, args.quantised, out=out,
-                                 first_tokens=None if dft is None else dft[j:j + B])
+        if dft is not None:
+            ft_stage.copy_(hft[j:j + B], non_blocking=True)
+        if args.quantised:
+            store.retrieve_quantised(dq_stage, n, L, args.quantised, out=out, first_tokens=ft_stage)
+        else:
+            store.retrieve_filtered(dq_stage, ft_stage, n, L, out=out)
         for h, o_ in zip(hout, out):
             h.copy_(o_, non_blocking=True)
         torch.cuda.synchronize()
@@ -379,16 +394,25 @@ def run_ours(args):
     e2e_qps = dist_util.aggregate_throughput(B, args.steps, world, e2e_ms_total)
     eb = synth.DTYPE_BYTES[dtype]
     key_bytes = cfg["N"] * cfg["d"] * (1 if args.quantised else eb)   # algorithmic bytes of one scoring launch
+    if args.sorted_store and dft is not None:
+        # only the rows of the batch's distinct first tokens are scored: mean over the timed steps
+        counts = np.bincount(toks[:, 0])
+        rows = [sum(int(counts[t]) for t in set(cfg["first_tokens"][j:j + B].tolist()))
+                for j in ((q_first + (args.warmup + i) % nq) * B for i in range(args.steps))]
+        cfg["rows_scanned_per_step_mean"] = float(np.mean(rows))
+        key_bytes = cfg["rows_scanned_per_step_mean"] * cfg["d"] * (1 if args.quantised else eb)
     peak, peak_src = peaks()
     achieved = passes * key_bytes / (scan_ms_avg * 1e-3) / 1e9
     line = {
         "metric": metric_name(cfg) + (" -- 8-bit candidates, exact re-rank of %d" % args.quantised
-                                      if args.quantised else ""), "value": qps, "unit": "queries/s", "n_gpus": world,
+                                      if args.quantised else "")
+                  + (" -- rows sorted by first token, only the queries' token windows scanned"
+                     if "rows_scanned_per_step_mean" in cfg else ""), "value": qps, "unit": "queries/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate over %s keys" % dtype,
         "data": "synthetic", "config": workload_config(cfg),
         "e2e": {"value": e2e_qps, "unit": "queries/s",
-                "h2d_bytes_per_step": B * cfg.get("d_in", cfg["d"]) * eb,
+                "h2d_bytes_per_step": B * cfg.get("d_in", cfg["d"]) * eb + (4 * B if dft is not None else 0),
                 "d2h_bytes_per_step": B * n * (8 + 4 * L) + 4},
         "gpu_launches": launches,
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},

@@ -126,8 +126,22 @@ dresd_status dresd_retrieve(dresd_store *store, const void *queries, int B, int 
  *                 that query; NULL disables it for the call.
  * When fewer than top_n keys match, the missing neighbours are reported as
  * id -1, score -infinity, tokens -1.
+ *
+ * dresd_store_index_first_tokens() is for a datastore whose rows the caller has
+ * SORTED by first stored token (non-decreasing next_tokens[.][0]; row order
+ * carries no other meaning, ids are row indices).  It enables the filter if
+ * needed, checks the order on the device and builds a table of every token's
+ * row range (4 bytes x (largest first token + 2)); it synchronises `stream`.
+ * Afterwards a filtered call of the tensor-core path on 16-bit stores (exact or
+ * quantised) in which EVERY query names a token scans only those tokens' rows --
+ * the result is the one the full filtered scan gives, bit for bit, at a fraction
+ * of the bytes; a call with a negative entry in first_tokens scans everything as
+ * before.  Returns DRESD_ERR_INVALID when the rows are not sorted or a stored
+ * first token is negative, DRESD_ERR_UNSUPPORTED for first tokens >= 2^24.
+ * Store option "first_token_windows" = 0 switches the windows off again.
  */
 dresd_status dresd_store_enable_first_token_filter(dresd_store *store, void *stream);
+dresd_status dresd_store_index_first_tokens(dresd_store *store, void *stream);
 dresd_status dresd_retrieve_filtered(dresd_store *store, const void *queries, const int32_t *first_tokens,
                                      int B, int top_n, int draft_len, int32_t *out_ids, float *out_scores,
                                      int32_t *out_tokens, void *stream);

@@ -30,7 +30,7 @@ EXPORTS = (
     "dresd_store_destroy", "dresd_retrieve_noalloc", "dresd_store_enable_first_token_filter",
     "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
     "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore", "dresd_set_global_option", "dresd_quantise_keys", "dresd_store_attach_quantised",
-    "dresd_retrieve_quantised",
+    "dresd_retrieve_quantised", "dresd_store_index_first_tokens",
 )
 
 
@@ -82,6 +82,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_store_destroy.argtypes = [vp]
     lib.dresd_store_enable_first_token_filter.restype = i32
     lib.dresd_store_enable_first_token_filter.argtypes = [vp, vp]
+    lib.dresd_store_index_first_tokens.restype = i32
+    lib.dresd_store_index_first_tokens.argtypes = [vp, vp]
     lib.dresd_retrieve_filtered.restype = i32
     lib.dresd_retrieve_filtered.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_drafts_prepare.restype = i32
@@ -139,6 +141,10 @@ def dresd_retrieve(store: int, queries_ptr: int, B: int, top_n: int, draft_len: 
 
 def dresd_store_enable_first_token_filter(store: int, stream: int = 0) -> None:
     _check(load().dresd_store_enable_first_token_filter(store, stream))
+
+
+def dresd_store_index_first_tokens(store: int, stream: int = 0) -> None:
+    _check(load().dresd_store_index_first_tokens(store, stream))
 
 
 def dresd_retrieve_filtered(store: int, queries_ptr: int, first_tokens_ptr, B: int, top_n: int, draft_len: int,
@@ -314,6 +320,12 @@ class Store:
     def enable_first_token_filter(self, stream=None):
         s = (stream or _torch().cuda.current_stream()).cuda_stream
         dresd_store_enable_first_token_filter(self.handle, s)
+
+    def index_first_tokens(self, stream=None):
+        """For a store whose rows are sorted by first stored token: filtered calls then scan only
+        the rows of the queries' tokens."""
+        s = (stream or _torch().cuda.current_stream()).cuda_stream
+        dresd_store_index_first_tokens(self.handle, s)
 
     def retrieve_filtered(self, queries, first_tokens, top_n: int, draft_len: int, out=None, stream=None):
         """Like retrieve(), restricted per query to keys whose first stored token is first_tokens[b]."""

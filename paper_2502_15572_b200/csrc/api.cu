@@ -65,8 +65,6 @@ EncodeTiledFn encode_tiled_fn()
 
 size_t elem_bytes(int dtype) { return dtype == kF32 ? 4 : 2; }
 
-// 2-D map over a row-major [rows][cols] matrix; box = one 128-byte swizzle row
-// wide, box_rows tall; out-of-range elements read as zero.
 // Device-side address of a page-locked host buffer that the device can reach, else null.
 void *mapped_device_ptr(const void *host)
 {
@@ -78,6 +76,8 @@ void *mapped_device_ptr(const void *host)
     return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
 }
 
+// 2-D map over a row-major [rows][cols] matrix; box = one 128-byte swizzle row
+// wide, box_rows tall; out-of-range elements read as zero.
 bool make_map(CUtensorMap *map, const void *base, int dtype, long long rows, int cols, int box_rows)
 {
     EncodeTiledFn fn = encode_tiled_fn();
@@ -121,6 +121,8 @@ struct dresd_store {
     int *status;                 // device status word
     unsigned int *gtau;          // [kMaxBatch] grid-wide filter words
     int32_t *first_col;          // [N] first stored token of every key; allocated on request
+    int32_t *win_start;          // [win_vocab + 1] rows of every first token (sorted stores); on request
+    int win_vocab, opt_windows;
     int max_grid;
     // staging for dresd_retrieve_host (owned, device)
     void *q_stage;
@@ -137,7 +139,7 @@ struct dresd_store {
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     // options / bookkeeping
     int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m, opt_pack2;
-    double last_key_passes;      // passes over the key matrix in the last call (probe = 1/64)
+    double last_key_passes;      // passes over the key matrix in the last call (a probe pass counts 1/stride)
     const void *k8;              // 8-bit (E4M3) copy of the keys, borrowed; null = none attached
     void *qsplit8;               // [2 * kMaxBatch][dpad8] 8-bit query operand
     int dpad8;                   // d rounded up to 128 bytes
@@ -167,6 +169,7 @@ void free_store(dresd_store *s)
     cudaFree(s->status);
     cudaFree(s->gtau);
     cudaFree(s->first_col);
+    cudaFree(s->win_start);
     cudaFree(s->q_stage);
     cudaFree(s->proj_ws);
     cudaFree(s->qsplit8);
@@ -179,11 +182,21 @@ void free_store(dresd_store *s)
     delete s;
 }
 
+// A store launches on the device it was created on (its workspace and descriptors live there).
+dresd_status check_device(const dresd_store *s)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != s->device)
+        return fail(DRESD_ERR_INVALID, "the store belongs to device %d; the current device is %d", s->device, dev);
+    return DRESD_OK;
+}
+
 dresd_status check_retrieve_args(const dresd_store *s, const void *queries, int B, int top_n,
                                  int draft_len, const void *ids, const void *scores,
                                  const void *tokens, bool device_ptrs)
 {
     if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+    if (dresd_status ds = check_device(s)) return ds;
     if (B < 0) return fail(DRESD_ERR_INVALID, "B = %d is negative", B);
     if (top_n < 1 || top_n > s->N) return fail(DRESD_ERR_INVALID, "top_n = %d outside 1..N", top_n);
     if (draft_len < 1 || draft_len > s->stored_len)
@@ -256,8 +269,11 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // streaming kernel stays available as "scan_path" 1 and serves the allocation-free call.
     const bool umma = q8 || (!f32 && s->opt_path != 1);
     const int op_rows = umma ? scan_umma_operand_rows(pack2 ? 2 * B : B) : 0;
+    // sorted store with an index: the kernel with the keys as M scans the queries' token windows only
+    const bool windows = umma && first_tokens && s->win_start && s->opt_windows;
+    const int keys_as_m = (q8 || s->opt_keys_as_m || windows) ? 1 : 0;
     // the kernel with the keys as the N operand reads hi and lo of a query from one TMEM fragment
-    const int blocked = umma && !q8 && !s->opt_keys_as_m && scan_ummat_eligible(s->d, B);
+    const int blocked = umma && !keys_as_m && scan_ummat_eligible(s->d, B);
     // one CTA per operand query: two operand rows each, four in the packed 8-bit layout
     const int pre_rows = pack2 ? op_rows / 4 : umma ? op_rows / 2 : ((B + 7) / 8) * 8;
     dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, blocked, pack2 ? 2 : q8 ? 1 : 0);
@@ -266,7 +282,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // the 8-bit store is scanned as rows of d/2 two-byte units (packed: N/2 rows of 64 units)
     const int scan_d = pack2 ? 64 : q8 ? s->d / 2 : s->d;
     const long long scan_rows = pack2 ? s->N / 2 : s->N;
-    const int umma_rows = umma ? scan_umma_tile_rows(scan_d, pack2 ? 2 * B : B, q8 ? 1 : s->opt_keys_as_m) : 1;
+    const int umma_rows = umma ? scan_umma_tile_rows(scan_d, pack2 ? 2 * B : B, keys_as_m) : 1;
     const int n_tiles = umma ? (int)((scan_rows + umma_rows - 1) / umma_rows) : s->n_tiles;
     int grid = s->opt_grid > 0 ? s->opt_grid : s->num_sms;
     if (grid > s->max_grid) grid = s->max_grid;
@@ -294,7 +310,11 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.status = s->status;
         a.gtau = s->gtau;
         a.no_select = s->opt_no_select;
-        a.keys_as_m = q8 ? 1 : s->opt_keys_as_m;
+        a.keys_as_m = keys_as_m;
+        if (windows) {
+            a.win_start = s->win_start;
+            a.win_vocab = s->win_vocab;
+        }
         const CUtensorMap &kmap = pack2 ? s->map_k8p : q8 ? s->map_k8 : s->map_umma;
         const CUtensorMap *qmaps = q8 ? s->map_q8 : s->map_q;
         const int sel_n = a.top_n;
@@ -302,9 +322,9 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.want_first = first_tokens;
         const int mi = op_rows == 16 ? 0 : op_rows == 32 ? 1 : op_rows == 64 ? 2 : 3;
         cudaError_t e = cudaSuccess;
-        // Large batches on large stores: a probe pass over every 64th tile first.  Its
+        // Large batches on large stores: a probe pass over every pstride-th tile first.  Its
         // n-th best score per query seeds the grid-wide filter, so that the full pass
-        // queues ~64 n survivors per query GPU-wide instead of ~n ln(rows/n) per CTA.
+        // queues ~pstride n survivors per query GPU-wide instead of ~n ln(rows/n) per CTA.
         // The filter only rejects rows that cannot be in the result.
         const int pstride = s->opt_probe;
         if (pstride > 1 && !s->opt_no_select && B * sel_n >= 256 && n_tiles >= pstride * grid) {
@@ -448,6 +468,7 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
     s->max_grid = 2 * s->num_sms;
     s->opt_probe = kProbeStride;
     s->opt_pack2 = 1;
+    s->opt_windows = 1;
 
     s->tile_rows = dtype == DRESD_F32 ? scan_f32_tile_rows(d) : scan_mma_tile_rows(d);
     s->n_tiles = (int)((N + s->tile_rows - 1) / s->tile_rows);
@@ -588,6 +609,7 @@ dresd_status dresd_store_enable_first_token_filter(dresd_store *s, void *stream_
 {
     if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
     if (s->first_col) return DRESD_OK;
+    if (dresd_status ds = check_device(s)) return ds;
     int32_t *col = nullptr;
     if (cudaMalloc(&col, sizeof(int32_t) * (size_t)s->N) != cudaSuccess) {
         cudaGetLastError();
@@ -599,6 +621,48 @@ dresd_status dresd_store_enable_first_token_filter(dresd_store *s, void *stream_
         return fail_cuda(e, "first-token column launch");
     }
     s->first_col = col;
+    return DRESD_OK;
+}
+
+dresd_status dresd_store_index_first_tokens(dresd_store *s, void *stream_v)
+{
+    if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+    if (s->win_start) return DRESD_OK;
+    dresd_status st = dresd_store_enable_first_token_filter(s, stream_v);
+    if (st != DRESD_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    // sortedness and the largest token, through the status word's neighbour: a set-up call may synchronise
+    int *flag = nullptr;
+    if (cudaMalloc(&flag, sizeof(int)) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(DRESD_ERR_ALLOC, "allocation failed");
+    }
+    int word = 0, last = 0;
+    cudaError_t e = cudaMemsetAsync(flag, 0, sizeof(int), stream);
+    if (e == cudaSuccess) e = launch_check_sorted(s->first_col, s->N, flag, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&word, flag, sizeof(int), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(&last, s->first_col + (s->N - 1), sizeof(int), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    cudaFree(flag);
+    if (e != cudaSuccess) return fail_cuda(e, "first-token order check");
+    if (word & 2) return fail(DRESD_ERR_INVALID, "a stored first token is negative");
+    if (word & 1) return fail(DRESD_ERR_INVALID, "the rows are not sorted by first stored token");
+    if (last >= (1 << 24)) return fail(DRESD_ERR_UNSUPPORTED, "largest first token %d exceeds 2^24 - 1", last);
+    const int vocab = last + 1;
+    int32_t *ws = nullptr;
+    if (cudaMalloc(&ws, sizeof(int32_t) * ((size_t)vocab + 1)) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(DRESD_ERR_ALLOC, "allocation of the window table (%d entries) failed", vocab + 1);
+    }
+    e = launch_build_windows(s->first_col, s->N, vocab, ws, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) {
+        cudaFree(ws);
+        return fail_cuda(e, "window table launch");
+    }
+    s->win_start = ws;
+    s->win_vocab = vocab;
     return DRESD_OK;
 }
 
@@ -624,6 +688,7 @@ dresd_status dresd_preprocess(dresd_store *s, const void *queries, int B, float 
     if (B < 0) return fail(DRESD_ERR_INVALID, "B = %d is negative", B);
     if (B > DRESD_MAX_BATCH) return fail(DRESD_ERR_UNSUPPORTED, "B = %d exceeds DRESD_MAX_BATCH", B);
     if (B == 0) return DRESD_OK;
+    if (dresd_status ds = check_device(s)) return ds;
     if (!is_device_ptr(queries) || !is_device_ptr(out_qhat))
         return fail(DRESD_ERR_INVALID, "queries/out_qhat must be device pointers");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
@@ -677,6 +742,11 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
     if (strcmp(name, "pack2") == 0) {
         if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "pack2 takes 0 or 1");
         s->opt_pack2 = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "first_token_windows") == 0) {
+        if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "first_token_windows takes 0 or 1");
+        s->opt_windows = value;
         return DRESD_OK;
     }
     if (strcmp(name, "keys_as_m") == 0) {
@@ -869,6 +939,7 @@ dresd_status dresd_store_attach_quantised(dresd_store *s, const void *keys_q8)
     if (s->d > 2048) return fail(DRESD_ERR_UNSUPPORTED, "d = %d exceeds 2048 for the 8-bit copy", s->d);
     if (!is_device_ptr(keys_q8) || reinterpret_cast<uintptr_t>(keys_q8) % 16 != 0)
         return fail(DRESD_ERR_INVALID, "keys_q8 must be a 16-byte aligned device pointer");
+    s->k8 = nullptr;                  // a failed attach leaves no copy attached
     if (!s->qsplit8) {
         s->dpad8 = (s->d + 127) / 128 * 128;
         if (cudaMalloc(&s->qsplit8, (size_t)2 * kMaxBatch * s->dpad8) != cudaSuccess) {

@@ -64,6 +64,11 @@ struct ScanArgs {
     // with first_col[row] == want_first[q]; want_first[q] < 0 disables it for that query.
     const int32_t *first_col;   // [N] first stored token of every key (compact copy)
     const int32_t *want_first;  // [B] of this launch
+    // Store sorted by first token (tcgen05 kernel with the keys as M): win_start[t] .. win_start[t+1]
+    // are the rows whose first token is t, t < win_vocab.  When every query of the launch names a
+    // token, only those windows are scanned; the result is that of the filtered full scan.
+    const int32_t *win_start;   // [win_vocab + 1], null = always scan everything
+    int win_vocab;
     int stages;             // pipeline depth
     long long wait_cycles;  // bound of every device-side wait in cycles, 0 = default (~2 s)
     int debug_lose_stage;   // test hook (streaming kernel): CTA 0 never receives stage (value-1); 0 = off
@@ -111,6 +116,13 @@ cudaError_t launch_merge_tau(const unsigned long long *cand, int grid_lists, int
 // first_col[i] = next_tokens[i][0]: the compact column the first-token filter reads.
 cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, long long N,
                                  int32_t *first_col, cudaStream_t stream);
+
+// Index of a store whose rows are sorted by first token.  check: *flag gets bit 0 when
+// first_col is not non-decreasing, bit 1 when it holds a negative token.  build:
+// win_start[t] = first row with first token >= t for t = 0 .. vocab (vocab = last token + 1).
+cudaError_t launch_check_sorted(const int32_t *first_col, long long N, int *flag, cudaStream_t stream);
+cudaError_t launch_build_windows(const int32_t *first_col, long long N, int vocab, int32_t *win_start,
+                                 cudaStream_t stream);
 
 // ---- K6: draft matrix preparation and longest-match acceptance (Section 3.6) ----
 cudaError_t launch_drafts_prepare(const int32_t *tokens, const int32_t *ids, int B, int n, int L, int eos,

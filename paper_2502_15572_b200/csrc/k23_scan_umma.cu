@@ -94,6 +94,19 @@ struct EpiFlags {
     int overflow;
 };
 
+// First-token windows of a filtered launch over a store sorted by first token (Section 3.5:
+// only keys whose value starts with x_{t+1} can be drafted).  Entry b belongs to query b; it
+// has tiles only when b is the first query that names its token, so that every window is
+// scanned once.  lo/hi are key indices, tile0 the window's first tile, prefix the running
+// tile count: CTA c takes the tiles c, c + G, ... of the concatenated windows.
+struct Windows {
+    int on;                          // 0: scan the whole store (a query without a token, or no index)
+    int total;
+    int tile0[kMaxBatch], lo[kMaxBatch], hi[kMaxBatch];
+    int prefix[kMaxBatch + 1];
+    unsigned long long qmask[kMaxBatch];   // operand column pairs (queries) that name the window's token
+};
+
 // PACK2 (8-bit keys of 64 elements): a 128-byte row of the store holds TWO keys.  Query j then
 // owns four operand rows -- (h1|0), (h2|0), (0|h1), (0|h2) -- i.e. two "virtual" queries 2j, 2j+1
 // that score the even and the odd key of a row; both feed the lists and the filter of query j,
@@ -134,11 +147,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     uint64_t *qbar = tempty + 2;                            // resident query operand landed
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(qbar + 1);
     EpiFlags *flags = reinterpret_cast<EpiFlags *>(tmem_slot + 2);
+    Windows *win = reinterpret_cast<Windows *>(flags + 3);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
-    const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
-    const int n_it = my_tiles * gpt;
     constexpr int kRowsPerTile = kTileRows * TSUB;
 
     if (tid == 0) {
@@ -176,10 +188,56 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             }
         }
     }
+    // Sorted store and a token for every query: scan those tokens' windows only.
+    const bool windowed = a.win_start != nullptr && a.first_col != nullptr && a.tile_stride == 1 && !a.probe_max;
+    if (windowed) {
+        if (tid < kMaxBatch) {
+            int t0 = 0, nt = 0, lo = 0, hi = 0;
+            unsigned long long qm = 0ull;
+            if (tid < a.B) {
+                const int tok = a.want_first[tid];
+                bool owner = tok >= 0 && tok < a.win_vocab;          // no row holds a token >= win_vocab
+                for (int b = 0; b < tid && owner; ++b) owner = a.want_first[b] != tok;
+                if (owner) {
+                    lo = a.win_start[tok];
+                    hi = a.win_start[tok + 1];
+                    if (hi > lo) {
+                        constexpr int kKeysPerTile = PACK2 ? 2 * kRowsPerTile : kRowsPerTile;
+                        t0 = lo / kKeysPerTile;
+                        nt = (hi - 1) / kKeysPerTile - t0 + 1;
+                        // every key of the window starts with `tok`: the token test is this constant mask
+                        for (int q = tid; q < a.B; ++q)
+                            if (a.want_first[q] == tok) qm |= PACK2 ? 3ull << (2 * q) : 1ull << q;
+                    }
+                }
+            }
+            win->tile0[tid] = t0;
+            win->lo[tid] = lo;
+            win->hi[tid] = hi;
+            win->qmask[tid] = qm;
+            win->prefix[tid + 1] = nt;                               // counts; summed below
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int sum = 0, wild = 0;
+            win->prefix[0] = 0;
+            for (int b = 0; b < a.B; ++b) {                          // entries beyond B are never looked at
+                sum += win->prefix[b + 1];
+                win->prefix[b + 1] = sum;
+                if (a.want_first[b] < 0) wild = 1;                   // that query needs every row
+            }
+            win->total = sum;
+            win->on = !wild;
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const bool win_on = windowed && win->on;
+    const int n_tiles = win_on ? win->total : a.n_tiles;
+    const int my_tiles = cta < n_tiles ? (n_tiles - cta + G - 1) / G : 0;
+    const int n_it = my_tiles * gpt;
 
     if (warp == 0) {
         // ---------------------------------- producer ----------------------------------
@@ -191,14 +249,18 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 for (int s = 0; s < dslabs; ++s)
                     tma_load_2d(qres + (size_t)s * kQSlabBytes, &q_map, s * kSlabElems, 0, qbar);
             }
-            int issued = 0;
+            int issued = 0, wk = 0;
             for (int it = 0; it < n_it; ++it) {
                 const int s = it % n_stages;
                 if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
                     report_timeout(a.status);
                     break;
                 }
-                const int tile = (cta + (it / gpt) * G) * a.tile_stride;
+                int tile = (cta + (it / gpt) * G) * a.tile_stride;
+                if (win_on) {                                    // tile of the concatenated windows -> tile of the store
+                    while (win->prefix[wk + 1] <= tile) ++wk;
+                    tile = win->tile0[wk] + (tile - win->prefix[wk]);
+                }
                 uint8_t *dst = stages + (size_t)s * stage_bytes;
                 if constexpr (TSUB > 1) {
                     // narrow rows: every slab of every sub-tile (rows past N read as zeros)
@@ -300,7 +362,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         const float inv = a.lo_inv_scale;
         const float4 *tau4 = reinterpret_cast<const float4 *>(tau + qbase);
         const int4 *want4 = reinterpret_cast<const int4 *>(want_s + qbase);
-        const bool filtered = a.first_col != nullptr;
+        const bool filtered = a.first_col != nullptr && !win_on;    // windows carry their token
+        uint32_t wmatch = 0xFFFFFFFFu;                      // this warp's queries that the tile's window serves
         uint32_t wild = 0u;                                 // this warp's queries without a token filter
         for (int j = 0; j < QW; ++j) wild |= (want_s[qbase + j] < 0) ? (1u << j) : 0u;
         // A warp whose wait expired goes "dead": it does no more work and no more
@@ -308,10 +371,19 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         bool dead = false;
         int round = 0;                                      // barrier-A count: selects the flag slot
         EpiFlags *fl = &flags[0];
+        int wk = 0;
         for (int tl = 0; tl < my_tiles; ++tl) {
             const int acc = tl & 1, use = tl >> 1;
-            const long long row0 =
-                (long long)(cta + tl * G) * a.tile_stride * kRowsPerTile + lane_grp * 32 + lane;
+            long long tile = (long long)(cta + tl * G) * a.tile_stride;
+            long long klo = 0, khi = PACK2 ? 2 * a.N : a.N;  // keys of this tile that count
+            if (win_on) {
+                while (win->prefix[wk + 1] <= tile) ++wk;
+                tile = win->tile0[wk] + (tile - win->prefix[wk]);
+                klo = win->lo[wk];
+                khi = win->hi[wk];
+                wmatch = (uint32_t)(win->qmask[wk] >> qbase);
+            }
+            const long long row0 = tile * kRowsPerTile + lane_grp * 32 + lane;
             // first stored token of this thread's rows (filtered calls), requested before the wait
             // (PACK2: of the row's two keys -- first_col is indexed by key, two per row)
             int tok[TSUB], tok1[TSUB];
@@ -398,7 +470,12 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
 #pragma unroll
                 for (int sub = 0; sub < TSUB; ++sub) {
                     const long long row = row0 + sub * kTileRows;
-                    const bool row_ok = !dead && row < a.N;
+                    uint32_t okmask;                        // columns whose key lies in the window (or the store)
+                    if constexpr (PACK2)
+                        okmask = ((2 * row >= klo && 2 * row < khi) ? 0x55555555u : 0u) |
+                                 ((2 * row + 1 >= klo && 2 * row + 1 < khi) ? 0xAAAAAAAAu : 0u);
+                    else
+                        okmask = (row >= klo && row < khi) ? 0xFFFFFFFFu : 0u;
                     // warp-uniform decision: tcgen05.ld needs the whole warp
                     if (dead || !(first || __any_sync(0xFFFFFFFFu, pending[sub] != 0u))) continue;
                     uint32_t r[CW];
@@ -430,7 +507,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         }
                         mask &= match;
                     }
-                    mask &= first ? (row_ok ? 0xFFFFFFFFu : 0u) : pending[sub];
+                    mask &= first ? (okmask & wmatch) : pending[sub];
                     pending[sub] = 0u;
                     // Cold part (rare once the filter is warm), kept out of the hot code:
                     // a warp-uniform loop over the queries that have a survivor in some
@@ -533,7 +610,7 @@ Plan make_plan(int d, int B)
     p.q_resident = qbytes <= (size_t)kResidentLimit;
     const size_t fixed = 1024 + (p.q_resident ? qbytes : 0) + sizeof(WarpTopN) * (p.ncols / 2) +
                          (sizeof(float) + sizeof(int) + 4 * p.tsub * sizeof(unsigned long long)) * (p.ncols / 2) +
-                         sizeof(uint64_t) * (2 * kMaxStages + 5) + 64;
+                         sizeof(uint64_t) * (2 * kMaxStages + 5) + 64 + sizeof(Windows);
     const size_t slab = kKeyStageBytes + (p.q_resident ? 0 : (size_t)p.ncols * kSlabBytes);
     if (p.tsub > 1) {
         p.gs = p.tsub * dslabs;

@@ -83,7 +83,54 @@ __global__ void extract_first_kernel(const int32_t *__restrict__ next_tokens, in
         first_col[i] = next_tokens[i * stored_len];
 }
 
+// Index of a store sorted by first token (Section 3.5: only keys whose value starts with
+// x_{t+1} can be drafted, so a sorted store needs to be scanned over that token's rows only).
+__global__ void check_sorted_kernel(const int32_t *__restrict__ first_col, long long N, int *flag)
+{
+    int bad = 0;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < N;
+         i += (long long)gridDim.x * blockDim.x) {
+        const int cur = first_col[i];
+        if (cur < 0) bad |= 2;
+        if (i > 0 && first_col[i - 1] > cur) bad |= 1;
+    }
+    if (bad) atomicOr(flag, bad);
+}
+
+// Row i opens the windows of every token in (first_col[i-1], first_col[i]]: tokens without
+// rows get an empty window at the next present token's first row.  Sorted input only.
+__global__ void build_windows_kernel(const int32_t *__restrict__ first_col, long long N, int vocab,
+                                     int32_t *__restrict__ win_start)
+{
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i <= N;
+         i += (long long)gridDim.x * blockDim.x) {
+        if (i == N) {
+            win_start[vocab] = (int32_t)N;
+            continue;
+        }
+        const int prev = i > 0 ? first_col[i - 1] : -1, cur = first_col[i];
+        for (int t = prev + 1; t <= cur && t < vocab; ++t) win_start[t] = (int32_t)i;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_check_sorted(const int32_t *first_col, long long N, int *flag, cudaStream_t stream)
+{
+    long long blocks = (N + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    check_sorted_kernel<<<(int)blocks, 256, 0, stream>>>(first_col, N, flag);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_build_windows(const int32_t *first_col, long long N, int vocab, int32_t *win_start,
+                                 cudaStream_t stream)
+{
+    long long blocks = (N + 1 + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    build_windows_kernel<<<(int)blocks, 256, 0, stream>>>(first_col, N, vocab, win_start);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, long long N, int32_t *first_col,
                                  cudaStream_t stream)

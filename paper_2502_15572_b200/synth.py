@@ -155,6 +155,13 @@ def make_store(seed: int, N: int, d: int, C: int, dtype: str, stored_len: int,
     return keys, toks
 
 
+def sort_by_first_token(keys: np.ndarray, toks: np.ndarray):
+    """The same datastore with its rows in order of first stored token (stable): the layout
+    dresd_store_index_first_tokens() asks for.  A permutation only."""
+    order = np.argsort(toks[:, 0], kind="stable")
+    return np.ascontiguousarray(keys[order]), np.ascontiguousarray(toks[order])
+
+
 def make_queries(seed: int, keys: np.ndarray, dtype: str, B: int, sigma: float):
     """Queries drawn near datastore keys.  Returns ``(queries, source_rows)``.
 

@@ -132,3 +132,53 @@ def test_config2_quantised_full_size():
         safe = np.flatnonzero(approx[k] >= cut + 5e-4)
         nth = exact[k][got[-1]]
         assert not [i for i in safe if exact[k][i] > nth + 2e-5 and i not in set(got.tolist())]
+
+
+def test_paper_shaped_sorted_store_full_size():
+    """46.3M x 64 fp16 with its rows sorted by first stored token, as
+    `bench.py --workload paper_46m_d64_f16 --first-token-filter --sorted-store` issues them:
+    24 single-query calls and 2 calls of 16, each scanning only its tokens' rows.  Every call
+    must equal the filtered scan of the whole store bit for bit; all rows carry the wanted
+    token, distinct, scores in order and equal to the oracle's score of the row, tokens the
+    stored ones; 2 queries element by element against the oracle's filtered search."""
+    import torch
+    w = synth.make_workload("paper_46m_d64_f16")
+    dtype, n, L = "f16", w["top_n"], w["draft_len"]
+    q, src = synth.make_queries(w["seed"] + 300, w["keys"], dtype, 56, w["sigma"])
+    ft = np.ascontiguousarray(w["next_tokens"][src, 0]).astype(np.int32)
+    keys, toks = synth.sort_by_first_token(w["keys"], w["next_tokens"])
+    del w
+    st = gpu_store(keys, toks, dtype)
+    try:
+        st.index_first_tokens()
+        dq, dft = binding.to_device(q, dtype), torch.from_numpy(ft).cuda()
+        calls = [(j, j + 1) for j in range(24)] + [(24, 40), (40, 56)]
+        outs = []
+        for a, b in calls:
+            st.set_option("first_token_windows", 1)
+            win = [t.clone() for t in st.retrieve_filtered(dq[a:b], dft[a:b], n, L)]
+            st.set_option("first_token_windows", 0)
+            full = st.retrieve_filtered(dq[a:b], dft[a:b], n, L)
+            torch.cuda.synchronize()
+            for x, y in zip(win, full):
+                assert torch.equal(x, y)
+            outs.append([t.cpu().numpy() for t in win])
+        st.status()
+    finally:
+        st.close()
+    ids = np.concatenate([o[0] for o in outs])
+    sc = np.concatenate([o[1] for o in outs])
+    tok = np.concatenate([o[2] for o in outs])
+    qh = oracle.preprocess(q, dtype)
+    for b in range(q.shape[0]):
+        k = int(np.sum(ids[b] >= 0))
+        assert k == min(n, int(np.sum(toks[:, 0] == ft[b]))) and np.all(ids[b, k:] == -1)
+        got = ids[b, :k]
+        assert len(set(got.tolist())) == k and np.all(toks[got, 0] == ft[b])
+        assert np.all(np.diff(sc[b, :k]) <= 0) and np.array_equal(tok[b, :k], toks[got][:, :L])
+        assert np.max(np.abs(_row_scores(keys, dtype, qh[b], got) - sc[b, :k])) <= checker.TOL[dtype]
+    sample = [3, 30]
+    o = oracle.retrieve(keys, toks, dtype, q[sample], n, L, first_token=ft[sample], want_full_scores=True,
+                        threads=oracle.dresd_oracle.default_threads())
+    for k, b in enumerate(sample):
+        checker.check_query_filtered(o.full_scores[k], toks, ids[b], sc[b], tok[b], dtype, n, L, int(ft[b]))
