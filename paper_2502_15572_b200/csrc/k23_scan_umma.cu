@@ -87,6 +87,13 @@ template <int C, int O> struct WarpColumnMax {
         }
     }
 };
+// *p = max(*p, v) for floats shared by several warps (no NaN): non-negative floats order like
+// signed integers, negative ones inversely like unsigned integers.
+__device__ __forceinline__ void raise_float(float *p, float v)
+{
+    if (v >= 0.f) atomicMax(reinterpret_cast<int *>(p), __float_as_int(v));
+    else atomicMin(reinterpret_cast<unsigned int *>(p), __float_as_uint(v));
+}
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory"); }
 
 struct EpiFlags {
@@ -371,7 +378,16 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         bool dead = false;
         int round = 0;                                      // barrier-A count: selects the flag slot
         EpiFlags *fl = &flags[0];
-        int wk = 0;
+        // Cold start.  While a query has no filter score, every row is a candidate and the 32-entry
+        // queues overflow round after round (a 512-row tile: 16 rounds of barriers and merges, ~4 us).
+        // So on the first tile of a scan, and of every window, the tile is cut into 32 groups of rows
+        // per query; the n-th largest of the 32 group maxima is reached by n rows of the tile (one per
+        // group), hence by the final n-th best too, and becomes the filter score before the tile is
+        // scored in earnest: about n rows then pass, one merge instead of sixteen.
+        uint32_t active = 0u;                               // this warp's column pairs that belong to real queries
+        for (int j = 0; j < QW; ++j)
+            if ((PACK2 ? (qbase + j) >> 1 : qbase + j) < a.B && !a.no_select) active |= 1u << j;
+        int wk = 0, wk_seen = -1;
         for (int tl = 0; tl < my_tiles; ++tl) {
             const int acc = tl & 1, use = tl >> 1;
             long long tile = (long long)(cta + tl * G) * a.tile_stride;
@@ -383,6 +399,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 khi = win->hi[wk];
                 wmatch = (uint32_t)(win->qmask[wk] >> qbase);
             }
+            const bool cold_tile = !a.no_select && !a.probe_max && (tl == 0 || wk != wk_seen);   // same in all warps
+            wk_seen = wk;
             const long long row0 = tile * kRowsPerTile + lane_grp * 32 + lane;
             // first stored token of this thread's rows (filtered calls), requested before the wait
             // (PACK2: of the row's two keys -- first_col is indexed by key, two per row)
@@ -462,6 +480,69 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 if (lane == 0) mbar_arrive(&tempty[acc]);
                 continue;
             }
+            auto okmask_of = [&](long long row) -> uint32_t {   // columns whose key lies in the window (or the store)
+                if constexpr (PACK2)
+                    return ((2 * row >= klo && 2 * row < khi) ? 0x55555555u : 0u) |
+                           ((2 * row + 1 >= klo && 2 * row + 1 < khi) ? 0xAAAAAAAAu : 0u);
+                else
+                    return (row >= klo && row < khi) ? 0xFFFFFFFFu : 0u;
+            };
+            if (cold_tile) {
+                constexpr int kGroupRows = 4 * TSUB;        // 32 groups over the tile's 128 * TSUB rows
+                constexpr int kGroupsPerUnit = 32 / kGroupRows;
+                epi_bar();                                  // tau[] is settled: every warp sees the same cold queries
+                uint32_t todo = 0u;
+                for (uint32_t m = active & wmatch; m; m &= m - 1) {
+                    const int j = __ffs(m) - 1;
+                    if (!(tau[qbase + j] > -INFINITY)) todo |= 1u << j;
+                }
+#pragma unroll
+                for (int sub = 0; sub < TSUB; ++sub) {
+                    const uint32_t ok = okmask_of(row0 + sub * kTileRows);
+                    const int slot = (sub * 4 + lane_grp) * kGroupsPerUnit + lane / kGroupRows;
+                    for (uint32_t m = todo; m; m &= m - 1) {            // warp-uniform
+                        const int j = __ffs(m) - 1;
+                        uint32_t key = 0u;
+                        if (!dead) {
+                            uint32_t v0, v1;
+                            tmem_ld2(acc_addr + (uint32_t)(sub * NCOLS + 2 * j), v0, v1);
+                            tmem_ld_wait();
+                            const float sc = fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
+                            bool valid = ((ok >> j) & 1u) && sc > -INFINITY;            // false for NaN
+                            if (filtered) {
+                                const int w = want_s[qbase + j];
+                                const int tkj = (PACK2 && (j & 1)) ? tok1[sub] : tok[sub];
+                                valid = valid && (w < 0 || tkj == w);
+                            }
+                            key = valid ? float_to_ordered(sc + 0.0f) : 0u;
+                            const uint32_t grp = ((1u << kGroupRows) - 1u) << (lane & ~(kGroupRows - 1));
+                            key = __reduce_max_sync(grp, key);
+                        }
+                        // the queue is empty on a cold tile: its first 128 bytes take the group maxima
+                        if (lane % kGroupRows == 0) reinterpret_cast<uint32_t *>(sel[qbase + j].queue)[slot] = key;
+                    }
+                }
+                epi_bar();
+                const unsigned long long wq = win_on ? win->qmask[wk] : ~0ull;
+                for (int q = ew; q < NQ; q += kEpiWarps) {
+                    const int rq = PACK2 ? q >> 1 : q;
+                    if (rq >= a.B || !((wq >> q) & 1ull) || tau[q] > -INFINITY) continue;   // warp-uniform
+                    unsigned long long x = reinterpret_cast<const uint32_t *>(sel[q].queue)[lane];
+                    __syncwarp();
+                    x = warp_sort_desc(x, lane);
+                    const uint32_t nth = (uint32_t)shfl_u64(x, a.top_n - 1);
+                    if (lane == 0 && nth) {
+                        const float t = share_tau(&a.gtau[rq], ordered_to_float(nth));
+                        if constexpr (PACK2) {               // the even and the odd keys feed one query
+                            raise_float(&tau[2 * rq], t);
+                            raise_float(&tau[2 * rq + 1], t);
+                        } else {
+                            tau[q] = t;
+                        }
+                    }
+                }
+                epi_bar();
+            }
             uint32_t pending[TSUB];                         // queries whose candidate found the queue full
 #pragma unroll
             for (int sub = 0; sub < TSUB; ++sub) pending[sub] = 0u;
@@ -470,12 +551,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
 #pragma unroll
                 for (int sub = 0; sub < TSUB; ++sub) {
                     const long long row = row0 + sub * kTileRows;
-                    uint32_t okmask;                        // columns whose key lies in the window (or the store)
-                    if constexpr (PACK2)
-                        okmask = ((2 * row >= klo && 2 * row < khi) ? 0x55555555u : 0u) |
-                                 ((2 * row + 1 >= klo && 2 * row + 1 < khi) ? 0xAAAAAAAAu : 0u);
-                    else
-                        okmask = (row >= klo && row < khi) ? 0xFFFFFFFFu : 0u;
+                    const uint32_t okmask = okmask_of(row);
                     // warp-uniform decision: tcgen05.ld needs the whole warp
                     if (dead || !(first || __any_sync(0xFFFFFFFFu, pending[sub] != 0u))) continue;
                     uint32_t r[CW];

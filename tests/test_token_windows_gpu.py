@@ -133,3 +133,30 @@ def test_quantised_search_over_windows_equals_the_full_filtered_search(dtype, d,
         rows = np.flatnonzero(toks[:, 0] == ft[b])
         k = min(n, len(rows))
         assert np.all(np.isin(ids[b, :k], rows)) and np.all(ids[b, k:] == -1)
+
+
+def test_calls_whose_windows_are_empty_or_shared():
+    """No row at all for the call's tokens (no CTA has a tile), and all queries naming one token."""
+    import torch
+    keys, toks = _sorted_store(9980, 20011, 64, "f16", 3, 30, missing=5)
+    st = gpu_store(keys, toks, "f16")
+    try:
+        st.index_first_tokens()
+        q = binding.to_device(keys[:4], "f16")
+        for ft in ([5], [1000], [5, 1000, 5, 31]):
+            d = torch.tensor(ft, dtype=torch.int32, device="cuda")
+            ids, sc, tok = st.retrieve_filtered(q[:len(ft)], d, 4, 3)
+            torch.cuda.synchronize()
+            assert torch.all(ids == -1) and torch.all(torch.isinf(sc)) and torch.all(tok == -1)
+        t0 = int(toks[0, 0])
+        d = torch.full((4,), t0, dtype=torch.int32, device="cuda")
+        ids, _, _ = st.retrieve_filtered(q, d, 4, 3)
+        torch.cuda.synchronize()
+        ids = ids.cpu().numpy()
+        rows = np.flatnonzero(toks[:, 0] == t0)
+        assert np.all(np.isin(ids, rows))
+        for b in range(4):                            # rows 0..3 start with t0 (sorted): each query finds its own key
+            assert np.array_equal(keys[ids[b, 0]], keys[b]) or toks[b, 0] != t0
+        st.status()
+    finally:
+        st.close()
