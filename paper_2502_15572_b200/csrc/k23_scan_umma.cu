@@ -161,6 +161,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     constexpr int kRowsPerTile = kTileRows * TSUB;
 
     if (tid == 0) {
+        tma_prefetch_desc(&keys_map);                       // kernel parameters: nothing to wait for
+        tma_prefetch_desc(&q_map);
         for (int s = 0; s < n_stages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
@@ -249,8 +251,6 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     if (warp == 0) {
         // ---------------------------------- producer ----------------------------------
         if (lane == 0) {
-            tma_prefetch_desc(&keys_map);
-            tma_prefetch_desc(&q_map);
             if (q_resident) {
                 mbar_arrive_expect_tx(qbar, (uint32_t)(dslabs * kQSlabBytes));
                 for (int s = 0; s < dslabs; ++s)

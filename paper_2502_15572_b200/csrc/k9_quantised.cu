@@ -91,19 +91,19 @@ merge_rerank_kernel(const unsigned long long *__restrict__ cand, int lists, int 
     pdl_launch_dependents();
 
     unsigned long long m = 0ull;
-    int g = warp;
-    for (; g + 3 * kRerankWarps < lists; g += 4 * kRerankWarps) {
-        unsigned long long l0 = cand[((size_t)(g + 0 * kRerankWarps) * B + b) * kCandStride + lane];
-        unsigned long long l1 = cand[((size_t)(g + 1 * kRerankWarps) * B + b) * kCandStride + lane];
-        unsigned long long l2 = cand[((size_t)(g + 2 * kRerankWarps) * B + b) * kCandStride + lane];
-        unsigned long long l3 = cand[((size_t)(g + 3 * kRerankWarps) * B + b) * kCandStride + lane];
-        m = warp_merge_top32(m, l0, lane);
-        m = warp_merge_top32(m, l1, lane);
-        m = warp_merge_top32(m, l2, lane);
-        m = warp_merge_top32(m, l3, lane);
+    // eight lists in flight per warp before the dependent merge chain; empty lists (CTAs that saw
+    // no candidate: short scans, token windows) are skipped
+    for (int g0 = warp; g0 < lists; g0 += 8 * kRerankWarps) {
+        unsigned long long l[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int g = g0 + k * kRerankWarps;
+            l[k] = g < lists ? cand[((size_t)g * B + b) * kCandStride + lane] : 0ull;
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (shfl_u64(l[k], 0) != 0ull) m = warp_merge_top32(m, l[k], lane);      // sorted: slot 0 is the best
     }
-    for (; g < lists; g += kRerankWarps)
-        m = warp_merge_top32(m, cand[((size_t)g * B + b) * kCandStride + lane], lane);
     part[warp][lane] = m;
     __syncthreads();
     for (int span = kRerankWarps / 2; span >= 1; span >>= 1) {
