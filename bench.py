@@ -47,6 +47,10 @@ def parse_args():
     ap.add_argument("--rows", type=int, default=None, help="override N (debugging; not a bench value)")
     ap.add_argument("--batch", type=int, default=None, help="override B (debugging; not a bench value)")
     ap.add_argument("--top-n", type=int, default=None, help="override top_n (debugging; not a bench value)")
+    ap.add_argument("--shard-rows", action="store_true",
+                    help="N > 1: the rows of ONE datastore are split over the ranks (every rank answers every query "
+                         "from its rows, the per-rank results are all-gathered and merged on the device): strong scaling. "
+                         "Default: every rank holds a replica and serves its own slice of the query stream (weak)")
     ap.add_argument("--oracle-queries", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--build-keys", action="store_true",
@@ -96,6 +100,7 @@ def workload_config(cfg):
             "key_dtype": cfg["dtype"],
             "batch": cfg["B"], "top_n": cfg["top_n"], "draft_len": cfg["draft_len"],
             "first_token_filter": bool(cfg.get("filter_on", False)),
+            "multi_gpu": cfg.get("multi_gpu", "replicas: every rank serves its own slice of the query stream"),
             "sorted_by_first_token": "rows_scanned_per_step_mean" in cfg,
             "rows_scanned_per_step_mean": cfg.get("rows_scanned_per_step_mean"),
             "mixture_components": cfg["C"], "query_noise_sigma": cfg["sigma"], "seed": cfg["seed"],
@@ -233,11 +238,21 @@ def run_ours(args):
     cfg, keys, toks, q = make_inputs(args)
     cfg["filter_on"] = args.first_token_filter
     B, n, L, dtype = cfg["B"], cfg["top_n"], cfg["draft_len"], cfg["dtype"]
+    shard = None
+    if args.shard_rows:
+        if args.first_token_filter or args.quantised:
+            raise SystemExit("--shard-rows times the exact, unfiltered call")
+        shard = dist_util.shard_rows(cfg["N"], rank, world)      # this rank's contiguous rows of the one datastore
+        cfg["multi_gpu"] = "rows of one datastore sharded over the ranks; all-gather of the per-rank results + device merge"
+        keys, toks = keys[shard.start:shard.stop], toks[shard.start:shard.stop]
     dkeys = binding.to_device(keys, dtype)
-    dtoks = torch.from_numpy(toks).cuda()
+    dtoks = torch.from_numpy(np.ascontiguousarray(toks)).cuda()
     dq = binding.to_device(q, dtype)                       # [nq][d] resident in HBM
-    # every rank serves its own slice of the query stream against its own replica
-    batches = dist_util.query_slice(dq.shape[0] // B, rank, world)
+    if shard is None:
+        # every rank serves its own slice of the query stream against its own replica
+        batches = dist_util.query_slice(dq.shape[0] // B, rank, world)
+    else:
+        batches = range(dq.shape[0] // B)                  # every rank sees every query
     nq, q_first = max(1, len(batches)), batches.start
     store = binding.Store(dkeys, dtoks, dtype)
     if "W" in cfg:
@@ -275,11 +290,15 @@ def run_ours(args):
                 tot += len(want)
         recall = hit / tot
 
+    sharded = None if shard is None else dist_util.ShardedRetriever(store, shard.start, n, L)
+
     def step(i):
         j = (q_first + i % nq) * B
         if args.quantised:
             store.retrieve_quantised(dq[j:j + B], n, L, args.quantised, out=out,
                                      first_tokens=None if dft is None else dft[j:j + B])
+        elif shard is not None:
+            sharded(dq[j:j + B])
         elif dft is None:
             store.retrieve(dq[j:j + B], n, L, out=out)
         else:
@@ -313,7 +332,7 @@ def run_ours(args):
     ev1.record()
     barrier()
     ms_total = ev0.elapsed_time(ev1)
-    launches = store.last_launches() * args.steps
+    launches = (store.last_launches() + (1 if shard is not None else 0)) * args.steps   # + the shard merge kernel
     passes = store.last_key_passes()                       # passes over the keys per call
     scan_ms, scan_calls = store.profile_read()
     store.set_option("profile", 0)
@@ -355,6 +374,14 @@ def run_ours(args):
     ft_stage = None if dft is None else dft[:B].clone()
 
     def host_call(j):
+        if shard is not None:
+            dq_stage.view(torch.int16 if dtype != "f32" else torch.float32).copy_(
+                hq[j:j + B].view(torch.int16 if dtype != "f32" else torch.float32), non_blocking=True)
+            res = sharded(dq_stage)
+            for h, o_ in zip(hout, res):
+                h.copy_(o_, non_blocking=True)
+            torch.cuda.synchronize()
+            return
         if not args.quantised and dft is None:
             store.retrieve_host(hq[j:j + B], n, L, hout)
             return
@@ -390,10 +417,13 @@ def run_ours(args):
         return
 
     ms_step = ms_total / args.steps
-    qps = dist_util.aggregate_throughput(B, args.steps, world, ms_total)
-    e2e_qps = dist_util.aggregate_throughput(B, args.steps, world, e2e_ms_total)
+    # replicas: every rank answered its own B queries per step; sharded rows: all ranks together answered B
+    qps = dist_util.aggregate_throughput(B, args.steps, 1 if shard is not None else world, ms_total)
+    e2e_qps = dist_util.aggregate_throughput(B, args.steps, 1 if shard is not None else world, e2e_ms_total)
     eb = synth.DTYPE_BYTES[dtype]
     key_bytes = cfg["N"] * cfg["d"] * (1 if args.quantised else eb)   # algorithmic bytes of one scoring launch
+    if shard is not None:
+        key_bytes = len(shard) * cfg["d"] * eb             # rank 0's kernel reads its shard
     if args.sorted_store and dft is not None:
         # only the rows of the batch's distinct first tokens are scored: mean over the timed steps
         counts = np.bincount(toks[:, 0])
@@ -409,7 +439,7 @@ def run_ours(args):
                   + (" -- rows sorted by first token, only the queries' token windows scanned"
                      if "rows_scanned_per_step_mean" in cfg else ""), "value": qps, "unit": "queries/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32 accumulate over %s keys" % dtype,
+        "scaling": "strong" if shard is not None else "weak", "vs_baseline": None, "dtype": "f32 accumulate over %s keys" % dtype,
         "data": "synthetic", "config": workload_config(cfg),
         "e2e": {"value": e2e_qps, "unit": "queries/s",
                 "h2d_bytes_per_step": B * cfg.get("d_in", cfg["d"]) * eb + (4 * B if dft is not None else 0),

@@ -283,6 +283,18 @@ dresd_status dresd_merge_shards(const int32_t *ids, const float *scores, const i
                                 int32_t *out_ids, float *out_scores, int32_t *out_tokens, void *stream);
 
 /*
+ * The same merge for results that were exchanged in ONE all-gather (the message is
+ * latency-bound: 480 bytes per shard at B = 1, n = 10, L = 10): shard p's block
+ * of B * top_n * (2 + draft_len) 32-bit words is
+ *     ids [B][top_n] int32 | scores [B][top_n] fp32 | tokens [B][top_n][draft_len] int32
+ * and `packed` (device) holds the P blocks back to back, as an all-gather of the
+ * blocks leaves them.  Everything else as for dresd_merge_shards().
+ */
+dresd_status dresd_merge_shards_packed(const int32_t *packed, const int64_t *row_offsets, int P, int B,
+                                       int top_n, int draft_len, int32_t *out_ids, float *out_scores,
+                                       int32_t *out_tokens, void *stream);
+
+/*
  * The same call for callers whose queries and results live in HOST memory, and
  * waits for `stream`.  When all four buffers are page-locked and mapped (e.g.
  * cudaHostAlloc, cudaHostRegister, a pinned framework tensor), the kernels read the

@@ -30,7 +30,7 @@ EXPORTS = (
     "dresd_store_destroy", "dresd_retrieve_noalloc", "dresd_store_enable_first_token_filter",
     "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
     "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore", "dresd_set_global_option", "dresd_quantise_keys", "dresd_store_attach_quantised",
-    "dresd_retrieve_quantised", "dresd_store_index_first_tokens",
+    "dresd_retrieve_quantised", "dresd_store_index_first_tokens", "dresd_merge_shards_packed",
 )
 
 
@@ -92,6 +92,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_drafts_accept.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_merge_shards.restype = i32
     lib.dresd_merge_shards.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+    lib.dresd_merge_shards_packed.restype = i32
+    lib.dresd_merge_shards_packed.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_build_keys.restype = i32
     lib.dresd_build_keys.argtypes = [vp, i64, i32, i32, vp, vp, f32, vp, i32, vp, vp, vp]
     lib.dresd_quantise_keys.restype = i32
@@ -162,6 +164,12 @@ def dresd_drafts_accept(drafts_ptr: int, valid_ptr: int, llm_ptr: int, B: int, n
                         out_best_ptr: int, out_len_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
     _check(load().dresd_drafts_accept(drafts_ptr, valid_ptr, llm_ptr, B, n, L, out_best_ptr, out_len_ptr,
                                       out_tokens_ptr, stream))
+
+
+def dresd_merge_shards_packed(packed_ptr: int, offsets_ptr: int, P: int, B: int, top_n: int, draft_len: int,
+                              out_ids_ptr: int, out_scores_ptr: int, out_tokens_ptr: int, stream: int = 0) -> None:
+    _check(load().dresd_merge_shards_packed(packed_ptr, offsets_ptr, P, B, top_n, draft_len, out_ids_ptr,
+                                            out_scores_ptr, out_tokens_ptr, stream))
 
 
 def dresd_merge_shards(ids_ptr: int, scores_ptr: int, tokens_ptr: int, offsets_ptr: int, P: int, B: int,

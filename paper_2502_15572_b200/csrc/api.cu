@@ -850,9 +850,27 @@ dresd_status dresd_merge_shards(const int32_t *ids, const float *scores, const i
     if (!is_device_ptr(ids) || !is_device_ptr(scores) || !is_device_ptr(tokens) || !is_device_ptr(row_offsets) ||
         !is_device_ptr(out_ids) || !is_device_ptr(out_scores) || !is_device_ptr(out_tokens))
         return fail(DRESD_ERR_INVALID, "all buffers must be device pointers");
-    cudaError_t e = launch_merge_shards(ids, scores, tokens, reinterpret_cast<const long long *>(row_offsets), P, B,
-                                        top_n, draft_len, out_ids, out_scores, out_tokens,
+    cudaError_t e = launch_merge_shards(ids, scores, tokens, (size_t)B * top_n, (size_t)B * top_n,
+                                        (size_t)B * top_n * draft_len, reinterpret_cast<const long long *>(row_offsets), P,
+                                        B, top_n, draft_len, out_ids, out_scores, out_tokens,
                                         static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "merge_shards launch");
+}
+
+dresd_status dresd_merge_shards_packed(const int32_t *packed, const int64_t *row_offsets, int P, int B, int top_n,
+                                       int draft_len, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
+                                       void *stream)
+{
+    if (P < 1 || B < 0 || top_n < 1 || draft_len < 1) return fail(DRESD_ERR_INVALID, "bad P/B/top_n/draft_len");
+    if (top_n > DRESD_MAX_TOP_N) return fail(DRESD_ERR_UNSUPPORTED, "top_n = %d exceeds DRESD_MAX_TOP_N", top_n);
+    if (B == 0) return DRESD_OK;
+    if (!is_device_ptr(packed) || !is_device_ptr(row_offsets) || !is_device_ptr(out_ids) || !is_device_ptr(out_scores) ||
+        !is_device_ptr(out_tokens))
+        return fail(DRESD_ERR_INVALID, "all buffers must be device pointers");
+    const size_t bn = (size_t)B * top_n, block = bn * (2 + (size_t)draft_len);
+    cudaError_t e = launch_merge_shards(packed, reinterpret_cast<const float *>(packed + bn), packed + 2 * bn, block, block,
+                                        block, reinterpret_cast<const long long *>(row_offsets), P, B, top_n, draft_len,
+                                        out_ids, out_scores, out_tokens, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "merge_shards launch");
 }
 

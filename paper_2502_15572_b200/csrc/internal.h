@@ -132,9 +132,10 @@ cudaError_t launch_drafts_accept(const int32_t *drafts, const int32_t *valid, co
                                  cudaStream_t stream);
 
 // Exchange step of a row-sharded datastore: P per-shard top-n lists -> the global top-n.
-cudaError_t launch_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens,
-                                const long long *offsets, int P, int B, int n, int L, int32_t *out_ids,
-                                float *out_scores, int32_t *out_tokens, cudaStream_t stream);
+cudaError_t launch_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens, size_t stride_ids,
+                                size_t stride_scores, size_t stride_tokens, const long long *offsets, int P, int B,
+                                int n, int L, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
+                                cudaStream_t stream);
 
 // ---- K7: datastore-side preprocessing (Eq. 1 -> v W -> Eq. 2 over N rows), a tcgen05 GEMM ----
 // `terms` = 2 multiplies by W' = hi + lo (needed when Eq. 1 scales the weights), 1 by hi alone

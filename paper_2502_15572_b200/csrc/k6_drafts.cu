@@ -101,8 +101,11 @@ cudaError_t launch_drafts_accept(const int32_t *drafts, const int32_t *valid, co
 namespace dresd {
 namespace {
 
+// stride_x: distance in elements between two shards' blocks of array x (dense arrays: B n and
+// B n L; results packed per shard for a single all-gather: the packed block size for all three).
 __global__ void merge_shards_kernel(const int32_t *__restrict__ ids, const float *__restrict__ scores,
-                                    const int32_t *__restrict__ tokens, const long long *__restrict__ offsets,
+                                    const int32_t *__restrict__ tokens, size_t stride_ids, size_t stride_scores,
+                                    size_t stride_tokens, const long long *__restrict__ offsets,
                                     int P, int B, int n, int L, int32_t *__restrict__ out_ids,
                                     float *__restrict__ out_scores, int32_t *__restrict__ out_tokens)
 {
@@ -111,8 +114,8 @@ __global__ void merge_shards_kernel(const int32_t *__restrict__ ids, const float
     for (int p = 0; p < P; ++p) {
         unsigned long long v = 0ull;
         if (lane < n) {
-            const int32_t id = ids[((size_t)p * B + b) * n + lane];
-            if (id >= 0) v = pack_candidate(scores[((size_t)p * B + b) * n + lane], (uint32_t)(id + offsets[p]));
+            const int32_t id = ids[p * stride_ids + (size_t)b * n + lane];
+            if (id >= 0) v = pack_candidate(scores[p * stride_scores + (size_t)b * n + lane], (uint32_t)(id + offsets[p]));
         }
         // a shard's list is sorted with its missing entries (id -1) last, so it is a valid input
         m = warp_merge_top32(m, v, lane);
@@ -130,21 +133,23 @@ __global__ void merge_shards_kernel(const int32_t *__restrict__ ids, const float
         while (p + 1 < P && offsets[p + 1] <= gid) ++p;
         const int32_t local = (int32_t)(gid - offsets[p]);
         for (int k = 0; k < n; ++k)
-            if (ids[((size_t)p * B + b) * n + k] == local) { r = k; break; }
+            if (ids[p * stride_ids + (size_t)b * n + k] == local) { r = k; break; }
     }
     if (lane < n)
         for (int t = 0; t < L; ++t)
             out_tokens[((size_t)b * n + lane) * L + t] =
-                r >= 0 ? tokens[(((size_t)p * B + b) * n + r) * L + t] : -1;
+                r >= 0 ? tokens[p * stride_tokens + (((size_t)b * n + r) * L + t)] : -1;
 }
 
 }  // namespace
 
-cudaError_t launch_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens,
-                                const long long *offsets, int P, int B, int n, int L, int32_t *out_ids,
-                                float *out_scores, int32_t *out_tokens, cudaStream_t stream)
+cudaError_t launch_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens, size_t stride_ids,
+                                size_t stride_scores, size_t stride_tokens, const long long *offsets, int P, int B,
+                                int n, int L, int32_t *out_ids, float *out_scores, int32_t *out_tokens,
+                                cudaStream_t stream)
 {
-    merge_shards_kernel<<<B, 32, 0, stream>>>(ids, scores, tokens, offsets, P, B, n, L, out_ids, out_scores, out_tokens);
+    merge_shards_kernel<<<B, 32, 0, stream>>>(ids, scores, tokens, stride_ids, stride_scores, stride_tokens, offsets, P, B,
+                                              n, L, out_ids, out_scores, out_tokens);
     return cudaGetLastError();
 }
 

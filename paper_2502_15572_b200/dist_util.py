@@ -7,8 +7,10 @@ Two ways to use several GPUs:
   benchmark's timing protocol (barrier on both sides, maximum of the per-rank times);
 * by ROWS (`sharded_retrieve`): the datastore is split into contiguous row shards, one
   per rank; every rank retrieves from its shard, the small per-shard results are
-  all-gathered (B * n * (8 + 4 L) bytes per rank -- latency-bound, so one collective)
-  and merged on the device by `dresd_merge_shards`.
+  all-gathered (B * n * (8 + 4 L) bytes per rank -- latency-bound, so ONE collective over a
+  packed block, `PackedExchange` / `ShardedRetriever`) and merged on the device by
+  `dresd_merge_shards_packed`.  `sharded_retrieve` is the plain form of the same step
+  (three all-gathers, nothing kept between calls).
 
 The collectives are torch.distributed calls, so the plumbing can be exercised on CPU
 with the gloo backend; the merge itself is a CUDA kernel.
@@ -88,3 +90,65 @@ def sharded_retrieve(store, row_offset: int, queries, top_n: int, draft_len: int
     binding.dresd_merge_shards(g_ids.data_ptr(), g_scores.data_ptr(), g_tokens.data_ptr(), offsets.data_ptr(),
                                P, B, top_n, draft_len, out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), s)
     return out
+
+
+class PackedExchange:
+    """Buffers of the exchange step for a fixed (B, top_n, draft_len): this rank's results live in
+    ONE block of B * n * (2 + L) 32-bit words -- ids | scores | tokens, the layout
+    dresd_merge_shards_packed() reads -- so that a call needs a single all-gather; the row
+    offsets of the shards are exchanged once, here.  Works on any device (CPU + gloo in the tests)."""
+
+    def __init__(self, B: int, top_n: int, draft_len: int, row_offset: int, device, group=None):
+        import torch
+        import torch.distributed as dist
+        self.group = group
+        self.P = dist.get_world_size(group) if dist.is_available() and dist.is_initialized() else 1
+        bn = B * top_n
+        self.words = bn * (2 + draft_len)
+        self.local = torch.empty(self.words, dtype=torch.int32, device=device)
+        self.ids = self.local[:bn].view(B, top_n)
+        self.scores = self.local[bn:2 * bn].view(torch.float32).view(B, top_n)
+        self.tokens = self.local[2 * bn:].view(B, top_n, draft_len)
+        off = torch.tensor([row_offset], dtype=torch.int64, device=device)
+        if self.P == 1:
+            self.gathered, self.offsets = self.local, off
+        else:
+            self.gathered = torch.empty(self.P * self.words, dtype=torch.int32, device=device)
+            self.offsets = torch.empty(self.P, dtype=torch.int64, device=device)
+            dist.all_gather_into_tensor(self.offsets, off, group=group)
+
+    def exchange(self):
+        """All ranks' blocks, back to back: int32 [P * words]."""
+        if self.P > 1:
+            import torch.distributed as dist
+            dist.all_gather_into_tensor(self.gathered, self.local, group=self.group)
+        return self.gathered
+
+
+class ShardedRetriever:
+    """dresd_retrieve over a datastore whose rows are sharded over the ranks of `group`: the local
+    call writes into the packed block, one all-gather, one merge kernel.  Buffers are kept per
+    batch size; every rank gets the global result (ids are global row indices)."""
+
+    def __init__(self, store, row_offset: int, top_n: int, draft_len: int, group=None):
+        self.store, self.row_offset, self.n, self.L, self.group = store, row_offset, top_n, draft_len, group
+        self._by_batch = {}
+
+    def __call__(self, queries, stream=None):
+        import torch
+        from . import binding
+        B = queries.shape[0]
+        st = self._by_batch.get(B)
+        if st is None:
+            ex = PackedExchange(B, self.n, self.L, self.row_offset, queries.device, self.group)
+            out = (torch.empty((B, self.n), dtype=torch.int32, device=queries.device),
+                   torch.empty((B, self.n), dtype=torch.float32, device=queries.device),
+                   torch.empty((B, self.n, self.L), dtype=torch.int32, device=queries.device))
+            st = self._by_batch[B] = (ex, out)
+        ex, out = st
+        self.store.retrieve(queries, self.n, self.L, out=(ex.ids, ex.scores, ex.tokens), stream=stream)
+        packed = ex.exchange()
+        s = (stream or torch.cuda.current_stream()).cuda_stream
+        binding.dresd_merge_shards_packed(packed.data_ptr(), ex.offsets.data_ptr(), ex.P, B, self.n, self.L,
+                                          out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), s)
+        return out

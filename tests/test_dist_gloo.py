@@ -100,3 +100,50 @@ def test_two_ranks_gloo_gather_of_shard_results():
     assert ids[0][0] == [0, 1, 2, 3] and ids[1][0] == [100, 101, 102, 103]
     assert scores[0][0][0] == 0.0 and scores[1][0][0] == 1.0
     assert tokens[0][0][0] == [7, 7] and tokens[1][0][0] == [8, 8]
+
+
+def _packed_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      LOCAL_RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        B, n, L = 3, 4, 2
+        rows = dist_util.shard_rows(1001, rank, world)
+        ex = dist_util.PackedExchange(B, n, L, rows.start, "cpu")
+        ex.ids.copy_(torch.arange(B * n, dtype=torch.int32).reshape(B, n) + 100 * rank)
+        ex.scores.fill_(0.5 + rank)
+        ex.tokens.fill_(7 + rank)
+        first = ex.exchange().clone()
+        ex.scores.fill_(2.5 + rank)                    # the buffers are reused by the next call
+        second = ex.exchange().clone()
+        out.put((rank, ex.words, ex.offsets.tolist(), first.tolist(), second.view(torch.float32).tolist()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_gloo_packed_exchange_is_one_block_per_rank():
+    """The single-collective form of the exchange step: the three result arrays of a rank travel
+    as one block ids | scores | tokens, the layout the packed merge kernel reads."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_packed_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    B, n, L = 3, 4, 2
+    bn = B * n
+    assert res[0][1:] == res[1][1:]                                # both ranks hold the same view
+    _, words, offsets, first, second = res[0]
+    assert words == bn * (2 + L) and offsets == [0, 501] and len(first) == 2 * words
+    for r in range(2):
+        blk = first[r * words:(r + 1) * words]
+        assert blk[:bn] == [i + 100 * r for i in range(bn)]        # ids
+        assert torch.tensor(blk[bn:2 * bn], dtype=torch.int32).view(torch.float32).tolist() == [0.5 + r] * bn
+        assert blk[2 * bn:] == [7 + r] * (bn * L)                  # tokens
+        assert second[r * words + bn:r * words + 2 * bn] == [2.5 + r] * bn

@@ -112,6 +112,15 @@ def test_row_sharded_merge_equals_whole_store(filtered):
     torch.cuda.synchronize()
     for a, b in zip(out, whole):
         assert torch.equal(a, b)
+    # the same exchange as ONE block per shard (ids | scores | tokens), the single-all-gather form
+    packed = torch.cat([torch.cat([p[0].reshape(-1), p[1].reshape(-1).view(torch.int32), p[2].reshape(-1)])
+                        for p in parts]).contiguous()
+    out2 = (torch.empty_like(whole[0]), torch.empty_like(whole[1]), torch.empty_like(whole[2]))
+    binding.dresd_merge_shards_packed(packed.data_ptr(), offsets.data_ptr(), 3, B, n, L, out2[0].data_ptr(),
+                                      out2[1].data_ptr(), out2[2].data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for a, b in zip(out2, whole):
+        assert torch.equal(a, b)
     if filtered:
         assert (whole[0] == -1).any()          # scarce tokens: some queries have fewer than n matches
 
@@ -127,4 +136,9 @@ def test_sharded_retrieve_single_process():
     got = dist_util.sharded_retrieve(st, 1000, dq, 5, 3)
     torch.cuda.synchronize()
     assert torch.equal(got[0], ref[0] + 1000) and torch.equal(got[1], ref[1]) and torch.equal(got[2], ref[2])
+    sharded = dist_util.ShardedRetriever(st, 1000, 5, 3)
+    for _ in range(2):                                  # the second call reuses the buffers
+        got = sharded(dq)
+        torch.cuda.synchronize()
+        assert torch.equal(got[0], ref[0] + 1000) and torch.equal(got[1], ref[1]) and torch.equal(got[2], ref[2])
     st.close()
