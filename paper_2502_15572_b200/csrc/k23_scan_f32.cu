@@ -4,23 +4,28 @@
 //
 // Same skeleton as the 16-bit streaming kernel: a producer thread streams
 // 128-row key tiles into shared memory with TMA (128-byte swizzle, two
-// 32-float slabs per stage) through an mbarrier ring; four consumer warps own
-// one row per thread, read it with conflict-free LDS.128 against queries
-// broadcast from shared memory, and keep four partial sums per query so that
-// the accumulation error stays near d/4 ulps.  Up to QB queries per launch.
+// 32-float slabs per stage) through an mbarrier ring; eight consumer warps in
+// two groups: a thread owns one row of the tile and half of the launch's
+// queries (two warps per scheduler hide the latency of the shared-memory reads
+// that one warp alone left exposed), reads the row with conflict-free LDS.128
+// against queries broadcast from shared memory, and keeps four partial sums per
+// query so that the accumulation error stays near d/4 ulps.  Up to QB queries per launch.
 // The running top-n lists are shared by the CTA (one per query): survivors of
 // the filter are queued with a shared-memory atomic, a named barrier per tile
 // publishes them, and a queue that reaches 16 entries is folded by one warp
-// (the four warps fold different queries at once).  Per-warp lists would cost
-// a small store four cold starts per query instead of one.
+// (the warps fold different queries at once).  Per-warp lists would cost a small
+// store four cold starts per query instead of one; the one cold start left is
+// bounded by taking the n-th largest of 32 group maxima of the first tile as the
+// first filter score (n rows reach it, so the final n-th best does too).
 #include "common.cuh"
 #include "internal.h"
 
 namespace dresd {
 namespace {
 
-constexpr int kConsumerWarps = 4;
-constexpr int kRows = kConsumerWarps * 32;       // 128 rows per stage, one per thread
+constexpr int kQueryGroups = 2;                   // warp groups; each takes QB / 2 of the queries
+constexpr int kRows = 128;                        // rows per stage, one per thread of a group
+constexpr int kConsumerWarps = kQueryGroups * kRows / 32;
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kSlabBytes = 128;                   // 32 floats
 constexpr int kSlabElems = 32;
@@ -110,25 +115,27 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 }
         }
     } else {
-        const int row_in_tile = tid;                  // 0..127
+        constexpr int QT = QB / kQueryGroups;         // queries per thread
+        const int row_in_tile = tid & (kRows - 1);    // 0..127
+        const int q0 = (tid / kRows) * QT;            // this thread's first query
         const uint32_t swz = (uint32_t)(row_in_tile & 7);
         // A warp whose wait expired goes "dead": it does no more work and no more waits,
         // but keeps taking part in every barrier so that nobody is left behind.
         bool dead = false;
         int round = 0;                                 // barrier-A count: selects the flag slot
         SelFlags *fl = &flags[0];
-        int want[QB];                                  // first-token filter, -1 = off
+        int want[QT];                                  // first-token filter, -1 = off
 #pragma unroll
-        for (int q = 0; q < QB; ++q) want[q] = (a.first_col && q < a.B) ? a.want_first[q] : -1;
+        for (int j = 0; j < QT; ++j) want[j] = (a.first_col && q0 + j < a.B) ? a.want_first[q0 + j] : -1;
         for (int tl = 0; tl < my_tiles; ++tl) {
             // this row's first stored token, requested before the tile is waited for
             const long long row = (long long)(cta + tl * G) * kRows + row_in_tile;
             const int tok = (a.first_col && row < a.N) ? a.first_col[row] : 0;
-            float acc[QB][4];
+            float acc[QT][4];
 #pragma unroll
-            for (int q = 0; q < QB; ++q)
+            for (int j = 0; j < QT; ++j)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[q][i] = 0.f;
+                for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
             for (int kc = 0; kc < kch; ++kc) {
                 const int it = tl * kch + kc;
                 const int s = it % n_stages;
@@ -141,18 +148,18 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 const uint8_t *rowp = stages + (size_t)s * kStageBytes + (size_t)row_in_tile * kSlabBytes;
                 const int nsl = min(kSlabsPerStage, dslabs - kc * kSlabsPerStage);
                 for (int sl = 0; sl < nsl; ++sl) {
-                    const float *qbase = qs + (kc * kSlabsPerStage + sl) * kSlabElems;
+                    const float *qbase = qs + (size_t)q0 * dpad + (kc * kSlabsPerStage + sl) * kSlabElems;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         const float4 k4 = *reinterpret_cast<const float4 *>(
                             rowp + (size_t)sl * kRows * kSlabBytes + ((c ^ swz) << 4));
 #pragma unroll
-                        for (int q = 0; q < QB; ++q) {
-                            const float4 q4 = *reinterpret_cast<const float4 *>(qbase + (size_t)q * dpad + c * 4);
-                            acc[q][0] = fmaf(q4.x, k4.x, acc[q][0]);
-                            acc[q][1] = fmaf(q4.y, k4.y, acc[q][1]);
-                            acc[q][2] = fmaf(q4.z, k4.z, acc[q][2]);
-                            acc[q][3] = fmaf(q4.w, k4.w, acc[q][3]);
+                        for (int j = 0; j < QT; ++j) {
+                            const float4 q4 = *reinterpret_cast<const float4 *>(qbase + (size_t)j * dpad + c * 4);
+                            acc[j][0] = fmaf(q4.x, k4.x, acc[j][0]);
+                            acc[j][1] = fmaf(q4.y, k4.y, acc[j][1]);
+                            acc[j][2] = fmaf(q4.z, k4.z, acc[j][2]);
+                            acc[j][3] = fmaf(q4.w, k4.w, acc[j][3]);
                         }
                     }
                 }
@@ -162,31 +169,61 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
             if ((tl & 3) == 0 && tid < a.B && tid < QB) sel[tid].tau = peek_tau(&a.gtau[tid], sel[tid].tau);
 
-            float sc[QB];
+            float sc[QT];
+#pragma unroll
+            for (int j = 0; j < QT; ++j) sc[j] = (acc[j][0] + acc[j][1]) + (acc[j][2] + acc[j][3]);
+            if (tl == 0) {
+                // Cold start: 32 groups of 4 rows per query; the n-th largest group maximum is reached by
+                // n rows of this tile and becomes the first filter score, so that about n rows are queued
+                // instead of all 128 (four overflow rounds of barriers and merges otherwise).
+#pragma unroll
+                for (int j = 0; j < QT; ++j) {
+                    const int q = q0 + j;
+                    const bool valid = !dead && q < a.B && row < a.N && sc[j] > -INFINITY &&      // false for NaN
+                                       (want[j] < 0 || tok == want[j]);
+                    uint32_t key = valid ? float_to_ordered(sc[j] + 0.0f) : 0u;
+                    key = __reduce_max_sync(0xFu << (lane & ~3), key);
+                    // the queue is still empty: its first 128 bytes take the group maxima
+                    if ((lane & 3) == 0)
+                        reinterpret_cast<uint32_t *>(sel[q].queue)[(warp & 3) * 8 + (lane >> 2)] = key;
+                }
+                consumer_bar();
+                for (int q = warp; q < QB; q += kConsumerWarps) {
+                    if (q >= a.B || sel[q].tau > -INFINITY) continue;                              // warp-uniform
+                    unsigned long long x = reinterpret_cast<const uint32_t *>(sel[q].queue)[lane];
+                    __syncwarp();
+                    x = warp_sort_desc(x, lane);
+                    const uint32_t nth = (uint32_t)shfl_u64(x, a.top_n - 1);
+                    if (lane == 0 && nth) sel[q].tau = share_tau(&a.gtau[q], ordered_to_float(nth));
+                }
+                consumer_bar();
+            }
             uint32_t pend = 0u;                        // queries for which this row is (still) a candidate
 #pragma unroll
-            for (int q = 0; q < QB; ++q) {
-                sc[q] = (acc[q][0] + acc[q][1]) + (acc[q][2] + acc[q][3]);
-                const bool take = !dead && q < a.B && row < a.N && sc[q] >= sel[q].tau && (want[q] < 0 || tok == want[q]);
-                pend |= take ? (1u << q) : 0u;
+            for (int j = 0; j < QT; ++j) {
+                const int q = q0 + j;
+                const bool take = !dead && q < a.B && row < a.N && sc[j] >= sel[q].tau && (want[j] < 0 || tok == want[j]);
+                pend |= take ? (1u << j) : 0u;
             }
             // Queue the survivors; when a queue is full the candidate waits (`pend`) until the CTA
             // has folded the queues, so that adversarial row orders stay exact.
             while (true) {
                 // claim the slots first (independent shared-memory atomics in flight together), then fill them
-                int slot[QB];
+                int slot[QT];
 #pragma unroll
-                for (int q = 0; q < QB; ++q) {
-                    if (((pend >> q) & 1u) && !(sc[q] >= sel[q].tau)) pend &= ~(1u << q);   // the filter has tightened
-                    slot[q] = ((pend >> q) & 1u) ? atomicAdd(&sel[q].count, 1) : 0;
+                for (int j = 0; j < QT; ++j) {
+                    const int q = q0 + j;
+                    if (((pend >> j) & 1u) && !(sc[j] >= sel[q].tau)) pend &= ~(1u << j);   // the filter has tightened
+                    slot[j] = ((pend >> j) & 1u) ? atomicAdd(&sel[q].count, 1) : 0;
                 }
 #pragma unroll
-                for (int q = 0; q < QB; ++q) {
-                    if ((pend >> q) & 1u) {
-                        if (slot[q] < kQueueCap) {
-                            sel[q].queue[slot[q]] = pack_candidate(sc[q], (uint32_t)row);
-                            if (slot[q] + 1 >= kMergeLevel) fl->need_merge = 1;
-                            pend &= ~(1u << q);
+                for (int j = 0; j < QT; ++j) {
+                    const int q = q0 + j;
+                    if ((pend >> j) & 1u) {
+                        if (slot[j] < kQueueCap) {
+                            sel[q].queue[slot[j]] = pack_candidate(sc[j], (uint32_t)row);
+                            if (slot[j] + 1 >= kMergeLevel) fl->need_merge = 1;
+                            pend &= ~(1u << j);
                         } else {
                             fl->overflow = 1;
                         }
