@@ -472,7 +472,7 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
 
     s->tile_rows = dtype == DRESD_F32 ? scan_f32_tile_rows(d) : scan_mma_tile_rows(d);
     s->n_tiles = (int)((N + s->tile_rows - 1) / s->tile_rows);
-    if (!make_map(&s->map_stream, keys, s->dtype, N, d, s->tile_rows)) {
+    if (!make_map(&s->map_stream, keys, s->dtype, N, d, dtype == DRESD_F32 ? scan_f32_box_rows(d) : s->tile_rows)) {
         free_store(s);
         return fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the key matrix");
     }

@@ -98,7 +98,8 @@ bool scan_ummat_eligible(int d, int B);
 cudaError_t launch_scan_ummat(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
                               int grid, cudaStream_t stream);
 
-int scan_f32_tile_rows(int d);
+int scan_f32_tile_rows(int d);   // rows per tile (tile count)
+int scan_f32_box_rows(int d);    // rows per TMA box of the key map (a tile is fetched as several boxes)
 int scan_f32_queries_per_launch(int d, int B);
 cudaError_t launch_scan_f32(const CUtensorMap &keys_map, const ScanArgs &a, int grid,
                             cudaStream_t stream);

@@ -2,50 +2,58 @@
 // in plain fp32 FMA (tensor cores would round fp32 operands to 10-11 mantissa
 // bits, far outside the 1e-5 score tolerance), fused with the per-CTA top-n.
 //
-// Same skeleton as the 16-bit streaming kernel: a producer thread streams
-// 128-row key tiles into shared memory with TMA (128-byte swizzle, two
-// 32-float slabs per stage) through an mbarrier ring; eight consumer warps in
-// two groups: a thread owns one row of the tile and half of the launch's
-// queries (two warps per scheduler hide the latency of the shared-memory reads
-// that one warp alone left exposed), reads the row with conflict-free LDS.128
-// against queries broadcast from shared memory, and keeps four partial sums per
-// query so that the accumulation error stays near d/4 ulps.  Up to QB queries per launch.
+// Same skeleton as the 16-bit streaming kernel: a producer thread streams key
+// tiles into shared memory with TMA (128-byte swizzle, one 32-float slab of 512
+// rows per stage) through an mbarrier ring; four consumer warps score them.
+// The loop is register-tiled: a thread owns FOUR rows of the tile and all QB
+// queries of the launch, so that per four elements of k it issues 4 LDS.128 of
+// its rows and QB broadcast LDS.128 of the queries for 16 QB FMAs.  With one row
+// per thread (the first form) the loop was bound by shared-memory instruction
+// issue, 5 LDS.128 per 16 FMAs: 2.5 TB/s on a large store at any batch.  Four
+// partial sums per (row, query) keep the accumulation error near d/4 ulps.
+// QB is the batch rounded up to 1, 2, 4 or 8: a single query pays for one.  Eight
+// queries are split over two groups of four warps (the same rows, four queries each):
+// 128 accumulators per thread would leave no registers for the loads in flight.
+//
 // The running top-n lists are shared by the CTA (one per query): survivors of
 // the filter are queued with a shared-memory atomic, a named barrier per tile
 // publishes them, and a queue that reaches 16 entries is folded by one warp
-// (the warps fold different queries at once).  Per-warp lists would cost a small
-// store four cold starts per query instead of one; the one cold start left is
-// bounded by taking the n-th largest of 32 group maxima of the first tile as the
-// first filter score (n rows reach it, so the final n-th best does too).
+// (the warps fold different queries at once).  The cold start is bounded by
+// taking the n-th largest of 32 group maxima of the first tile as the first
+// filter score (n rows reach it, so the final n-th best does too).
 #include "common.cuh"
 #include "internal.h"
 
 namespace dresd {
 namespace {
 
-constexpr int kQueryGroups = 2;                   // warp groups; each takes QB / 2 of the queries
-constexpr int kRows = 128;                        // rows per stage, one per thread of a group
-constexpr int kConsumerWarps = kQueryGroups * kRows / 32;
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kSlabBytes = 128;                   // 32 floats
+constexpr int kGroupWarps = 4;
+constexpr int kRowsPerThread = 4;
+constexpr int kLanes = kGroupWarps * 32;                     // 128 threads share the rows of a tile
+constexpr int kRows = kLanes * kRowsPerThread;               // 512 rows per tile
+constexpr int kBoxRows = 256;                                // a TMA box is at most 256 rows tall
+constexpr int groups_of(int QB) { return QB > 4 ? 2 : 1; }   // query groups (each: kGroupWarps warps)
+constexpr int kSlabBytes = 128;                              // 32 floats
 constexpr int kSlabElems = 32;
-constexpr int kSlabsPerStage = 2;
-constexpr int kStageBytes = kRows * kSlabsPerStage * kSlabBytes;   // 32 KB
-constexpr int kMaxStages = 6;
+constexpr int kStageBytes = kRows * kSlabBytes;              // one slab of the tile: 64 KB
+constexpr int kMaxStages = 3;
 
 struct SelFlags {
     int need_merge;
     int overflow;
 };
-__device__ __forceinline__ void consumer_bar()
+template <int NTHREADS> __device__ __forceinline__ void consumer_bar()
 {
-    asm volatile("bar.sync 2, %0;" ::"n"(kConsumerWarps * 32) : "memory");
+    asm volatile("bar.sync 2, %0;" ::"n"(NTHREADS) : "memory");
 }
 
 template <int QB>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__((groups_of(QB) * kGroupWarps + 1) * 32, 1)
 scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
 {
+    constexpr int kConsumerWarps = groups_of(QB) * kGroupWarps;
+    constexpr int kThreads = (kConsumerWarps + 1) * 32;
+    constexpr int QT = QB / groups_of(QB);                   // queries per thread
     extern __shared__ uint8_t smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -55,7 +63,8 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
     uint64_t *full = reinterpret_cast<uint64_t *>(sel + QB);
     uint64_t *empty = full + kMaxStages;
     SelFlags *flags = reinterpret_cast<SelFlags *>(empty + kMaxStages);   // [3], rotating
-    float *qs = reinterpret_cast<float *>(flags + 4);              // [QB][dpad]
+    float *qs = reinterpret_cast<float *>(                         // [QB][dpad], read as float4
+        (reinterpret_cast<uintptr_t>(flags + 4) + 15) & ~static_cast<uintptr_t>(15));
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
@@ -63,6 +72,7 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
     const int dpad = dslabs * kSlabElems;
 
     if (tid == 0) {
+        tma_prefetch_desc(&keys_map);
         for (int s = 0; s < n_stages; ++s) {
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], kConsumerWarps);
@@ -84,13 +94,11 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
     }
     __syncthreads();
 
-    const int kch = (dslabs + kSlabsPerStage - 1) / kSlabsPerStage;
     const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
-    const int n_it = my_tiles * kch;
+    const int n_it = my_tiles * dslabs;                // one slab of one tile per stage
 
     if (warp == kConsumerWarps) {
         if (lane == 0) {
-            tma_prefetch_desc(&keys_map);
             int issued = 0;
             for (int it = 0; it < n_it; ++it) {
                 const int s = it % n_stages;
@@ -98,14 +106,13 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                     report_timeout(a.status);
                     break;
                 }
-                const int tile = cta + (it / kch) * G;
-                const int kc = it % kch;
-                const int nsl = min(kSlabsPerStage, dslabs - kc * kSlabsPerStage);
-                mbar_arrive_expect_tx(&full[s], (uint32_t)(nsl * kRows * kSlabBytes));
+                const int tile = cta + (it / dslabs) * G;
+                const int sl = it % dslabs;
+                mbar_arrive_expect_tx(&full[s], (uint32_t)kStageBytes);     // rows past N arrive as zeros
                 uint8_t *dst = stages + (size_t)s * kStageBytes;
-                for (int sl = 0; sl < nsl; ++sl)
-                    tma_load_2d(dst + (size_t)sl * kRows * kSlabBytes, &keys_map,
-                                (kc * kSlabsPerStage + sl) * kSlabElems, tile * kRows, &full[s]);
+                for (int h = 0; h < kRows / kBoxRows; ++h)
+                    tma_load_2d(dst + (size_t)h * kBoxRows * kSlabBytes, &keys_map, sl * kSlabElems,
+                                tile * kRows + h * kBoxRows, &full[s]);
                 issued = it + 1;
             }
             for (int it = max(0, issued - n_stages); it < issued; ++it)
@@ -115,10 +122,11 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 }
         }
     } else {
-        constexpr int QT = QB / kQueryGroups;         // queries per thread
-        const int row_in_tile = tid & (kRows - 1);    // 0..127
-        const int q0 = (tid / kRows) * QT;            // this thread's first query
-        const uint32_t swz = (uint32_t)(row_in_tile & 7);
+        constexpr int R = kRowsPerThread;
+        // this thread's rows of a tile: rt, rt + 128, rt + 256, rt + 384 (the same swizzle phase);
+        // its queries: q0 .. q0 + QT - 1
+        const int rt = tid & (kLanes - 1), q0 = (tid / kLanes) * QT;
+        const uint32_t swz = (uint32_t)(rt & 7);
         // A warp whose wait expired goes "dead": it does no more work and no more waits,
         // but keeps taking part in every barrier so that nobody is left behind.
         bool dead = false;
@@ -128,16 +136,23 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
 #pragma unroll
         for (int j = 0; j < QT; ++j) want[j] = (a.first_col && q0 + j < a.B) ? a.want_first[q0 + j] : -1;
         for (int tl = 0; tl < my_tiles; ++tl) {
-            // this row's first stored token, requested before the tile is waited for
-            const long long row = (long long)(cta + tl * G) * kRows + row_in_tile;
-            const int tok = (a.first_col && row < a.N) ? a.first_col[row] : 0;
-            float acc[QT][4];
+            const long long row0 = (long long)(cta + tl * G) * kRows + rt;
+            // the rows' first stored tokens, requested before the tile is waited for
+            int tok[R];
 #pragma unroll
-            for (int j = 0; j < QT; ++j)
+            for (int ri = 0; ri < R; ++ri) {
+                const long long row = row0 + ri * kLanes;
+                tok[ri] = (a.first_col && row < a.N) ? a.first_col[row] : 0;
+            }
+            float acc[R][QT][4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
-            for (int kc = 0; kc < kch; ++kc) {
-                const int it = tl * kch + kc;
+            for (int ri = 0; ri < R; ++ri)
+#pragma unroll
+                for (int q = 0; q < QT; ++q)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[ri][q][i] = 0.f;
+            for (int sl = 0; sl < dslabs; ++sl) {
+                const int it = tl * dslabs + sl;
                 const int s = it % n_stages;
                 if (!dead && !mbar_wait(&full[s], (it / n_stages) & 1)) {
                     report_timeout(a.status);
@@ -145,21 +160,23 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 }
                 dead = __any_sync(0xFFFFFFFFu, dead);
                 if (dead) continue;
-                const uint8_t *rowp = stages + (size_t)s * kStageBytes + (size_t)row_in_tile * kSlabBytes;
-                const int nsl = min(kSlabsPerStage, dslabs - kc * kSlabsPerStage);
-                for (int sl = 0; sl < nsl; ++sl) {
-                    const float *qbase = qs + (size_t)q0 * dpad + (kc * kSlabsPerStage + sl) * kSlabElems;
+                const uint8_t *rowp = stages + (size_t)s * kStageBytes + (size_t)rt * kSlabBytes;
+                const float *qbase = qs + (size_t)q0 * dpad + sl * kSlabElems;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const float4 k4 = *reinterpret_cast<const float4 *>(
-                            rowp + (size_t)sl * kRows * kSlabBytes + ((c ^ swz) << 4));
+                for (int c = 0; c < 8; ++c) {
+                    float4 k4[R];
 #pragma unroll
-                        for (int j = 0; j < QT; ++j) {
-                            const float4 q4 = *reinterpret_cast<const float4 *>(qbase + (size_t)j * dpad + c * 4);
-                            acc[j][0] = fmaf(q4.x, k4.x, acc[j][0]);
-                            acc[j][1] = fmaf(q4.y, k4.y, acc[j][1]);
-                            acc[j][2] = fmaf(q4.z, k4.z, acc[j][2]);
-                            acc[j][3] = fmaf(q4.w, k4.w, acc[j][3]);
+                    for (int ri = 0; ri < R; ++ri)
+                        k4[ri] = *reinterpret_cast<const float4 *>(rowp + (size_t)ri * kLanes * kSlabBytes + ((c ^ swz) << 4));
+#pragma unroll
+                    for (int q = 0; q < QT; ++q) {
+                        const float4 q4 = *reinterpret_cast<const float4 *>(qbase + (size_t)q * dpad + c * 4);
+#pragma unroll
+                        for (int ri = 0; ri < R; ++ri) {
+                            acc[ri][q][0] = fmaf(q4.x, k4[ri].x, acc[ri][q][0]);
+                            acc[ri][q][1] = fmaf(q4.y, k4[ri].y, acc[ri][q][1]);
+                            acc[ri][q][2] = fmaf(q4.z, k4[ri].z, acc[ri][q][2]);
+                            acc[ri][q][3] = fmaf(q4.w, k4[ri].w, acc[ri][q][3]);
                         }
                     }
                 }
@@ -169,25 +186,33 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
             if ((tl & 3) == 0 && tid < a.B && tid < QB) sel[tid].tau = peek_tau(&a.gtau[tid], sel[tid].tau);
 
-            float sc[QT];
+            float sc[R][QT];
+            uint32_t okbits = 0u;                      // bit ri * QT + j: the row may be a result of query q0 + j
 #pragma unroll
-            for (int j = 0; j < QT; ++j) sc[j] = (acc[j][0] + acc[j][1]) + (acc[j][2] + acc[j][3]);
+            for (int ri = 0; ri < R; ++ri)
+#pragma unroll
+                for (int q = 0; q < QT; ++q) {
+                    sc[ri][q] = (acc[ri][q][0] + acc[ri][q][1]) + (acc[ri][q][2] + acc[ri][q][3]);
+                    const bool ok = !dead && q0 + q < a.B && row0 + ri * kLanes < a.N && sc[ri][q] > -INFINITY &&   // false for NaN
+                                    (want[q] < 0 || tok[ri] == want[q]);
+                    okbits |= ok ? (1u << (ri * QT + q)) : 0u;
+                }
             if (tl == 0) {
-                // Cold start: 32 groups of 4 rows per query; the n-th largest group maximum is reached by
-                // n rows of this tile and becomes the first filter score, so that about n rows are queued
-                // instead of all 128 (four overflow rounds of barriers and merges otherwise).
+                // Cold start: 32 groups of 16 rows per query (a thread's four rows and those of its three
+                // neighbours); the n-th largest group maximum is reached by n rows of this tile and becomes
+                // the first filter score, so that about n rows are queued instead of all 512.
 #pragma unroll
-                for (int j = 0; j < QT; ++j) {
-                    const int q = q0 + j;
-                    const bool valid = !dead && q < a.B && row < a.N && sc[j] > -INFINITY &&      // false for NaN
-                                       (want[j] < 0 || tok == want[j]);
-                    uint32_t key = valid ? float_to_ordered(sc[j] + 0.0f) : 0u;
+                for (int q = 0; q < QT; ++q) {
+                    uint32_t key = 0u;
+#pragma unroll
+                    for (int ri = 0; ri < R; ++ri)
+                        if ((okbits >> (ri * QT + q)) & 1u) key = max(key, float_to_ordered(sc[ri][q] + 0.0f));
                     key = __reduce_max_sync(0xFu << (lane & ~3), key);
                     // the queue is still empty: its first 128 bytes take the group maxima
                     if ((lane & 3) == 0)
-                        reinterpret_cast<uint32_t *>(sel[q].queue)[(warp & 3) * 8 + (lane >> 2)] = key;
+                        reinterpret_cast<uint32_t *>(sel[q0 + q].queue)[(warp & (kGroupWarps - 1)) * 8 + (lane >> 2)] = key;
                 }
-                consumer_bar();
+                consumer_bar<kConsumerWarps * 32>();
                 for (int q = warp; q < QB; q += kConsumerWarps) {
                     if (q >= a.B || sel[q].tau > -INFINITY) continue;                              // warp-uniform
                     unsigned long long x = reinterpret_cast<const uint32_t *>(sel[q].queue)[lane];
@@ -196,40 +221,42 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                     const uint32_t nth = (uint32_t)shfl_u64(x, a.top_n - 1);
                     if (lane == 0 && nth) sel[q].tau = share_tau(&a.gtau[q], ordered_to_float(nth));
                 }
-                consumer_bar();
+                consumer_bar<kConsumerWarps * 32>();
             }
-            uint32_t pend = 0u;                        // queries for which this row is (still) a candidate
+            uint32_t pend = 0u;                        // (row, query) pairs that are (still) candidates
 #pragma unroll
-            for (int j = 0; j < QT; ++j) {
-                const int q = q0 + j;
-                const bool take = !dead && q < a.B && row < a.N && sc[j] >= sel[q].tau && (want[j] < 0 || tok == want[j]);
-                pend |= take ? (1u << j) : 0u;
-            }
+            for (int ri = 0; ri < R; ++ri)
+#pragma unroll
+                for (int q = 0; q < QT; ++q)
+                    if (((okbits >> (ri * QT + q)) & 1u) && sc[ri][q] >= sel[q0 + q].tau) pend |= 1u << (ri * QT + q);
             // Queue the survivors; when a queue is full the candidate waits (`pend`) until the CTA
             // has folded the queues, so that adversarial row orders stay exact.
             while (true) {
-                // claim the slots first (independent shared-memory atomics in flight together), then fill them
-                int slot[QT];
+                uint32_t todo = pend;
+                while (todo) {                          // rare once the filter is warm
+                    const int b = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const int ri = b / QT, q = q0 + b % QT;
+                    float s = 0.f;                      // the pair's score without dynamic register indexing
 #pragma unroll
-                for (int j = 0; j < QT; ++j) {
-                    const int q = q0 + j;
-                    if (((pend >> j) & 1u) && !(sc[j] >= sel[q].tau)) pend &= ~(1u << j);   // the filter has tightened
-                    slot[j] = ((pend >> j) & 1u) ? atomicAdd(&sel[q].count, 1) : 0;
-                }
+                    for (int i = 0; i < R; ++i)
 #pragma unroll
-                for (int j = 0; j < QT; ++j) {
-                    const int q = q0 + j;
-                    if ((pend >> j) & 1u) {
-                        if (slot[j] < kQueueCap) {
-                            sel[q].queue[slot[j]] = pack_candidate(sc[j], (uint32_t)row);
-                            if (slot[j] + 1 >= kMergeLevel) fl->need_merge = 1;
-                            pend &= ~(1u << j);
-                        } else {
-                            fl->overflow = 1;
-                        }
+                        for (int j = 0; j < QT; ++j)
+                            if (i * QT + j == b) s = sc[i][j];
+                    if (!(s >= sel[q].tau)) {           // the filter has tightened
+                        pend &= ~(1u << b);
+                        continue;
+                    }
+                    const int slot = atomicAdd(&sel[q].count, 1);
+                    if (slot < kQueueCap) {
+                        sel[q].queue[slot] = pack_candidate(s, (uint32_t)(row0 + ri * kLanes));
+                        if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
+                        pend &= ~(1u << b);
+                    } else {
+                        fl->overflow = 1;
                     }
                 }
-                consumer_bar();                         // A: every push of this pass is visible
+                consumer_bar<kConsumerWarps * 32>();                         // A: every push of this pass is visible
                 const int need = fl->need_merge, over = fl->overflow;
                 // Flags rotate over three slots: the slot of the previous pass was read by everyone
                 // before arriving at A and is not written again before the next A.
@@ -247,12 +274,12 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                         if (lane == 0 && q < a.B) sel[q].tau = share_tau(&a.gtau[q], sel[q].tau);
                     }
                 }
-                consumer_bar();                         // C: lists, counts and tau are settled
+                consumer_bar<kConsumerWarps * 32>();                         // C: lists, counts and tau are settled
                 if (!over) break;
             }
         }
         // flush and publish this CTA's lists
-        consumer_bar();
+        consumer_bar<kConsumerWarps * 32>();
         for (int q = warp; q < min(QB, a.B); q += kConsumerWarps) {
             if (sel[q].count > 0) warp_topn_merge(&sel[q], a.top_n, lane);
             unsigned long long m = sel[q].list[lane];
@@ -266,7 +293,7 @@ template <int QB>
 size_t smem_bytes(int d, int *stages_out)
 {
     const int dpad = ((d + kSlabElems - 1) / kSlabElems) * kSlabElems;
-    size_t fixed = 1024 + sizeof(WarpTopN) * QB + 2 * kMaxStages * sizeof(uint64_t) + 4 * sizeof(SelFlags) +
+    size_t fixed = 1024 + sizeof(WarpTopN) * QB + 2 * kMaxStages * sizeof(uint64_t) + 4 * sizeof(SelFlags) + 16 +
                    sizeof(float) * (size_t)QB * dpad;
     int stages = (int)((227 * 1024 - (long long)fixed) / kStageBytes);
     if (stages > kMaxStages) stages = kMaxStages;
@@ -284,19 +311,24 @@ cudaError_t launch_one(const CUtensorMap &map, ScanArgs a, int grid, cudaStream_
     auto kernel = scan_f32_kernel<QB>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kernel<<<grid, kThreads, smem, stream>>>(map, a);
+    kernel<<<grid, (groups_of(QB) * kGroupWarps + 1) * 32, smem, stream>>>(map, a);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 int scan_f32_tile_rows(int) { return kRows; }
+int scan_f32_box_rows(int) { return kBoxRows; }
+// the queries of a launch sit in shared memory beside at least two 64 KB stages
 int scan_f32_queries_per_launch(int d, int) { return d <= 1024 ? 8 : 4; }
 
 cudaError_t launch_scan_f32(const CUtensorMap &map, const ScanArgs &a, int grid, cudaStream_t stream)
 {
-    return scan_f32_queries_per_launch(a.d, a.B) == 8 ? launch_one<8>(map, a, grid, stream)
-                                                       : launch_one<4>(map, a, grid, stream);
+    const int cap = scan_f32_queries_per_launch(a.d, a.B);
+    if (a.B <= 1) return launch_one<1>(map, a, grid, stream);
+    if (a.B <= 2) return launch_one<2>(map, a, grid, stream);
+    if (a.B <= 4 || cap == 4) return launch_one<4>(map, a, grid, stream);
+    return launch_one<8>(map, a, grid, stream);
 }
 
 }  // namespace dresd

@@ -149,7 +149,7 @@ extern "C" dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *
     const int tile_rows = f32 ? scan_f32_tile_rows(d) : scan_mma_tile_rows(d);
     const int n_tiles = (int)((N + tile_rows - 1) / tile_rows);
     CUtensorMap map;
-    if (!encode_key_map(&map, keys, (int)dtype, N, d, tile_rows))
+    if (!encode_key_map(&map, keys, (int)dtype, N, d, f32 ? scan_f32_box_rows(d) : tile_rows))
         return na_fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the key matrix");
 
     // The workspace keeps the previous call's contents.  Only the status word
