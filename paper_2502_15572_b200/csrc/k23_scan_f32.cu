@@ -10,7 +10,8 @@
 // its rows and QB broadcast LDS.128 of the queries for 16 QB FMAs.  With one row
 // per thread (the first form) the loop was bound by shared-memory instruction
 // issue, 5 LDS.128 per 16 FMAs: 2.5 TB/s on a large store at any batch.  Four
-// partial sums per (row, query) keep the accumulation error near d/4 ulps.
+// partial sums per (row, query), advanced in pairs by packed FMAs (fma.rn.f32x2),
+// keep the accumulation error near d/4 ulps.
 // QB is the batch rounded up to 1, 2, 4 or 8: a single query pays for one.  Eight
 // queries are split over two groups of four warps (the same rows, four queries each):
 // 128 accumulators per thread would leave no registers for the loads in flight.
@@ -144,13 +145,15 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 const long long row = row0 + ri * kLanes;
                 tok[ri] = (a.first_col && row < a.N) ? a.first_col[row] : 0;
             }
-            float acc[R][QT][4];
+            // four partial sums per (row, query), held as two pairs: one packed FMA (two IEEE fp32
+            // FMAs in one instruction) advances a pair
+            float2 acc[R][QT][2];
 #pragma unroll
             for (int ri = 0; ri < R; ++ri)
 #pragma unroll
                 for (int q = 0; q < QT; ++q)
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) acc[ri][q][i] = 0.f;
+                    for (int i = 0; i < 2; ++i) acc[ri][q][i] = make_float2(0.f, 0.f);
             for (int sl = 0; sl < dslabs; ++sl) {
                 const int it = tl * dslabs + sl;
                 const int s = it % n_stages;
@@ -173,10 +176,8 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                         const float4 q4 = *reinterpret_cast<const float4 *>(qbase + (size_t)q * dpad + c * 4);
 #pragma unroll
                         for (int ri = 0; ri < R; ++ri) {
-                            acc[ri][q][0] = fmaf(q4.x, k4[ri].x, acc[ri][q][0]);
-                            acc[ri][q][1] = fmaf(q4.y, k4[ri].y, acc[ri][q][1]);
-                            acc[ri][q][2] = fmaf(q4.z, k4[ri].z, acc[ri][q][2]);
-                            acc[ri][q][3] = fmaf(q4.w, k4[ri].w, acc[ri][q][3]);
+                            acc[ri][q][0] = __ffma2_rn(make_float2(q4.x, q4.y), make_float2(k4[ri].x, k4[ri].y), acc[ri][q][0]);
+                            acc[ri][q][1] = __ffma2_rn(make_float2(q4.z, q4.w), make_float2(k4[ri].z, k4[ri].w), acc[ri][q][1]);
                         }
                     }
                 }
@@ -192,7 +193,7 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             for (int ri = 0; ri < R; ++ri)
 #pragma unroll
                 for (int q = 0; q < QT; ++q) {
-                    sc[ri][q] = (acc[ri][q][0] + acc[ri][q][1]) + (acc[ri][q][2] + acc[ri][q][3]);
+                    sc[ri][q] = (acc[ri][q][0].x + acc[ri][q][0].y) + (acc[ri][q][1].x + acc[ri][q][1].y);
                     const bool ok = !dead && q0 + q < a.B && row0 + ri * kLanes < a.N && sc[ri][q] > -INFINITY &&   // false for NaN
                                     (want[q] < 0 || tok[ri] == want[q]);
                     okbits |= ok ? (1u << (ri * QT + q)) : 0u;
