@@ -333,7 +333,7 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "pack2"      1 (default): the quantised search of a store with d = 64 scans the 8-bit copy
  *                as rows of two keys (one 128-byte line), up to 32 queries per call; 0 = one
  *                key per row.  Results do not change.
- *   "keys_as_m"  0 (default): batches of 33-64 queries on rows of 129-256 elements run the
+ *   "keys_as_m"  0 (default): batches of 17-64 queries on rows of 129-256 elements run the
  *                tcgen05 kernel with the queries as the M = 128 and the keys as the
  *                N = 256 operand of the instruction; 1 = keys as the M operand at every
  *                batch size (the form all other shapes use).  Results do not change.

@@ -268,12 +268,13 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // against 6.7-6.8 for the streaming mma.sync kernel), so it is the default; the
     // streaming kernel stays available as "scan_path" 1 and serves the allocation-free call.
     const bool umma = q8 || (!f32 && s->opt_path != 1);
-    const int op_rows = umma ? scan_umma_operand_rows(pack2 ? 2 * B : B) : 0;
     // sorted store with an index: the kernel with the keys as M scans the queries' token windows only
     const bool windows = umma && first_tokens && s->win_start && s->opt_windows;
     const int keys_as_m = (q8 || s->opt_keys_as_m || windows) ? 1 : 0;
-    // the kernel with the keys as the N operand reads hi and lo of a query from one TMEM fragment
+    // the kernel with the keys as the N operand reads hi and lo of a query from one TMEM fragment;
+    // its operand always has 128 rows (64 hi, 64 lo), whatever the batch
     const int blocked = umma && !keys_as_m && scan_ummat_eligible(s->d, B);
+    const int op_rows = !umma ? 0 : blocked ? 2 * kMaxBatch : scan_umma_operand_rows(pack2 ? 2 * B : B);
     // one CTA per operand query: two operand rows each, four in the packed 8-bit layout
     const int pre_rows = pack2 ? op_rows / 4 : umma ? op_rows / 2 : ((B + 7) / 8) * 8;
     dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, blocked, pack2 ? 2 : q8 ? 1 : 0);

@@ -92,7 +92,7 @@ int scan_umma_operand_rows(int B);
 cudaError_t launch_scan_umma(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
                              int grid, cudaStream_t stream);
 
-// Same path for 33-64 queries on rows of 129-256 elements: queries as the M = 128 operand,
+// Same path for 17-64 queries on rows of 129-256 elements: queries as the M = 128 operand,
 // keys as the N = 256 operand (256-key tiles).  launch_scan_umma() dispatches to it.
 bool scan_ummat_eligible(int d, int B);
 cudaError_t launch_scan_ummat(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,

@@ -1,4 +1,4 @@
-// K2+K3 for 33-64 queries on 16-bit keys of 129-256 elements -- Eq. 3 of the paper for
+// K2+K3 for 17-64 queries on 16-bit keys of 129-256 elements -- Eq. 3 of the paper for
 // every key, fused with the per-CTA top-n, with the operand roles of the tensor-core
 // instruction swapped: the QUERIES are the M = 128 operand (two rows per query: q = hi +
 // lo/scale) and the KEYS are the N = 256 operand.
@@ -460,13 +460,16 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
 
 }  // namespace
 
-// This kernel serves 33-64 queries on rows of three or four 64-element slabs (129-256 elements).
+// This kernel serves 17-64 queries on rows of three or four 64-element slabs (129-256 elements):
+// its cost does not depend on the batch (the operand always has 128 rows), and from 17 queries on it
+// beats the form with the keys as M (10M x 256 bf16: 0.75 against 0.90 ms at 17-32 queries; 9-16
+// queries measured equal or slightly worse, 0.742-0.748 against 0.736-0.738 ms).
 // On narrower rows it works too but measured no better than the other tcgen05 kernel (the
 // epilogue, ~2.7 k cycles per 256 keys, is then slower than the memory stream in both).
 bool scan_ummat_eligible(int d, int B)
 {
     const int dslabs = (d + kSlabElems - 1) / kSlabElems;
-    return B > 32 && B <= kNQ && dslabs >= 3 && dslabs <= 4;
+    return B > 16 && B <= kNQ && dslabs >= 3 && dslabs <= 4;
 }
 
 cudaError_t launch_scan_ummat(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a_in, int grid,
