@@ -324,14 +324,19 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                             for (int j = 0; j < dslabs; ++j) {
                                 const uint64_t a_desc = make_desc(st_addr + (uint32_t)((sub * dslabs + j) * slab_bytes));
                                 const uint64_t b_desc = make_desc(smem_u32(qres + (size_t)j * kQSlabBytes));
+                                // a last slab that the row fills only in part (zeros beyond d) needs only
+                                // the 32-byte steps that hold data
+                                const int ksteps = min(4, (a.d - j * kSlabElems + 15) / 16);
 #pragma unroll
-                                for (int k = 0; k < 4; ++k)
+                                for (int k = 0; k < 4; ++k) {
+                                    if (k >= ksteps) break;
                                     if constexpr (kIs8)
                                         umma_f8(d_tmem + (uint32_t)(sub * NCOLS), a_desc + 2 * k, b_desc + 2 * k, idesc,
                                                 (j + k) != 0);
                                     else
                                         umma_f16(d_tmem + (uint32_t)(sub * NCOLS), a_desc + 2 * k, b_desc + 2 * k, idesc,
                                                  (j + k) != 0);
+                                }
                             }
                     } else {
                         const int sl0 = g * gs;
@@ -341,10 +346,13 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                             const uint32_t b_addr = q_resident ? smem_u32(qres + (size_t)(sl0 + j) * kQSlabBytes)
                                                                : a_addr + kKeyStageBytes;
                             const uint64_t a_desc = make_desc(a_addr), b_desc = make_desc(b_addr);
+                            const int ksteps = min(4, (a.d - (sl0 + j) * kSlabElems + 15) / 16);
 #pragma unroll
-                            for (int k = 0; k < 4; ++k)   // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
+                            for (int k = 0; k < 4; ++k) {  // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
+                                if (k >= ksteps) break;
                                 if constexpr (kIs8) umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
                                 else umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
+                            }
                         }
                     }
                     tc_commit(&empty[s]);             // group reusable once these MMAs have read it
@@ -695,8 +703,8 @@ Plan make_plan(int d, int B)
     } else {
         // Largest slab group (fewest barrier round trips per tile) that still leaves
         // at least three groups in flight.
-        for (int gs = 4; gs >= 1; gs >>= 1) {
-            if (gs > dslabs && gs > 1) continue;
+        for (int gs = 4; gs >= 1; --gs) {
+            if (gs > dslabs && gs > 1) continue;          // three-slab rows: one group of three per tile
             long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)(gs * slab);
             if (s > kMaxStages) s = kMaxStages;
             p.gs = gs;

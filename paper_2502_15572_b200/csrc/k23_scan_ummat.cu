@@ -214,9 +214,12 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
                     tc_fence_after();
                     const uint64_t a_desc = make_desc(smem_u32(qres + (size_t)ks * kQSlabBytes));
                     const uint64_t b_desc = make_desc(smem_u32(stages + (size_t)s * kStageBytes));
+                    // 4 x K=16 inside the 128-byte swizzle row, +32 bytes each; a last slab that the row
+                    // fills only in part (zeros beyond d) needs only the steps that hold data
+                    const int ksteps = min(4, (a.d - ks * kSlabElems + 15) / 16);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)      // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
-                        umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (ks | k) != 0);
+                    for (int k = 0; k < 4; ++k)
+                        if (k < ksteps) umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (ks | k) != 0);
                     tc_commit(&empty[s]);            // slab reusable once these MMAs have read it
                 }
                 if (!ok) break;
