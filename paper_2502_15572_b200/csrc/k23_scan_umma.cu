@@ -372,8 +372,12 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         const int lane_grp = warp & 3;
         const int half = ew >> 2;
         const int et = ew * 32 + lane;
-        const int qbase = half * QW;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(half * CW);
+        // Few queries on narrow rows (all of them within one warp's columns, several sub-tiles per
+        // tile): the two warps of a lane group split the SUB-TILES instead, so that neither spends
+        // its time on columns of padding.
+        const bool split_subs = TSUB >= 2 && (PACK2 ? 2 * a.B : a.B) <= QW;
+        const int qbase = split_subs ? 0 : half * QW;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(qbase * 2);
         const float inv = a.lo_inv_scale;
         const float4 *tau4 = reinterpret_cast<const float4 *>(tau + qbase);
         const int4 *want4 = reinterpret_cast<const int4 *>(want_s + qbase);
@@ -445,6 +449,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 // largest of all CTAs' bests is a valid filter: at least n rows reach it.
 #pragma unroll
                 for (int sub = 0; sub < TSUB; ++sub) {
+                    if (split_subs && (sub & 1) != half) continue;
                     const long long row = row0 + sub * kTileRows;
                     const bool row_ok = row < a.N;
                     unsigned long long *slot = tilemax + (size_t)(sub * 4 + lane_grp) * NQ + qbase;
@@ -506,6 +511,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 }
 #pragma unroll
                 for (int sub = 0; sub < TSUB; ++sub) {
+                    if (split_subs && (sub & 1) != half) continue;
                     const uint32_t ok = okmask_of(row0 + sub * kTileRows);
                     const int slot = (sub * 4 + lane_grp) * kGroupsPerUnit + lane / kGroupRows;
                     for (uint32_t m = todo; m; m &= m - 1) {            // warp-uniform
@@ -561,7 +567,9 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     const long long row = row0 + sub * kTileRows;
                     const uint32_t okmask = okmask_of(row);
                     // warp-uniform decision: tcgen05.ld needs the whole warp
-                    if (dead || !(first || __any_sync(0xFFFFFFFFu, pending[sub] != 0u))) continue;
+                    if (dead || (split_subs && (sub & 1) != half) ||
+                        !(first || __any_sync(0xFFFFFFFFu, pending[sub] != 0u)))
+                        continue;
                     uint32_t r[CW];
                     tmem_ld_cols<CW>(acc_addr + (uint32_t)(sub * NCOLS), r);
                     tmem_ld_wait();
