@@ -31,7 +31,15 @@ namespace dresd {
 namespace {
 
 constexpr int kEpiWarps = 8;
-constexpr int kThreads = (2 + kEpiWarps) * 32;
+// Two threads issue the MMAs where the instruction stream would otherwise set the pace (one
+// tcgen05.mma per ~85 ns from one thread = 4 KB of keys, level with what HBM delivers): on narrow rows they
+// take alternate sub-tiles; on wide rows with at most 16 queries alternate 64-element slabs, into two
+// accumulator sets that the epilogue adds.
+constexpr bool dual_possible(int tsub, int ncols) { return tsub == 1 && ncols <= 32; }
+constexpr int threads_of(int tsub, bool dual) { return (2 + kEpiWarps + ((tsub > 1 || dual) ? 1 : 0)) * 32; }
+// Measured against one issuer on 3 GB stores at 1 and 8 queries: rows of 3-6 slabs 5-14 % faster (d = 256:
+// 0.775 -> 0.739 ms on 10M rows), 16 and more slabs 2-6 % faster, 8 and 12 slabs 4-6 % slower.
+inline bool dual_pays(int dslabs) { return dslabs <= 6 || dslabs >= 16; }
 constexpr int kTileRows = 128;
 constexpr int kSlabBytes = 128;
 constexpr int kSlabElems = 64;
@@ -119,13 +127,14 @@ struct Windows {
 // that score the even and the odd key of a row; both feed the lists and the filter of query j,
 // and a candidate's id is 2 * row + parity.  tau[] is kept per virtual query (two equal
 // entries per query) so that the hot loop is the same code.
-template <typename T, int NCOLS, int TSUB, bool PACK2 = false>
-__global__ void __launch_bounds__(kThreads, 1)
+template <typename T, int NCOLS, int TSUB, bool PACK2 = false, bool DUAL = false>
+__global__ void __launch_bounds__(threads_of(TSUB, DUAL), 1)
 scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_constant__ CUtensorMap q_map,
                  const ScanArgs a, const int q_resident, const int gs)
 {
     constexpr int NQ = NCOLS / 2;                           // queries (padded)
-    constexpr int kAccCols = TSUB * NCOLS;                  // one accumulator buffer
+    static_assert(!DUAL || dual_possible(TSUB, NCOLS), "two accumulator sets: wide rows, at most 16 queries");
+    constexpr int kAccCols = TSUB * NCOLS * (DUAL ? 2 : 1); // one accumulator buffer
     constexpr int kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;
     static_assert(kTmemCols <= 512, "TMEM has 512 columns");
     constexpr int kQSlabBytes = NCOLS * kSlabBytes;
@@ -159,16 +168,20 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
     constexpr int kRowsPerTile = kTileRows * TSUB;
+    // Narrow rows: the sub-tiles of a tile have accumulators of their own, so two threads (warps 1
+    // and 10) issue the MMAs of alternate sub-tiles; each commits to the barriers for its share.
+    constexpr int kIssuers = (TSUB > 1 || DUAL) ? 2 : 1;
+    constexpr int kIssuer2Warp = 2 + kEpiWarps;
 
     if (tid == 0) {
         tma_prefetch_desc(&keys_map);                       // kernel parameters: nothing to wait for
         tma_prefetch_desc(&q_map);
         for (int s = 0; s < n_stages; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&empty[s], 1);
+            mbar_init(&empty[s], kIssuers);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&tfull[b], 1);
+            mbar_init(&tfull[b], kIssuers);
             mbar_init(&tempty[b], kEpiWarps);
         }
         mbar_init(qbar, 1);
@@ -186,7 +199,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     // (the query operand, the reset filter words).
     pdl_wait();
     pdl_launch_dependents();
-    if (warp >= 2) {
+    if (warp >= 2 && warp < kIssuer2Warp) {
         for (int q = warp - 2; q < NQ; q += kEpiWarps) {
             warp_topn_init(&sel[q], lane);
             // start from whatever the grid already knows; padding columns never pass
@@ -298,9 +311,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 }
             if (q_resident && !mbar_wait(qbar, 0)) report_timeout(a.status);
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == kIssuer2Warp) {
         // ---------------------------------- MMA issuer ----------------------------------
-        if (lane == 0) {
+        const int issuer = warp == 1 ? 0 : 1;
+        if (lane == 0 && issuer < kIssuers) {
             // operand formats: kind::f16 -- 0 = fp16, 1 = bf16; kind::f8f6f4 -- 0 = E4M3
             constexpr bool kIs8 = std::is_same<T, E4M3Keys>::value;
             constexpr uint32_t kFmt = std::is_same<T, __nv_bfloat16>::value ? 1u : 0u;
@@ -320,7 +334,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     tc_fence_after();
                     const uint32_t st_addr = smem_u32(stages + (size_t)s * stage_bytes);
                     if constexpr (TSUB > 1) {
-                        for (int sub = 0; sub < TSUB; ++sub)
+                        for (int sub = issuer; sub < TSUB; sub += kIssuers)
                             for (int j = 0; j < dslabs; ++j) {
                                 const uint64_t a_desc = make_desc(st_addr + (uint32_t)((sub * dslabs + j) * slab_bytes));
                                 const uint64_t b_desc = make_desc(smem_u32(qres + (size_t)j * kQSlabBytes));
@@ -342,6 +356,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         const int sl0 = g * gs;
                         const int nsl = min(gs, dslabs - sl0);
                         for (int j = 0; j < nsl; ++j) {
+                            if (DUAL && ((sl0 + j) & 1) != issuer) continue;      // the other thread's slab
                             const uint32_t a_addr = st_addr + (uint32_t)(j * slab_bytes);
                             const uint32_t b_addr = q_resident ? smem_u32(qres + (size_t)(sl0 + j) * kQSlabBytes)
                                                                : a_addr + kKeyStageBytes;
@@ -350,8 +365,11 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {  // 4 x K=16 inside the 128-byte swizzle row: +32 bytes each
                                 if (k >= ksteps) break;
-                                if constexpr (kIs8) umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
-                                else umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (sl0 + j + k) != 0);
+                                // a set starts afresh with the first step of its first slab (slab 0 or 1)
+                                const uint32_t d_set = d_tmem + (DUAL ? (uint32_t)(issuer * NCOLS) : 0u);
+                                const bool accumulate = (DUAL ? (sl0 + j - issuer) : (sl0 + j)) + k != 0;
+                                if constexpr (kIs8) umma_f8(d_set, a_desc + 2 * k, b_desc + 2 * k, idesc, accumulate);
+                                else umma_f16(d_set, a_desc + 2 * k, b_desc + 2 * k, idesc, accumulate);
                             }
                         }
                     }
@@ -362,7 +380,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             }
             if (!ok) report_timeout(a.status);
         }
-    } else {
+    } else if (warp < kIssuer2Warp) {
         // ---------------------------------- epilogue ----------------------------------
         // Eight warps: warp w may read TMEM lanes 32*(w&3)..+31 (one key row per thread and
         // sub-tile); the two warps that share a lane group split the accumulator columns.
@@ -379,6 +397,28 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         const int qbase = split_subs ? 0 : half * QW;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(qbase * 2);
         const float inv = a.lo_inv_scale;
+        // accumulator reads (issued only; the caller waits): with two sets, set B (NCOLS columns further)
+        // is added to set A -- the sum of the even and of the odd slabs' partial products
+        auto ld_cols = [&](uint32_t addr, uint32_t (&r)[CW]) {
+            tmem_ld_cols<CW>(addr, r);
+            if constexpr (DUAL) {
+                uint32_t r2[CW];
+                tmem_ld_cols<CW>(addr + NCOLS, r2);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < CW; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+            }
+        };
+        auto ld_pair = [&](uint32_t addr, uint32_t &v0, uint32_t &v1) {
+            tmem_ld2(addr, v0, v1);
+            if constexpr (DUAL) {
+                uint32_t w0, w1;
+                tmem_ld2(addr + NCOLS, w0, w1);
+                tmem_ld_wait();
+                v0 = __float_as_uint(__uint_as_float(v0) + __uint_as_float(w0));
+                v1 = __float_as_uint(__uint_as_float(v1) + __uint_as_float(w1));
+            }
+        };
         const float4 *tau4 = reinterpret_cast<const float4 *>(tau + qbase);
         const int4 *want4 = reinterpret_cast<const int4 *>(want_s + qbase);
         const bool filtered = a.first_col != nullptr && !win_on;    // windows carry their token
@@ -455,7 +495,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     unsigned long long *slot = tilemax + (size_t)(sub * 4 + lane_grp) * NQ + qbase;
                     if (!dead) {
                         uint32_t r[CW];
-                        tmem_ld_cols<CW>(acc_addr + (uint32_t)(sub * NCOLS), r);
+                        ld_cols(acc_addr + (uint32_t)(sub * NCOLS), r);
                         tmem_ld_wait();
                         unsigned long long v[QW];
 #pragma unroll
@@ -519,7 +559,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         uint32_t key = 0u;
                         if (!dead) {
                             uint32_t v0, v1;
-                            tmem_ld2(acc_addr + (uint32_t)(sub * NCOLS + 2 * j), v0, v1);
+                            ld_pair(acc_addr + (uint32_t)(sub * NCOLS + 2 * j), v0, v1);
                             tmem_ld_wait();
                             const float sc = fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
                             bool valid = ((ok >> j) & 1u) && sc > -INFINITY;            // false for NaN
@@ -571,7 +611,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         !(first || __any_sync(0xFFFFFFFFu, pending[sub] != 0u)))
                         continue;
                     uint32_t r[CW];
-                    tmem_ld_cols<CW>(acc_addr + (uint32_t)(sub * NCOLS), r);
+                    ld_cols(acc_addr + (uint32_t)(sub * NCOLS), r);
                     tmem_ld_wait();
                     // Hot part, branch-free and compact: one bit per query whose score
                     // reaches the filter.
@@ -609,7 +649,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         const int j = __ffs(wm) - 1;
                         wm &= wm - 1;
                         uint32_t v0, v1;
-                        tmem_ld2(acc_addr + (uint32_t)(sub * NCOLS + 2 * j), v0, v1);
+                        ld_pair(acc_addr + (uint32_t)(sub * NCOLS + 2 * j), v0, v1);
                         tmem_ld_wait();
                         if ((mask >> j) & 1u) {
                             const float s = fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
@@ -731,10 +771,21 @@ cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const S
     if constexpr (2 * TSUB * NCOLS > 512) {
         return cudaErrorInvalidValue;
     } else {
-        auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2>;
+        const int dslabs = (a.d + kSlabElems - 1) / kSlabElems;
+        if constexpr (dual_possible(TSUB, NCOLS)) {
+            if (dual_pays(dslabs)) {
+                auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, true>;
+                cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
+                if (e != cudaSuccess) return e;
+                return launch_dependent(kernel, dim3(grid), dim3(threads_of(TSUB, true)), p.smem, stream, kmap, qmap, a,
+                                        p.q_resident, p.gs);
+            }
+        }
+        auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, false>;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
         if (e != cudaSuccess) return e;
-        return launch_dependent(kernel, dim3(grid), dim3(kThreads), p.smem, stream, kmap, qmap, a, p.q_resident, p.gs);
+        return launch_dependent(kernel, dim3(grid), dim3(threads_of(TSUB, false)), p.smem, stream, kmap, qmap, a,
+                                p.q_resident, p.gs);
     }
 }
 
