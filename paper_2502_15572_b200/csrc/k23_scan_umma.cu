@@ -33,13 +33,14 @@ namespace {
 constexpr int kEpiWarps = 8;
 // Two threads issue the MMAs where the instruction stream would otherwise set the pace (one
 // tcgen05.mma per ~85 ns from one thread = 4 KB of keys, level with what HBM delivers): on narrow rows they
-// take alternate sub-tiles; on wide rows with at most 16 queries alternate 64-element slabs, into two
+// take alternate sub-tiles; on wide rows alternate 64-element slabs, into two
 // accumulator sets that the epilogue adds.
-constexpr bool dual_possible(int tsub, int ncols) { return tsub == 1 && ncols <= 32; }
+constexpr bool dual_possible(int tsub, int ncols) { return tsub == 1 && 4 * ncols <= 512; }
 constexpr int threads_of(int tsub, bool dual) { return (2 + kEpiWarps + ((tsub > 1 || dual) ? 1 : 0)) * 32; }
-// Measured against one issuer on 3 GB stores at 1 and 8 queries: rows of 3-6 slabs 5-14 % faster (d = 256:
-// 0.775 -> 0.739 ms on 10M rows), 16 and more slabs 2-6 % faster, 8 and 12 slabs 4-6 % slower.
-inline bool dual_pays(int dslabs) { return dslabs <= 6 || dslabs >= 16; }
+// Measured against one issuer on 3 GB stores.  Up to 16 queries: rows of 3-6 slabs 5-14 % faster (d = 256:
+// 0.775 -> 0.739 ms on 10M rows), 16 and more slabs 2-6 % faster, 8 and 12 slabs 4-6 % slower.  17-64 queries
+// (rows wider than 256 elements): 10-25 % faster at every width.
+inline bool dual_pays(int dslabs, int ncols) { return ncols >= 64 || dslabs <= 6 || dslabs >= 16; }
 constexpr int kTileRows = 128;
 constexpr int kSlabBytes = 128;
 constexpr int kSlabElems = 64;
@@ -133,7 +134,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                  const ScanArgs a, const int q_resident, const int gs)
 {
     constexpr int NQ = NCOLS / 2;                           // queries (padded)
-    static_assert(!DUAL || dual_possible(TSUB, NCOLS), "two accumulator sets: wide rows, at most 16 queries");
+    static_assert(!DUAL || dual_possible(TSUB, NCOLS), "two accumulator sets: wide rows only");
     constexpr int kAccCols = TSUB * NCOLS * (DUAL ? 2 : 1); // one accumulator buffer
     constexpr int kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;
     static_assert(kTmemCols <= 512, "TMEM has 512 columns");
@@ -402,11 +403,16 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         auto ld_cols = [&](uint32_t addr, uint32_t (&r)[CW]) {
             tmem_ld_cols<CW>(addr, r);
             if constexpr (DUAL) {
-                uint32_t r2[CW];
-                tmem_ld_cols<CW>(addr + NCOLS, r2);
-                tmem_ld_wait();
+                constexpr int CH = CW < 16 ? CW : 16;       // set B in chunks: 16 registers, not CW more
 #pragma unroll
-                for (int i = 0; i < CW; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+                for (int c = 0; c < CW / CH; ++c) {
+                    uint32_t r2[CH];
+                    tmem_ld_cols<CH>(addr + NCOLS + c * CH, r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < CH; ++i)
+                        r[c * CH + i] = __float_as_uint(__uint_as_float(r[c * CH + i]) + __uint_as_float(r2[i]));
+                }
             }
         };
         auto ld_pair = [&](uint32_t addr, uint32_t &v0, uint32_t &v1) {
@@ -773,7 +779,7 @@ cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const S
     } else {
         const int dslabs = (a.d + kSlabElems - 1) / kSlabElems;
         if constexpr (dual_possible(TSUB, NCOLS)) {
-            if (dual_pays(dslabs)) {
+            if (dual_pays(dslabs, NCOLS)) {
                 auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, true>;
                 cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
                 if (e != cudaSuccess) return e;
