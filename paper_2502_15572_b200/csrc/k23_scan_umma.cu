@@ -40,7 +40,12 @@ constexpr int threads_of(int tsub, bool dual) { return (2 + kEpiWarps + ((tsub >
 // Measured against one issuer on 3 GB stores.  Up to 16 queries: rows of 3-6 slabs 5-14 % faster (d = 256:
 // 0.775 -> 0.739 ms on 10M rows), 16 and more slabs 2-6 % faster, 8 and 12 slabs 4-6 % slower.  17-64 queries
 // (rows wider than 256 elements): 10-25 % faster at every width.
-inline bool dual_pays(int dslabs, int ncols) { return ncols >= 64 || dslabs <= 6 || dslabs >= 16; }
+// Rows of 3-4 slabs with more than 16 queries normally run the kernel with the keys as N; when they come
+// here (token windows, "keys_as_m") they keep one accumulator set, whose sums are bit-identical to that kernel's.
+inline bool dual_pays(int dslabs, int ncols)
+{
+    return ncols >= 64 ? dslabs > 4 : (dslabs <= 6 || dslabs >= 16);
+}
 constexpr int kTileRows = 128;
 constexpr int kSlabBytes = 128;
 constexpr int kSlabElems = 64;
