@@ -37,14 +37,16 @@ constexpr int kEpiWarps = 8;
 // accumulator sets that the epilogue adds.
 constexpr bool dual_possible(int tsub, int ncols) { return tsub == 1 && 4 * ncols <= 512; }
 constexpr int threads_of(int tsub, bool dual) { return (2 + kEpiWarps + ((tsub > 1 || dual) ? 1 : 0)) * 32; }
-// Measured against one issuer on 3 GB stores.  Up to 16 queries: rows of 3-6 slabs 5-14 % faster (d = 256:
-// 0.775 -> 0.739 ms on 10M rows), 16 and more slabs 2-6 % faster, 8 and 12 slabs 4-6 % slower.  17-64 queries
-// (rows wider than 256 elements): 10-25 % faster at every width.
+// Measured against one issuer on 3 GB stores.  Up to 8 queries: rows of 3-6 slabs 5-14 % faster (d = 256:
+// 0.775 -> 0.739 ms on 10M rows), 15 and more slabs 2-6 % faster, 7-12 slabs 4-10 % slower.  9-16 queries:
+// faster at every width (d = 512: 0.51 -> 0.45 ms).  17-64 queries (rows wider than 256): 10-25 % faster.
 // Rows of 3-4 slabs with more than 16 queries normally run the kernel with the keys as N; when they come
 // here (token windows, "keys_as_m") they keep one accumulator set, whose sums are bit-identical to that kernel's.
 inline bool dual_pays(int dslabs, int ncols)
 {
-    return ncols >= 64 ? dslabs > 4 : (dslabs <= 6 || dslabs >= 16);
+    if (ncols >= 64) return dslabs > 4;
+    if (ncols == 32) return true;                     // 9-16 queries: 6-20 % faster at every width measured
+    return dslabs <= 6 || dslabs >= 15;               // up to 8 queries: 7-12 slabs measured 4-10 % slower
 }
 constexpr int kTileRows = 128;
 constexpr int kSlabBytes = 128;
