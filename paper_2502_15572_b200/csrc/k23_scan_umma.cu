@@ -403,6 +403,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         // its time on columns of padding.
         const bool split_subs = TSUB >= 2 && (PACK2 ? 2 * a.B : a.B) <= QW;
         const int qbase = split_subs ? 0 : half * QW;
+        // a warp whose columns are all padding (few queries, one sub-tile per tile) only keeps the barriers
+        const bool no_cols = qbase >= (PACK2 ? 2 * a.B : a.B);
         const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(qbase * 2);
         const float inv = a.lo_inv_scale;
         // accumulator reads (issued only; the caller waits): with two sets, set B (NCOLS columns further)
@@ -502,7 +504,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 // largest of all CTAs' bests is a valid filter: at least n rows reach it.
 #pragma unroll
                 for (int sub = 0; sub < TSUB; ++sub) {
-                    if (split_subs && (sub & 1) != half) continue;
+                    if ((split_subs && (sub & 1) != half) || no_cols) continue;
                     const long long row = row0 + sub * kTileRows;
                     const bool row_ok = row < a.N;
                     unsigned long long *slot = tilemax + (size_t)(sub * 4 + lane_grp) * NQ + qbase;
@@ -564,7 +566,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 }
 #pragma unroll
                 for (int sub = 0; sub < TSUB; ++sub) {
-                    if (split_subs && (sub & 1) != half) continue;
+                    if ((split_subs && (sub & 1) != half) || no_cols) continue;
                     const uint32_t ok = okmask_of(row0 + sub * kTileRows);
                     const int slot = (sub * 4 + lane_grp) * kGroupsPerUnit + lane / kGroupRows;
                     for (uint32_t m = todo; m; m &= m - 1) {            // warp-uniform
@@ -620,7 +622,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     const long long row = row0 + sub * kTileRows;
                     const uint32_t okmask = okmask_of(row);
                     // warp-uniform decision: tcgen05.ld needs the whole warp
-                    if (dead || (split_subs && (sub & 1) != half) ||
+                    if (dead || no_cols || (split_subs && (sub & 1) != half) ||
                         !(first || __any_sync(0xFFFFFFFFu, pending[sub] != 0u)))
                         continue;
                     uint32_t r[CW];
