@@ -4,7 +4,7 @@
 // ridge): tensor cores are used so that the arithmetic of B queries hides
 // under ONE pass over the keys.
 //
-// One persistent CTA per SM, ten warps:
+// One persistent CTA per SM, ten or eleven warps:
 //   warp 0    producer: one thread streams 128-row x 64-column key slabs
 //             (16 KB, 128-byte swizzle) with TMA through an mbarrier ring and,
 //             when the query operand is too large to stay resident, the
@@ -14,7 +14,9 @@
 //             instruction, fp32 accumulators in TMEM, two accumulator buffers
 //             so that the epilogue of tile t overlaps the MMAs of tile t+1);
 //             tcgen05.commit releases shared-memory stages and publishes
-//             finished accumulators;
+//             finished accumulators; where the instruction stream would set the pace, a
+//             second issuing thread (warp 10) takes half of the instructions (see
+//             threads_of() below);
 //   warps 2-9 epilogue: each thread owns one key row of the tile and half of
 //             its N accumulator columns (two warps share a TMEM lane group),
 //             reads them with tcgen05.ld, combines hi and lo, filters against
