@@ -337,6 +337,9 @@ dresd_status dresd_store_status(dresd_store *store);
  *                tcgen05 kernel with the queries as the M = 128 and the keys as the
  *                N = 256 operand of the instruction; 1 = keys as the M operand at every
  *                batch size (the form all other shapes use).  Results do not change.
+ *   "first_token_windows"  1 (default): on a store indexed by dresd_store_index_first_tokens()
+ *                filtered calls scan only the rows of their queries' tokens; 0 = scan every row.
+ *                Results do not change.
  *   "wait_ms"    bound of the device-side waits of the streaming kernels in
  *                milliseconds (0 = default, about 2 s).
  *   "debug_lose_stage"  test hook: in the next calls the streaming 16-bit kernel's
