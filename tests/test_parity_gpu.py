@@ -44,6 +44,38 @@ def test_parity_shapes(dtype, d, B, n, L, N):
     _check(keys, toks, dtype, q, n, L)
 
 
+# One case per form of the tcgen05 kernel's MMA issue and of the fp32 loop: two issuer threads on
+# alternate sub-tiles (narrow rows), on alternate slabs into two accumulator sets (wide rows), the
+# single-issuer exceptions, ragged last slabs (steps beyond the row width are skipped), three-slab
+# stage groups, the epilogue's sub-tile split for few queries, 17-32 queries with the keys as N,
+# and every fp32 register tile (1, 2, 4, 8 queries; more than 8 = several passes).
+@pytest.mark.parametrize("dtype,d,B,n,L,N", [
+    ("f16", 32, 1, 10, 4, 148 * 512 + 301),     # half-filled slab, 4 sub-tiles, sub-tile split
+    ("bf16", 96, 3, 10, 4, 60013),              # 1.5 slabs, 2 sub-tiles
+    ("f16", 160, 1, 10, 4, 40009),              # 2.5 slabs: one group of three per tile, two sets
+    ("bf16", 192, 12, 16, 4, 40009),            # three full slabs, 9-16 queries
+    ("f16", 256, 16, 10, 4, 148 * 128 * 2 + 9), # two sets, 32 accumulator columns
+    ("bf16", 256, 20, 10, 4, 40009),            # 17-32 queries: keys as the N operand
+    ("f16", 200, 32, 32, 4, 30011),
+    ("bf16", 512, 2, 10, 4, 30011),             # 8 slabs, few queries: one issuer
+    ("f16", 512, 12, 10, 4, 30011),             # 8 slabs, 9-16 queries: two sets
+    ("bf16", 960, 3, 10, 4, 10007),             # 15 slabs, few queries: two sets
+    ("f16", 320, 24, 10, 4, 20011),             # 17-32 queries, wider than 256: two sets, 64 columns
+    ("bf16", 448, 64, 32, 4, 20011),            # 64 queries, 7 slabs: two sets, 128 columns (all of TMEM)
+    ("f16", 1024, 48, 10, 4, 6007),
+    ("f32", 128, 1, 10, 4, 148 * 512 * 2 + 77),
+    ("f32", 96, 2, 10, 4, 60013),
+    ("f32", 256, 4, 32, 4, 40009),
+    ("f32", 64, 8, 10, 4, 148 * 512 + 5),
+    ("f32", 2048, 3, 10, 4, 3001),              # wide fp32 rows: four queries per launch
+    ("f32", 40, 13, 5, 2, 20011),
+])
+def test_parity_kernel_forms(dtype, d, B, n, L, N):
+    keys, toks = synth.make_store(7300 + d + B, N, d, 32, dtype, L + 1)
+    q, _ = synth.make_queries(7400 + d + B, keys, dtype, B, 0.1)
+    _check(keys, toks, dtype, q, n, L)
+
+
 # Both 16-bit scoring kernels at every batch size: path 1 = streaming mma.sync kernel
 # (several passes when B > 8), path 2 = tcgen05/TMEM kernel (one pass, operand padded).
 @pytest.mark.parametrize("path", [1, 2])
