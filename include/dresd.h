@@ -237,7 +237,8 @@ dresd_status dresd_fit_zscore(const void *sample, int64_t N, int d_in, dresd_dty
  * The `candidates` rows with the largest a[i] (ties to the lower row) are scored exactly
  * against the 16-bit keys (fp32) and the top_n best of them returned like dresd_retrieve().
  * The result is NOT always the exact top_n: a true neighbour whose approximate score falls
- * below the candidate cut is missed (recall is measured by bench.py --quantised).
+ * below the candidate cut is missed; how often depends on `candidates` and on how close the
+ * neighbours' scores lie (recall = the share of dresd_retrieve()'s rows that come back).
  *
  * dresd_quantise_keys       keys: device [N][d] fp16/bf16, d a multiple of 16; out_q8: device
  *                           [N][d] bytes; both 16-byte aligned.  Asynchronous on `stream`.
@@ -275,7 +276,10 @@ dresd_status dresd_set_global_option(const char *name, int value);
  *   ids, scores, tokens  device, [P][B][top_n] / [P][B][top_n] / [P][B][top_n][draft_len]:
  *                        the shards' outputs, ids LOCAL to each shard (-1 = missing)
  *   row_offsets          device, int64 [P]: global row index of each shard's row 0,
- *                        ascending; global ids must stay below 2^31
+ *                        ascending.  Output ids are int32: the shards may hold at most
+ *                        2^31 - 1 rows in all (offset + rows of every shard <= 2^31 - 1);
+ *                        the call cannot see the shards' sizes, so the caller checks this
+ *                        where the offsets are made
  *   out_*                as for dresd_retrieve(), ids global.
  */
 dresd_status dresd_merge_shards(const int32_t *ids, const float *scores, const int32_t *tokens,
@@ -391,9 +395,15 @@ const char *dresd_last_error(void);
  * their 16-bit split, per-CTA candidate lists, status word) is a fixed
  * ~576 KB array inside the library image, held by every GPU that loads the
  * library until the process exits.  It calls no cudaMalloc/cudaFree and no
- * allocating library routine; it computes exactly what dresd_retrieve() does
- * on a store without z-scoring or projection (Eq. 2, Eq. 3, Section 3.5),
- * with the same kernels, so results are identical.
+ * allocating library routine; it computes what dresd_retrieve() computes
+ * on a store without z-scoring or projection (Eq. 2, Eq. 3, Section 3.5).
+ * fp32 stores run the kernel dresd_retrieve() runs.  16-bit stores run the
+ * STREAMING scoring kernel (the one store option "scan_path" 1 selects), not the
+ * tcgen05 kernel that dresd_retrieve() uses by default: its workspace is smaller
+ * and it needs no query-operand descriptor.  Both accumulate in fp32 and meet the
+ * same tolerances, but in a different order, so against the default store path
+ * scores can differ in the last bits and rows that tie within that rounding can
+ * swap; against a store with "scan_path" 1 results are identical.
  *
  *   keys, next_tokens, N, d, dtype, stored_len   as for dresd_store_create();
  *   queries [B][d], B, top_n, draft_len, out_*   as for dresd_retrieve()
@@ -409,13 +419,20 @@ const char *dresd_last_error(void);
  * contents (the call clears the one word that must start at zero): two calls
  * whose kernels overlap on the GPU -- different streams, or threads -- race
  * on it and return garbage.  Serialise them on one stream.  Asynchronous on
- * `stream` like dresd_retrieve(); device-side timeouts are not reported here.
+ * `stream` like dresd_retrieve().
+ *
+ * dresd_noalloc_status() is dresd_store_status() for this call: it waits for
+ * `stream`, reads the workspace's status word with a 4-byte copy (no allocation
+ * either) and returns DRESD_OK, or DRESD_ERR_TIMEOUT when a bounded device-side
+ * wait of the last call expired (the word is then cleared).  Call it after a
+ * dresd_retrieve_noalloc() and before the next one, which resets the word.
  */
 enum { DRESD_NOALLOC_MAX_BATCH = 8 };
 dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *next_tokens, int64_t N, int d,
                                     dresd_dtype dtype, int stored_len, const void *queries, int B,
                                     int top_n, int draft_len, int32_t *out_ids, float *out_scores,
                                     int32_t *out_tokens, void *stream);
+dresd_status dresd_noalloc_status(void *stream);
 
 /* Frees the workspace only, never caller memory.  NULL is allowed. */
 void dresd_store_destroy(dresd_store *store);

@@ -31,6 +31,7 @@ EXPORTS = (
     "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
     "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore", "dresd_set_global_option", "dresd_quantise_keys", "dresd_store_attach_quantised",
     "dresd_retrieve_quantised", "dresd_store_index_first_tokens", "dresd_merge_shards_packed",
+    "dresd_noalloc_status",
 )
 
 
@@ -108,6 +109,8 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_fit_zscore.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     lib.dresd_retrieve_noalloc.restype = i32
     lib.dresd_retrieve_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.dresd_noalloc_status.restype = i32
+    lib.dresd_noalloc_status.argtypes = [vp]
     if path is None:
         _lib = lib
     return lib
@@ -259,6 +262,12 @@ def dresd_retrieve_noalloc(keys_ptr: int, next_tokens_ptr: int, N: int, d: int, 
     _check(load().dresd_retrieve_noalloc(keys_ptr, next_tokens_ptr, N, d, dtype, stored_len, queries_ptr,
                                          B, top_n, draft_len, out_ids_ptr, out_scores_ptr, out_tokens_ptr,
                                          stream))
+
+
+def dresd_noalloc_status(stream: int = 0) -> None:
+    """Waits for `stream`; raises DRESD_ERR_TIMEOUT if a device-side wait of the last
+    dresd_retrieve_noalloc() call expired."""
+    _check(load().dresd_noalloc_status(stream))
 
 
 # ---- torch convenience ----------------------------------------------------------

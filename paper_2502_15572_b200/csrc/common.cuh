@@ -415,16 +415,6 @@ __device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols)
 {
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
-// Arrives on the barrier at the same shared-memory offset in every CTA of `mask` once all
-// MMAs issued so far by this thread have retired.
-__device__ __forceinline__ void tc_commit2(uint64_t *bar, uint16_t mask)
-{
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
-            smem_u32(bar)),
-        "h"(mask)
-        : "memory");
-}
 __device__ __forceinline__ void umma2_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate)
 {
@@ -436,7 +426,7 @@ __device__ __forceinline__ void umma2_f16(uint32_t d_tmem, uint64_t a_desc, uint
         : "memory");
 }
 // TMA load into this CTA's shared memory whose completion bytes are counted on a barrier of
-// the pair's leader CTA (`bar_cluster_addr` from mapa_rank).  No multicast.
+// the pair's leader CTA (`bar_cluster_addr` from mapa_rank); the data go to this CTA only.
 __device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, int x, int y,
                                                  uint32_t bar_cluster_addr)
 {

@@ -25,6 +25,17 @@
 namespace dresd {
 namespace {
 
+// Arrives on the barrier at the same shared-memory offset in every CTA of `mask` once all
+// MMAs issued so far by this thread have retired.
+__device__ __forceinline__ void tc_commit2(uint64_t *bar, uint16_t mask)
+{
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+            smem_u32(bar)),
+        "h"(mask)
+        : "memory");
+}
+
 constexpr int kThreads = 10 * 32;
 constexpr int kSubRows = 128;
 constexpr int kTileRows = 2 * kSubRows;

@@ -50,18 +50,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+EncodeTiledFn g_encode = nullptr;                      // resolved in setup_device(), under g_mutex
+
 // Host-side descriptor of the key matrix (no device memory involved).
 bool encode_key_map(CUtensorMap *map, const void *base, int dtype, long long rows, int cols, int box_rows)
 {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            return false;
-        fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+    EncodeTiledFn fn = g_encode;
+    if (!fn) return false;
     const size_t eb = dtype == kF32 ? 4 : 2;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)cols * eb};
@@ -96,6 +91,14 @@ dresd_status setup_device(int dev, unsigned char **ptr_out, int *sms_out)
         int sms = 0;
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess || sms <= 0) return na_fail(DRESD_ERR_CUDA, "cannot query the SM count");
+        if (!g_encode) {
+            void *p = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+                q != cudaDriverEntryPointSuccess)
+                return na_fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled is not available");
+            g_encode = reinterpret_cast<EncodeTiledFn>(p);
+        }
         g_num_sms[dev] = sms;
         g_scratch_ptr[dev] = ptr;
     }
@@ -199,5 +202,33 @@ extern "C" dresd_status dresd_retrieve_noalloc(const void *keys, const int32_t *
     if (launch_merge_gather(cand, grid, B, top_n, out_ids, out_scores, next_tokens, stored_len, N, draft_len,
                             out_tokens, stream) != cudaSuccess)
         return na_fail(DRESD_ERR_CUDA, "merge/gather launch failed");
+    return DRESD_OK;
+}
+
+// The status word of the static workspace: the scoring kernels' bounded waits record a give-up
+// there.  Reading it needs a 4-byte copy into the caller's stack and nothing else.
+extern "C" dresd_status dresd_noalloc_status(void *stream_v)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return na_fail(DRESD_ERR_CUDA, "cudaGetDevice failed");
+    if (dev < 0 || dev >= kMaxDevices) return na_fail(DRESD_ERR_UNSUPPORTED, "device ordinal beyond 63");
+    unsigned char *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        scratch = g_scratch_ptr[dev];
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    if (!scratch) {                                     // no call was made on this device yet
+        if (cudaStreamSynchronize(stream) != cudaSuccess) return na_fail(DRESD_ERR_CUDA, "stream synchronize failed");
+        return DRESD_OK;
+    }
+    int word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, scratch + kOffStatus, sizeof(int), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return na_fail(DRESD_ERR_CUDA, "status read failed");
+    if (word != 0) {
+        cudaMemsetAsync(scratch + kOffStatus, 0, sizeof(int), stream);
+        return na_fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
+    }
     return DRESD_OK;
 }

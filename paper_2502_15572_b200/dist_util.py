@@ -55,14 +55,87 @@ def shard_rows(N: int, rank: int, world: int) -> range:
     return query_slice(N, rank, world)
 
 
-def gather_shard_results(ids, scores, tokens, row_offset: int, group=None):
+MAX_GLOBAL_ROWS = 2 ** 31 - 1          # merged ids are int32 row indices
+
+
+def check_global_rows(offsets, rows) -> None:
+    """Raises ValueError when some shard's rows would get global ids beyond int32: the merge
+    kernels write ids as int32, so a sharded datastore may hold at most 2^31 - 1 rows in all."""
+    for off, n in zip(offsets, rows):
+        if off < 0 or n < 0 or off + n > MAX_GLOBAL_ROWS:
+            raise ValueError(f"shard at row offset {off} with {n} rows passes the largest global row id "
+                             f"({MAX_GLOBAL_ROWS - 1}): a sharded datastore holds at most 2^31 - 1 rows")
+
+
+def _on_stream(stream):
+    """Context in which torch.distributed collectives are enqueued on `stream` (torch orders a
+    collective after the CURRENT stream, so kernels launched on another stream would race it)."""
+    import contextlib
+    import torch
+    if stream is None or not torch.cuda.is_available():
+        return contextlib.nullcontext()
+    return torch.cuda.stream(stream)
+
+
+def broadcast_array(array, src: int = 0, device="cuda", group=None):
+    """A numpy array that only rank `src` holds (the others pass None) -> a tensor on `device`
+    on every rank, moved by one broadcast: a replica of the datastore is generated once, not
+    once per rank.  16-bit bit patterns travel as int16."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    multi = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
+    rank = dist.get_rank(group) if multi else src
+    meta = [None]
+    if rank == src:
+        a = np.ascontiguousarray(array)
+        if a.dtype in (np.float16, np.uint16):
+            a = a.view(np.int16)
+        meta = [(tuple(a.shape), a.dtype.str)]
+    if multi:
+        dist.broadcast_object_list(meta, src=src, group=group)
+    shape, dt = meta[0]
+    # the payload travels as bytes (every backend moves uint8) and is re-viewed on arrival
+    if rank == src:
+        t = torch.from_numpy(a.reshape(-1).view(np.uint8)).to(device)
+    else:
+        t = torch.empty(int(np.prod(shape)) * np.dtype(dt).itemsize, dtype=torch.uint8, device=device)
+    if multi:
+        dist.broadcast(t, src=src, group=group)
+    return t.view(torch.from_numpy(np.empty(0, dtype=np.dtype(dt))).dtype).reshape(shape)
+
+
+def collect_rows(local_rows, first_row: int, wanted, group=None, device="cpu"):
+    """Rows `wanted` (global indices, the same list on every rank) of a matrix whose rows are
+    sharded over the ranks: this rank holds rows first_row .. first_row + len(local_rows) - 1
+    as the numpy array `local_rows`.  Every rank gets all wanted rows, bit for bit (each row
+    is contributed by its one owner and the others add zero bytes).  numpy in, numpy out."""
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    local_rows = np.ascontiguousarray(local_rows)
+    wanted = np.asarray(wanted, dtype=np.int64)
+    row_bytes = local_rows.shape[1] * local_rows.dtype.itemsize
+    buf = np.zeros((len(wanted), row_bytes), dtype=np.uint8)
+    mine = (wanted >= first_row) & (wanted < first_row + local_rows.shape[0])
+    buf[mine] = local_rows[wanted[mine] - first_row].view(np.uint8).reshape(-1, row_bytes)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        t = torch.from_numpy(buf).to(device)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
+        buf = t.cpu().numpy()
+    return buf.view(local_rows.dtype).reshape(len(wanted), local_rows.shape[1])
+
+
+def gather_shard_results(ids, scores, tokens, row_offset: int, group=None, n_rows: int = 0):
     """All-gather the per-shard results.  Returns ``(ids [P][B][n], scores [P][B][n],
     tokens [P][B][n][L], offsets int64 [P])`` on the inputs' device; with one process
-    the inputs come back with a leading axis of 1."""
+    the inputs come back with a leading axis of 1.  `n_rows` (this shard's row count), when
+    given, is exchanged with the offsets and every rank checks that global ids fit int32."""
     import torch
     import torch.distributed as dist
     off = torch.tensor([row_offset], dtype=torch.int64, device=ids.device)
     if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        check_global_rows([row_offset], [n_rows])
         return ids[None], scores[None], tokens[None], off
     P = dist.get_world_size(group)
 
@@ -72,7 +145,9 @@ def gather_shard_results(ids, scores, tokens, row_offset: int, group=None):
         dist.all_gather_into_tensor(out, t.contiguous(), group=group)
         return out.reshape((P,) + tuple(t.shape))
 
-    return gather(ids), gather(scores), gather(tokens), gather(off).reshape(P)
+    meta = gather(torch.tensor([[row_offset, n_rows]], dtype=torch.int64, device=ids.device)).reshape(P, 2)
+    check_global_rows(meta[:, 0].tolist(), meta[:, 1].tolist())
+    return gather(ids), gather(scores), gather(tokens), meta[:, 0].contiguous()
 
 
 def sharded_retrieve(store, row_offset: int, queries, top_n: int, draft_len: int, group=None, stream=None):
@@ -83,7 +158,9 @@ def sharded_retrieve(store, row_offset: int, queries, top_n: int, draft_len: int
     import torch
     from . import binding
     ids, scores, tokens = store.retrieve(queries, top_n, draft_len, stream=stream)
-    g_ids, g_scores, g_tokens, offsets = gather_shard_results(ids, scores, tokens, row_offset, group)
+    with _on_stream(stream):
+        g_ids, g_scores, g_tokens, offsets = gather_shard_results(ids, scores, tokens, row_offset, group,
+                                                                  n_rows=getattr(store, "N", 0))
     P, B = g_ids.shape[0], g_ids.shape[1]
     out = (torch.empty_like(ids), torch.empty_like(scores), torch.empty_like(tokens))
     s = (stream or torch.cuda.current_stream()).cuda_stream
@@ -98,7 +175,7 @@ class PackedExchange:
     dresd_merge_shards_packed() reads -- so that a call needs a single all-gather; the row
     offsets of the shards are exchanged once, here.  Works on any device (CPU + gloo in the tests)."""
 
-    def __init__(self, B: int, top_n: int, draft_len: int, row_offset: int, device, group=None):
+    def __init__(self, B: int, top_n: int, draft_len: int, row_offset: int, device, group=None, n_rows: int = 0):
         import torch
         import torch.distributed as dist
         self.group = group
@@ -109,13 +186,17 @@ class PackedExchange:
         self.ids = self.local[:bn].view(B, top_n)
         self.scores = self.local[bn:2 * bn].view(torch.float32).view(B, top_n)
         self.tokens = self.local[2 * bn:].view(B, top_n, draft_len)
-        off = torch.tensor([row_offset], dtype=torch.int64, device=device)
+        off = torch.tensor([row_offset, n_rows], dtype=torch.int64, device=device)
         if self.P == 1:
-            self.gathered, self.offsets = self.local, off
+            self.gathered, meta = self.local, off.view(1, 2)
         else:
             self.gathered = torch.empty(self.P * self.words, dtype=torch.int32, device=device)
-            self.offsets = torch.empty(self.P, dtype=torch.int64, device=device)
-            dist.all_gather_into_tensor(self.offsets, off, group=group)
+            meta = torch.empty(self.P * 2, dtype=torch.int64, device=device)
+            dist.all_gather_into_tensor(meta, off, group=group)
+            meta = meta.view(self.P, 2)
+        # every rank sees every shard's extent, so every rank raises (or none does)
+        check_global_rows(meta[:, 0].tolist(), meta[:, 1].tolist())
+        self.offsets = meta[:, 0].contiguous()
 
     def exchange(self):
         """All ranks' blocks, back to back: int32 [P * words]."""
@@ -140,14 +221,16 @@ class ShardedRetriever:
         B = queries.shape[0]
         st = self._by_batch.get(B)
         if st is None:
-            ex = PackedExchange(B, self.n, self.L, self.row_offset, queries.device, self.group)
+            ex = PackedExchange(B, self.n, self.L, self.row_offset, queries.device, self.group,
+                                n_rows=getattr(self.store, "N", 0))
             out = (torch.empty((B, self.n), dtype=torch.int32, device=queries.device),
                    torch.empty((B, self.n), dtype=torch.float32, device=queries.device),
                    torch.empty((B, self.n, self.L), dtype=torch.int32, device=queries.device))
             st = self._by_batch[B] = (ex, out)
         ex, out = st
         self.store.retrieve(queries, self.n, self.L, out=(ex.ids, ex.scores, ex.tokens), stream=stream)
-        packed = ex.exchange()
+        with _on_stream(stream):                       # the collective follows the kernels of `stream`
+            packed = ex.exchange()
         s = (stream or torch.cuda.current_stream()).cuda_stream
         binding.dresd_merge_shards_packed(packed.data_ptr(), ex.offsets.data_ptr(), ex.P, B, self.n, self.L,
                                           out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(), s)

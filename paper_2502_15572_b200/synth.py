@@ -114,44 +114,51 @@ def _n_threads(threads):
 # datastore
 # ----------------------------------------------------------------------------
 def make_store(seed: int, N: int, d: int, C: int, dtype: str, stored_len: int,
-               vocab: int = 32000, rho: float = 0.5, threads=None):
+               vocab: int = 32000, rho: float = 0.5, threads=None, rows=None):
     """Return ``(keys, next_tokens)``.
 
     ``keys``: ``[N][d]`` in the store dtype's container (see module doc).
     ``next_tokens``: ``[N][stored_len]`` int32 in ``[0, vocab)``.
+    ``rows = (lo, hi)``: only rows lo .. hi-1 of the N-row store are made and returned
+    (the same values the whole store holds there: every 65,536-row chunk has a random
+    stream of its own), so that a process that holds a shard generates only its shard.
     """
     if dtype not in DTYPES:
         raise ValueError(f"unknown dtype {dtype!r}")
+    r_lo, r_hi = (0, N) if rows is None else (int(rows[0]), int(rows[1]))
+    if not (0 <= r_lo <= r_hi <= N):
+        raise ValueError("rows must satisfy 0 <= lo <= hi <= N")
     M = centres(seed, C, d).astype(np.float32)
     cdf = zipf_cdf(vocab)
-    keys = _store_empty((N, d), dtype)
-    toks = np.empty((N, stored_len), dtype=np.int32)
+    keys = _store_empty((r_hi - r_lo, d), dtype)
+    toks = np.empty((r_hi - r_lo, stored_len), dtype=np.int32)
     scale = np.float32(rho / np.sqrt(d))
-    n_chunks = (N + CHUNK_ROWS - 1) // CHUNK_ROWS
+    chunks = range(r_lo // CHUNK_ROWS, (r_hi + CHUNK_ROWS - 1) // CHUNK_ROWS) if r_hi > r_lo else range(0)
 
     def work(ci: int):
         lo = ci * CHUNK_ROWS
         hi = min(N, lo + CHUNK_ROWS)
-        rows = hi - lo
+        n_rows = hi - lo
         rng = _stream(seed, 1 + ci)
-        comp = rng.integers(0, C, size=rows)
-        g = rng.standard_normal((rows, d), dtype=np.float32)
+        comp = rng.integers(0, C, size=n_rows)
+        g = rng.standard_normal((n_rows, d), dtype=np.float32)
         g *= scale
         g += M[comp]
         g = _normalise_rows(g)
-        keys[lo:hi] = cast_to_store(g, dtype)
-        u = rng.random((rows, stored_len))
+        a, b = max(lo, r_lo), min(hi, r_hi)              # the part of the chunk that is asked for
+        keys[a - r_lo:b - r_lo] = cast_to_store(g[a - lo:b - lo], dtype)
+        u = rng.random((n_rows, stored_len))
         t = np.searchsorted(cdf, u, side="right")
         np.minimum(t, vocab - 1, out=t)
-        toks[lo:hi] = t.astype(np.int32)
+        toks[a - r_lo:b - r_lo] = t[a - lo:b - lo].astype(np.int32)
 
-    nt = min(_n_threads(threads), n_chunks)
+    nt = min(_n_threads(threads), max(1, len(chunks)))
     if nt <= 1:
-        for ci in range(n_chunks):
+        for ci in chunks:
             work(ci)
     else:
         with ThreadPoolExecutor(nt) as ex:
-            list(ex.map(work, range(n_chunks)))
+            list(ex.map(work, chunks))
     return keys, toks
 
 
@@ -169,12 +176,26 @@ def make_queries(seed: int, keys: np.ndarray, dtype: str, B: int, sigma: float):
     int64 ``[B]``.  The source row is usually, not always, the best match.
     """
     N, d = keys.shape
+    src = query_sources(seed, N, B)
+    return queries_from_rows(seed, keys[src], dtype, N, sigma), src
+
+
+def query_sources(seed: int, N: int, B: int) -> np.ndarray:
+    """The source rows ``make_queries(seed, keys[N], ..., B, ...)`` draws: int64 ``[B]``."""
+    return _stream(seed, 0).integers(0, N, size=B).astype(np.int64)
+
+
+def queries_from_rows(seed: int, source_keys: np.ndarray, dtype: str, N: int, sigma: float) -> np.ndarray:
+    """The queries of ``make_queries`` given only the keys of their source rows
+    (``source_keys[b] = keys[query_sources(seed, N, B)[b]]``): for processes that hold a
+    shard of the rows and collect the source rows from their owners."""
+    B, d = source_keys.shape
     rng = _stream(seed, 0)
-    src = rng.integers(0, N, size=B)
-    base = store_to_float32(keys[src], dtype).astype(np.float64)
+    rng.integers(0, N, size=B)                           # the draw that chose the source rows
+    base = store_to_float32(source_keys, dtype).astype(np.float64)
     q = base + sigma * rng.standard_normal((B, d))
     q = _normalise_rows(q)
-    return cast_to_store(q.astype(np.float32), dtype), src.astype(np.int64)
+    return cast_to_store(q.astype(np.float32), dtype)
 
 
 def make_hidden_queries(seed: int, B: int, d_in: int, dtype: str,
@@ -224,6 +245,9 @@ WORKLOADS = {
                               draft_len=10, stored_len=20, sigma=0.1, seed=1010),
     "paper_46m_d64_f16_b16": dict(N=46_300_000, d=64, dtype="f16", C=4096, B=16, top_n=10,
                                   draft_len=10, stored_len=20, sigma=0.1, seed=1010),
+    # the paper's smaller datastore (Table 1 / Section 5.6: 19M tokens, 6.49 GB on disk), same reduced width
+    "paper_19m_d64_f16": dict(N=19_000_000, d=64, dtype="f16", C=4096, B=1, top_n=10,
+                              draft_len=10, stored_len=20, sigma=0.1, seed=1011),
     "c5b_projected_bf16": dict(N=4_000_000, d=256, dtype="bf16", C=1024, B=16, top_n=10,
                                draft_len=10, stored_len=10, sigma=0.1, seed=1006,
                                d_in=4096, proj_seed=1007),

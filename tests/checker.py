@@ -15,6 +15,12 @@ the oracle's order, ``n`` = top_n):
 * tokens are bit-exact copies of the stored continuation of the returned id.
 
 ``tol`` is 2e-3 for 16-bit keys and 1e-5 for fp32 keys; ``band`` is 2e-3.
+
+``eps_acc`` is stated for unit-length keys.  The accumulation error of an inner
+product is proportional to the sum of |q_j k_ij|, which the key's length bounds
+(the query has unit length), so for stores whose keys are not unit vectors the
+caller passes ``key_scale`` = the largest key norm and ``eps_acc`` is multiplied
+by it (never below 1).  ``tol`` and ``band`` stay absolute.
 """
 from __future__ import annotations
 
@@ -42,13 +48,13 @@ def oracle_order(full_scores: np.ndarray, k: int) -> np.ndarray:
 
 
 def check_query(s: np.ndarray, next_tokens: np.ndarray, g_ids, g_scores, g_tokens, dtype: str,
-                top_n: int, draft_len: int, oracle_ids=None):
+                top_n: int, draft_len: int, oracle_ids=None, key_scale: float = 1.0):
     """Raises AssertionError with a description on the first violation.
 
     Returns the number of ranks whose id equals the oracle's.
     """
     N = s.shape[0]
-    tol, band, eps = TOL[dtype], BAND, EPS_ACC[dtype]
+    tol, band, eps = TOL[dtype], BAND, EPS_ACC[dtype] * max(1.0, float(key_scale))
     g_ids = np.asarray(g_ids).astype(np.int64)
     g_scores = np.asarray(g_scores).astype(np.float64)
     g_tokens = np.asarray(g_tokens)
@@ -94,14 +100,15 @@ def check_query(s: np.ndarray, next_tokens: np.ndarray, g_ids, g_scores, g_token
     return exact
 
 
-def check_batch(full_scores, next_tokens, ids, scores, tokens, dtype, top_n, draft_len, oracle_ids=None):
+def check_batch(full_scores, next_tokens, ids, scores, tokens, dtype, top_n, draft_len, oracle_ids=None,
+                key_scale: float = 1.0):
     """All queries of a batch; returns the fraction of ranks identical to the oracle."""
     B = full_scores.shape[0]
     exact = 0
     for b in range(B):
         try:
             exact += check_query(full_scores[b], next_tokens, ids[b], scores[b], tokens[b], dtype,
-                                 top_n, draft_len, None if oracle_ids is None else oracle_ids[b])
+                                 top_n, draft_len, None if oracle_ids is None else oracle_ids[b], key_scale)
         except AssertionError as e:
             raise AssertionError(f"query {b}: {e}") from None
     return exact / float(B * top_n)

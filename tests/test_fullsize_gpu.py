@@ -35,6 +35,17 @@ def _properties(keys, toks, dtype, q, ids, sc, tok, n, L):
         assert np.max(np.abs(want - sc[b])) <= tol
 
 
+_CACHE = {}
+
+
+def _workload(name):
+    """The named workload; the last one made stays in memory for the next test that asks for it."""
+    if name not in _CACHE:
+        _CACHE.clear()
+        _CACHE[name] = synth.make_workload(name)
+    return _CACHE[name]
+
+
 def _sampled_parity(w, sample, q=None):
     import torch
     keys, toks, dtype = w["keys"], w["next_tokens"], w["dtype"]
@@ -62,35 +73,9 @@ def _sampled_parity(w, sample, q=None):
 
 def test_config2_decode_batch1_full_size():
     """10M x 256 fp16, single queries: 64 calls checked by properties, 3 against the oracle."""
-    w = synth.make_workload("c2_decode_b1_f16")
+    w = _workload("c2_decode_b1_f16")
     q, _ = synth.make_queries(w["seed"] + 100, w["keys"], "f16", 64, w["sigma"])
     rate = _sampled_parity(w, sample=[0, 17, 63], q=q)
-    assert rate >= 0.9
-
-
-def test_config3_batched_full_size():
-    """10M x 256 bf16, one batch of 64 (tensor-core kernel with its probe pass): 3 queries against the oracle."""
-    w = synth.make_workload("c3_batched_bf16")
-    rate = _sampled_parity(w, sample=[0, 31, 63])
-    assert rate >= 0.9
-
-
-def test_config5b_projected_full_size():
-    """4M x 256 bf16 with the 4096 -> 256 projection, batch 16: all 16 queries against the oracle."""
-    import torch
-    w = synth.make_workload("c5b_projected_bf16")
-    keys, toks, dtype, n, L = w["keys"], w["next_tokens"], w["dtype"], w["top_n"], w["draft_len"]
-    st = gpu_store(keys, toks, dtype)
-    dW = binding.to_device(w["W"], dtype)
-    st.set_preprocess(w["d_in"], W=dW)
-    ids, sc, tok = st.retrieve(binding.to_device(w["queries"], dtype), n, L)
-    torch.cuda.synchronize()
-    st.status()
-    ids, sc, tok = ids.cpu().numpy(), sc.cpu().numpy(), tok.cpu().numpy()
-    st.close()
-    o = oracle.retrieve(keys, toks, dtype, w["queries"], n, L, W=w["W"], want_full_scores=True,
-                        threads=oracle.dresd_oracle.default_threads())
-    rate = checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids)
     assert rate >= 0.9
 
 
@@ -100,7 +85,7 @@ def test_config2_quantised_full_size():
     properties (rows distinct and in range, exact scores in order, stored tokens), 3 against
     the oracle's statement of the same rules, and the recall of the exact path's rows."""
     import torch
-    w = synth.make_workload("c2_decode_b1_f16")
+    w = _workload("c2_decode_b1_f16")
     keys, toks, dtype, n, L, m = w["keys"], w["next_tokens"], "f16", w["top_n"], w["draft_len"], 32
     q, _ = synth.make_queries(w["seed"] + 200, keys, dtype, 32, w["sigma"])
     st = gpu_store(keys, toks, dtype)
@@ -134,6 +119,51 @@ def test_config2_quantised_full_size():
         assert not [i for i in safe if exact[k][i] > nth + 2e-5 and i not in set(got.tolist())]
 
 
+def test_config3_batched_full_size():
+    """10M x 256 bf16, one batch of 64 (tensor-core kernel with its probe pass): 3 queries against the oracle."""
+    w = synth.make_workload("c3_batched_bf16")
+    rate = _sampled_parity(w, sample=[0, 31, 63])
+    assert rate >= 0.9
+
+
+def test_config4_large_full_size():
+    """50M x 128 fp16 (12.8 GB of keys, the largest row count of the configurations), one batch
+    of 4 as bench.py issues it: all 4 queries by properties and against the oracle's full result."""
+    _CACHE.clear()
+    w = synth.make_workload("c4_large_f16")
+    rate = _sampled_parity(w, sample=[0, 1, 2, 3])
+    assert rate >= 0.9
+
+
+def test_config5a_unreduced_full_size():
+    """4M x 4096 bf16 (32.8 GB of keys, 8 KB rows: the query operand travels with every key slab,
+    64 slabs per row, the largest byte offsets of the configurations), one batch of 16, no
+    projection: all 16 queries by properties, 4 of them against the oracle's full result."""
+    _CACHE.clear()
+    w = synth.make_workload("c5a_hidden_bf16")
+    rate = _sampled_parity(w, sample=[0, 5, 10, 15])
+    assert rate >= 0.9
+
+
+def test_config5b_projected_full_size():
+    """4M x 256 bf16 with the 4096 -> 256 projection, batch 16: all 16 queries against the oracle."""
+    import torch
+    w = synth.make_workload("c5b_projected_bf16")
+    keys, toks, dtype, n, L = w["keys"], w["next_tokens"], w["dtype"], w["top_n"], w["draft_len"]
+    st = gpu_store(keys, toks, dtype)
+    dW = binding.to_device(w["W"], dtype)
+    st.set_preprocess(w["d_in"], W=dW)
+    ids, sc, tok = st.retrieve(binding.to_device(w["queries"], dtype), n, L)
+    torch.cuda.synchronize()
+    st.status()
+    ids, sc, tok = ids.cpu().numpy(), sc.cpu().numpy(), tok.cpu().numpy()
+    st.close()
+    o = oracle.retrieve(keys, toks, dtype, w["queries"], n, L, W=w["W"], want_full_scores=True,
+                        threads=oracle.dresd_oracle.default_threads())
+    rate = checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids)
+    assert rate >= 0.9
+
+
 def test_paper_shaped_sorted_store_full_size():
     """46.3M x 64 fp16 with its rows sorted by first stored token, as
     `bench.py --workload paper_46m_d64_f16 --first-token-filter --sorted-store` issues them:
@@ -142,6 +172,7 @@ def test_paper_shaped_sorted_store_full_size():
     token, distinct, scores in order and equal to the oracle's score of the row, tokens the
     stored ones; 2 queries element by element against the oracle's filtered search."""
     import torch
+    _CACHE.clear()
     w = synth.make_workload("paper_46m_d64_f16")
     dtype, n, L = "f16", w["top_n"], w["draft_len"]
     q, src = synth.make_queries(w["seed"] + 300, w["keys"], dtype, 56, w["sigma"])

@@ -98,6 +98,35 @@ def test_parity_both_16bit_paths(path, dtype, d, B, n, L, N):
     _check(keys, toks, dtype, q, n, L, options={"scan_path": path})
 
 
+def _rescaled(keys, dtype, seed, lo=0.25, hi=4.0):
+    """The same rows with lengths spread log-uniformly over lo..hi (store dtype after scaling)."""
+    rng = np.random.default_rng(seed)
+    f = np.exp(rng.uniform(np.log(lo), np.log(hi), size=keys.shape[0])).astype(np.float32)
+    scaled = synth.store_to_float32(keys, dtype) * f[:, None]
+    return synth.cast_to_store(scaled, dtype), float(f.max()) * 1.01
+
+
+# Keys that are NOT unit vectors: Eq. 3 is read as the inner product of the unit query with the
+# key as stored (keys are never renormalised), so a long key can outrank a better-aligned short
+# one.  One case per dtype and scoring kernel, lengths 0.25 .. 4.
+@pytest.mark.parametrize("dtype,d,B,n,L,N,options", [
+    ("f32", 128, 5, 10, 4, 40009, None),
+    ("f16", 256, 3, 10, 4, 40009, None),                       # tcgen05, keys as M
+    ("bf16", 64, 16, 10, 4, 60013, None),                      # narrow rows, sub-tiles
+    ("bf16", 256, 40, 32, 4, 30011, None),                     # keys as the N operand
+    ("f16", 128, 6, 10, 4, 40009, {"scan_path": 1}),           # streaming mma.sync kernel
+    ("bf16", 512, 64, 16, 4, 20011, None),                     # 64 queries on wide rows
+    ("f16", 64, 64, 10, 4, 60013, None),                       # 64 queries on narrow rows
+])
+def test_parity_keys_not_unit_length(dtype, d, B, n, L, N, options):
+    keys, toks = synth.make_store(7500 + d + B, N, d, 32, dtype, L + 1)
+    keys, kmax = _rescaled(keys, dtype, 7501 + d)
+    q, _ = synth.make_queries(7502 + d + B, keys, dtype, B, 0.1)
+    ids, sc, tok, o = run_both(keys, toks, dtype, q, n, L, options=options)
+    assert np.max(np.abs(o.full_scores)) > 2.0                  # the spread is really there
+    checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids, key_scale=kmax)
+
+
 @pytest.mark.parametrize("path", [1, 2])
 def test_adversarial_order_both_paths(path):
     # ascending scores in memory: every row beats all rows before it (queue overflow path)
