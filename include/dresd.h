@@ -261,6 +261,12 @@ dresd_status dresd_retrieve_quantised(dresd_store *store, const void *queries, c
  *   "build_keys_pairs"  1 (default): dresd_build_keys runs on CTA pairs -- clusters of two
  *                       CTAs, one tensor-core instruction spanning both SMs, each CTA staging
  *                       half of the weight slab; 0: one CTA per tile.  Results are identical.
+ *   "build_keys_wait_ms"  bound of the device-side waits of dresd_build_keys in milliseconds
+ *                       (0 = default, about 2 s).
+ *   "build_keys_debug_lose_stage"  test hook: in the next dresd_build_keys calls the first CTA (the
+ *                       leader of the first pair) never receives the copies of pipeline stage
+ *                       (value-1), so its waits run out: the kernel returns in an orderly way and
+ *                       the call returns DRESD_ERR_TIMEOUT.  0 = off.
  * Unknown names and values outside the stated set return DRESD_ERR_INVALID.
  */
 dresd_status dresd_set_global_option(const char *name, int value);
@@ -344,12 +350,13 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "first_token_windows"  1 (default): on a store indexed by dresd_store_index_first_tokens()
  *                filtered calls scan only the rows of their queries' tokens; 0 = scan every row.
  *                Results do not change.
- *   "wait_ms"    bound of the device-side waits of the streaming kernels in
+ *   "wait_ms"    bound of the device-side waits of the scoring kernels in
  *                milliseconds (0 = default, about 2 s).
- *   "debug_lose_stage"  test hook: in the next calls the streaming 16-bit kernel's
- *                first CTA never receives the copies of pipeline stage (value-1),
- *                so its waits run out: the kernel returns in an orderly way and
- *                dresd_store_status() reports DRESD_ERR_TIMEOUT.  0 = off.
+ *   "debug_lose_stage"  test hook: in the next calls the first CTA of the scoring kernel
+ *                (whichever kernel the call selects) never receives the copies of pipeline
+ *                stage (value-1), so its waits run out: the kernel returns in an orderly way,
+ *                frees its tensor memory, and dresd_store_status() reports
+ *                DRESD_ERR_TIMEOUT; the results of such a call are incomplete.  0 = off.
  *   "debug_no_select"  measurement hook: the tcgen05 scoring kernel streams and scores
  *                every key but lets nothing pass its filter (results are empty); the
  *                time of such a call is the floor against which the cost of

@@ -312,6 +312,8 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.gtau = s->gtau;
         a.no_select = s->opt_no_select;
         a.keys_as_m = keys_as_m;
+        a.wait_cycles = (long long)s->opt_wait_ms * 2000000LL;     // ~2 GHz
+        a.debug_lose_stage = s->opt_lose_stage;
         if (windows) {
             a.win_start = s->win_start;
             a.win_vocab = s->win_vocab;
@@ -404,6 +406,8 @@ uint8_t *g_scratch_ptr[kScratchDevices] = {};
 size_t g_scratch_size[kScratchDevices] = {};
 
 std::atomic<int> g_build_pairs{1};      // dresd_build_keys on CTA pairs (cta_group::2); 0 = one CTA per tile
+std::atomic<int> g_build_wait_ms{0};    // bound of dresd_build_keys' device-side waits, 0 = default
+std::atomic<int> g_build_lose_stage{0}; // test hook: the first CTA (pair) never receives stage (value-1)
 
 uint8_t *device_scratch(int dev, size_t need)
 {
@@ -922,7 +926,8 @@ dresd_status dresd_build_keys(const void *hidden, int64_t N, int d_in, dresd_dty
                                                  stream)) != cudaSuccess)
         st = fail_cuda(e, "build prep launch");
     if (st == DRESD_OK && (e = launch_build_keys(h_map, whi_map, wlo_map, (int)dtype, N, d_in, d, mean ? 2 : 1, pair, bias, out_keys,
-                                                 kEpsNorm, status, sms, stream)) != cudaSuccess)
+                                                 kEpsNorm, status, sms, stream, (long long)g_build_wait_ms.load() * 2000000LL,
+                                                 g_build_lose_stage.load())) != cudaSuccess)
         st = fail_cuda(e, "build keys launch");
     int word = 0;
     if (st == DRESD_OK && (e = cudaMemcpyAsync(&word, status, sizeof(int), cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
@@ -1005,6 +1010,16 @@ dresd_status dresd_set_global_option(const char *name, int value)
     if (std::strcmp(name, "build_keys_pairs") == 0) {
         if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "build_keys_pairs takes 0 or 1");
         g_build_pairs.store(value);
+        return DRESD_OK;
+    }
+    if (std::strcmp(name, "build_keys_wait_ms") == 0) {
+        if (value < 0 || value > 60000) return fail(DRESD_ERR_INVALID, "build_keys_wait_ms = %d outside 0..60000", value);
+        g_build_wait_ms.store(value);
+        return DRESD_OK;
+    }
+    if (std::strcmp(name, "build_keys_debug_lose_stage") == 0) {
+        if (value < 0) return fail(DRESD_ERR_INVALID, "build_keys_debug_lose_stage = %d is negative", value);
+        g_build_lose_stage.store(value);
         return DRESD_OK;
     }
     return fail(DRESD_ERR_INVALID, "unknown global option '%s'", name);

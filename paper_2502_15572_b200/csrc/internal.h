@@ -71,7 +71,7 @@ struct ScanArgs {
     int win_vocab;
     int stages;             // pipeline depth
     long long wait_cycles;  // bound of every device-side wait in cycles, 0 = default (~2 s)
-    int debug_lose_stage;   // test hook (streaming kernel): CTA 0 never receives stage (value-1); 0 = off
+    int debug_lose_stage;   // test hook (every scan kernel): CTA 0 never receives stage (value-1); 0 = off
     int tile_stride;        // tcgen05 kernel: visit every tile_stride-th tile (probe pass), default 1
     int probe_max;          // tcgen05 kernel, probe pass: keep only each tile's best row per query
     int no_select;          // tcgen05 kernel, measurement only: nothing passes the filter (scan floor)
@@ -148,7 +148,8 @@ cudaError_t launch_build_prep(const void *W, int dtype, const float *mean, const
                               cudaStream_t stream);
 cudaError_t launch_build_keys(const CUtensorMap &h_map, const CUtensorMap &whi_map, const CUtensorMap &wlo_map,
                               int dtype, long long N, int d_in, int d, int terms, int pair, const float *bias,
-                              void *out, float eps_n, int *status, int grid, cudaStream_t stream);
+                              void *out, float eps_n, int *status, int grid, cudaStream_t stream,
+                              long long wait_cycles = 0, int lose_stage = 0);
 
 // ---- K8: statistics of Eq. 1 (Section 3.2) from a sample of embeddings, one streaming pass ----
 size_t fit_zscore_workspace_bytes(long long N, int d_in, int sms);

@@ -97,13 +97,14 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
 
     const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
     const int n_it = my_tiles * dslabs;                // one slab of one tile per stage
+    const long long wl = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;   // bound of every wait below
 
     if (warp == kConsumerWarps) {
         if (lane == 0) {
             int issued = 0;
             for (int it = 0; it < n_it; ++it) {
                 const int s = it % n_stages;
-                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
+                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1, wl)) {
                     report_timeout(a.status);
                     break;
                 }
@@ -111,13 +112,15 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 const int sl = it % dslabs;
                 mbar_arrive_expect_tx(&full[s], (uint32_t)kStageBytes);     // rows past N arrive as zeros
                 uint8_t *dst = stages + (size_t)s * kStageBytes;
-                for (int h = 0; h < kRows / kBoxRows; ++h)
+                // Test hook: CTA 0 "loses" the copies of one stage, so that the waits on it run out.
+                const bool lose = a.debug_lose_stage > 0 && cta == 0 && it == a.debug_lose_stage - 1;
+                for (int h = 0; h < kRows / kBoxRows && !lose; ++h)
                     tma_load_2d(dst + (size_t)h * kBoxRows * kSlabBytes, &keys_map, sl * kSlabElems,
                                 tile * kRows + h * kBoxRows, &full[s]);
                 issued = it + 1;
             }
             for (int it = max(0, issued - n_stages); it < issued; ++it)
-                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1)) {
+                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1, wl)) {
                     report_timeout(a.status);
                     break;
                 }
@@ -157,7 +160,7 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             for (int sl = 0; sl < dslabs; ++sl) {
                 const int it = tl * dslabs + sl;
                 const int s = it % n_stages;
-                if (!dead && !mbar_wait(&full[s], (it / n_stages) & 1)) {
+                if (!dead && !mbar_wait(&full[s], (it / n_stages) & 1, wl)) {
                     report_timeout(a.status);
                     dead = true;
                 }

@@ -177,6 +177,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, G = gridDim.x;
+    const long long wl = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;   // bound of every wait below
     constexpr int kRowsPerTile = kTileRows * TSUB;
     // Narrow rows: the sub-tiles of a tile have accumulators of their own, so two threads (warps 1
     // and 10) issue the MMAs of alternate sub-tiles; each commits to the barriers for its share.
@@ -282,7 +283,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             int issued = 0, wk = 0;
             for (int it = 0; it < n_it; ++it) {
                 const int s = it % n_stages;
-                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
+                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1, wl)) {
                     report_timeout(a.status);
                     break;
                 }
@@ -292,10 +293,13 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     tile = win->tile0[wk] + (tile - win->prefix[wk]);
                 }
                 uint8_t *dst = stages + (size_t)s * stage_bytes;
+                // Test hook: CTA 0 "loses" the copies of one stage (they are announced to the barrier
+                // but never issued), so that every wait that depends on it runs out.
+                const bool lose = a.debug_lose_stage > 0 && cta == 0 && it == a.debug_lose_stage - 1;
                 if constexpr (TSUB > 1) {
                     // narrow rows: every slab of every sub-tile (rows past N read as zeros)
                     mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
-                    for (int sub = 0; sub < TSUB; ++sub)
+                    for (int sub = 0; sub < TSUB && !lose; ++sub)
                         for (int j = 0; j < dslabs; ++j)
                             tma_load_2d(dst + (size_t)(sub * dslabs + j) * slab_bytes, &keys_map, j * kSlabElems,
                                         tile * kRowsPerTile + sub * kTileRows, &full[s]);
@@ -303,7 +307,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     const int sl0 = (it % gpt) * gs;
                     const int nsl = min(gs, dslabs - sl0);
                     mbar_arrive_expect_tx(&full[s], (uint32_t)(nsl * slab_bytes));
-                    for (int j = 0; j < nsl; ++j) {
+                    for (int j = 0; j < nsl && !lose; ++j) {
                         tma_load_2d(dst + (size_t)j * slab_bytes, &keys_map, (sl0 + j) * kSlabElems,
                                     tile * kTileRows, &full[s]);
                         if (!q_resident)
@@ -315,11 +319,11 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             }
             // Do not leave while copies into this CTA's shared memory are in flight.
             for (int it = max(0, issued - n_stages); it < issued; ++it)
-                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1)) {
+                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1, wl)) {
                     report_timeout(a.status);
                     break;
                 }
-            if (q_resident && !mbar_wait(qbar, 0)) report_timeout(a.status);
+            if (q_resident && !mbar_wait(qbar, 0, wl)) report_timeout(a.status);
         }
     } else if (warp == 1 || warp == kIssuer2Warp) {
         // ---------------------------------- MMA issuer ----------------------------------
@@ -331,16 +335,16 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             constexpr uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(NCOLS >> 3) << 17) |
                                        ((uint32_t)(kTileRows >> 4) << 24);
             bool ok = true;
-            if (q_resident && my_tiles > 0) ok = mbar_wait(qbar, 0);
+            if (q_resident && my_tiles > 0) ok = mbar_wait(qbar, 0, wl);
             for (int tl = 0; tl < my_tiles && ok; ++tl) {
                 const int acc = tl & 1, use = tl >> 1;
-                if (use >= 1 && !mbar_wait(&tempty[acc], (use - 1) & 1)) { ok = false; break; }
+                if (use >= 1 && !mbar_wait(&tempty[acc], (use - 1) & 1, wl)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
                 for (int g = 0; g < gpt; ++g) {
                     const int it = tl * gpt + g;
                     const int s = it % n_stages;
-                    if (!mbar_wait(&full[s], (it / n_stages) & 1)) { ok = false; break; }
+                    if (!mbar_wait(&full[s], (it / n_stages) & 1, wl)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t st_addr = smem_u32(stages + (size_t)s * stage_bytes);
                     if constexpr (TSUB > 1) {
@@ -488,7 +492,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     }
                 }
             }
-            if (!dead && !mbar_wait(&tfull[acc], use & 1)) {
+            if (!dead && !mbar_wait(&tfull[acc], use & 1, wl)) {
                 report_timeout(a.status);
                 dead = true;
             }

@@ -121,6 +121,7 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
     const int cta = blockIdx.x, G = gridDim.x;
     const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
     const int n_it = my_tiles * dslabs;
+    const long long wl = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;   // bound of every wait below
 
     if (tid == 0) {
         for (int s = 0; s < n_stages; ++s) {
@@ -172,7 +173,7 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
             int issued = 0;
             for (int it = 0; it < n_it; ++it) {
                 const int s = it % n_stages;
-                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
+                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1, wl)) {
                     report_timeout(a.status);
                     break;
                 }
@@ -181,17 +182,22 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
                 uint8_t *dst = stages + (size_t)s * kStageBytes;
                 // rows past N read as zeros (a box may start past the end)
                 mbar_arrive_expect_tx(&full[s], (uint32_t)kStageBytes);
+                // Test hook: CTA 0 "loses" the copies of one stage, so that the waits on it run out.
+                if (a.debug_lose_stage > 0 && cta == 0 && it == a.debug_lose_stage - 1) {
+                    issued = it + 1;
+                    continue;
+                }
                 tma_load_2d(dst, &keys_map, ks * kSlabElems, tile * kTileKeys, &full[s]);
                 tma_load_2d(dst + kBoxBytes, &keys_map, ks * kSlabElems, tile * kTileKeys + 128, &full[s]);
                 issued = it + 1;
             }
             // Do not leave while copies into this CTA's shared memory are in flight.
             for (int it = max(0, issued - n_stages); it < issued; ++it)
-                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1)) {
+                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1, wl)) {
                     report_timeout(a.status);
                     break;
                 }
-            if (!mbar_wait(qbar, 0)) report_timeout(a.status);
+            if (!mbar_wait(qbar, 0, wl)) report_timeout(a.status);
         }
     } else if (warp == 1) {
         // ---------------------------------- MMA issuer ----------------------------------
@@ -201,16 +207,16 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
             constexpr uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(kTileKeys >> 3) << 17) |
                                        ((uint32_t)(kOpRows >> 4) << 24);
             bool ok = true;
-            if (my_tiles > 0) ok = mbar_wait(qbar, 0);
+            if (my_tiles > 0) ok = mbar_wait(qbar, 0, wl);
             for (int tl = 0; tl < my_tiles && ok; ++tl) {
                 const int acc = tl & 1, use = tl >> 1;
-                if (use >= 1 && !mbar_wait(&tempty[acc], (use - 1) & 1)) { ok = false; break; }
+                if (use >= 1 && !mbar_wait(&tempty[acc], (use - 1) & 1, wl)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccCols);
                 for (int ks = 0; ks < dslabs; ++ks) {
                     const int it = tl * dslabs + ks;
                     const int s = it % n_stages;
-                    if (!mbar_wait(&full[s], (it / n_stages) & 1)) { ok = false; break; }
+                    if (!mbar_wait(&full[s], (it / n_stages) & 1, wl)) { ok = false; break; }
                     tc_fence_after();
                     const uint64_t a_desc = make_desc(smem_u32(qres + (size_t)ks * kQSlabBytes));
                     const uint64_t b_desc = make_desc(smem_u32(stages + (size_t)s * kStageBytes));
@@ -259,7 +265,7 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
             // first stored token of the tile's keys (filtered calls), requested before the wait
             int tk = -1;
             if (filtered && tile_key0 + et < a.N) tk = a.first_col[tile_key0 + et];
-            if (!dead && !mbar_wait(&tfull[acc], use & 1)) {
+            if (!dead && !mbar_wait(&tfull[acc], use & 1, wl)) {
                 report_timeout(a.status);
                 dead = true;
             }

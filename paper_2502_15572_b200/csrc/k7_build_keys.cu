@@ -148,6 +148,8 @@ struct BuildArgs {
     void *out;               // [N][d] store dtype
     float eps_n;
     int *status;
+    long long wait_cycles;   // bound of every device-side wait in cycles, 0 = default
+    int lose_stage;          // test hook: the first CTA (pair) never receives stage (value-1); 0 = off
 };
 
 template <typename T>
@@ -174,6 +176,7 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
     const int cta = blockIdx.x, G = gridDim.x;
     const int my_tiles = cta < a.n_tiles ? (a.n_tiles - cta + G - 1) / G : 0;
     const int n_it = my_tiles * kslabs;
+    const long long wl = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;   // bound of every wait below
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * a.d) tmem_cols <<= 1;
 
@@ -204,7 +207,7 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
             int issued = 0;
             for (int it = 0; it < n_it; ++it) {
                 const int s = it % n_stages;
-                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
+                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1, wl)) {
                     report_timeout(a.status);
                     break;
                 }
@@ -212,6 +215,11 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
                 const int ks = it % kslabs;
                 uint8_t *dst = stages + (size_t)s * stage_bytes;
                 mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
+                // Test hook: CTA 0 "loses" the copies of one stage, so that the waits on it run out.
+                if (a.lose_stage > 0 && cta == 0 && it == a.lose_stage - 1) {
+                    issued = it + 1;
+                    continue;
+                }
                 tma_load_2d(dst, &h_map, ks * kSlabElems, tile * kTileRows, &full[s]);
                 tma_load_2d(dst + kASlab, &h_map, ks * kSlabElems, tile * kTileRows + kSubRows, &full[s]);
                 tma_load_2d(dst + 2 * kASlab, &whi_map, ks * kSlabElems, 0, &full[s]);
@@ -219,7 +227,7 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
                 issued = it + 1;
             }
             for (int it = max(0, issued - n_stages); it < issued; ++it)
-                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1)) {
+                if (!mbar_wait(&full[it % n_stages], (it / n_stages) & 1, wl)) {
                     report_timeout(a.status);
                     break;
                 }
@@ -233,12 +241,12 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
             const bool two = a.terms == 2;
             for (int tl = 0; tl < my_tiles && ok; ++tl) {
                 // one accumulator set: wait until the epilogue has drained the previous tile
-                if (tl >= 1 && !mbar_wait(tempty, (tl - 1) & 1)) { ok = false; break; }
+                if (tl >= 1 && !mbar_wait(tempty, (tl - 1) & 1, wl)) { ok = false; break; }
                 tc_fence_after();
                 for (int ks = 0; ks < kslabs; ++ks) {
                     const int it = tl * kslabs + ks;
                     const int s = it % n_stages;
-                    if (!mbar_wait(&full[s], (it / n_stages) & 1)) { ok = false; break; }
+                    if (!mbar_wait(&full[s], (it / n_stages) & 1, wl)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
                     const uint64_t bhi = make_desc(st + 2 * kASlab), blo = make_desc(st + 2 * kASlab + b_slab);
@@ -268,7 +276,7 @@ build_keys_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_consta
         T *out = static_cast<T *>(a.out);
         bool dead = false;
         for (int tl = 0; tl < my_tiles; ++tl) {
-            if (!dead && !mbar_wait(tfull, tl & 1)) {
+            if (!dead && !mbar_wait(tfull, tl & 1, wl)) {
                 report_timeout(a.status);
                 dead = true;
             }
@@ -329,6 +337,7 @@ build_keys_pair_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_c
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int my_tiles = pair < a.n_tiles ? (a.n_tiles - pair + n_pairs - 1) / n_pairs : 0;   // 512-row pair tiles
     const int n_it = my_tiles * kslabs;
+    const long long wl = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;   // bound of every wait below
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * a.d) tmem_cols <<= 1;
 
@@ -360,7 +369,7 @@ build_keys_pair_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_c
             bool ok = true;
             for (int it = 0; it < n_it; ++it) {
                 const int s = it % n_stages;
-                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1)) {
+                if (it >= n_stages && !mbar_wait(&empty[s], ((it / n_stages) - 1) & 1, wl)) {
                     report_timeout(a.status);
                     ok = false;
                     break;
@@ -371,6 +380,9 @@ build_keys_pair_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_c
                 uint8_t *dst = stages + (size_t)s * stage_bytes;
                 const uint32_t lead_full = mapa_rank(smem_u32(&full[s]), 0);
                 if (rank == 0) mbar_arrive_expect_tx(&full[s], (uint32_t)(2 * stage_bytes));
+                // Test hook: the leader of pair 0 "loses" its copies of one stage (the peer's still
+                // arrive), so that the leader's barrier never completes and the waits on it run out.
+                if (a.lose_stage > 0 && pair == 0 && rank == 0 && it == a.lose_stage - 1) continue;
                 tma_load_2d_pair(dst, &h_map, ks * kSlabElems, row0, lead_full);
                 tma_load_2d_pair(dst + kASlab, &h_map, ks * kSlabElems, row0 + kSubRows, lead_full);
                 tma_load_2d_pair(dst + 2 * kASlab, &whi_map, ks * kSlabElems, (int)rank * (a.d / 2), lead_full);
@@ -394,12 +406,12 @@ build_keys_pair_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_c
             const bool two = a.terms == 2;
             for (int tl = 0; tl < my_tiles && ok; ++tl) {
                 // one accumulator set: both epilogues have drained the previous tile
-                if (tl >= 1 && !mbar_wait(tempty, (tl - 1) & 1)) { ok = false; break; }
+                if (tl >= 1 && !mbar_wait(tempty, (tl - 1) & 1, wl)) { ok = false; break; }
                 tc_fence_after();
                 for (int ks = 0; ks < kslabs; ++ks) {
                     const int it = tl * kslabs + ks;
                     const int s = it % n_stages;
-                    if (!mbar_wait(&full[s], (it / n_stages) & 1)) { ok = false; break; }
+                    if (!mbar_wait(&full[s], (it / n_stages) & 1, wl)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t st = smem_u32(stages + (size_t)s * stage_bytes);
                     const uint64_t bhi = make_desc(st + 2 * kASlab), blo = make_desc(st + 2 * kASlab + b_half);
@@ -430,7 +442,7 @@ build_keys_pair_kernel(const __grid_constant__ CUtensorMap h_map, const __grid_c
         T *out = static_cast<T *>(a.out);
         bool dead = false;
         for (int tl = 0; tl < my_tiles; ++tl) {
-            if (!dead && !mbar_wait(tfull, tl & 1)) {
+            if (!dead && !mbar_wait(tfull, tl & 1, wl)) {
                 report_timeout(a.status);
                 dead = true;
             }
@@ -481,9 +493,12 @@ cudaError_t launch_build_prep(const void *W, int dtype, const float *mean, const
 
 cudaError_t launch_build_keys(const CUtensorMap &h_map, const CUtensorMap &whi_map, const CUtensorMap &wlo_map,
                               int dtype, long long N, int d_in, int d, int terms, int pair, const float *bias,
-                              void *out, float eps_n, int *status, int grid, cudaStream_t stream)
+                              void *out, float eps_n, int *status, int grid, cudaStream_t stream, long long wait_cycles,
+                              int lose_stage)
 {
     BuildArgs a{};
+    a.wait_cycles = wait_cycles;
+    a.lose_stage = lose_stage;
     a.terms = terms == 1 ? 1 : 2;
     a.N = N;
     a.d_in = d_in;
