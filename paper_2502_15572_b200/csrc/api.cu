@@ -138,7 +138,7 @@ struct dresd_store {
     CUtensorMap map_umma;
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     // options / bookkeeping
-    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m, opt_pack2;
+    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m, opt_pack2, opt_merged;
     double last_key_passes;      // passes over the key matrix in the last call (a probe pass counts 1/stride)
     const void *k8;              // 8-bit (E4M3) copy of the keys, borrowed; null = none attached
     void *qsplit8;               // [2 * kMaxBatch][dpad8] 8-bit query operand
@@ -274,16 +274,19 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // the kernel with the keys as the N operand reads hi and lo of a query from one TMEM fragment;
     // its operand always has 128 rows (64 hi, 64 lo), whatever the batch
     const int blocked = umma && !keys_as_m && scan_ummat_eligible(s->d, B);
+    // more than 16 queries on the other widths: one accumulator column per query (half the epilogue's work)
+    const int merged = umma && !q8 && !blocked && s->opt_merged != 2 &&
+                       (s->opt_merged == 1 ? B > 16 : scan_umma_merged_eligible(s->d, B, s->dtype));
     const int op_rows = !umma ? 0 : blocked ? 2 * kMaxBatch : scan_umma_operand_rows(pack2 ? 2 * B : B);
     // one CTA per operand query: two operand rows each, four in the packed 8-bit layout
     const int pre_rows = pack2 ? op_rows / 4 : umma ? op_rows / 2 : ((B + 7) / 8) * 8;
-    dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, blocked, pack2 ? 2 : q8 ? 1 : 0);
+    dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, merged ? 2 : blocked, pack2 ? 2 : q8 ? 1 : 0);
     if (st != DRESD_OK) return st;
 
     // the 8-bit store is scanned as rows of d/2 two-byte units (packed: N/2 rows of 64 units)
     const int scan_d = pack2 ? 64 : q8 ? s->d / 2 : s->d;
     const long long scan_rows = pack2 ? s->N / 2 : s->N;
-    const int umma_rows = umma ? scan_umma_tile_rows(scan_d, pack2 ? 2 * B : B, keys_as_m) : 1;
+    const int umma_rows = umma ? scan_umma_tile_rows(scan_d, pack2 ? 2 * B : B, keys_as_m, merged) : 1;
     const int n_tiles = umma ? (int)((scan_rows + umma_rows - 1) / umma_rows) : s->n_tiles;
     int grid = s->opt_grid > 0 ? s->opt_grid : s->num_sms;
     if (grid > s->max_grid) grid = s->max_grid;
@@ -312,6 +315,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.gtau = s->gtau;
         a.no_select = s->opt_no_select;
         a.keys_as_m = keys_as_m;
+        a.merged = merged;
         a.wait_cycles = (long long)s->opt_wait_ms * 2000000LL;     // ~2 GHz
         a.debug_lose_stage = s->opt_lose_stage;
         if (windows) {
@@ -731,7 +735,7 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
         return DRESD_OK;
     }
     if (strcmp(name, "debug_no_select") == 0) {
-        s->opt_no_select = value != 0;
+        s->opt_no_select = value;
         return DRESD_OK;
     }
     if (strcmp(name, "wait_ms") == 0) {
@@ -752,6 +756,11 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
     if (strcmp(name, "first_token_windows") == 0) {
         if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "first_token_windows takes 0 or 1");
         s->opt_windows = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "merged_columns") == 0) {
+        if (value < 0 || value > 2) return fail(DRESD_ERR_INVALID, "merged_columns = %d outside 0..2", value);
+        s->opt_merged = value;
         return DRESD_OK;
     }
     if (strcmp(name, "keys_as_m") == 0) {

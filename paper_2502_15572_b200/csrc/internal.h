@@ -31,7 +31,8 @@ struct PreprocessArgs {
     int rows;               // CTAs launched: B rounded up to the operand row count
     float lo_scale;
     unsigned int *gtau;     // [rows] grid-wide filter words, reset to 0 ("nothing known") here
-    int split_blocked;      // qsplit rows: 0 = (2b, 2b+1); 1 = 16-row blocks, hi rows 0-7, lo rows 8-15
+    int split_blocked;      // qsplit rows: 0 = (2b, 2b+1); 1 = 16-row blocks, hi rows 0-7, lo rows 8-15;
+                            // 2 = rows b and `rows` + b hold S hi and S (q - hi), S = lo_scale (one column per query)
     // Split projection (W given): `slices` CTAs of `rows_per_slice` rows of W each write
     // partial[slice][B][d]; null = every query's CTA walks all of W itself.
     float *partial;
@@ -76,6 +77,7 @@ struct ScanArgs {
     int probe_max;          // tcgen05 kernel, probe pass: keep only each tile's best row per query
     int no_select;          // tcgen05 kernel, measurement only: nothing passes the filter (scan floor)
     int keys_as_m;          // tcgen05 kernels: never use the form with the keys as the N = 256 operand
+    int merged;             // tcgen05 kernel, keys as M: one accumulator column per query (operand: hi' rows, then lo' rows)
     int pack2;              // 8-bit keys of 64 elements: a 128-byte row holds two keys (N = rows, ids = 2 row + parity)
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.
@@ -87,7 +89,10 @@ cudaError_t launch_scan_mma(const CUtensorMap &keys_map, const ScanArgs &a, int 
 
 // Batched tensor-core kernel (tcgen05/TMEM, 16-bit keys): 128-row tiles; the query
 // operand holds 2 rows per query, padded to 16/32/64/128 rows.
-int scan_umma_tile_rows(int d, int B, int keys_as_m);   // rows per tile of the kernel that will run
+int scan_umma_tile_rows(int d, int B, int keys_as_m, int merged);   // rows per tile of the kernel that will run
+bool scan_umma_merged_eligible(int d, int B, int dtype);            // one accumulator column per query
+cudaError_t launch_scan_umma_merged(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
+                                    int grid, cudaStream_t stream);
 int scan_umma_operand_rows(int B);
 cudaError_t launch_scan_umma(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
                              int grid, cudaStream_t stream);

@@ -177,8 +177,10 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
     pdl_launch_dependents();              // the scan may set itself up while this kernel runs
     // operand rows of query b: (2b, 2b+1), or -- blocked layout -- rows (b % 8) and 8 + (b % 8)
     // of the 16-row block b / 8, so that a 16-lane TMEM fragment holds hi and lo of 8 queries
-    const int row_hi = a.split_blocked ? 16 * (b >> 3) + (b & 7) : 2 * b;
-    const int row_lo = a.split_blocked ? row_hi + 8 : row_hi + 1;
+    // or -- merged layout -- rows b and rows + b, both terms scaled by lo_scale
+    const bool merged = a.split_blocked == 2;
+    const int row_hi = merged ? b : a.split_blocked ? 16 * (b >> 3) + (b & 7) : 2 * b;
+    const int row_lo = merged ? a.rows + b : a.split_blocked ? row_hi + 8 : row_hi + 1;
     T *split_hi = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)row_hi * a.dpad : nullptr;
     T *split_lo = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)row_lo * a.dpad : nullptr;
     float *qrow = a.qhat + (size_t)b * a.d;
@@ -275,6 +277,7 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
         if (split_hi) {
             T hi = from_f32<T>(x);
             float r = (x - to_f32<T>(hi)) * a.lo_scale;
+            if (merged) hi = from_f32<T>(to_f32<T>(hi) * a.lo_scale);     // exact: a power of two, |hi| <= 1
             split_hi[c] = hi;
             split_lo[c] = from_f32<T>(r);
         }
