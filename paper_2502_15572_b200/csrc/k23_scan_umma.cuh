@@ -710,31 +710,44 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         // yields a filter score, never a result row), so the maximum is one redux.sync per
                         // query on the order-preserving integer image of the score; the row that goes with
                         // it is any row of this sub-tile and lane group (distinct per entry, never returned).
+                        // Lane j keeps query j's maximum and stores it after the loop: no store inside the
+                        // loop, so that the reductions of different queries overlap.
+                        int wants[QW];
+#pragma unroll
+                        for (int j4 = 0; j4 < QW / 4; ++j4) {
+                            const int4 w = want4[j4];
+                            wants[4 * j4] = w.x; wants[4 * j4 + 1] = w.y; wants[4 * j4 + 2] = w.z; wants[4 * j4 + 3] = w.w;
+                        }
+                        uint32_t mine = 0u;
 #pragma unroll
                         for (int j = 0; j < QW; ++j) {
                             const float s = score_at(r, j);
-                            const int w = want_s[qbase + j];
                             const int tkj = (PACK2 && ((qbase + j) & 1)) ? tok1[sub] : tok[sub];
-                            const bool ok = row_ok && (w < 0 || tkj == w) && s > -INFINITY;        // false for NaN
+                            const bool ok = row_ok && (wants[j] < 0 || tkj == wants[j]) && s > -INFINITY;   // false for NaN
                             const uint32_t best = __reduce_max_sync(0xFFFFFFFFu, ok ? float_to_ordered(s + 0.0f) : 0u);
-                            if (lane == j % 32) {
-                                const uint32_t id = PACK2 ? (uint32_t)(2 * row + ((qbase + j) & 1)) : (uint32_t)row;
-                                slot[j] = best ? ((unsigned long long)best << 32) | (0xFFFFFFFFu - id) : 0ull;
-                            }
+                            if (lane == j) mine = best;
+                        }
+                        if (lane < QW) {
+                            const uint32_t id = PACK2 ? (uint32_t)(2 * row + ((qbase + lane) & 1)) : (uint32_t)row;
+                            slot[lane] = mine ? ((unsigned long long)mine << 32) | (0xFFFFFFFFu - id) : 0ull;
                         }
                     } else if (lane < QW) {
                         slot[lane] = 0ull;
                     }
                 }
                 epi_bar();                                   // all lane groups have written
-                for (int q = ew; q < a.B; q += kEpiWarps) {
-                    if (lane == 0) {
-                        for (int sub = 0; sub < TSUB; ++sub) {
-                            const unsigned long long *m = tilemax + (size_t)(sub * 4) * NQ + (PACK2 ? 2 * q : q);
-                            unsigned long long v = umax64(umax64(m[0], m[NQ]), umax64(m[2 * NQ], m[3 * NQ]));
-                            if constexpr (PACK2)               // the odd keys of the same rows
-                                v = umax64(v, umax64(umax64(m[1], m[NQ + 1]), umax64(m[2 * NQ + 1], m[3 * NQ + 1])));
-                            if (v && sel[q].count < kQueueCap) sel[q].queue[sel[q].count++] = v;
+                // a lane per (query of this warp, sub-tile): the best of the four lane groups joins the queue
+                {
+                    const int q = ew + kEpiWarps * (lane / TSUB), sub = lane % TSUB;
+                    if (q < a.B) {
+                        const unsigned long long *m = tilemax + (size_t)(sub * 4) * NQ + (PACK2 ? 2 * q : q);
+                        unsigned long long v = umax64(umax64(m[0], m[NQ]), umax64(m[2 * NQ], m[3 * NQ]));
+                        if constexpr (PACK2)               // the odd keys of the same rows
+                            v = umax64(v, umax64(umax64(m[1], m[NQ + 1]), umax64(m[2 * NQ + 1], m[3 * NQ + 1])));
+                        if (v) {
+                            const int at = atomicAdd(&sel[q].count, 1);
+                            if (at < kQueueCap) sel[q].queue[at] = v;
+                            else atomicSub(&sel[q].count, 1);
                         }
                     }
                 }
