@@ -85,7 +85,7 @@ __host__ __device__ inline Layout make_layout(int n_stages, int dslabs)
     l.tok_off = l.want_off + (int)sizeof(int) * kNQ;
     l.best_off = l.tok_off + (int)sizeof(int) * kTileKeys;
     l.bar_off = l.best_off + (int)sizeof(unsigned long long) * kNQ;
-    l.total = l.bar_off + (int)sizeof(uint64_t) * (2 * kMaxStages + 5) + 8 + (int)sizeof(EpiFlags) * 4;
+    l.total = l.bar_off + (int)sizeof(uint64_t) * (2 * kMaxStages + 5) + 8 + (int)sizeof(EpiFlags) * 3;
     return l;
 }
 
@@ -133,7 +133,7 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
             mbar_init(&tempty[b], kEpiWarps);
         }
         mbar_init(qbar, 1);
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 3; ++i) {
             flags[i].need_merge = 0;
             flags[i].overflow = 0;
         }
@@ -256,44 +256,6 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
         bool dead = false;
         int round = 0;                                      // barrier-A count: selects the flag slot
         EpiFlags *fl = &flags[0];
-        int *done_warps = &flags[3].need_merge;             // epilogue warps that are through all their tiles
-        // Rounds on demand, as in the kernel with the keys as M (k23_scan_umma.cuh): the warps do not
-        // meet at every tile; a warp goes to barrier A when a flag word of the current round is set, which
-        // it checks at the end of a tile and while it waits for an accumulator.  Calls with the
-        // first-token filter (the tile's tokens are staged in shared memory behind a barrier) and the
-        // probe pass keep a round per tile.
-        const bool free_run = !filtered && !a.probe_max;
-        int last_over = 0, last_done = 0;
-        auto round_wanted = [&]() -> bool {
-            return (*reinterpret_cast<volatile int *>(&fl->need_merge) | *reinterpret_cast<volatile int *>(&fl->overflow)) != 0;
-        };
-        auto one_round = [&]() -> int {
-            epi_bar();                                       // A: every push so far is visible
-            const int need = fl->need_merge, over = fl->overflow;
-            last_done = *reinterpret_cast<volatile int *>(done_warps);
-            last_over = over;
-            // Flags rotate over three slots: the slot of the previous round was read by
-            // everyone before arriving at A and is not written again before the next A.
-            if (et == 0) {
-                EpiFlags *prev = &flags[(round + 2) % 3];
-                prev->need_merge = 0;
-                prev->overflow = 0;
-            }
-            round += 1;
-            fl = &flags[round % 3];
-            if (need | over) {
-                for (int qq = ew; qq < kNQ; qq += kEpiWarps) {
-                    if (sel[qq].count > 0) {
-                        warp_topn_merge(&sel[qq], a.top_n, lane);
-                        if (lane == 0 && qq < a.B) tau[qq] = share_tau(&a.gtau[qq], sel[qq].tau);
-                    }
-                }
-            }
-            // C: lists, counts and tau are settled; free-running warps hold it in every round, so that
-            // nobody leaves a round (and counts itself done) before all have read its flags
-            if ((need | over) || free_run) epi_bar();
-            return over;
-        };
 
         for (int tl = 0; tl < my_tiles; ++tl) {
             const int acc = tl & 1, use = tl >> 1;
@@ -303,31 +265,14 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
             // first stored token of the tile's keys (filtered calls), requested before the wait
             int tk = -1;
             if (filtered && tile_key0 + et < a.N) tk = a.first_col[tile_key0 + et];
-            // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best); the
-            // word comes from L2: requested before the wait for the accumulator, used after it
-            const bool pull = (tl & 3) == 0 && et < a.B && !a.no_select;
-            unsigned int gword = 0u;
-            if (pull) gword = *reinterpret_cast<const volatile unsigned int *>(&a.gtau[et]);
-            if (!dead && !mbar_try_wait(&tfull[acc], use & 1)) {
-                const long long t0 = clock64();
-                while (!mbar_try_wait(&tfull[acc], use & 1)) {
-                    // a warp that waits at the round's barrier holds its accumulator buffer, which this
-                    // wait may depend on: rounds are attended from here too
-                    if (free_run && round_wanted())
-                        while (one_round()) {}
-                    if (clock64() - t0 > wl) {
-                        report_timeout(a.status);
-                        dead = true;
-                        break;
-                    }
-                }
+            if (!dead && !mbar_wait(&tfull[acc], use & 1, wl)) {
+                report_timeout(a.status);
+                dead = true;
             }
             dead = __any_sync(0xFFFFFFFFu, dead);
             tc_fence_after();
-            if (pull && gword) {
-                const float g = ordered_to_float(gword);
-                if (g > tau[et]) tau[et] = g;
-            }
+            // every fourth tile, pull the grid-wide filter (other CTAs may know a better n-th best)
+            if ((tl & 3) == 0 && et < a.B && !a.no_select) tau[et] = peek_tau(&a.gtau[et], tau[et]);
             if (filtered) {
                 tok_s[et] = tk;                             // readers of the previous tile are past its barrier A
                 epi_bar();
@@ -450,7 +395,6 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
                 return false;
             };
             bool first_round = true;
-            int must = 0;                                   // the last round left an overflow: the next one is attended too
             while (true) {
                 const float tau0 = tau[qq0], tau1 = tau[qq0 + 8];
                 if (!dead && first_round) {
@@ -479,27 +423,33 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
                     next_unit = u;
                 }
                 first_round = false;
-                // nobody has asked for a round (no queue at the merge level, none overflowed): no barrier
-                const bool mine = __any_sync(0xFFFFFFFFu, resume);
-                if (free_run && !must && !mine && !round_wanted()) break;
-                must = one_round();
-                if (!must) break;
+                epi_bar();                                   // A: every push of this round is visible
+                const int need = fl->need_merge, over = fl->overflow;
+                // Flags rotate over three slots: the slot of the previous round was read by
+                // everyone before arriving at A and is not written again before the next A.
+                if (et == 0) {
+                    EpiFlags *prev = &flags[(round + 2) % 3];
+                    prev->need_merge = 0;
+                    prev->overflow = 0;
+                }
+                round += 1;
+                fl = &flags[round % 3];
+                if (!(need | over)) break;
+                for (int qq = ew; qq < kNQ; qq += kEpiWarps) {
+                    if (sel[qq].count > 0) {
+                        warp_topn_merge(&sel[qq], a.top_n, lane);
+                        if (lane == 0 && qq < a.B) tau[qq] = share_tau(&a.gtau[qq], sel[qq].tau);
+                    }
+                }
+                epi_bar();                                   // C: lists, counts and tau are settled
+                if (!over) break;
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty[acc]);
         }
-        // Through all tiles.  Other warps may still ask for rounds: they are attended until every warp is here.
-        if (free_run) {
-            if (lane == 0) atomicAdd(done_warps, 1);
-            while (true) {
-                one_round();
-                if (last_done == kEpiWarps && !last_over) break;
-            }
-        } else {
-            epi_bar();
-        }
         // flush and publish this CTA's lists
+        epi_bar();
         for (int qq = ew; qq < kNQ; qq += kEpiWarps) {
             if (sel[qq].count > 0) warp_topn_merge(&sel[qq], a.top_n, lane);
             if (qq < a.B) {
