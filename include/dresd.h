@@ -340,9 +340,10 @@ dresd_status dresd_store_status(dresd_store *store);
  *   "probe"      large batches on large stores first run a probe pass over every
  *                value-th key tile to seed the selection filter; 0 = never,
  *                1 = default stride (128).
- *   "pack2"      1 (default): the quantised search of a store with d = 64 scans the 8-bit copy
- *                as rows of two keys (one 128-byte line), up to 32 queries per call; 0 = one
- *                key per row.  Results do not change.
+ *   "pack2"      1 (default): 64-byte keys are scanned as rows of two keys (one 128-byte line) --
+ *                the 8-bit copy of a store with d = 64 in the quantised search (up to 32 queries
+ *                per call), and a 16-bit store with d = 32 and an even number of rows in the exact
+ *                search (up to 16 queries per call); 0 = one key per row.  Results do not change.
  *   "keys_as_m"  0 (default): batches of 17-64 queries on rows of 129-256 elements run the
  *                tcgen05 kernel with the queries as the M = 128 and the keys as the
  *                N = 256 operand of the instruction; 1 = keys as the M operand at every

@@ -138,7 +138,7 @@ struct dresd_store {
     CUtensorMap map_umma;
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     // options / bookkeeping
-    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m, opt_pack2, opt_merged;
+    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m, opt_pack2, opt_merged, opt_round_per_tile;
     double last_key_passes;      // passes over the key matrix in the last call (a probe pass counts 1/stride)
     const void *k8;              // 8-bit (E4M3) copy of the keys, borrowed; null = none attached
     void *qsplit8;               // [2 * kMaxBatch][dpad8] 8-bit query operand
@@ -146,6 +146,8 @@ struct dresd_store {
     CUtensorMap map_k8, map_q8[4];
     CUtensorMap map_k8p;         // d = 64: the 8-bit copy as N/2 rows of two keys (128 bytes)
     int k8_packable;
+    CUtensorMap map_k16p;        // 16-bit keys, d = 32, even N: the store as N/2 rows of two keys (128 bytes)
+    int k16_packable;
     int prof_stride, prof_calls;
     float *proj_ws;              // partial products of the split projection (allocated with W)
     size_t proj_ws_bytes;
@@ -258,7 +260,11 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // tcgen05 kernel, other instruction kind), then exact re-ranking of the quantised_m best
     const bool q8 = quantised_m > 0;
     // 64-element keys are 64 bytes in the 8-bit copy: two per 128-byte row, two column pairs per query
-    const bool pack2 = q8 && s->k8_packable && B <= kMaxBatch / 2 && s->opt_pack2;
+    const bool pack8 = q8 && s->k8_packable && B <= kMaxBatch / 2 && s->opt_pack2;
+    // 32-element 16-bit keys are 64 bytes as well: the same two-keys-per-row scan for up to 16 queries
+    // (more run the form with one accumulator column per query)
+    const bool pack16 = !q8 && s->dtype != kF32 && s->opt_path != 1 && s->k16_packable && B <= 16 && s->opt_pack2;
+    const bool pack2 = pack8 || pack16;
     s->last_stream = stream;
     s->last_launches = 0;
     s->last_key_passes = 0.0;
@@ -275,12 +281,13 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     // its operand always has 128 rows (64 hi, 64 lo), whatever the batch
     const int blocked = umma && !keys_as_m && scan_ummat_eligible(s->d, B);
     // more than 16 queries on the other widths: one accumulator column per query (half the epilogue's work)
-    const int merged = umma && !q8 && !blocked && s->opt_merged != 2 &&
+    const int merged = umma && !q8 && !blocked && !pack16 && s->opt_merged != 2 &&
                        (s->opt_merged == 1 ? B > 16 : scan_umma_merged_eligible(s->d, B, s->dtype));
     const int op_rows = !umma ? 0 : blocked ? 2 * kMaxBatch : scan_umma_operand_rows(pack2 ? 2 * B : B);
     // one CTA per operand query: two operand rows each, four in the packed 8-bit layout
     const int pre_rows = pack2 ? op_rows / 4 : umma ? op_rows / 2 : ((B + 7) / 8) * 8;
-    dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, merged ? 2 : blocked, pack2 ? 2 : q8 ? 1 : 0);
+    dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, pack16 ? 3 : merged ? 2 : blocked,
+                                     pack8 ? 2 : q8 ? 1 : 0);
     if (st != DRESD_OK) return st;
 
     // the 8-bit store is scanned as rows of d/2 two-byte units (packed: N/2 rows of 64 units)
@@ -316,13 +323,14 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.no_select = s->opt_no_select;
         a.keys_as_m = keys_as_m;
         a.merged = merged;
+        a.round_per_tile = s->opt_round_per_tile;
         a.wait_cycles = (long long)s->opt_wait_ms * 2000000LL;     // ~2 GHz
         a.debug_lose_stage = s->opt_lose_stage;
         if (windows) {
             a.win_start = s->win_start;
             a.win_vocab = s->win_vocab;
         }
-        const CUtensorMap &kmap = pack2 ? s->map_k8p : q8 ? s->map_k8 : s->map_umma;
+        const CUtensorMap &kmap = pack8 ? s->map_k8p : pack16 ? s->map_k16p : q8 ? s->map_k8 : s->map_umma;
         const CUtensorMap *qmaps = q8 ? s->map_q8 : s->map_q;
         const int sel_n = a.top_n;
         a.first_col = first_tokens ? s->first_col : nullptr;
@@ -385,7 +393,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     if (q8) {
         // fold the approximate lists, score the m survivors exactly, sort, gather: one launch
         cudaError_t e = launch_merge_rerank(s->cand, grid, B, s->keys, s->dtype, s->d, s->N, s->qhat, quantised_m, top_n,
-                                            pack2 && (s->N & 1) ? s->N - 1 : -1, first_tokens, s->next_tokens, s->stored_len,
+                                            pack8 && (s->N & 1) ? s->N - 1 : -1, first_tokens, s->next_tokens, s->stored_len,
                                             draft_len, out_ids, out_scores, out_tokens, stream);
         if (e != cudaSuccess) return fail_cuda(e, "merge / re-rank launch");
         s->last_launches += 1;
@@ -499,6 +507,11 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
         bool mok = make_map(&s->map_umma, keys, s->dtype, N, d, 128);
         for (int i = 0; i < 4; ++i)
             mok = mok && make_map(&s->map_q[i], s->qsplit, s->dtype, 2 * kMaxBatch, s->dpad, 16 << i);
+        // 32-element keys are 64 bytes: an even-sized store is also seen as N/2 rows of two keys
+        if (mok && d == 32 && N >= 2 && (N & 1) == 0) {
+            mok = make_map(&s->map_k16p, keys, s->dtype, N / 2, 64, 128);
+            s->k16_packable = mok ? 1 : 0;
+        }
         if (!mok) {
             free_store(s);
             return fail(DRESD_ERR_CUDA, "cuTensorMapEncodeTiled failed for the tensor-core path");
@@ -756,6 +769,11 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
     if (strcmp(name, "first_token_windows") == 0) {
         if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "first_token_windows takes 0 or 1");
         s->opt_windows = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "round_per_tile") == 0) {
+        if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "round_per_tile takes 0 or 1");
+        s->opt_round_per_tile = value;
         return DRESD_OK;
     }
     if (strcmp(name, "merged_columns") == 0) {

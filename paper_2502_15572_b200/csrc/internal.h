@@ -32,7 +32,8 @@ struct PreprocessArgs {
     float lo_scale;
     unsigned int *gtau;     // [rows] grid-wide filter words, reset to 0 ("nothing known") here
     int split_blocked;      // qsplit rows: 0 = (2b, 2b+1); 1 = 16-row blocks, hi rows 0-7, lo rows 8-15;
-                            // 2 = rows b and `rows` + b hold S hi and S (q - hi), S = lo_scale (one column per query)
+                            // 2 = rows b and `rows` + b hold S hi and S (q - hi), S = lo_scale (one column per query);
+                            // 3 = d = 32 keys scanned two per 64-element row: rows 4b .. 4b+3 = (hi|0), (lo|0), (0|hi), (0|lo)
     // Split projection (W given): `slices` CTAs of `rows_per_slice` rows of W each write
     // partial[slice][B][d]; null = every query's CTA walks all of W itself.
     float *partial;
@@ -77,8 +78,9 @@ struct ScanArgs {
     int probe_max;          // tcgen05 kernel, probe pass: keep only each tile's best row per query
     int no_select;          // tcgen05 kernel, measurement only: nothing passes the filter (scan floor)
     int keys_as_m;          // tcgen05 kernels: never use the form with the keys as the N = 256 operand
+    int round_per_tile;     // tcgen05 kernel, keys as M: the epilogue warps meet at every tile (measurement)
     int merged;             // tcgen05 kernel, keys as M: one accumulator column per query (operand: hi' rows, then lo' rows)
-    int pack2;              // 8-bit keys of 64 elements: a 128-byte row holds two keys (N = rows, ids = 2 row + parity)
+    int pack2;              // 64-byte keys (8-bit d = 64, 16-bit d = 32): a 128-byte row holds two keys (N = rows, ids = 2 row + parity)
 };
 // Tile heights (rows per TMA stage) so that api.cu can build matching tensor maps.
 int scan_mma_tile_rows(int d);
@@ -91,6 +93,9 @@ cudaError_t launch_scan_mma(const CUtensorMap &keys_map, const ScanArgs &a, int 
 // operand holds 2 rows per query, padded to 16/32/64/128 rows.
 int scan_umma_tile_rows(int d, int B, int keys_as_m, int merged);   // rows per tile of the kernel that will run
 bool scan_umma_merged_eligible(int d, int B, int dtype);            // one accumulator column per query
+// 16-bit keys of 32 elements scanned as rows of two keys (the packed forms of the kernel for 16-bit operands)
+cudaError_t launch_scan_umma_pack16(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
+                                    int grid, cudaStream_t stream);
 cudaError_t launch_scan_umma_merged(const CUtensorMap &keys_map, const CUtensorMap &q_map, const ScanArgs &a,
                                     int grid, cudaStream_t stream);
 int scan_umma_operand_rows(int B);

@@ -177,10 +177,12 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
     pdl_launch_dependents();              // the scan may set itself up while this kernel runs
     // operand rows of query b: (2b, 2b+1), or -- blocked layout -- rows (b % 8) and 8 + (b % 8)
     // of the 16-row block b / 8, so that a 16-lane TMEM fragment holds hi and lo of 8 queries
-    // or -- merged layout -- rows b and rows + b, both terms scaled by lo_scale
-    const bool merged = a.split_blocked == 2;
-    const int row_hi = merged ? b : a.split_blocked ? 16 * (b >> 3) + (b & 7) : 2 * b;
-    const int row_lo = merged ? a.rows + b : a.split_blocked ? row_hi + 8 : row_hi + 1;
+    // or -- merged layout -- rows b and rows + b, both terms scaled by lo_scale;
+    // or -- packed layout, two 32-element keys per 64-element store row -- rows 4b .. 4b+3 =
+    // (hi|0), (lo|0), (0|hi), (0|lo): two column pairs that score the even and the odd key of a row
+    const bool merged = a.split_blocked == 2, packed = a.split_blocked == 3;
+    const int row_hi = packed ? 4 * b : merged ? b : a.split_blocked ? 16 * (b >> 3) + (b & 7) : 2 * b;
+    const int row_lo = merged ? a.rows + b : a.split_blocked == 1 ? row_hi + 8 : row_hi + 1;
     T *split_hi = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)row_hi * a.dpad : nullptr;
     T *split_lo = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)row_lo * a.dpad : nullptr;
     float *qrow = a.qhat + (size_t)b * a.d;
@@ -192,6 +194,10 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
             for (int c = tid; c < a.dpad; c += blockDim.x) {
                 split_hi[c] = from_f32<T>(0.f);
                 split_lo[c] = from_f32<T>(0.f);
+                if (packed) {
+                    split_hi[2 * a.dpad + c] = from_f32<T>(0.f);
+                    split_lo[2 * a.dpad + c] = from_f32<T>(0.f);
+                }
             }
         if (a.qsplit8)
             for (int c = tid; c < a.dpad8; c += blockDim.x) store_query_e4m3(a.qsplit8, a.dpad8, a.pack2, b, c, 0.f);
@@ -278,6 +284,22 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
             T hi = from_f32<T>(x);
             float r = (x - to_f32<T>(hi)) * a.lo_scale;
             if (merged) hi = from_f32<T>(to_f32<T>(hi) * a.lo_scale);     // exact: a power of two, |hi| <= 1
+            if (packed) {
+                // c < 32: the query's element c, for the even key (columns c) and the odd key (columns 32 + c);
+                // the other half of every operand row is zero
+                if (c < 32) {
+                    const T z = from_f32<T>(0.f), lo = from_f32<T>(r);
+                    split_hi[c] = hi;
+                    split_hi[32 + c] = z;
+                    split_lo[c] = lo;
+                    split_lo[32 + c] = z;
+                    split_hi[2 * a.dpad + c] = z;
+                    split_hi[2 * a.dpad + 32 + c] = hi;
+                    split_lo[2 * a.dpad + c] = z;
+                    split_lo[2 * a.dpad + 32 + c] = lo;
+                }
+                continue;
+            }
             split_hi[c] = hi;
             split_lo[c] = from_f32<T>(r);
         }

@@ -130,6 +130,7 @@ cudaError_t launch_scan_umma(const CUtensorMap &kmap, const CUtensorMap &qmap, c
     if (!a_in.keys_as_m && a_in.dtype != kE4M3 && scan_ummat_eligible(a_in.d, a_in.B))
         return launch_scan_ummat(kmap, qmap, a_in, grid, stream);
     if (a_in.merged) return launch_scan_umma_merged(kmap, qmap, a_in, grid, stream);
+    if (a_in.pack2 && a_in.dtype != kE4M3) return launch_scan_umma_pack16(kmap, qmap, a_in, grid, stream);
     ScanArgs a = a_in;
     if (a.tile_stride < 1) a.tile_stride = 1;
     const bool h = a.dtype == kF16, q8 = a.dtype == kE4M3;

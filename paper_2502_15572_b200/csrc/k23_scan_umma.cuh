@@ -592,7 +592,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         // every round (bar.sync counts them), whichever tile each is at; they are never more than two
         // tiles apart (two accumulator buffers).  Token windows and the probe pass, whose tiles have
         // barriers of their own, keep a round per tile.
-        const bool free_run = !win_on && !a.probe_max;
+        const bool free_run = !win_on && !a.probe_max && !a.round_per_tile;
         int last_over = 0, last_done = 0;
         auto round_wanted = [&]() -> bool {
             return (*reinterpret_cast<volatile int *>(&fl->need_merge) | *reinterpret_cast<volatile int *>(&fl->overflow)) != 0;

@@ -54,6 +54,9 @@ def _run(dtype, d, B, n, L, N, vocab, path, seed):
     ("bf16", 512, 6, 10, 3, 20011, 50, 1),
     ("f32", 128, 8, 10, 10, 40009, 50, 0),
     ("f32", 64, 11, 32, 2, 20011, 3000, 0),
+    ("f16", 32, 6, 10, 2, 50022, 50, 0),           # two keys per row: a token per key of the row
+    ("bf16", 32, 16, 10, 2, 50022, 3000, 0),
+    ("f16", 32, 30, 10, 2, 50022, 50, 0),          # one column per query
 ])
 def test_first_token_filter_parity(dtype, d, B, n, L, N, vocab, path):
     _run(dtype, d, B, n, L, N, vocab, path, 9500 + d + B)

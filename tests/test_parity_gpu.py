@@ -127,6 +127,33 @@ def test_parity_keys_not_unit_length(dtype, d, B, n, L, N, options):
     checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids, key_scale=kmax)
 
 
+# 32-element 16-bit keys are 64 bytes: an even-sized store is scanned as rows of two keys (up to 16
+# queries; more run the one-column-per-query form).  Against the oracle, and bit for bit against
+# the one-key-per-row scan ("pack2" 0): the zero halves of the operand rows add exact zeros.
+@pytest.mark.parametrize("dtype,B,n,N", [
+    ("f16", 1, 10, 148 * 1024 * 2 + 302),      # several 1024-key tiles per CTA, ragged tail
+    ("bf16", 4, 10, 60014),
+    ("f16", 8, 32, 60014),                     # 32 accumulator columns
+    ("bf16", 16, 10, 148 * 1024 + 6),          # 64 columns
+    ("f16", 16, 16, 2 * 148 * 128 * 1024 // 128 + 2),   # B * n = 256: with the probe pass when large enough
+    ("f16", 3, 5, 2),                          # a single row of two keys
+    ("bf16", 2, 10, 1022),
+    ("f16", 5, 10, 60013),                     # odd size: the one-key-per-row scan
+    ("f16", 24, 10, 60014),                    # more than 16 queries: one column per query
+])
+def test_parity_two_keys_per_row(dtype, B, n, N):
+    import torch
+    d, L = 32, 3
+    keys, toks = synth.make_store(7600 + B, N, d, 16, dtype, L)
+    q, _ = synth.make_queries(7601 + B, keys, dtype, B, 0.1)
+    n = min(n, N)
+    ids, sc, tok, o = run_both(keys, toks, dtype, q, n, L)
+    checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, L, oracle_ids=o.ids)
+    i0, s0, t0, _ = run_both(keys, toks, dtype, q, n, L, options={"pack2": 0, "merged_columns": 2})
+    if B <= 16:
+        assert np.array_equal(ids, i0) and np.array_equal(sc, s0) and np.array_equal(tok, t0)
+
+
 @pytest.mark.parametrize("path", [1, 2])
 def test_adversarial_order_both_paths(path):
     # ascending scores in memory: every row beats all rows before it (queue overflow path)

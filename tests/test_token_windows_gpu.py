@@ -39,6 +39,9 @@ def _tokens(rng, B, vocab, missing):
     ("bf16", 256, 64, 32, 4, 30011, 12),             # the batch that otherwise runs with the keys as N
     ("f16", 64, 5, 5, 2, 50021, 50),
     ("bf16", 192, 9, 16, 3, 20011, 7),
+    ("f16", 32, 7, 10, 2, 50022, 50),                # two keys per row: a window edge may fall inside a row
+    ("bf16", 32, 16, 5, 2, 50022, 3000),
+    ("f16", 64, 48, 10, 2, 50021, 50),               # one column per query, windows
 ])
 def test_windows_equal_filtered_full_scan_and_oracle(dtype, d, B, n, L, N, vocab):
     import torch
