@@ -53,6 +53,10 @@ int umma_queries_padded(int B) { return B <= 8 ? 8 : B <= 16 ? 16 : B <= 32 ? 32
 int umma_tsub_of(int d, int ncols)
 {
     const int dslabs = (d + kSlabElems - 1) / kSlabElems;
+    // 33-64 queries (two columns each) on rows wider than 256: the 16 KB operand slab does not stay in
+    // shared memory (128 rows x d) and would come from L2 once per 16 KB key slab; with two sub-tiles per
+    // tile one operand slab serves 32 KB of keys (and the two sub-tiles have an MMA-issuing thread each)
+    if (dslabs > 4 && ncols == 128) return 2;
     if (dslabs > 2) return 1;
     int t = 4 / dslabs;                              // 4 slabs per stage
     while (2 * t * ncols > 512) t >>= 1;             // two accumulator buffers in 512 TMEM columns
@@ -86,9 +90,13 @@ UmmaPlan umma_make_plan(int d, int B, bool merged)
                          sizeof(uint64_t) * (2 * kMaxStages + 5) + 64 + sizeof(Windows);
     const size_t slab = kKeyStageBytes + (p.q_resident ? 0 : op_slab);
     if (p.tsub > 1) {
-        p.gs = p.tsub * dslabs;
-        long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)(p.gs * slab);
+        // narrow rows: the whole tile is one group; wide rows (operand not resident): one slab index per group
+        p.gs = dslabs <= 2 ? dslabs : 1;
+        const size_t group = (size_t)p.gs * (p.tsub * kKeyStageBytes + (p.q_resident ? 0 : op_slab));
+        long long s = ((long long)227 * 1024 - (long long)fixed) / (long long)group;
         p.stages = (int)(s > kMaxStages ? kMaxStages : s);
+        p.smem = fixed + (size_t)(p.stages > 0 ? p.stages : 0) * group;
+        return p;
     } else {
         // Largest slab group (fewest barrier round trips per tile) that still leaves
         // at least three groups in flight.

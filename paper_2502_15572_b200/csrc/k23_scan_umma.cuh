@@ -253,9 +253,11 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     // tile, i.e. all slabs of all its sub-tiles.
     const int n_stages = a.stages;
     const int dslabs = (a.d + kSlabElems - 1) / kSlabElems;
-    const int gpt = TSUB > 1 ? 1 : (dslabs + gs - 1) / gs;  // groups per tile
+    const int gpt = (dslabs + gs - 1) / gs;                 // groups per tile (narrow rows: gs = dslabs, one group)
     const int slab_bytes = kKeyStageBytes + (q_resident ? 0 : kQSlabBytes);
-    const int stage_bytes = (TSUB > 1 ? TSUB * dslabs : gs) * slab_bytes;
+    // TSUB > 1: a group holds the slabs sl0 .. sl0+gs-1 of ALL sub-tiles, [sub][slab], then (query operand
+    // not resident) the gs operand slabs, which the sub-tiles share -- one operand slab per TSUB key slabs
+    const int stage_bytes = TSUB > 1 ? gs * (TSUB * kKeyStageBytes + (q_resident ? 0 : kQSlabBytes)) : gs * slab_bytes;
     uint8_t *stages = base;
     uint8_t *qres = stages + (size_t)n_stages * stage_bytes;                 // resident query operand
     WarpTopN *sel = reinterpret_cast<WarpTopN *>(qres + (q_resident ? (size_t)dslabs * kQSlabBytes : 0));
@@ -401,12 +403,18 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 // but never issued), so that every wait that depends on it runs out.
                 const bool lose = a.debug_lose_stage > 0 && cta == 0 && it == a.debug_lose_stage - 1;
                 if constexpr (TSUB > 1) {
-                    // narrow rows: every slab of every sub-tile (rows past N read as zeros)
-                    mbar_arrive_expect_tx(&full[s], (uint32_t)stage_bytes);
+                    // the group's slabs of every sub-tile (rows past N read as zeros), then its operand slabs
+                    const int sl0 = (it % gpt) * gs;
+                    const int nsl = min(gs, dslabs - sl0);
+                    mbar_arrive_expect_tx(&full[s], (uint32_t)(nsl * (TSUB * kKeyStageBytes + (q_resident ? 0 : kQSlabBytes))));
                     for (int sub = 0; sub < TSUB && !lose; ++sub)
-                        for (int j = 0; j < dslabs; ++j)
-                            tma_load_2d(dst + (size_t)(sub * dslabs + j) * slab_bytes, &keys_map, j * kSlabElems,
+                        for (int j = 0; j < nsl; ++j)
+                            tma_load_2d(dst + (size_t)(sub * gs + j) * kKeyStageBytes, &keys_map, (sl0 + j) * kSlabElems,
                                         tile * kRowsPerTile + sub * kTileRows, &full[s]);
+                    if (!q_resident)
+                        for (int j = 0; j < nsl && !lose; ++j)
+                            tma_load_2d(dst + (size_t)TSUB * gs * kKeyStageBytes + (size_t)j * kQSlabBytes, &q_map,
+                                        (sl0 + j) * kSlabElems, 0, &full[s]);
                 } else {
                     const int sl0 = (it % gpt) * gs;
                     const int nsl = min(gs, dslabs - sl0);
@@ -452,10 +460,15 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     tc_fence_after();
                     const uint32_t st_addr = smem_u32(stages + (size_t)s * stage_bytes);
                     if constexpr (TSUB > 1) {
+                        const int sl0 = g * gs;
+                        const int nsl = min(gs, dslabs - sl0);
                         for (int sub = issuer; sub < TSUB; sub += kIssuers)
-                            for (int j = 0; j < dslabs; ++j) {
-                                const uint64_t a_desc = make_desc(st_addr + (uint32_t)((sub * dslabs + j) * slab_bytes));
-                                const uint64_t b_desc = make_desc(smem_u32(qres + (size_t)j * kQSlabBytes));
+                            for (int jj = 0; jj < nsl; ++jj) {
+                                const int j = sl0 + jj;                       // slab of the row
+                                const uint64_t a_desc = make_desc(st_addr + (uint32_t)((sub * gs + jj) * kKeyStageBytes));
+                                const uint64_t b_desc = make_desc(
+                                    q_resident ? smem_u32(qres + (size_t)j * kQSlabBytes)
+                                               : st_addr + (uint32_t)(TSUB * gs * kKeyStageBytes + jj * kQSlabBytes));
                                 // a last slab that the row fills only in part (zeros beyond d) needs only
                                 // the 32-byte steps that hold data
                                 const int ksteps = min(4, (a.d - j * kSlabElems + 15) / 16);
