@@ -36,7 +36,8 @@ typedef enum {
     DRESD_ERR_UNSUPPORTED = -2, /* valid request outside the built kernel range       */
     DRESD_ERR_ALLOC = -3,       /* workspace allocation failed                        */
     DRESD_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed                  */
-    DRESD_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (see _status)   */
+    DRESD_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (see _status)   */
+    DRESD_ERR_INTERNAL = -6     /* debug build: a bounds check inside a kernel failed */
 } dresd_status;
 
 enum {
@@ -331,6 +332,24 @@ dresd_status dresd_preprocess(dresd_store *store, const void *queries, int B, fl
  * that word: DRESD_OK or DRESD_ERR_TIMEOUT.
  */
 dresd_status dresd_store_status(dresd_store *store);
+
+/*
+ * Bounds-checked debug build.  The library is also built as libdresd_debug.so with
+ * -DDRESD_DEBUG_BOUNDS (the Python binding loads it when the environment variable
+ * DRESD_DEBUG is 1): every global index and pipeline-ring slot that the kernels form -- stage
+ * slots and tile coordinates of the loaders, rows of the first-token column, entries of the
+ * window table, positions in the candidate array, the row ids of candidates and winners -- is
+ * checked where it is formed; a violation skips the access and records its site in the status
+ * word, and dresd_store_status() then returns DRESD_ERR_INTERNAL with the site number in the
+ * message.  It stands in for a memory checker on systems where none can be run; it is a few per
+ * cent slower and otherwise computes the same results.
+ *   dresd_debug_build()            1 in the debug build, 0 in the release build.
+ *   dresd_store_debug_selftest()   debug build: one thread fails check 7 on purpose (no access is
+ *                                  attempted), so that the reporting path can be seen to work;
+ *                                  release build: DRESD_ERR_UNSUPPORTED.
+ */
+int dresd_debug_build(void);
+dresd_status dresd_store_debug_selftest(dresd_store *store, void *stream);
 
 /*
  * Kernel-selection knobs for tests and measurements (set between calls).

@@ -14,12 +14,14 @@ import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libdresd.so")
+LIB_DEBUG_PATH = os.path.join(_HERE, "libdresd_debug.so")    # loaded instead when DRESD_DEBUG=1 (bounds-checked build)
 
 DRESD_F32, DRESD_F16, DRESD_BF16 = 0, 1, 2
 DTYPE_CODE = {"f32": DRESD_F32, "f16": DRESD_F16, "bf16": DRESD_BF16}
 DRESD_OK = 0
 STATUS_NAME = {0: "DRESD_OK", -1: "DRESD_ERR_INVALID", -2: "DRESD_ERR_UNSUPPORTED",
-               -3: "DRESD_ERR_ALLOC", -4: "DRESD_ERR_CUDA", -5: "DRESD_ERR_TIMEOUT"}
+               -3: "DRESD_ERR_ALLOC", -4: "DRESD_ERR_CUDA", -5: "DRESD_ERR_TIMEOUT",
+               -6: "DRESD_ERR_INTERNAL"}
 MAX_BATCH, MAX_TOP_N, MAX_DIM = 64, 32, 4096
 
 EXPORTS = (
@@ -31,7 +33,7 @@ EXPORTS = (
     "dresd_retrieve_filtered", "dresd_drafts_prepare", "dresd_drafts_accept",
     "dresd_merge_shards", "dresd_build_keys", "dresd_fit_zscore", "dresd_set_global_option", "dresd_quantise_keys", "dresd_store_attach_quantised",
     "dresd_retrieve_quantised", "dresd_store_index_first_tokens", "dresd_merge_shards_packed",
-    "dresd_noalloc_status",
+    "dresd_noalloc_status", "dresd_debug_build", "dresd_store_debug_selftest",
 )
 
 
@@ -50,7 +52,7 @@ def load(path: str | None = None) -> ctypes.CDLL:
     global _lib
     if _lib is not None and path is None:
         return _lib
-    p = path or LIB_PATH
+    p = path or (LIB_DEBUG_PATH if os.environ.get("DRESD_DEBUG") == "1" else LIB_PATH)
     if not os.path.exists(p):
         raise DresdError(-4, f"{p} not found: build it with `python -m paper_2502_15572_b200.build` "
                              "(there is no CPU fallback)")
@@ -111,6 +113,10 @@ def load(path: str | None = None) -> ctypes.CDLL:
     lib.dresd_retrieve_noalloc.argtypes = [vp, vp, i64, i32, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.dresd_noalloc_status.restype = i32
     lib.dresd_noalloc_status.argtypes = [vp]
+    lib.dresd_debug_build.restype = i32
+    lib.dresd_debug_build.argtypes = []
+    lib.dresd_store_debug_selftest.restype = i32
+    lib.dresd_store_debug_selftest.argtypes = [vp, vp]
     if path is None:
         _lib = lib
     return lib
@@ -262,6 +268,15 @@ def dresd_retrieve_noalloc(keys_ptr: int, next_tokens_ptr: int, N: int, d: int, 
     _check(load().dresd_retrieve_noalloc(keys_ptr, next_tokens_ptr, N, d, dtype, stored_len, queries_ptr,
                                          B, top_n, draft_len, out_ids_ptr, out_scores_ptr, out_tokens_ptr,
                                          stream))
+
+
+def dresd_debug_build() -> int:
+    """1 when the loaded library is the bounds-checked debug build."""
+    return int(load().dresd_debug_build())
+
+
+def dresd_store_debug_selftest(store: int, stream: int = 0) -> None:
+    _check(load().dresd_store_debug_selftest(store, stream))
 
 
 def dresd_noalloc_status(stream: int = 0) -> None:

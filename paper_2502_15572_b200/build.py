@@ -16,6 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libdresd.so")
+LIB_DEBUG = os.path.join(HERE, "libdresd_debug.so")      # the same sources with -DDRESD_DEBUG_BOUNDS
 OBJ_DIR = os.path.join(HERE, "build")
 
 NVCC_FLAGS = [
@@ -33,22 +34,26 @@ def _deps():
         glob.glob(os.path.join(INCLUDE, "*.h"))
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB):
+def is_stale(debug: bool = False) -> bool:
+    lib = LIB_DEBUG if debug else LIB
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(p) > t for p in _deps())
 
 
-def build(force: bool = False, ptxas: bool = False, verbose: bool = False) -> str:
-    if not force and not ptxas and not is_stale():
-        return LIB
-    os.makedirs(OBJ_DIR, exist_ok=True)
+def build(force: bool = False, ptxas: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Builds the release library, or with ``debug=True`` the bounds-checked one (libdresd_debug.so)."""
+    lib = LIB_DEBUG if debug else LIB
+    if not force and not ptxas and not is_stale(debug):
+        return lib
+    obj_dir = OBJ_DIR + ("_debug" if debug else "")
+    os.makedirs(obj_dir, exist_ok=True)
     nvcc = os.environ.get("NVCC", "nvcc")
-    extra = ["-Xptxas", "-v"] if ptxas else []
+    extra = (["-Xptxas", "-v"] if ptxas else []) + (["-DDRESD_DEBUG_BOUNDS"] if debug else [])
 
     def compile_one(src):
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
@@ -59,15 +64,15 @@ def build(force: bool = False, ptxas: bool = False, verbose: bool = False) -> st
 
     with ThreadPoolExecutor(max(1, min(8, os.cpu_count() or 1))) as ex:
         objs = list(ex.map(compile_one, sources()))
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = lib + f".tmp{os.getpid()}"
     link = [nvcc, "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a",
             "-o", tmp, *objs]
     r = subprocess.run(link, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, ptxas="--ptxas" in sys.argv, verbose=True))
+    print(build(force="--force" in sys.argv, ptxas="--ptxas" in sys.argv, verbose=True, debug="--debug" in sys.argv))

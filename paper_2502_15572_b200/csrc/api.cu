@@ -400,7 +400,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         return DRESD_OK;
     }
     cudaError_t e = launch_merge_gather(s->cand, grid, B, top_n, out_ids, out_scores, s->next_tokens, s->stored_len,
-                                        s->N, draft_len, out_tokens, stream);
+                                        s->N, draft_len, out_tokens, stream, s->status);
     if (e != cudaSuccess) return fail_cuda(e, "merge/gather launch");
     s->last_launches += 1;
     return DRESD_OK;
@@ -734,9 +734,34 @@ dresd_status dresd_store_status(dresd_store *s)
     if (e != cudaSuccess) return fail_cuda(e, "status read");
     if (word != 0) {
         cudaMemset(s->status, 0, sizeof(int));
+        if (word <= -1000)
+            return fail(DRESD_ERR_INTERNAL, "debug build: bounds check %d failed (an index or ring slot out of range)",
+                        -1000 - word);
         return fail(DRESD_ERR_TIMEOUT, "a device-side wait expired");
     }
     return DRESD_OK;
+}
+
+int dresd_debug_build(void)
+{
+#ifdef DRESD_DEBUG_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+dresd_status dresd_store_debug_selftest(dresd_store *s, void *stream)
+{
+    if (!valid(s)) return fail(DRESD_ERR_INVALID, "store handle is NULL or destroyed");
+#ifdef DRESD_DEBUG_BOUNDS
+    s->last_stream = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_debug_selftest(s->status, s->last_stream);
+    return e == cudaSuccess ? DRESD_OK : fail_cuda(e, "selftest launch");
+#else
+    (void)stream;
+    return fail(DRESD_ERR_UNSUPPORTED, "this is the release build: no bounds checks are compiled in");
+#endif
 }
 
 dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)

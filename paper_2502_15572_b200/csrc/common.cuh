@@ -446,4 +446,19 @@ __device__ __forceinline__ void report_timeout(int *status_word)
     atomicExch(status_word, kStatusTimeout);
 }
 
+// Bounds-checked debug build (-DDRESD_DEBUG_BOUNDS, libdresd_debug.so): every global index and every
+// pipeline-ring slot that the kernels form is checked where it is formed; a violation records
+// -(1000 + site) in the status word (the first one wins) and the caller SKIPS the access.  In the
+// release build the function is the constant `true` and the checks compile to nothing.
+constexpr int kStatusBoundsBase = -1000;
+#ifdef DRESD_DEBUG_BOUNDS
+__device__ __forceinline__ bool debug_check(bool ok, int *status_word, int site)
+{
+    if (!ok && status_word) atomicCAS(status_word, 0, kStatusBoundsBase - site);
+    return ok;
+}
+#else
+__device__ __forceinline__ bool debug_check(bool, int *, int) { return true; }
+#endif
+
 }  // namespace dresd

@@ -118,7 +118,7 @@ cudaError_t launch_scan_f32(const CUtensorMap &keys_map, const ScanArgs &a, int 
 // Merge of the per-CTA lists and gather of the winners' stored tokens, one kernel.
 cudaError_t launch_merge_gather(const unsigned long long *cand, int grid_lists, int B, int top_n, int32_t *out_ids,
                                 float *out_scores, const int32_t *next_tokens, int stored_len, long long N,
-                                int draft_len, int32_t *out_tokens, cudaStream_t stream);
+                                int draft_len, int32_t *out_tokens, cudaStream_t stream, int *status = nullptr);
 // Same merge, but only the n-th best score of each query is kept, as a grid-wide
 // filter word (see share_tau); 0 when fewer than top_n candidates exist.
 cudaError_t launch_merge_tau(const unsigned long long *cand, int grid_lists, int B, int top_n,
@@ -175,6 +175,9 @@ cudaError_t launch_merge_rerank(const unsigned long long *cand, int lists, int B
                                 long long N, const float *qhat, int mcand, int top_n, long long extra_id,
                                 const int32_t *want_first, const int32_t *next_tokens, int stored_len, int draft_len,
                                 int32_t *out_ids, float *out_scores, int32_t *out_tokens, cudaStream_t stream);
+
+// Debug build only: one thread fails check 7 on purpose (no access is attempted), to show the reporting path.
+cudaError_t launch_debug_selftest(int *status, cudaStream_t stream);
 
 // Stores `msg` as the calling thread's dresd_last_error() text.
 void set_last_error(const char *msg);

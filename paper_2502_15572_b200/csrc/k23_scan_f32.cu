@@ -112,6 +112,7 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 const int sl = it % dslabs;
                 mbar_arrive_expect_tx(&full[s], (uint32_t)kStageBytes);     // rows past N arrive as zeros
                 uint8_t *dst = stages + (size_t)s * kStageBytes;
+                if (!debug_check(s >= 0 && s < n_stages && tile >= 0 && (long long)tile * kRows < a.N + kRows, a.status, 21)) break;
                 // Test hook: CTA 0 "loses" the copies of one stage, so that the waits on it run out.
                 const bool lose = a.debug_lose_stage > 0 && cta == 0 && it == a.debug_lose_stage - 1;
                 for (int h = 0; h < kRows / kBoxRows && !lose; ++h)
@@ -288,7 +289,8 @@ scan_f32_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             if (sel[q].count > 0) warp_topn_merge(&sel[q], a.top_n, lane);
             unsigned long long m = sel[q].list[lane];
             if (lane >= a.top_n) m = 0ull;
-            a.cand[((size_t)cta * a.cand_batch + q) * kCandStride + lane] = m;
+            if (debug_check(q < a.cand_batch && (m == 0ull || (long long)candidate_id(m) < a.N), a.status, 24))
+                a.cand[((size_t)cta * a.cand_batch + q) * kCandStride + lane] = m;
         }
     }
 }

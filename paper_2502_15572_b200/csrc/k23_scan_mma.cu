@@ -143,6 +143,7 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
                 const int nsl = KS > 0 ? KS : min(4, dslabs - kc * 4);
                 mbar_arrive_expect_tx(&full[s], (uint32_t)(nsl * S::kRows * kSlabBytes));
                 uint8_t *dst = stages + (size_t)s * kStageBytes;
+                if (!debug_check(s >= 0 && s < n_stages && tile >= 0 && (long long)tile * S::kRows < a.N + S::kRows, a.status, 31)) break;
                 // Test hook: one CTA "loses" the copies of one stage, so that the waits on it
                 // run out and the timeout path (status word, orderly exit) can be exercised.
                 const bool lose = a.debug_lose_stage > 0 && cta == 0 && it == a.debug_lose_stage - 1;
@@ -313,7 +314,8 @@ scan_mma_kernel(const __grid_constant__ CUtensorMap keys_map, const ScanArgs a)
             for (int w = 1; w < kConsumerWarps; ++w)
                 m = warp_merge_top32(m, sel[w * NQ + q].list[lane], lane);
             if (lane >= a.top_n) m = 0ull;
-            a.cand[((size_t)cta * a.cand_batch + q) * kCandStride + lane] = m;
+            if (debug_check(q < a.cand_batch && (m == 0ull || (long long)candidate_id(m) < a.N), a.status, 34))
+                a.cand[((size_t)cta * a.cand_batch + q) * kCandStride + lane] = m;
         }
     }
 }

@@ -338,8 +338,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 bool owner = tok >= 0 && tok < a.win_vocab;          // no row holds a token >= win_vocab
                 for (int b = 0; b < tid && owner; ++b) owner = a.want_first[b] != tok;
                 if (owner) {
-                    lo = a.win_start[tok];
-                    hi = a.win_start[tok + 1];
+                    if (debug_check(tok >= 0 && tok + 1 <= a.win_vocab, a.status, 3)) {
+                        lo = a.win_start[tok];
+                        hi = a.win_start[tok + 1];
+                    }
                     if (hi > lo) {
                         constexpr int kKeysPerTile = PACK2 ? 2 * kRowsPerTile : kRowsPerTile;
                         t0 = lo / kKeysPerTile;
@@ -399,6 +401,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     tile = win->tile0[wk] + (tile - win->prefix[wk]);
                 }
                 uint8_t *dst = stages + (size_t)s * stage_bytes;
+                // debug build: the ring slot lies inside the stage area, the tile inside the key matrix
+                if (!debug_check(s >= 0 && s < n_stages && dst + stage_bytes <= qres && tile >= 0 &&
+                                     (long long)tile * kRowsPerTile < a.N + kRowsPerTile, a.status, 1))
+                    break;
                 // Test hook: CTA 0 "loses" the copies of one stage (they are announced to the barrier
                 // but never issued), so that every wait that depends on it runs out.
                 const bool lose = a.debug_lose_stage > 0 && cta == 0 && it == a.debug_lose_stage - 1;
@@ -672,7 +678,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         tok[sub] = t.x;
                         tok1[sub] = t.y;
                     } else {
-                        tok[sub] = a.first_col[r];
+                        if (debug_check(r >= 0 && r < a.N, a.status, 2)) tok[sub] = a.first_col[r];
                     }
                 }
             }
@@ -957,7 +963,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             if (q < a.B) {
                 unsigned long long m = sel[q].list[lane];
                 if (lane >= a.top_n) m = 0ull;
-                a.cand[((size_t)cta * a.cand_batch + q) * kCandStride + lane] = m;
+                // debug build: the list lies in this launch's part of the candidate array, its rows in the store
+                if (debug_check(q < a.cand_batch && (m == 0ull || (long long)candidate_id(m) < (PACK2 ? 2 * a.N + 1 : a.N)),
+                                a.status, 4))
+                    a.cand[((size_t)cta * a.cand_batch + q) * kCandStride + lane] = m;
             }
         }
     }

@@ -180,6 +180,9 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
                 const int tile = (cta + (it / dslabs) * G) * a.tile_stride;
                 const int ks = it % dslabs;
                 uint8_t *dst = stages + (size_t)s * kStageBytes;
+                if (!debug_check(s >= 0 && s < n_stages && dst + kStageBytes <= qres && tile >= 0 &&
+                                     (long long)tile * kTileKeys < a.N + kTileKeys, a.status, 11))
+                    break;
                 // rows past N read as zeros (a box may start past the end)
                 mbar_arrive_expect_tx(&full[s], (uint32_t)kStageBytes);
                 // Test hook: CTA 0 "loses" the copies of one stage, so that the waits on it run out.
@@ -455,7 +458,8 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
             if (qq < a.B) {
                 unsigned long long m = sel[qq].list[lane];
                 if (lane >= a.top_n) m = 0ull;
-                a.cand[((size_t)cta * a.cand_batch + qq) * kCandStride + lane] = m;
+                if (debug_check(qq < a.cand_batch && (m == 0ull || (long long)candidate_id(m) < a.N), a.status, 14))
+                    a.cand[((size_t)cta * a.cand_batch + qq) * kCandStride + lane] = m;
             }
         }
     }

@@ -20,7 +20,7 @@ __global__ void __launch_bounds__(kMergeWarps * 32)
 merge_gather_kernel(const unsigned long long *__restrict__ cand, int lists, int B, int top_n,
                     int32_t *__restrict__ out_ids, float *__restrict__ out_scores, unsigned int *__restrict__ gtau,
                     const int32_t *__restrict__ next_tokens, int stored_len, long long N, int draft_len,
-                    int32_t *__restrict__ out_tokens)
+                    int32_t *__restrict__ out_tokens, int *status)
 {
     __shared__ unsigned long long part[kMergeWarps][kListLen];
     __shared__ int win[kListLen];
@@ -58,7 +58,8 @@ merge_gather_kernel(const unsigned long long *__restrict__ cand, int lists, int 
         return;
     }
     if (warp == 0 && lane < top_n) {
-        const int id = m ? (int32_t)candidate_id(m) : -1;
+        int id = m ? (int32_t)candidate_id(m) : -1;
+        if (!debug_check(id >= -1 && id < N, status, 41)) id = -1;     // debug build: a winner is a row of the store
         out_ids[(size_t)b * top_n + lane] = id;
         out_scores[(size_t)b * top_n + lane] = m ? candidate_score(m) : -INFINITY;
         win[lane] = id;
@@ -142,12 +143,24 @@ cudaError_t launch_extract_first(const int32_t *next_tokens, int stored_len, lon
     return cudaGetLastError();
 }
 
+__global__ void debug_selftest_kernel(int *status)
+{
+    const int index = 5, limit = 4;                    // an index that is out of range; the access is skipped
+    if (debug_check(index < limit, status, 7)) status[index] = 0;
+}
+
+cudaError_t launch_debug_selftest(int *status, cudaStream_t stream)
+{
+    debug_selftest_kernel<<<1, 1, 0, stream>>>(status);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_merge_gather(const unsigned long long *cand, int lists, int B, int top_n, int32_t *out_ids,
                                 float *out_scores, const int32_t *next_tokens, int stored_len, long long N,
-                                int draft_len, int32_t *out_tokens, cudaStream_t stream)
+                                int draft_len, int32_t *out_tokens, cudaStream_t stream, int *status)
 {
     return launch_dependent(merge_gather_kernel, dim3(B), dim3(kMergeWarps * 32), 0, stream, cand, lists, B, top_n, out_ids,
-                            out_scores, (unsigned int *)nullptr, next_tokens, stored_len, N, draft_len, out_tokens);
+                            out_scores, (unsigned int *)nullptr, next_tokens, stored_len, N, draft_len, out_tokens, status);
 }
 
 cudaError_t launch_merge_tau(const unsigned long long *cand, int lists, int B, int top_n, unsigned int *gtau,
@@ -155,7 +168,7 @@ cudaError_t launch_merge_tau(const unsigned long long *cand, int lists, int B, i
 {
     return launch_dependent(merge_gather_kernel, dim3(B), dim3(kMergeWarps * 32), 0, stream, cand, lists, B, top_n,
                             (int32_t *)nullptr, (float *)nullptr, gtau, (const int32_t *)nullptr, 0, 0LL, 0,
-                            (int32_t *)nullptr);
+                            (int32_t *)nullptr, (int *)nullptr);
 }
 
 }  // namespace dresd
