@@ -352,6 +352,22 @@ scan_ummat_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_con
             // scores of one unit against the filter, survivors queued; true = stop here (queue full)
             auto process = [&](int u, const uint32_t (&r)[32], float tau_r) -> bool {
                 const int q = qq0 + 8 * (u >> 1);
+                if (!resume && !a.no_fast_reject) {
+                    // Fast rejection: hi + lo/S for two keys at a time (packed fp32, the same rounding as the
+                    // exact step below), plus -tau; the sign bit of that sum is clear exactly when the score
+                    // reaches the filter (a sum of two floats is never rounded across zero).  The sign bits
+                    // are ANDed; a warp in which no key of the unit reaches its query's filter is done with it.
+                    const float2 iv = make_float2(inv, inv), nt = make_float2(-tau_r, -tau_r);
+                    uint32_t neg = 0x80000000u;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        const float2 s2 = __ffma2_rn(make_float2(__uint_as_float(r[4 * g + 2]), __uint_as_float(r[4 * g + 3])), iv,
+                                                     make_float2(__uint_as_float(r[4 * g]), __uint_as_float(r[4 * g + 1])));
+                        const float2 t2 = __fadd2_rn(s2, nt);
+                        neg &= __float_as_uint(t2.x) & __float_as_uint(t2.y);
+                    }
+                    if (!__any_sync(0xFFFFFFFFu, (neg & 0x80000000u) == 0u)) return false;
+                }
                 uint32_t m = 0u;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
