@@ -286,8 +286,11 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
     const int op_rows = !umma ? 0 : blocked ? 2 * kMaxBatch : scan_umma_operand_rows(pack2 ? 2 * B : B);
     // one CTA per operand query: two operand rows each, four in the packed 8-bit layout
     const int pre_rows = pack2 ? op_rows / 4 : umma ? op_rows / 2 : ((B + 7) / 8) * 8;
-    dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, pack16 ? 3 : merged ? 2 : blocked,
-                                     pack8 ? 2 : q8 ? 1 : 0);
+    // operand layouts (PreprocessArgs::split_blocked): the tcgen05 kernel with the keys as M takes the hi rows of all
+    // queries first, then the lo rows (4); its one-column form both scaled (2); 32-element keys two per row (3);
+    // the kernel with the keys as N 16-row blocks (1); the streaming kernel and the 8-bit search pairs (0)
+    const int layout = pack16 ? 3 : merged ? 2 : blocked ? 1 : (umma && !q8) ? 4 : 0;
+    dresd_status st = run_preprocess(s, queries, B, pre_rows, stream, layout, pack8 ? 2 : q8 ? 1 : 0);
     if (st != DRESD_OK) return st;
 
     // the 8-bit store is scanned as rows of d/2 two-byte units (packed: N/2 rows of 64 units)

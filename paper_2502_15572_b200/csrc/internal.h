@@ -33,6 +33,7 @@ struct PreprocessArgs {
     unsigned int *gtau;     // [rows] grid-wide filter words, reset to 0 ("nothing known") here
     int split_blocked;      // qsplit rows: 0 = (2b, 2b+1); 1 = 16-row blocks, hi rows 0-7, lo rows 8-15;
                             // 2 = rows b and `rows` + b hold S hi and S (q - hi), S = lo_scale (one column per query);
+                            // 4 = rows b and `rows` + b hold hi and S (q - hi): two columns per query, hi columns first;
                             // 3 = d = 32 keys scanned two per 64-element row: rows 4b .. 4b+3 = (hi|0), (lo|0), (0|hi), (0|lo)
     // Split projection (W given): `slices` CTAs of `rows_per_slice` rows of W each write
     // partial[slice][B][d]; null = every query's CTA walks all of W itself.

@@ -180,9 +180,10 @@ __global__ void __launch_bounds__(kThreads) preprocess_kernel(PreprocessArgs a)
     // or -- merged layout -- rows b and rows + b, both terms scaled by lo_scale;
     // or -- packed layout, two 32-element keys per 64-element store row -- rows 4b .. 4b+3 =
     // (hi|0), (lo|0), (0|hi), (0|lo): two column pairs that score the even and the odd key of a row
-    const bool merged = a.split_blocked == 2, packed = a.split_blocked == 3;
-    const int row_hi = packed ? 4 * b : merged ? b : a.split_blocked ? 16 * (b >> 3) + (b & 7) : 2 * b;
-    const int row_lo = merged ? a.rows + b : a.split_blocked == 1 ? row_hi + 8 : row_hi + 1;
+    // or -- halves layout -- rows b (hi) and rows + b (lo), the hi rows of all queries first
+    const bool merged = a.split_blocked == 2, packed = a.split_blocked == 3, halves = a.split_blocked == 4;
+    const int row_hi = packed ? 4 * b : (merged || halves) ? b : a.split_blocked ? 16 * (b >> 3) + (b & 7) : 2 * b;
+    const int row_lo = (merged || halves) ? a.rows + b : a.split_blocked == 1 ? row_hi + 8 : row_hi + 1;
     T *split_hi = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)row_hi * a.dpad : nullptr;
     T *split_lo = a.qsplit ? static_cast<T *>(a.qsplit) + (size_t)row_lo * a.dpad : nullptr;
     float *qrow = a.qhat + (size_t)b * a.d;

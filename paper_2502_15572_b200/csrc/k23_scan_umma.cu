@@ -11,20 +11,22 @@ template <typename T, int NCOLS, int TSUB, bool PACK2 = false>
 cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const ScanArgs &a, const UmmaPlan &p,
                        int grid, cudaStream_t stream)
 {
+    // 16-bit keys, one key per row: the operand rows come as hi block | lo block (K1 layout 4)
+    constexpr bool HALVES = !PACK2 && !std::is_same<T, E4M3Keys>::value;
     if constexpr (2 * TSUB * NCOLS > 512) {
         return cudaErrorInvalidValue;
     } else {
         const int dslabs = (a.d + kSlabElems - 1) / kSlabElems;
         if constexpr (dual_possible(TSUB, NCOLS)) {
             if (umma_dual_pays(dslabs, NCOLS)) {
-                auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, true>;
+                auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, true, false, HALVES>;
                 cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
                 if (e != cudaSuccess) return e;
                 return launch_dependent(kernel, dim3(grid), dim3(threads_of(TSUB, true)), p.smem, stream, kmap, qmap, a,
                                         p.q_resident, p.gs);
             }
         }
-        auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, false>;
+        auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, false, false, HALVES>;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
         if (e != cudaSuccess) return e;
         return launch_dependent(kernel, dim3(grid), dim3(threads_of(TSUB, false)), p.smem, stream, kmap, qmap, a,

@@ -73,15 +73,27 @@ __device__ __forceinline__ void tmem_ld16p(uint32_t taddr, uint32_t *r)
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
 }
-// CW consecutive accumulator columns of this thread's TMEM lane -> registers.
-template <int CW> __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[CW])
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t *r)
 {
-    if constexpr (CW == 8) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(taddr));
+}
+// C consecutive accumulator columns of this thread's TMEM lane -> registers (C = 4, 8, 16, 32, 64).
+template <int C> __device__ __forceinline__ void tmem_ld_n(uint32_t taddr, uint32_t *r)
+{
+    if constexpr (C == 4) {
+        tmem_ld4(taddr, r);
+    } else if constexpr (C == 8) {
         tmem_ld8(taddr, r);
     } else {
 #pragma unroll
-        for (int c = 0; c < CW / 16; ++c) tmem_ld16p(taddr + 16 * c, r + 16 * c);
+        for (int c = 0; c < C / 16; ++c) tmem_ld16p(taddr + 16 * c, r + 16 * c);
     }
+}
+template <int CW> __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[CW])
+{
+    tmem_ld_n<CW>(taddr, r);
 }
 // Column-wise maximum over the 32 lanes of a warp for C values per lane, with C-1
 // exchanges in total instead of 5 per value: at each step a lane keeps one half of its
@@ -134,53 +146,70 @@ struct Windows {
     unsigned long long qmask[kMaxBatch];   // operand column pairs (queries) that name the window's token
 };
 
-// CW accumulator columns of this thread's lane; with two accumulator sets, set B (NCOLS columns
-// further) is added to set A -- the sum of the even and of the odd slabs' partial products.
-template <int CW, int NCOLS, bool DUAL> __device__ __forceinline__ void tmem_ld_acc(uint32_t addr, uint32_t (&r)[CW])
+// The accumulator columns of this warp's QW queries -> registers.  Layouts of a sub-tile's NCOLS columns:
+//   pairs  (PACK2 and the 8-bit copy)   query j: columns 2j (hi) and 2j+1 (lo);  CW = 2 QW consecutive columns
+//   HALVES (16-bit keys, two columns)   query j: column j (hi) and column NQ + j (lo): r[0..QW) = hi, r[QW..2QW) = lo
+//   MERGED (one column per query)       query j: column j;  CW = QW
+// With two accumulator sets, set B (NCOLS columns further) is added to set A -- the sum of the even and of the
+// odd slabs' partial products.  Loads are issued only; the caller waits.
+template <int CW, int QW, int NQ, int NCOLS, bool DUAL, bool HALVES>
+__device__ __forceinline__ void tmem_ld_acc(uint32_t addr, uint32_t (&r)[CW])
 {
-    tmem_ld_cols<CW>(addr, r);
+    if constexpr (HALVES) {
+        tmem_ld_n<QW>(addr, r);
+        tmem_ld_n<QW>(addr + NQ, r + QW);
+    } else {
+        tmem_ld_n<CW>(addr, r);
+    }
     if constexpr (DUAL) {
-        constexpr int CH = CW < 16 ? CW : 16;       // set B in chunks: 16 registers, not CW more
+        constexpr int PART = HALVES ? QW : CW;        // consecutive columns per load
+        constexpr int CH = PART < 16 ? PART : 16;     // set B in chunks: 16 registers, not CW more
 #pragma unroll
         for (int c = 0; c < CW / CH; ++c) {
             uint32_t r2[CH];
-            tmem_ld_cols<CH>(addr + NCOLS + c * CH, r2);
+            const int first = c * CH;                  // register index of the chunk
+            const uint32_t col = HALVES ? (uint32_t)(first < QW ? first : NQ + first - QW) : (uint32_t)first;
+            tmem_ld_n<CH>(addr + NCOLS + col, r2);
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < CH; ++i)
-                r[c * CH + i] = __float_as_uint(__uint_as_float(r[c * CH + i]) + __uint_as_float(r2[i]));
+                r[first + i] = __float_as_uint(__uint_as_float(r[first + i]) + __uint_as_float(r2[i]));
         }
     }
 }
 
-// The exact selection step of the one-column-per-query forms for ONE sub-tile of one warp: the
-// columns are read again, compared with the filter scores, and the survivors queued.  Kept out
-// of line on purpose: it runs for a few per cent of the sub-tiles, and a single copy that all
+// The exact selection step of the forms with a fast rejection (HALVES, MERGED) for ONE sub-tile of one
+// warp: the columns are read again, compared with the filter scores, and the survivors queued.  Kept
+// out of line on purpose: it runs for a few per cent of the sub-tiles, and a single copy that all
 // warps and sub-tiles share stays in the instruction cache, where copies inlined into every
 // unrolled sub-tile were fetched cold each time (measured: 0.74 -> 1.38 ms per call when the
 // rare path was unrolled in place).  `allow` = the queries this thread's row may feed (window,
 // range and, on a resumed round, the candidates that found their queue full); returns the
 // queries whose candidate found the queue full now.
-template <int CW, int NCOLS, bool DUAL>
-static __device__ __noinline__ uint32_t epi_select_merged(uint32_t addr, const float *tau_q, const int *want_q, int tok,
-                                                          uint32_t wild, int filtered, uint32_t allow, float inv,
-                                                          WarpTopN *sel_q, uint32_t row, EpiFlags *fl)
+template <int CW, int QW, int NQ, int NCOLS, bool DUAL, bool MERGED>
+static __device__ __noinline__ uint32_t epi_select(uint32_t addr, const float *tau_q, const int *want_q, int tok,
+                                                   uint32_t wild, int filtered, uint32_t allow, float inv,
+                                                   WarpTopN *sel_q, uint32_t row, EpiFlags *fl)
 {
     uint32_t r[CW];
-    tmem_ld_acc<CW, NCOLS, DUAL>(addr, r);
+    tmem_ld_acc<CW, QW, NQ, NCOLS, DUAL, !MERGED>(addr, r);
     tmem_ld_wait();
+    auto score = [&](int j) -> float {
+        if constexpr (MERGED) return __uint_as_float(r[j]) * inv;
+        else return fmaf(__uint_as_float(r[QW + j]), inv, __uint_as_float(r[j]));
+    };
     uint32_t mask = 0u;
 #pragma unroll
-    for (int j4 = 0; j4 < CW / 4; ++j4) {
+    for (int j4 = 0; j4 < QW / 4; ++j4) {
         const float4 t = reinterpret_cast<const float4 *>(tau_q)[j4];
         const float tt[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) mask |= (__uint_as_float(r[4 * j4 + i]) * inv >= tt[i]) ? (1u << (4 * j4 + i)) : 0u;
+        for (int i = 0; i < 4; ++i) mask |= (score(4 * j4 + i) >= tt[i]) ? (1u << (4 * j4 + i)) : 0u;
     }
     if (filtered) {                                     // Section 3.5: drafts must start with x_{t+1}
         uint32_t match = wild;
 #pragma unroll
-        for (int j4 = 0; j4 < CW / 4; ++j4) {
+        for (int j4 = 0; j4 < QW / 4; ++j4) {
             const int4 w = reinterpret_cast<const int4 *>(want_q)[j4];
             match |= ((tok == w.x ? 1u : 0u) | (tok == w.y ? 2u : 0u) | (tok == w.z ? 4u : 0u) | (tok == w.w ? 8u : 0u))
                      << (4 * j4);
@@ -193,22 +222,25 @@ static __device__ __noinline__ uint32_t epi_select_merged(uint32_t addr, const f
     while (wm) {                                        // warp-uniform: tcgen05.ld needs the whole warp
         const int j = __ffs(wm) - 1;
         wm &= wm - 1;
-        uint32_t v0;
+        // the registers cannot be indexed by a run-time j: the score's columns are read once more
+        uint32_t v0, v1 = 0u;
         tmem_ld1(addr + (uint32_t)j, v0);
-        float acc;
+        if constexpr (!MERGED) tmem_ld1(addr + (uint32_t)(NQ + j), v1);
         if constexpr (DUAL) {
-            uint32_t w0;
+            uint32_t w0, w1 = 0u;
             tmem_ld1(addr + (uint32_t)j + NCOLS, w0);
+            if constexpr (!MERGED) tmem_ld1(addr + (uint32_t)(NQ + j) + NCOLS, w1);
             tmem_ld_wait();
-            acc = __uint_as_float(v0) + __uint_as_float(w0);
+            v0 = __float_as_uint(__uint_as_float(v0) + __uint_as_float(w0));
+            v1 = __float_as_uint(__uint_as_float(v1) + __uint_as_float(w1));
         } else {
             tmem_ld_wait();
-            acc = __uint_as_float(v0);
         }
+        const float sc = MERGED ? __uint_as_float(v0) * inv : fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
         if ((mask >> j) & 1u) {
             const int slot = atomicAdd(&sel_q[j].count, 1);
             if (slot < kQueueCap) {
-                sel_q[j].queue[slot] = pack_candidate(acc * inv, row);
+                sel_q[j].queue[slot] = pack_candidate(sc, row);
                 if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
             } else {
                 pend |= 1u << j;
@@ -231,7 +263,13 @@ static __device__ __noinline__ uint32_t epi_select_merged(uint32_t addr, const f
 // the SAME columns, and the accumulator is S times the score.  Half the accumulator columns means
 // half the TMEM reads and compares of the epilogue, at twice the instructions: the form for
 // batches whose epilogue, not the instruction stream, sets the pace (more than 16 queries).
-template <typename T, int NCOLS, int TSUB, bool PACK2 = false, bool DUAL = false, bool MERGED = false>
+//
+// HALVES: two columns per query, but the hi columns of all queries first and the lo columns after them
+// (K1 writes the operand rows in that order), so that hi and lo of NEIGHBOURING queries sit in neighbouring
+// registers and packed fp32 instructions can combine them: the same one-and-a-half instructions per score
+// fast rejection -- fma.f32x2 (hi + lo/S), add.f32x2 (-tau), sign bits ANDed -- for every two-column form.
+template <typename T, int NCOLS, int TSUB, bool PACK2 = false, bool DUAL = false, bool MERGED = false,
+          bool HALVES = false>
 __global__ void __launch_bounds__(threads_of(TSUB, DUAL, MERGED), 1)
 scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_constant__ CUtensorMap q_map,
                  const ScanArgs a, const int q_resident, const int gs)
@@ -239,6 +277,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     constexpr int NQ = MERGED ? NCOLS : NCOLS / 2;          // queries (padded)
     constexpr int CPQ = MERGED ? 1 : 2;                     // accumulator columns per query
     static_assert(!(MERGED && PACK2), "the packed 8-bit layout keeps two columns per query");
+    static_assert(!(HALVES && (MERGED || PACK2)), "hi block | lo block: a layout of the plain two-column forms");
+    constexpr bool FAST = MERGED || HALVES;                 // forms with the packed sign-bit rejection
     static_assert(!DUAL || dual_possible(TSUB, NCOLS), "two accumulator sets: wide rows only");
     constexpr int kAccCols = TSUB * NCOLS * (DUAL ? 2 : 1); // one accumulator buffer
     constexpr int kTmemCols = 2 * kAccCols < 32 ? 32 : 2 * kAccCols;
@@ -262,7 +302,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     uint8_t *qres = stages + (size_t)n_stages * stage_bytes;                 // resident query operand
     WarpTopN *sel = reinterpret_cast<WarpTopN *>(qres + (q_resident ? (size_t)dslabs * kQSlabBytes : 0));
     float *tau = reinterpret_cast<float *>(sel + NQ);
-    float *ntau = tau + NQ;                                 // MERGED: -S tau, what the hot loop adds to an accumulator
+    float *ntau = tau + NQ;                                 // -tau (MERGED: -S tau), what the fast rejection adds to a score
     int *want_s = reinterpret_cast<int *>(ntau + NQ);       // first-token filter per query, -1 = off
     unsigned long long *tilemax = reinterpret_cast<unsigned long long *>(want_s + NQ);   // probe: [sub][lane group][query]
     uint64_t *full = reinterpret_cast<uint64_t *>(tilemax + 4 * TSUB * NQ);
@@ -282,6 +322,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     auto set_tau = [&](int q, float t) {
         tau[q] = t;
         if constexpr (MERGED) ntau[q] = -t * acc_scale;
+        else if constexpr (HALVES) ntau[q] = -t;
     };
     const long long wl = a.wait_cycles > 0 ? a.wait_cycles : kWaitCycles;   // bound of every wait below
     constexpr int kRowsPerTile = kTileRows * TSUB;
@@ -544,16 +585,17 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         const int qbase = split_subs ? 0 : half * QW;
         // a warp whose columns are all padding (few queries, one sub-tile per tile) only keeps the barriers
         const bool no_cols = qbase >= (PACK2 ? 2 * a.B : a.B);
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(qbase * CPQ);
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(qbase * (HALVES ? 1 : CPQ));
         const float inv = a.lo_inv_scale;
         // score of this warp's j-th query from the registers of ld_cols: hi + lo / S, or acc / S
         auto score_at = [&](const uint32_t (&r)[CW], int j) -> float {
             if constexpr (MERGED) return __uint_as_float(r[j]) * inv;
+            else if constexpr (HALVES) return fmaf(__uint_as_float(r[QW + j]), inv, __uint_as_float(r[j]));
             else return fmaf(__uint_as_float(r[2 * j + 1]), inv, __uint_as_float(r[2 * j]));
         };
         // accumulator reads (issued only; the caller waits): with two sets, set B (NCOLS columns further)
         // is added to set A -- the sum of the even and of the odd slabs' partial products
-        auto ld_cols = [&](uint32_t addr, uint32_t (&r)[CW]) { tmem_ld_acc<CW, NCOLS, DUAL>(addr, r); };
+        auto ld_cols = [&](uint32_t addr, uint32_t (&r)[CW]) { tmem_ld_acc<CW, QW, NQ, NCOLS, DUAL, HALVES>(addr, r); };
         // the same score re-read from TMEM: `addr` = the sub-tile's first column of this warp, j = its query
         auto ld_score = [&](uint32_t addr, int j) -> float {
             if constexpr (MERGED) {
@@ -567,6 +609,20 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                 }
                 tmem_ld_wait();
                 return __uint_as_float(v0) * inv;
+            } else if constexpr (HALVES) {
+                uint32_t v0, v1;
+                tmem_ld1(addr + (uint32_t)j, v0);
+                tmem_ld1(addr + (uint32_t)(NQ + j), v1);
+                if constexpr (DUAL) {
+                    uint32_t w0, w1;
+                    tmem_ld1(addr + (uint32_t)j + NCOLS, w0);
+                    tmem_ld1(addr + (uint32_t)(NQ + j) + NCOLS, w1);
+                    tmem_ld_wait();
+                    v0 = __float_as_uint(__uint_as_float(v0) + __uint_as_float(w0));
+                    v1 = __float_as_uint(__uint_as_float(v1) + __uint_as_float(w1));
+                }
+                tmem_ld_wait();
+                return fmaf(__uint_as_float(v1), inv, __uint_as_float(v0));
             } else {
                 uint32_t v0, v1;
                 tmem_ld2(addr + (uint32_t)(2 * j), v0, v1);
@@ -851,31 +907,38 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                     if (dead || no_cols || (split_subs && (sub & 1) != half) ||
                         !(first || __any_sync(0xFFFFFFFFu, pending[sub] != 0u)))
                         continue;
-                    if constexpr (MERGED) {
-                        // Fast rejection, one instruction per score: accumulator + (-S tau) has its sign
-                        // bit clear exactly when the score reaches the filter (the sum of two floats is never
-                        // rounded across zero), packed adds take two columns at a time, and the sign bits
-                        // are ANDed three words per instruction.  A warp in which no row reaches any
-                        // filter -- the usual case once the filter is warm -- is done with the sub-tile.
+                    if constexpr (FAST) {
+                        // Fast rejection, one instruction per score (one and a half with two columns per query):
+                        // score + (-tau) has its sign bit clear exactly when the score reaches the filter (the
+                        // sum of two floats is never rounded across zero); packed fp32 instructions take two
+                        // queries at a time -- MERGED: accumulator + (-S tau); HALVES: hi + lo/S, rounded as in
+                        // the exact step, then + (-tau) -- and the sign bits are ANDed three words per
+                        // instruction.  A warp in which no row reaches any filter -- the usual case once the
+                        // filter is warm -- is done with the sub-tile.
                         if (first) {
                             uint32_t r[CW];
                             ld_cols(acc_addr + (uint32_t)(sub * NCOLS), r);
                             tmem_ld_wait();
                             uint32_t neg = 0x80000000u;
                             const float4 *nt4 = reinterpret_cast<const float4 *>(ntau + qbase);
+                            const float2 iv = make_float2(inv, inv);
 #pragma unroll
                             for (int j4 = 0; j4 < QW / 4; ++j4) {
                                 const float4 t = nt4[j4];
-                                const float2 x = __fadd2_rn(make_float2(__uint_as_float(r[4 * j4]), __uint_as_float(r[4 * j4 + 1])),
-                                                            make_float2(t.x, t.y));
-                                const float2 y = __fadd2_rn(make_float2(__uint_as_float(r[4 * j4 + 2]), __uint_as_float(r[4 * j4 + 3])),
-                                                            make_float2(t.z, t.w));
+                                float2 s0 = make_float2(__uint_as_float(r[4 * j4]), __uint_as_float(r[4 * j4 + 1]));
+                                float2 s1 = make_float2(__uint_as_float(r[4 * j4 + 2]), __uint_as_float(r[4 * j4 + 3]));
+                                if constexpr (HALVES) {
+                                    s0 = __ffma2_rn(make_float2(__uint_as_float(r[QW + 4 * j4]), __uint_as_float(r[QW + 4 * j4 + 1])), iv, s0);
+                                    s1 = __ffma2_rn(make_float2(__uint_as_float(r[QW + 4 * j4 + 2]), __uint_as_float(r[QW + 4 * j4 + 3])), iv, s1);
+                                }
+                                const float2 x = __fadd2_rn(s0, make_float2(t.x, t.y));
+                                const float2 y = __fadd2_rn(s1, make_float2(t.z, t.w));
                                 neg &= __float_as_uint(x.x) & __float_as_uint(x.y);
                                 neg &= __float_as_uint(y.x) & __float_as_uint(y.y);
                             }
                             if (!__any_sync(0xFFFFFFFFu, (neg & 0x80000000u) == 0u)) continue;
                         }
-                        pending[sub] = epi_select_merged<CW, NCOLS, DUAL>(
+                        pending[sub] = epi_select<CW, QW, NQ, NCOLS, DUAL, MERGED>(
                             acc_addr + (uint32_t)(sub * NCOLS), tau + qbase, want_s + qbase, tok[sub], wild, filtered ? 1 : 0,
                             first ? (okmask & wmatch) : pending[sub], inv, sel + qbase, (uint32_t)row, fl);
                         continue;
