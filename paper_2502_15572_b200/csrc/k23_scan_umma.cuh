@@ -19,11 +19,16 @@
 //             second issuing thread (warp 10) takes half of the instructions (see
 //             threads_of() below);
 //   warps 2-9 epilogue: each thread owns one key row of the tile and half of
-//             its N accumulator columns (two warps share a TMEM lane group),
-//             reads them with tcgen05.ld, combines hi and lo, filters against
-//             the CTA's running n-th best per query and queues survivors;
-//             queues are folded into sorted 32-lane lists with shuffle-based
-//             bitonic merges.
+//             the queries' accumulator columns (two warps share a TMEM lane group),
+//             reads them with tcgen05.ld and rejects the sub-tile with a packed
+//             sign-bit test of score - tau when no row reaches any filter; else
+//             the exact step combines hi and lo, compares with the CTA's running
+//             n-th best per query and queues the survivors; queues are folded into
+//             sorted 32-lane lists with shuffle-based bitonic merges, in rounds that
+//             the warps hold on demand (they do not meet at every tile).
+// Forms (template parameters): TSUB sub-tiles per tile (narrow rows; 33-64 queries on wide
+// rows), DUAL accumulator sets with two issuing threads (wide rows), PACK2 (64-byte keys,
+// two per row), MERGED (one accumulator column per query), HALVES (hi columns, then lo columns).
 // Every wait is bounded; TMEM is freed on every path.
 #pragma once
 #include <type_traits>
