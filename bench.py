@@ -440,10 +440,11 @@ def run_ours(args):
     # so the two are compared burst by burst; medians).
     floor_ms = normal_ms = None
     if dtype != "f32" and args.scan_path != 1:
-        burst, rounds = max(4, min(args.steps, 20)), 7
+        burst, rounds = max(4, min(args.steps, 20)), 12
         t_floor, t_norm = [], []
         for r in range(rounds):
-            for flag, acc in ((1, t_floor), (0, t_norm)):
+            order = ((1, t_floor), (0, t_norm)) if r % 2 == 0 else ((0, t_norm), (1, t_floor))
+            for flag, acc in order:
                 store.set_option("debug_no_select", flag)
                 step(r)
                 f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
