@@ -5,7 +5,7 @@ draft (a serving runtime that owns all device memory through its own pool, a
 plug-in inside another program's budget).  For them the library carries one
 entry point whose workspace is a fixed array inside the library image.  This
 test calls it through the C ABI twice in a row -- the second call finds the
-first call's leftovers in the shared workspace -- and judges each call against
+first call's leftovers in the shared workspace -- and checks each call against
 the CPU oracle with the checker every parity test uses.  As a second check it
 compares with the store-based dresd_retrieve(): for 16-bit stores the
 allocation-free call runs the streaming scoring kernel, so the store is put on
