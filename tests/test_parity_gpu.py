@@ -165,6 +165,26 @@ def test_adversarial_order_both_paths(path):
     _check(keys[order], toks[order], dtype, q, 10, 2, options={"scan_path": path})
 
 
+# Ascending scores in memory (every row beats all rows before it: the queues overflow round after round)
+# for every form of the tcgen05 kernel's epilogue -- rounds on demand with warps at different tiles, the
+# fast rejection and its out-of-line exact step, sub-tiles, two keys per row, keys as N.
+@pytest.mark.parametrize("dtype,d,B,n,N", [
+    ("f16", 64, 64, 32, 148 * 512 + 3000),      # one column per query, four sub-tiles
+    ("bf16", 64, 16, 10, 148 * 512 + 3000),     # hi block | lo block, four sub-tiles
+    ("f16", 32, 8, 10, 148 * 1024 + 3000),      # two keys per row
+    ("bf16", 512, 40, 16, 40000),               # two sub-tiles sharing an operand slab
+    ("f16", 256, 3, 32, 40000),                 # two accumulator sets
+    ("bf16", 256, 33, 32, 60000),               # keys as N
+    ("f16", 1024, 20, 10, 20000),
+])
+def test_adversarial_order_every_epilogue_form(dtype, d, B, n, N):
+    keys, toks = synth.make_store(7280 + d + B, N, d, 4, dtype, 2)
+    q, _ = synth.make_queries(7281 + d + B, keys, dtype, B, 0.1)
+    s = oracle.scores(keys, dtype, oracle.preprocess(q[:1], dtype)[0])
+    order = np.argsort(s, kind="stable")
+    _check(keys[order], toks[order], dtype, q, n, 2)
+
+
 def test_config1_tiny_exact_knn_full():
     w = synth.make_workload("c1_tiny_f32")
     rate = _check(w["keys"], w["next_tokens"], "f32", w["queries"], w["top_n"], w["draft_len"])
