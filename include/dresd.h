@@ -373,6 +373,13 @@ dresd_status dresd_store_debug_selftest(dresd_store *store, void *stream);
  *                compare per key, twice the instructions); 1 = that form for every batch of more
  *                than 16 queries that the keys-as-N form does not take, 2 = never.  Scores agree with
  *                the two-column form to fp32 accumulation order (last bits), within the tolerances.
+ *   "epi_warps"  0 (default): the one-column form on rows of one slab runs sixteen selection warps;
+ *                8 = eight, as every other form.  Results do not change.
+ *   "round_per_tile"  0 (default): the selection warps of the tcgen05 kernel with the keys as M fold
+ *                their candidate queues in rounds held on demand; 1 = a round after every tile (the
+ *                earlier form; token windows and the probe pass always use it).  Results do not change.
+ *   "fast_reject"  1 (default): the kernel with the keys as N tests a unit of 16 scores with packed
+ *                sign-bit arithmetic before the exact compare; 0 = exact compare only.  Results do not change.
  *   "first_token_windows"  1 (default): on a store indexed by dresd_store_index_first_tokens()
  *                filtered calls scan only the rows of their queries' tokens; 0 = scan every row.
  *                Results do not change.

@@ -53,9 +53,9 @@ constexpr int issuers_of(int tsub, bool dual, bool merged = false)
 {
     return (tsub > 1 || dual) ? 2 : 1;
 }
-constexpr int threads_of(int tsub, bool dual, bool merged = false)
+constexpr int threads_of(int tsub, bool dual, bool merged = false, int epi_warps = kEpiWarps)
 {
-    return (2 + kEpiWarps + issuers_of(tsub, dual, merged) - 1) * 32;
+    return (2 + epi_warps + issuers_of(tsub, dual, merged) - 1) * 32;
 }
 constexpr int kTileRows = 128;
 constexpr int kSlabBytes = 128;
@@ -131,7 +131,7 @@ __device__ __forceinline__ void raise_float(float *p, float v)
     if (v >= 0.f) atomicMax(reinterpret_cast<int *>(p), __float_as_int(v));
     else atomicMin(reinterpret_cast<unsigned int *>(p), __float_as_uint(v));
 }
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory"); }
+template <int EW> __device__ __forceinline__ void epi_bar_n() { asm volatile("bar.sync 1, %0;" ::"n"(EW * 32) : "memory"); }
 
 struct EpiFlags {
     int need_merge;
@@ -273,9 +273,10 @@ static __device__ __noinline__ uint32_t epi_select(uint32_t addr, const float *t
 // (K1 writes the operand rows in that order), so that hi and lo of NEIGHBOURING queries sit in neighbouring
 // registers and packed fp32 instructions can combine them: the same one-and-a-half instructions per score
 // fast rejection -- fma.f32x2 (hi + lo/S), add.f32x2 (-tau), sign bits ANDed -- for every two-column form.
+// EW epilogue warps (8, or 16: four per TMEM lane group, a quarter of the columns each).
 template <typename T, int NCOLS, int TSUB, bool PACK2 = false, bool DUAL = false, bool MERGED = false,
-          bool HALVES = false>
-__global__ void __launch_bounds__(threads_of(TSUB, DUAL, MERGED), 1)
+          bool HALVES = false, int EW = kEpiWarps>
+__global__ void __launch_bounds__(threads_of(TSUB, DUAL, MERGED, EW), 1)
 scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_constant__ CUtensorMap q_map,
                  const ScanArgs a, const int q_resident, const int gs)
 {
@@ -334,7 +335,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     // Narrow rows: the sub-tiles of a tile have accumulators of their own, so two threads (warps 1
     // and 10) issue the MMAs of alternate sub-tiles; each commits to the barriers for its share.
     constexpr int kIssuers = issuers_of(TSUB, DUAL, MERGED);
-    constexpr int kIssuer2Warp = 2 + kEpiWarps;
+    constexpr int kIssuer2Warp = 2 + EW;
 
     if (tid == 0) {
         tma_prefetch_desc(&keys_map);                       // kernel parameters: nothing to wait for
@@ -345,7 +346,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&tfull[b], kIssuers);
-            mbar_init(&tempty[b], kEpiWarps);
+            mbar_init(&tempty[b], EW);
         }
         mbar_init(qbar, 1);
         for (int i = 0; i < 4; ++i) {
@@ -363,7 +364,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
     pdl_wait();
     pdl_launch_dependents();
     if (warp >= 2 && warp < kIssuer2Warp) {
-        for (int q = warp - 2; q < NQ; q += kEpiWarps) {
+        for (int q = warp - 2; q < NQ; q += EW) {
             warp_topn_init(&sel[q], lane);
             // start from whatever the grid already knows; padding columns never pass
             if (lane == 0) {
@@ -577,7 +578,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         // ---------------------------------- epilogue ----------------------------------
         // Eight warps: warp w may read TMEM lanes 32*(w&3)..+31 (one key row per thread and
         // sub-tile); the two warps that share a lane group split the accumulator columns.
-        constexpr int CW = NCOLS / 2;                       // columns per warp
+        constexpr int CW = NCOLS / (EW / 4);                // columns per warp
         constexpr int QW = CW / CPQ;                        // queries per warp
         const int ew = warp - 2;                            // 0..7
         const int lane_grp = warp & 3;
@@ -586,7 +587,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         // Few queries on narrow rows (all of them within one warp's columns, several sub-tiles per
         // tile): the two warps of a lane group split the SUB-TILES instead, so that neither spends
         // its time on columns of padding.
-        const bool split_subs = TSUB >= 2 && (PACK2 ? 2 * a.B : a.B) <= QW;
+        const bool split_subs = EW == 8 && TSUB >= 2 && (PACK2 ? 2 * a.B : a.B) <= QW;
         const int qbase = split_subs ? 0 : half * QW;
         // a warp whose columns are all padding (few queries, one sub-tile per tile) only keeps the barriers
         const bool no_cols = qbase >= (PACK2 ? 2 * a.B : a.B);
@@ -678,7 +679,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             return (*reinterpret_cast<volatile int *>(&fl->need_merge) | *reinterpret_cast<volatile int *>(&fl->overflow)) != 0;
         };
         auto one_round = [&]() -> int {
-            epi_bar();                                       // A: every push so far is visible
+            epi_bar_n<EW>();                                       // A: every push so far is visible
             const int need = fl->need_merge, over = fl->overflow;
             last_done = *reinterpret_cast<volatile int *>(done_warps);
             last_over = over;
@@ -692,7 +693,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             round += 1;
             fl = &flags[round % 3];
             if (need | over) {
-                for (int q = ew; q < NQ; q += kEpiWarps) {
+                for (int q = ew; q < NQ; q += EW) {
                     if (sel[q].count > 0) {
                         warp_topn_merge(&sel[q], a.top_n, lane);
                         if (lane == 0 && q < a.B) {
@@ -705,7 +706,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             }
             // C: lists, counts and filter scores are settled.  Free-running warps hold it in every round, so
             // that nobody leaves a round (and counts itself done) before all have read its flags.
-            if ((need | over) || free_run) epi_bar();
+            if ((need | over) || free_run) epi_bar_n<EW>();
             return over;
         };
         auto attend_rounds = [&]() {
@@ -815,10 +816,10 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         slot[lane] = 0ull;
                     }
                 }
-                epi_bar();                                   // all lane groups have written
+                epi_bar_n<EW>();                                   // all lane groups have written
                 // a lane per (query of this warp, sub-tile): the best of the four lane groups joins the queue
                 {
-                    const int q = ew + kEpiWarps * (lane / TSUB), sub = lane % TSUB;
+                    const int q = ew + EW * (lane / TSUB), sub = lane % TSUB;
                     if (q < a.B) {
                         const unsigned long long *m = tilemax + (size_t)(sub * 4) * NQ + (PACK2 ? 2 * q : q);
                         unsigned long long v = umax64(umax64(m[0], m[NQ]), umax64(m[2 * NQ], m[3 * NQ]));
@@ -831,7 +832,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         }
                     }
                 }
-                epi_bar();                                   // slots may be rewritten for the next tile
+                epi_bar_n<EW>();                                   // slots may be rewritten for the next tile
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&tempty[acc]);
@@ -847,7 +848,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             if (cold_tile) {
                 constexpr int kGroupRows = 4 * TSUB;        // 32 groups over the tile's 128 * TSUB rows
                 constexpr int kGroupsPerUnit = 32 / kGroupRows;
-                epi_bar();                                  // tau[] is settled: every warp sees the same cold queries
+                epi_bar_n<EW>();                                  // tau[] is settled: every warp sees the same cold queries
                 uint32_t todo = 0u;
                 for (uint32_t m = active & wmatch; m; m &= m - 1) {
                     const int j = __ffs(m) - 1;
@@ -877,9 +878,9 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         if (lane % kGroupRows == 0) reinterpret_cast<uint32_t *>(sel[qbase + j].queue)[slot] = key;
                     }
                 }
-                epi_bar();
+                epi_bar_n<EW>();
                 const unsigned long long wq = win_on ? win->qmask[wk] : ~0ull;
-                for (int q = ew; q < NQ; q += kEpiWarps) {
+                for (int q = ew; q < NQ; q += EW) {
                     const int rq = PACK2 ? q >> 1 : q;
                     if (rq >= a.B || !((wq >> q) & 1ull) || tau[q] > -INFINITY) continue;   // warp-uniform
                     unsigned long long x = reinterpret_cast<const uint32_t *>(sel[q].queue)[lane];
@@ -896,7 +897,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         }
                     }
                 }
-                epi_bar();
+                epi_bar_n<EW>();
             }
             uint32_t pending[TSUB];                         // queries whose candidate found the queue full
 #pragma unroll
@@ -1020,13 +1021,13 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             if (lane == 0) atomicAdd(done_warps, 1);
             while (true) {
                 one_round();
-                if (last_done == kEpiWarps && !last_over) break;
+                if (last_done == EW && !last_over) break;
             }
         } else {
-            epi_bar();
+            epi_bar_n<EW>();
         }
         // flush and publish this CTA's lists
-        for (int q = ew; q < NQ; q += kEpiWarps) {
+        for (int q = ew; q < NQ; q += EW) {
             if (sel[q].count > 0) warp_topn_merge(&sel[q], a.top_n, lane);
             if (q < a.B) {
                 unsigned long long m = sel[q].list[lane];

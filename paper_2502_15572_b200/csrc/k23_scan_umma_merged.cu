@@ -25,6 +25,20 @@ cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const S
                                         p.q_resident, p.gs);
             }
         }
+        if constexpr (NCOLS == 64 && TSUB == 4) {
+            // Sixteen epilogue warps (four per TMEM lane group, a quarter of the queries each) where the tile
+            // has four sub-tiles: the epilogue is bound by latency, not by issue slots (the schedulers
+            // issue 37 % of the time with eight), and twice the warps hide more of it.  Interleaved A/B,
+            // 3 GB fp16 stores, 8 -> 16 warps: d = 64, 64 queries 0.778 -> 0.746 ms, with n = 32
+            // 0.916 -> 0.807, 40 queries 0.734 -> 0.692; d = 32 1.132 -> 1.096.
+            if (a.epi_warps != 8) {
+                auto kernel = scan_umma_kernel<T, NCOLS, TSUB, false, false, true, false, 16>;
+                cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
+                if (e != cudaSuccess) return e;
+                return launch_dependent(kernel, dim3(grid), dim3(threads_of(TSUB, false, true, 16)), p.smem, stream, kmap,
+                                        qmap, a, p.q_resident, p.gs);
+            }
+        }
         auto kernel = scan_umma_kernel<T, NCOLS, TSUB, false, false, true>;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
         if (e != cudaSuccess) return e;

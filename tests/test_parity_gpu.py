@@ -185,6 +185,26 @@ def test_adversarial_order_every_epilogue_form(dtype, d, B, n, N):
     _check(keys[order], toks[order], dtype, q, n, 2)
 
 
+# Measurement switches that select another form of the same computation: results must not change.
+@pytest.mark.parametrize("dtype,d,B,n,N,options", [
+    ("f16", 64, 64, 32, 148 * 512 * 2 + 77, {"epi_warps": 8}),          # one column per query on eight warps
+    ("bf16", 64, 40, 10, 60013, {"epi_warps": 8}),
+    ("f16", 64, 16, 10, 148 * 512 * 2 + 77, {"round_per_tile": 1}),     # a round after every tile
+    ("bf16", 512, 64, 16, 30011, {"round_per_tile": 1}),
+    ("bf16", 256, 48, 32, 148 * 256 * 2 + 5, {"fast_reject": 0}),       # keys as N, exact compare only
+    ("f16", 64, 48, 10, 60013, {"merged_columns": 2}),                  # two columns per query
+    ("f16", 320, 24, 10, 30011, {"merged_columns": 1}),                 # one column per query on wide rows
+])
+def test_measurement_switches_do_not_change_results(dtype, d, B, n, N, options):
+    keys, toks = synth.make_store(7700 + d + B, N, d, 16, dtype, 3)
+    q, _ = synth.make_queries(7701 + d + B, keys, dtype, B, 0.1)
+    ids, sc, tok, o = run_both(keys, toks, dtype, q, n, 2, options=options)
+    checker.check_batch(o.full_scores, toks, ids, sc, tok, dtype, n, 2, oracle_ids=o.ids)
+    ids0, sc0, tok0, _ = run_both(keys, toks, dtype, q, n, 2)
+    assert np.array_equal(tok0, tok) or np.array_equal(ids0, ids)      # ids may swap only inside rounding ties
+    np.testing.assert_allclose(sc, sc0, atol=2 * checker.EPS_ACC[dtype], rtol=0)
+
+
 def test_config1_tiny_exact_knn_full():
     w = synth.make_workload("c1_tiny_f32")
     rate = _check(w["keys"], w["next_tokens"], "f32", w["queries"], w["top_n"], w["draft_len"])
