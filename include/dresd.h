@@ -373,8 +373,10 @@ dresd_status dresd_store_debug_selftest(dresd_store *store, void *stream);
  *                compare per key, twice the instructions); 1 = that form for every batch of more
  *                than 16 queries that the keys-as-N form does not take, 2 = never.  Scores agree with
  *                the two-column form to fp32 accumulation order (last bits), within the tolerances.
- *   "epi_warps"  0 (default): the one-column form on rows of one slab runs sixteen selection warps;
- *                8 = eight, as every other form.  Results do not change.
+ *   "epi_warps"  0 (default): the forms for 33-64 queries with several sub-tiles per tile (one column
+ *                per query on one-slab rows; two columns per query on rows of two slabs and on rows
+ *                wider than 256) run sixteen selection warps; 8 = eight, as every other form.
+ *                Results do not change.
  *   "round_per_tile"  0 (default): the selection warps of the tcgen05 kernel with the keys as M fold
  *                their candidate queues in rounds held on demand; 1 = a round after every tile (the
  *                earlier form; token windows and the probe pass always use it).  Results do not change.

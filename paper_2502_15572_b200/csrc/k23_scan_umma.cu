@@ -26,6 +26,20 @@ cudaError_t launch_one(const CUtensorMap &kmap, const CUtensorMap &qmap, const S
                                         p.q_resident, p.gs);
             }
         }
+        if constexpr (HALVES && TSUB > 1 && NCOLS == 128) {
+            // 33-64 queries, two sub-tiles per tile: sixteen selection warps (four per TMEM lane group, a
+            // quarter of the queries each) hide more of the epilogue's latency than eight.  Interleaved A/B,
+            // 3 GB stores, 8 -> 16 warps: d = 128 0.638 -> 0.632 ms (n = 32: 0.738 -> 0.676), d = 512
+            // 0.693 -> 0.671, d = 2048 0.634 -> 0.616, d = 1024 with 40 queries and n = 32 0.682 -> 0.640;
+            // with 17-32 queries (64 columns) eight warps stay ahead (d = 128: 0.521 against 0.540).
+            if (a.epi_warps != 8) {
+                auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, false, false, HALVES, 16>;
+                cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
+                if (e != cudaSuccess) return e;
+                return launch_dependent(kernel, dim3(grid), dim3(threads_of(TSUB, false, false, 16)), p.smem, stream, kmap,
+                                        qmap, a, p.q_resident, p.gs);
+            }
+        }
         auto kernel = scan_umma_kernel<T, NCOLS, TSUB, PACK2, false, false, HALVES>;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem);
         if (e != cudaSuccess) return e;

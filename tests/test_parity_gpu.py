@@ -189,6 +189,8 @@ def test_adversarial_order_every_epilogue_form(dtype, d, B, n, N):
 @pytest.mark.parametrize("dtype,d,B,n,N,options", [
     ("f16", 64, 64, 32, 148 * 512 * 2 + 77, {"epi_warps": 8}),          # one column per query on eight warps
     ("bf16", 64, 40, 10, 60013, {"epi_warps": 8}),
+    ("f16", 128, 64, 16, 60013, {"epi_warps": 8}),                      # two columns, two sub-tiles, eight warps
+    ("bf16", 1024, 48, 10, 20011, {"epi_warps": 8}),
     ("f16", 64, 16, 10, 148 * 512 * 2 + 77, {"round_per_tile": 1}),     # a round after every tile
     ("bf16", 512, 64, 16, 30011, {"round_per_tile": 1}),
     ("bf16", 256, 48, 32, 148 * 256 * 2 + 5, {"fast_reject": 0}),       # keys as N, exact compare only

@@ -25,7 +25,8 @@ pytestmark = pytest.mark.gpu
     ("bf16", 4096, 16, 2003, {}),                       # tcgen05, query operand travelling with the key slabs
     ("f16", 64, 40, 148 * 512 * 2 + 77, {}),            # tcgen05, one column per query, sixteen selection warps
     ("bf16", 32, 4, 148 * 1024 * 2 + 78, {}),           # tcgen05, two keys per row
-    ("f16", 512, 64, 60013, {}),                        # tcgen05, two sub-tiles sharing an operand slab
+    ("f16", 512, 64, 60013, {}),                        # tcgen05, two sub-tiles sharing an operand slab, sixteen warps
+    ("f16", 512, 64, 60013, {"epi_warps": 8}),
     ("bf16", 256, 40, 148 * 256 * 2 + 5, {}),           # tcgen05, keys as the N operand
     ("f16", 256, 40, 60013, {"keys_as_m": 1}),          # tcgen05, keys as M, 128 accumulator columns
     ("f32", 128, 4, 148 * 512 * 2 + 19, {}),            # fp32 keys, FFMA kernel
