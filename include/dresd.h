@@ -373,6 +373,8 @@ dresd_status dresd_store_debug_selftest(dresd_store *store, void *stream);
  *                compare per key, twice the instructions); 1 = that form for every batch of more
  *                than 16 queries that the keys-as-N form does not take, 2 = never.  Scores agree with
  *                the two-column form to fp32 accumulation order (last bits), within the tolerances.
+ *   "merge_level"  0 (default, = 24): the tcgen05 kernels fold a query's queue of 32 candidates into its
+ *                sorted list once it holds this many (1..32).  Results do not change.
  *   "epi_warps"  0 (default): the forms for 33-64 queries with several sub-tiles per tile (one column
  *                per query on one-slab rows; two columns per query on rows of two slabs and on rows
  *                wider than 256) run sixteen selection warps; 8 = eight, as every other form.

@@ -138,7 +138,7 @@ struct dresd_store {
     CUtensorMap map_umma;
     CUtensorMap map_q[4];        // box rows 16 / 32 / 64 / 128 over qsplit
     // options / bookkeeping
-    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m, opt_pack2, opt_merged, opt_round_per_tile, opt_no_fast_reject, opt_epi_warps;
+    int opt_path, opt_grid, opt_probe, opt_wait_ms, opt_lose_stage, opt_no_select, opt_keys_as_m, opt_pack2, opt_merged, opt_round_per_tile, opt_no_fast_reject, opt_epi_warps, opt_merge_level;
     double last_key_passes;      // passes over the key matrix in the last call (a probe pass counts 1/stride)
     const void *k8;              // 8-bit (E4M3) copy of the keys, borrowed; null = none attached
     void *qsplit8;               // [2 * kMaxBatch][dpad8] 8-bit query operand
@@ -329,6 +329,7 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         a.round_per_tile = s->opt_round_per_tile;
         a.no_fast_reject = s->opt_no_fast_reject;
         a.epi_warps = s->opt_epi_warps;
+        a.merge_level = s->opt_merge_level;
         a.wait_cycles = (long long)s->opt_wait_ms * 2000000LL;     // ~2 GHz
         a.debug_lose_stage = s->opt_lose_stage;
         if (windows) {
@@ -799,6 +800,11 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
     if (strcmp(name, "first_token_windows") == 0) {
         if (value != 0 && value != 1) return fail(DRESD_ERR_INVALID, "first_token_windows takes 0 or 1");
         s->opt_windows = value;
+        return DRESD_OK;
+    }
+    if (strcmp(name, "merge_level") == 0) {
+        if (value < 0 || value > 32) return fail(DRESD_ERR_INVALID, "merge_level outside 0..32");
+        s->opt_merge_level = value;
         return DRESD_OK;
     }
     if (strcmp(name, "epi_warps") == 0) {

@@ -79,6 +79,7 @@ struct ScanArgs {
     int probe_max;          // tcgen05 kernel, probe pass: keep only each tile's best row per query
     int no_select;          // tcgen05 kernel, measurement only: nothing passes the filter (scan floor)
     int keys_as_m;          // tcgen05 kernels: never use the form with the keys as the N = 256 operand
+    int merge_level;        // tcgen05 kernels: a round is asked for when a queue holds this many (0 = 16) (measurement)
     int epi_warps;          // tcgen05 kernel, one column per query: 16 = sixteen epilogue warps (measurement)
     int no_fast_reject;     // tcgen05 kernel, keys as N: skip the packed sign-bit rejection ahead of the exact compare (measurement)
     int round_per_tile;     // tcgen05 kernel, keys as M: the epilogue warps meet at every tile (measurement)

@@ -194,7 +194,7 @@ __device__ __forceinline__ void tmem_ld_acc(uint32_t addr, uint32_t (&r)[CW])
 template <int CW, int QW, int NQ, int NCOLS, bool DUAL, bool MERGED>
 static __device__ __noinline__ uint32_t epi_select(uint32_t addr, const float *tau_q, const int *want_q, int tok,
                                                    uint32_t wild, int filtered, uint32_t allow, float inv,
-                                                   WarpTopN *sel_q, uint32_t row, EpiFlags *fl)
+                                                   WarpTopN *sel_q, uint32_t row, EpiFlags *fl, int mlevel)
 {
     uint32_t r[CW];
     tmem_ld_acc<CW, QW, NQ, NCOLS, DUAL, !MERGED>(addr, r);
@@ -246,7 +246,7 @@ static __device__ __noinline__ uint32_t epi_select(uint32_t addr, const float *t
             const int slot = atomicAdd(&sel_q[j].count, 1);
             if (slot < kQueueCap) {
                 sel_q[j].queue[slot] = pack_candidate(sc, row);
-                if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
+                if (slot + 1 >= mlevel) fl->need_merge = 1;
             } else {
                 pend |= 1u << j;
                 fl->overflow = 1;
@@ -593,6 +593,8 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
         const bool no_cols = qbase >= (PACK2 ? 2 * a.B : a.B);
         const uint32_t lane_addr = tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(qbase * (HALVES ? 1 : CPQ));
         const float inv = a.lo_inv_scale;
+        // a round is asked for when a queue of 32 holds this many: 24 measured 1-4 % ahead of 16 (fewer rounds)
+        const int mlevel = a.merge_level > 0 ? a.merge_level : 24;
         // score of this warp's j-th query from the registers of ld_cols: hi + lo / S, or acc / S
         auto score_at = [&](const uint32_t (&r)[CW], int j) -> float {
             if constexpr (MERGED) return __uint_as_float(r[j]) * inv;
@@ -946,7 +948,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                         }
                         pending[sub] = epi_select<CW, QW, NQ, NCOLS, DUAL, MERGED>(
                             acc_addr + (uint32_t)(sub * NCOLS), tau + qbase, want_s + qbase, tok[sub], wild, filtered ? 1 : 0,
-                            first ? (okmask & wmatch) : pending[sub], inv, sel + qbase, (uint32_t)row, fl);
+                            first ? (okmask & wmatch) : pending[sub], inv, sel + qbase, (uint32_t)row, fl, mlevel);
                         continue;
                     }
                     uint32_t r[CW];
@@ -993,7 +995,7 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
                             const int slot = atomicAdd(&sel[q].count, 1);
                             if (slot < kQueueCap) {
                                 sel[q].queue[slot] = pack_candidate(s, id);
-                                if (slot + 1 >= kMergeLevel) fl->need_merge = 1;
+                                if (slot + 1 >= mlevel) fl->need_merge = 1;
                             } else {
                                 pending[sub] |= 1u << j;
                                 fl->overflow = 1;

@@ -195,6 +195,8 @@ def test_adversarial_order_every_epilogue_form(dtype, d, B, n, N):
     ("bf16", 512, 64, 16, 30011, {"round_per_tile": 1}),
     ("bf16", 256, 48, 32, 148 * 256 * 2 + 5, {"fast_reject": 0}),       # keys as N, exact compare only
     ("f16", 64, 48, 10, 60013, {"merged_columns": 2}),                  # two columns per query
+    ("bf16", 256, 64, 32, 60013, {"merge_level": 8}),                   # queues folded early ...
+    ("f16", 64, 20, 32, 60013, {"merge_level": 32}),                    # ... and only when full
     ("f16", 320, 24, 10, 30011, {"merged_columns": 1}),                 # one column per query on wide rows
 ])
 def test_measurement_switches_do_not_change_results(dtype, d, B, n, N, options):
