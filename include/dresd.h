@@ -358,7 +358,9 @@ dresd_status dresd_store_debug_selftest(dresd_store *store, void *stream);
  *   "grid"       CTAs of the scoring kernel, 0 = one per SM.
  *   "probe"      large batches on large stores first run a probe pass over every
  *                value-th key tile to seed the selection filter; 0 = never,
- *                1 = default stride (128).
+ *                1 (default) = a stride that follows the call: 64 (64 queries x top-32) to 256
+ *                (few results), less on a small store (at least one probe tile per CTA, no probe
+ *                pass below eight tiles per CTA).
  *   "pack2"      1 (default): 64-byte keys are scanned as rows of two keys (one 128-byte line) --
  *                the 8-bit copy of a store with d = 64 in the quantised search (up to 32 queries
  *                per call), and a 16-bit store with d = 32 and an even number of rows in the exact

@@ -31,7 +31,7 @@ dresd_status fail_cuda(cudaError_t e, const char *what)
 }
 
 constexpr uint32_t kMagic = 0xD2E5D001u;
-constexpr int kProbeStride = 128;    // default: the probe pass visits every 128th tile
+constexpr int kProbeAuto = 1;        // default: the stride follows the store (about four probe tiles per CTA)
 constexpr float kEpsNorm = 1e-12f;   // epsilon of Eq. 2 (the paper leaves it open)
 
 bool is_device_ptr(const void *p)
@@ -347,7 +347,20 @@ dresd_status run_retrieve(dresd_store *s, const void *queries, int B, int top_n,
         // n-th best score per query seeds the grid-wide filter, so that the full pass
         // queues ~pstride n survivors per query GPU-wide instead of ~n ln(rows/n) per CTA.
         // The filter only rejects rows that cannot be in the result.
-        const int pstride = s->opt_probe;
+        int pstride = s->opt_probe;
+        if (pstride == kProbeAuto) {
+            // The full pass queues ~pstride n survivors per query, the probe pass costs 1/pstride of a full
+            // pass plus its fixed part (launch, set-up, one tile's latency): the best stride falls with
+            // sqrt(B n) -- 64 measured best at 64 queries x top-32, 128-256 at top-10 -- and a small
+            // store still gets one probe tile per CTA.
+            const double t = 2900.0 / sqrt((double)B * sel_n);
+            pstride = t < 64.0 ? 64 : t > 256.0 ? 256 : (int)t;
+            // one best per 128 rows and CTA must fit the CTA's queue of 32 (the cheap form of the probe pass)
+            const long long fit = ((long long)n_tiles * (umma_rows / 128) + 32LL * grid - 1) / (32LL * grid);
+            if (pstride < fit) pstride = (int)fit;
+            if ((long long)pstride * grid > n_tiles) pstride = n_tiles / grid;
+            if (pstride < 2) pstride = 0;
+        }
         if (pstride > 1 && !s->opt_no_select && B * sel_n >= 256 && n_tiles >= pstride * grid) {
             ScanArgs pa = a;
             pa.tile_stride = pstride;
@@ -489,7 +502,7 @@ dresd_status dresd_store_create(const void *keys, const int32_t *next_tokens, in
     s->d_in = d;
     s->eps_z = 1e-5f;
     s->max_grid = 2 * s->num_sms;
-    s->opt_probe = kProbeStride;
+    s->opt_probe = kProbeAuto;
     s->opt_pack2 = 1;
     s->opt_windows = 1;
 
@@ -834,7 +847,7 @@ dresd_status dresd_store_set_option(dresd_store *s, const char *name, int value)
     }
     if (strcmp(name, "probe") == 0) {
         if (value < 0 || value > 65536) return fail(DRESD_ERR_INVALID, "probe = %d outside 0..65536", value);
-        s->opt_probe = value == 1 ? kProbeStride : value;
+        s->opt_probe = value;
         return DRESD_OK;
     }
     if (strcmp(name, "grid") == 0) {
