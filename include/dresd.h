@@ -369,7 +369,7 @@ dresd_status dresd_store_debug_selftest(dresd_store *store, void *stream);
  *                tcgen05 kernel with the queries as the M = 128 and the keys as the
  *                N = 256 operand of the instruction; 1 = keys as the M operand at every
  *                batch size (the form all other shapes use).  Results do not change.
- *   "merged_columns"  0 (default): batches of 17-64 queries on rows of at most 64 elements run the
+ *   "merged_columns"  0 (default): batches of 33-64 queries on rows of at most 64 elements run the
  *                tcgen05 kernel with ONE accumulator column per query (both 16-bit terms of the query
  *                are accumulated into the same column, scaled by a power of two; half the columns to
  *                compare per key, twice the instructions); 1 = that form for every batch of more

@@ -129,15 +129,18 @@ UmmaPlan umma_make_plan(int d, int B, bool merged)
     return p;
 }
 
-// One accumulator column per query: for more than 16 queries on rows of at most 64 elements (one
+// One accumulator column per query: for more than 32 queries on rows of at most 64 elements (one
 // slab), where the epilogue -- the compares per key and query -- sets the pace.  Measured on 3 GB
-// fp16 stores, two columns -> one column per query: d = 64, 64 queries 0.90 -> 0.68 ms, 32 queries
-// 0.65 -> 0.60; d = 32, 64 queries 1.72 -> 1.04.  From two slabs per row on, twice the instructions
-// cost more than half the columns save (d = 128, 64 queries: 0.58 against 0.64 ms; d = 512: 0.73
-// against 0.93).
+// fp16 stores, two columns -> one column per query: d = 64, 64 queries 0.90 -> 0.68 ms; d = 32,
+// 64 queries 1.72 -> 1.04.  With 17-32 queries the two-column form (hi block | lo block, one
+// instruction per K-step instead of two) is the faster one since its rejection test went to packed
+// arithmetic: d = 64, 17 / 24 / 32 queries 0.61 / 0.65 / 0.66 -> 0.54 / 0.58 / 0.58 ms, 46.3M rows at
+// 32 queries 1.24 -> 1.05; d = 48 0.80 -> 0.70; d = 32 0.88 -> 0.85 (interleaved A/B).  From two slabs
+// per row on, twice the instructions cost more than half the columns save (d = 128, 64 queries:
+// 0.58 against 0.64 ms; d = 512: 0.73 against 0.93).
 bool scan_umma_merged_eligible(int d, int B, int dtype)
 {
-    return dtype != kE4M3 && B > 16 && d <= kSlabElems;
+    return dtype != kE4M3 && B > 32 && d <= kSlabElems;
 }
 
 int scan_umma_tile_rows(int d, int B, int keys_as_m, int merged)

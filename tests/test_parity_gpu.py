@@ -171,6 +171,7 @@ def test_adversarial_order_both_paths(path):
 @pytest.mark.parametrize("dtype,d,B,n,N", [
     ("f16", 64, 64, 32, 148 * 512 + 3000),      # one column per query, four sub-tiles
     ("bf16", 64, 16, 10, 148 * 512 + 3000),     # hi block | lo block, four sub-tiles
+    ("f16", 64, 28, 10, 148 * 512 + 3000),      # the same with 64 columns (17-32 queries)
     ("f16", 32, 8, 10, 148 * 1024 + 3000),      # two keys per row
     ("bf16", 512, 40, 16, 40000),               # two sub-tiles sharing an operand slab
     ("f16", 256, 3, 32, 40000),                 # two accumulator sets
@@ -198,6 +199,7 @@ def test_adversarial_order_every_epilogue_form(dtype, d, B, n, N):
     ("bf16", 256, 64, 32, 60013, {"merge_level": 8}),                   # queues folded early ...
     ("f16", 64, 20, 32, 60013, {"merge_level": 32}),                    # ... and only when full
     ("f16", 320, 24, 10, 30011, {"merged_columns": 1}),                 # one column per query on wide rows
+    ("bf16", 64, 24, 10, 148 * 512 * 2 + 77, {"merged_columns": 1}),    # ... and for 17-32 queries (32 columns)
 ])
 def test_measurement_switches_do_not_change_results(dtype, d, B, n, N, options):
     keys, toks = synth.make_store(7700 + d + B, N, d, 16, dtype, 3)
