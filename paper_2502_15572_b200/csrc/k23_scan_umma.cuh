@@ -751,20 +751,21 @@ scan_umma_kernel(const __grid_constant__ CUtensorMap keys_map, const __grid_cons
             const bool pull = (tl & 3) == 0 && et < a.B && !a.no_select;
             unsigned int gword = 0u;
             if (pull) gword = *reinterpret_cast<const volatile unsigned int *>(&a.gtau[et]);
-            if (!dead && !mbar_try_wait(&tfull[acc], use & 1)) {
+            // The wait is decided warp-wide (votes): what follows -- rounds with their CTA barriers, tcgen05.ld --
+            // needs the whole warp, so no lane may leave the loop, or enter a round, on its own view of the barrier.
+            if (!__all_sync(0xFFFFFFFFu, dead || mbar_try_wait(&tfull[acc], use & 1))) {
                 const long long t0 = clock64();
-                while (!mbar_try_wait(&tfull[acc], use & 1)) {
+                while (!__all_sync(0xFFFFFFFFu, mbar_try_wait(&tfull[acc], use & 1))) {
                     // a warp that waits at the round's barrier holds its accumulator buffer, which this
                     // wait may depend on: rounds are attended from here too
-                    if (free_run && round_wanted()) attend_rounds();
-                    if (clock64() - t0 > wl) {
-                        report_timeout(a.status);
+                    if (free_run && __any_sync(0xFFFFFFFFu, round_wanted())) attend_rounds();
+                    if (__any_sync(0xFFFFFFFFu, clock64() - t0 > wl)) {
+                        if (lane == 0) report_timeout(a.status);
                         dead = true;
                         break;
                     }
                 }
             }
-            dead = __any_sync(0xFFFFFFFFu, dead);
             tc_fence_after();
             if (pull && gword) {
                 const float g = ordered_to_float(gword);
