@@ -186,6 +186,20 @@ def test_adversarial_order_every_epilogue_form(dtype, d, B, n, N):
     _check(keys[order], toks[order], dtype, q, n, 2)
 
 
+# Forty and more tiles per CTA without a probe pass: the lists fill from nothing in every CTA, rounds are asked
+# for tile after tile while the selection warps are at different tiles (two accumulator buffers apart), and the
+# warps that wait for an accumulator attend them from their polling loops.
+@pytest.mark.parametrize("dtype,d,B,n,N", [
+    ("f16", 64, 10, 10, 148 * 512 * 24 + 333),      # hi block | lo block, four sub-tiles
+    ("bf16", 64, 40, 16, 148 * 512 * 12 + 5),       # one column per query, sixteen selection warps
+    ("f16", 256, 5, 32, 148 * 128 * 40 + 77),       # two accumulator sets
+])
+def test_rounds_on_demand_over_many_tiles(dtype, d, B, n, N):
+    keys, toks = synth.make_store(7800 + d + B, N, d, 4, dtype, 2)
+    q, _ = synth.make_queries(7801 + d + B, keys, dtype, B, 0.1)
+    _check(keys, toks, dtype, q, n, 2, options={"probe": 0})
+
+
 # Measurement switches that select another form of the same computation: results must not change.
 @pytest.mark.parametrize("dtype,d,B,n,N,options", [
     ("f16", 64, 64, 32, 148 * 512 * 2 + 77, {"epi_warps": 8}),          # one column per query on eight warps
