@@ -53,7 +53,7 @@ def parse_args():
                     help="N > 1: the rows of ONE datastore are split over the ranks (every rank answers every query "
                          "from its rows, the per-rank results are all-gathered and merged on the device): strong scaling. "
                          "Default: every rank holds a replica and serves its own slice of the query stream (weak)")
-    ap.add_argument("--oracle-queries", type=int, default=2)
+    ap.add_argument("--oracle-queries", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--build-keys", action="store_true",
                     help="time dresd_build_keys (datastore-side Eq. 1 -> v W -> Eq. 2, a tensor-bound GEMM) instead")
