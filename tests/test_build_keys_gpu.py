@@ -53,6 +53,9 @@ def test_build_keys_matches_oracle_preprocess(dtype, N, d_in, d, zscore, centre,
         binding.dresd_set_global_option("build_keys_pairs", 1)
 
 
+_ORACLE = {}
+
+
 def _check_build(dtype, N, d_in, d, zscore, centre):
     mean, var, W = synth.make_preprocess(6100 + d, d_in, d, dtype)
     hidden = synth.make_hidden_queries(6200 + d, N, d_in, dtype)
@@ -64,7 +67,11 @@ def _check_build(dtype, N, d_in, d, zscore, centre):
                                                    "bf16": __import__("torch").int16}[dtype]).numpy()
                                    if dtype == "f16" else got.cpu().view(__import__("torch").int16).numpy().view(np.uint16),
                                    dtype).astype(np.float64)
-    want = oracle.preprocess(hidden, dtype, mean=mean, var=var, eps_z=1e-5, W=W, pca_mean=pm)
+    # the oracle's result does not depend on the launch form: computed once per case (seeded inputs; ~80 MB in all)
+    key = (dtype, N, d_in, d, zscore, centre)
+    if key not in _ORACLE:
+        _ORACLE[key] = oracle.preprocess(hidden, dtype, mean=mean, var=var, eps_z=1e-5, W=W, pca_mean=pm)
+    want = _ORACLE[key]
     # Stored values: the float64 result rounded to the store dtype, up to the arithmetic
     # error of the GEMM before that rounding.  That error is absolute (it scales with the
     # row, not the element): W / sigma is carried as two 16-bit terms (2^-17 relative per
